@@ -1,0 +1,345 @@
+"""Pins for the fp64 oracle: each test ties it to something other than itself --
+a reduction between the paper's own definitions, an independently written dense
+numpy routine on a special case, brute force on tiny inputs, or an invariant."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2608_14385_b200 import synth
+from tests.common import oracle_cfg, oracle_weights, silu, widen
+
+SMALL = synth.LayerShape("small", hidden=48, n_dept=3, experts_per_dept=4, ffn=40, priv=24, top_k=3,
+                         weight_dtype=1, act_dtype=1)
+
+
+def _layer(shape, seed=0, std=None):
+    w = synth.make_deamoe_weights(shape, seed)
+    if std is not None:       # larger weights so that non-linearities matter in small layers
+        for k in w:
+            if k != "router":
+                w[k] = (w[k].float() * (std / synth.W_STD)).to(w[k].dtype)
+    return w
+
+
+# ---------------------------------------------------------------- routing (Eq. 2, gate weights)
+
+def test_topk_is_max_sum_subset_bruteforce():
+    """Eq. (2): on tiny inputs the selected set must be the k-subset with the largest logit sum."""
+    shape = synth.LayerShape("t", hidden=16, n_dept=2, experts_per_dept=4, ffn=8, priv=0, top_k=3,
+                             weight_dtype=0, act_dtype=0)
+    cfg = oracle_cfg(shape)
+    for seed in range(5):
+        router = synth.normal((8, 16), 1.0, seed, "r").numpy()
+        tokens = synth.normal((6, 16), 1.0, seed, "x").numpy()
+        got = ref.route(cfg, router, tokens, want_logits=True)
+        np.testing.assert_allclose(got["logits"], tokens.astype(np.float64) @ router.astype(np.float64).T,
+                                   rtol=1e-12, atol=1e-12)
+        for t in range(6):
+            l = got["logits"][t]
+            best = max(itertools.combinations(range(8), 3), key=lambda s: sum(l[list(s)]))
+            assert set(got["idx"][t]) == set(best)
+            assert list(l[got["idx"][t]]) == sorted(l[got["idx"][t]], reverse=True)
+
+
+def test_topk_ties_go_to_lowest_index_all_permutations():
+    """Exactly representable logits with repeated values, every ordering of the experts."""
+    shape = synth.LayerShape("t", hidden=4, n_dept=1, experts_per_dept=5, ffn=8, priv=0, top_k=3,
+                             weight_dtype=0, act_dtype=0)
+    cfg = oracle_cfg(shape)
+    values = [2.0, 1.0, 1.0, 1.0, 0.5]
+    tokens = np.array([[1.0, 0.0, 0.0, 0.0]], np.float32)
+    for perm in itertools.permutations(range(5)):
+        router = np.zeros((5, 4), np.float32)
+        for slot, src in enumerate(perm):
+            router[slot, 0] = values[src]
+        got = ref.route(cfg, router, tokens)["idx"][0]
+        order = sorted(range(5), key=lambda i: (-router[i, 0], i))[:3]
+        assert list(got) == order
+    # all logits equal: the first k indices in order
+    got = ref.route(cfg, np.ones((5, 4), np.float32), tokens)
+    assert list(got["idx"][0]) == [0, 1, 2]
+    assert got["gap"][0] == 0.0
+
+
+def test_gate_weights_are_renormalised_full_softmax():
+    """p over the selection == softmax over all n followed by renormalisation; sum == route_scale;
+    norm_topk = 0 returns the plain full-softmax entries."""
+    shape = SMALL.with_(route_scale=2.5)
+    cfg = oracle_cfg(shape)
+    router = synth.normal((12, 48), 0.3, 1, "r").numpy()
+    tokens = synth.to_numpy(synth.make_tokens(shape, 5, 1))
+    got = ref.route(cfg, router, tokens, want_logits=True)
+    full = np.exp(got["logits"] - got["logits"].max(1, keepdims=True))
+    full /= full.sum(1, keepdims=True)
+    for t in range(5):
+        sel = full[t, got["idx"][t]]
+        np.testing.assert_allclose(got["w"][t], 2.5 * sel / sel.sum(), rtol=1e-12)
+        assert abs(got["w"][t].sum() - 2.5) < 1e-12
+    cfg0 = oracle_cfg(shape.with_(norm_topk=0, route_scale=1.0))
+    got0 = ref.route(cfg0, router, tokens)
+    for t in range(5):
+        np.testing.assert_allclose(got0["w"][t], full[t, got0["idx"][t]], rtol=1e-12)
+
+
+def test_group_limited_routing_bruteforce():
+    """k_dept cap: the selection is the flat top-k restricted to the k_dept departments with the
+    largest best logit, so it never spans more than k_dept departments; k_dept = m changes nothing."""
+    shape = synth.LayerShape("t", hidden=16, n_dept=4, experts_per_dept=3, ffn=8, priv=0, top_k=4,
+                             k_dept=2, weight_dtype=0, act_dtype=0)
+    router = synth.normal((12, 16), 1.0, 3, "r").numpy()
+    tokens = synth.normal((9, 16), 1.0, 3, "x").numpy()
+    got = ref.route(oracle_cfg(shape), router, tokens, want_logits=True)
+    flat = ref.route(oracle_cfg(shape.with_(k_dept=4)), router, tokens)
+    free = ref.route(oracle_cfg(shape.with_(k_dept=0)), router, tokens)
+    assert (flat["idx"] == free["idx"]).all()
+    for t in range(9):
+        l = got["logits"][t]
+        score = [max(l[j * 3:(j + 1) * 3]) for j in range(4)]
+        keep = sorted(range(4), key=lambda j: (-score[j], j))[:2]
+        cand = [i for i in range(12) if i // 3 in keep]
+        want = sorted(cand, key=lambda i: (-l[i], i))[:4]
+        assert list(got["idx"][t]) == want
+        assert len({i // 3 for i in got["idx"][t]}) <= 2
+
+
+# ---------------------------------------------------------------- Section 3.2 sets and lists
+
+def test_bucketing_matches_python_sets():
+    shape = SMALL
+    cfg = oracle_cfg(shape)
+    g, m, n = shape.experts_per_dept, shape.n_dept, shape.n_expert
+    for seed in range(4):
+        B = 1 + 3 * seed
+        picks = synth.uniform_ints(B * n, 1 << 20, seed, "pick")
+        idx = np.array([sorted(range(n), key=lambda i: (picks[t * n + i], i))[:shape.top_k]
+                        for t in range(B)], np.int32)
+        got = ref.bucket(cfg, idx)
+        for j in range(m):
+            want = [t for t in range(B) if any(i // g == j for i in idx[t])]
+            assert list(got["dept_tok"][got["dept_off"][j]:got["dept_off"][j + 1]]) == want
+            assert bool(int(got["dept_mask"][0]) >> j & 1) == bool(want)
+        for i in range(n):
+            want = [t for t in range(B) if i in idx[t]]
+            assert list(got["expert_tok"][got["expert_off"][i]:got["expert_off"][i + 1]]) == want
+        assert got["expert_off"][n] == B * shape.top_k
+
+
+# ---------------------------------------------------------------- reductions of Eq. (4)
+
+def test_one_expert_per_department_without_private_parts_is_vanilla_moe():
+    """g = 1, no private parameters, no interface non-linearity: Eq. (4) is Eq. (1), and the
+    DeaMoE layer must equal the standard MoE layer on the same matrices."""
+    shape = synth.LayerShape("p1", hidden=32, n_dept=6, experts_per_dept=1, ffn=24, priv=0, top_k=2,
+                             sigma=0, n_shared=1, shared_ffn=16)
+    cfg = oracle_cfg(shape)
+    w = oracle_weights(_layer(shape, 2, std=0.3))
+    tokens = synth.to_numpy(synth.make_tokens(shape, 5, 2))
+    a = ref.deamoe_forward(cfg, w, tokens)
+    b = ref.vanilla_forward(cfg, w, tokens)
+    assert (a["idx"] == b["idx"]).all()
+    np.testing.assert_allclose(a["out"], b["out"], rtol=1e-13, atol=1e-15)
+    assert np.abs(a["out"]).max() > 1e-3
+
+
+def _dense_swiglu(Wg, Wu, Wd, x):
+    """Eq. (1) with numpy matmuls on torch-widened matrices (independent of the oracle's loops)."""
+    return Wd.T @ (silu(Wg @ x) * (Wu @ x))
+
+
+def test_no_private_parameters_collapse_to_department_ffn():
+    """priv = 0 and sigma = none: every selected expert is its department's plain SwiGLU FFN, so
+    out_t = sum_j (sum of p over the picks in department j) * SwiGLU_j(x_t) (+ shared expert)."""
+    shape = SMALL.with_(priv=0, sigma=0, n_shared=1, shared_ffn=20)
+    cfg = oracle_cfg(shape)
+    wt = _layer(shape, 3, std=0.25)
+    tokens_t = synth.make_tokens(shape, 6, 3)
+    got = ref.deamoe_forward(cfg, oracle_weights(wt), synth.to_numpy(tokens_t))
+    X = widen(tokens_t)
+    Wg, Wu, Wd = (widen(wt[f"dept_{k}"]) for k in ("gate", "up", "down"))
+    Sg, Su, Sd = (widen(wt[f"shared_{k}"]) for k in ("gate", "up", "down"))
+    for t in range(6):
+        want = _dense_swiglu(Sg, Su, Sd, X[t])
+        for i, p in zip(got["idx"][t], got["w"][t]):
+            j = i // shape.experts_per_dept
+            want = want + p * _dense_swiglu(Wg[j], Wu[j], Wd[j], X[t])
+        np.testing.assert_allclose(got["out"][t], want, rtol=1e-11, atol=1e-14)
+    assert np.abs(got["out"]).max() > 1e-3
+
+
+def test_identity_private_matrices_give_the_department_backbone_and_zero_gives_zero():
+    """Square A = I with SiLU interfaces: every expert of department j computes
+    Wd^T SiLU( SiLU(SiLU(Wg x)) * SiLU(Wu x) ) -- the identity-initialisation property --
+    and equals the priv = 0 shorthand; A = 0 gives exactly 0."""
+    f = 40
+    shape = SMALL.with_(priv=f)
+    cfg = oracle_cfg(shape)
+    wt = _layer(shape, 4, std=0.3)
+    eye = torch.eye(f).to(torch.bfloat16).expand(shape.n_expert, f, f).contiguous()
+    for k in ("gate", "up", "down"):
+        wt[f"priv_{k}"] = eye
+    tokens_t = synth.make_tokens(shape, 4, 4)
+    tokens = synth.to_numpy(tokens_t)
+    got = ref.deamoe_forward(cfg, oracle_weights(wt), tokens)
+    X = widen(tokens_t)
+    Wg, Wu, Wd = (widen(wt[f"dept_{k}"]) for k in ("gate", "up", "down"))
+    for t in range(4):
+        want = np.zeros(shape.hidden)
+        for i, p in zip(got["idx"][t], got["w"][t]):
+            j = i // shape.experts_per_dept
+            want += p * (Wd[j].T @ silu(silu(silu(Wg[j] @ X[t])) * silu(Wu[j] @ X[t])))
+        np.testing.assert_allclose(got["out"][t], want, rtol=1e-11, atol=1e-14)
+    short = ref.deamoe_forward(oracle_cfg(shape.with_(priv=0)), oracle_weights(wt), tokens)
+    np.testing.assert_allclose(short["out"], got["out"], rtol=1e-13, atol=1e-16)
+    for k in ("gate", "up", "down"):
+        wt[f"priv_{k}"] = torch.zeros_like(eye)
+    zero = ref.deamoe_forward(cfg, oracle_weights(wt), tokens)
+    assert np.all(zero["out"] == 0.0)
+
+
+def test_selection_matrices_pin_orientation_of_private_transforms():
+    """Private matrices that are 0/1 selections: A_g picks G[pg], A_u picks U[pu] and A_d^T scatters
+    Y into Z, so Eq. (4) can be written with index arithmetic only.  Catches a transposed A_d, a
+    gate/up swap and a misplaced non-linearity."""
+    shape = SMALL.with_(n_dept=1, experts_per_dept=2, top_k=1)
+    cfg = oracle_cfg(shape)
+    h, f, r = shape.hidden, shape.ffn, shape.priv
+    wt = _layer(shape, 5, std=0.4)
+    pg = np.array(synth.uniform_ints(r, f, 5, "pg"))
+    pu = np.array(synth.uniform_ints(r, f, 5, "pu"))
+    pd = np.array(synth.uniform_ints(r, f, 5, "pd"))
+
+    def sel(p):
+        a = np.zeros((r, f), np.float32)
+        a[np.arange(r), p] = 1.0
+        return synth.to_numpy(torch.from_numpy(a).to(torch.bfloat16))
+    Wg, Wu, Wd = (widen(wt[f"dept_{k}"][0]) for k in ("gate", "up", "down"))
+    w0 = [synth.to_numpy(wt[f"dept_{k}"][0]) for k in ("gate", "up", "down")]
+    x = widen(synth.make_tokens(shape, 1, 5))[0]
+    out, G, U, Y, Z = ref.deamoe_expert(cfg, *w0, sel(pg), sel(pu), sel(pd), x, taps=True)
+    G_w, U_w = silu(Wg @ x), silu(Wu @ x)
+    Y_w = silu(G_w[pg]) * U_w[pu]
+    Zpre = np.zeros(f)
+    np.add.at(Zpre, pd, Y_w)
+    np.testing.assert_allclose(G, G_w, rtol=1e-12)
+    np.testing.assert_allclose(U, U_w, rtol=1e-12)
+    np.testing.assert_allclose(Y, Y_w, rtol=1e-12)
+    np.testing.assert_allclose(Z, silu(Zpre), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(out, Wd.T @ silu(Zpre), rtol=1e-11, atol=1e-14)
+
+
+# ---------------------------------------------------------------- invariants
+
+def test_layer_invariants():
+    """Row t of a batch equals the layer on token t alone; permuting tokens permutes rows;
+    relabelling the experts inside a department (router rows and private matrices together)
+    leaves the output unchanged; the routed part is linear in route_scale."""
+    shape = SMALL
+    cfg = oracle_cfg(shape)
+    wt = _layer(shape, 6, std=0.3)
+    w = oracle_weights(wt)
+    tok_t = synth.make_tokens(shape, 5, 6)
+    tok = synth.to_numpy(tok_t)
+    full = ref.deamoe_forward(cfg, w, tok)
+    assert np.abs(full["out"]).max() > 1e-4
+    for t in range(5):
+        one = ref.deamoe_forward(cfg, w, tok[t:t + 1])
+        assert (one["out"][0] == full["out"][t]).all()
+    sub = ref.deamoe_forward(cfg, w, tok, rows=[3, 1])
+    assert (sub["out"][[3, 1]] == full["out"][[3, 1]]).all() and (sub["out"][0] == 0).all()
+    perm = [4, 2, 0, 3, 1]
+    pf = ref.deamoe_forward(cfg, w, tok[perm])
+    assert (pf["out"] == full["out"][perm]).all()
+    # relabel experts inside each department
+    g = shape.experts_per_dept
+    relabel = np.concatenate([j * g + np.array([2, 0, 3, 1]) for j in range(shape.n_dept)])
+    w2 = dict(w)
+    for k in ("router", "priv_gate", "priv_up", "priv_down"):
+        w2[k] = np.ascontiguousarray(w[k][relabel])
+    rf = ref.deamoe_forward(cfg, w2, tok)
+    np.testing.assert_allclose(rf["out"], full["out"], rtol=1e-12, atol=1e-16)
+    assert (relabel[rf["idx"]] == full["idx"]).all()
+    scaled = ref.deamoe_forward(oracle_cfg(shape.with_(route_scale=3.0)), w, tok)
+    np.testing.assert_allclose(scaled["out"], 3.0 * full["out"], rtol=1e-12)
+    res = ref.deamoe_forward(oracle_cfg(shape.with_(residual=1)), w, tok)
+    np.testing.assert_allclose(res["out"], full["out"] + widen(tok_t), rtol=1e-12)
+
+
+def test_bf16_and_fp32_storage_agree_on_the_same_numbers():
+    """The same bf16-representable numbers stored as fp32 give the same output bit for bit."""
+    shape = SMALL
+    wt = _layer(shape, 7, std=0.3)
+    tok_t = synth.make_tokens(shape, 3, 7)
+    a = ref.deamoe_forward(oracle_cfg(shape), oracle_weights(wt), synth.to_numpy(tok_t))
+    w32 = {k: v.float() for k, v in wt.items()}
+    b = ref.deamoe_forward(oracle_cfg(shape.with_(weight_dtype=0, act_dtype=0)), oracle_weights(w32),
+                           synth.to_numpy(tok_t.float()))
+    assert (a["out"] == b["out"]).all()
+
+
+# ---------------------------------------------------------------- accounting (Table 1, Fig. 2)
+
+def _golden(name):
+    path = os.path.join(os.path.dirname(__file__), "golden", name)
+    return [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+
+
+def test_table1_budget_ratios_reproduce_to_the_printed_digit():
+    from oracle import accounting as acc
+    for name, kb, h, f, nb, m, n, kd, k, fx, px in _golden("table1_budget_ratios.txt"):
+        kb, h, f, nb, m, n, kd, k = map(int, (kb, h, f, nb, m, n, kd, k))
+        params = acc.deamoe_params(h, f, m, n) / acc.baseline_params(h, f, nb)
+        flops = acc.deamoe_flops(h, f, n, kd, k) / acc.baseline_flops(h, f, nb, kb)
+        assert abs(params - float(px)) <= 0.00051, (name, params)
+        if fx != "-":
+            assert abs(flops - float(fx)) <= 0.00051, (name, flops)
+
+
+def test_fig2_loading_ratio_range_for_the_deepseek_v3_row():
+    from oracle import accounting as acc
+    gold = {k: float(v) for k, v in _golden("fig2_loading_ratio.txt")}
+    ratios = [acc.expected_loading_ratio(T, 7168, 2048, 256, 8, 8, 864, 5, 10) for T in range(4, 65)]
+    assert abs(min(ratios) - gold["min_ratio_tokens_4_to_64"]) < 0.00051
+    assert abs(max(ratios) - gold["max_ratio_tokens_4_to_64"]) < 0.00051
+    assert abs((1 - min(ratios)) - gold["max_reduction"]) < 0.00051
+    # non-monotone: falls from 4 tokens to its minimum, then rises again towards 1
+    lo = ratios.index(min(ratios))
+    assert 0 < lo < len(ratios) - 1
+    assert acc.expected_loading_ratio(4096, 7168, 2048, 256, 8, 8, 864, 5, 10) > 0.97
+
+
+def test_expected_active_departments_matches_counted_routings():
+    """Hypergeometric closed form for flat uniform top-k against Monte-Carlo counting with the
+    oracle's own bucketing, at the DeepSeek-V3 benchmark layout (32 x 8 experts, top-8)."""
+    from oracle import accounting as acc
+    n, g, k, B, trials = 256, 8, 8, 8, 300
+    shape = synth.LayerShape("t", hidden=8, n_dept=32, experts_per_dept=8, ffn=8, priv=0, top_k=8)
+    cfg = oracle_cfg(shape)
+    rnd = synth.uniform_ints(trials * B * n, 1 << 30, 11, "mc")
+    tot_d = tot_e = 0
+    for s in range(trials):
+        idx = []
+        for t in range(B):
+            v = rnd[(s * B + t) * n:(s * B + t + 1) * n]
+            idx.append(sorted(range(n), key=lambda i: (v[i], i))[:k])
+        got = ref.bucket(cfg, np.array(idx, np.int32))
+        nd, ne, _ = acc.count_active(idx, g)
+        assert nd == bin(int(got["dept_mask"][0])).count("1")
+        assert ne == int((np.diff(got["expert_off"]) > 0).sum())
+        tot_d += nd
+        tot_e += ne
+    assert abs(tot_d / trials - acc.expected_active_depts(n, g, k, B)) < 0.25
+    assert abs(tot_e / trials - acc.expected_unique(n, k, B)) < 0.6
+    assert abs(acc.dept_miss_probability(256, 8, 8) - 0.7729) < 1e-4
+
+
+def test_unique_bytes_closed_form_against_vanilla():
+    from oracle import accounting as acc
+    h, f, r, n = 7168, 2048, 896, 256
+    dea = acc.unique_bytes_deamoe(7, 8, h, f, r, n, 2, 1, 2048)
+    van = acc.unique_bytes_vanilla(8, h, f, n, 2, 1, 2048)
+    assert dea == 7 * 88080384 + 8 * 11010048 + 88080384 + 7340032
+    assert van == 8 * 88080384 + 88080384 + 7340032
