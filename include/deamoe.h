@@ -1,0 +1,194 @@
+/*
+ * deamoe.h -- C ABI of the B200 (sm_100a) decode forward of one DeaMoE layer.
+ *
+ * One layer = a router, m departments that each own three large SwiGLU matrices
+ * shared by their experts, and n = m*g experts that each own three small private
+ * matrices (paper Section 3.1, Eq. (4)).  A decode step routes B tokens to their
+ * top-k experts (Eq. (2)), gathers the tokens of every department once, streams the
+ * department's matrices from HBM once for all of them, applies the selected experts'
+ * private matrices, and combines with the gate weights (Eq. (3)) -- the two-stage
+ * schedule of Section 3.2.  The same library builds the standard MoE layer of
+ * Eq. (1)-(3) at the same shape as a comparator.
+ *
+ * Conventions that hold for every entry point:
+ *  - Pointers marked DEVICE are CUDA device pointers of the current device; pointers
+ *    marked HOST are ordinary host pointers.  `cuda_stream` is a cudaStream_t passed as
+ *    void* (NULL = the legacy default stream).
+ *  - All matrices are dense, row-major, 16-byte aligned.
+ *  - Every call returns a deamoe_status_t; nothing aborts, traps or throws.  Argument
+ *    errors are detected on the host before anything is enqueued.
+ *  - deamoe_route / deamoe_forward only ENQUEUE work on the given stream; they never
+ *    synchronise and never allocate (all workspace is sized at create for max_batch).
+ *  - There is no CPU fallback and no other backend: without a CUDA device the create
+ *    calls fail with DEAMOE_ERR_CUDA.
+ */
+#ifndef DEAMOE_H
+#define DEAMOE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct deamoe_layer deamoe_layer_t; /* opaque, owned by the library */
+
+typedef enum {
+  DEAMOE_OK = 0,
+  DEAMOE_ERR_INVALID_ARG = 1, /* NULL pointer, inconsistent or non-positive sizes */
+  DEAMOE_ERR_UNSUPPORTED = 2, /* a valid request this build has no kernel for */
+  DEAMOE_ERR_ALLOC = 3,       /* device or host allocation failed */
+  DEAMOE_ERR_CUDA = 4,        /* a CUDA runtime call failed (no device, launch error) */
+  DEAMOE_ERR_BATCH = 5,       /* B < 0 or B > max_batch */
+  DEAMOE_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by get_stats) */
+} deamoe_status_t;
+
+typedef enum { DEAMOE_F32 = 0, DEAMOE_BF16 = 1 } deamoe_dtype_t;
+
+/* sigma of Section 3.1: the non-linearity between department and expert projections */
+typedef enum { DEAMOE_SIGMA_NONE = 0, DEAMOE_SIGMA_SILU = 1, DEAMOE_SIGMA_GELU = 2 } deamoe_sigma_t;
+
+/* how one forward is issued */
+typedef enum {
+  DEAMOE_SCHED_AUTO = 0,   /* the library's best schedule for the dtype */
+  DEAMOE_SCHED_PLAIN = 1,  /* one simple kernel per stage on the canonical layouts (any dtype) */
+  DEAMOE_SCHED_STAGED = 2, /* bf16 weight-streaming kernel, one launch per stage */
+  DEAMOE_SCHED_FUSED = 3   /* bf16 weight-streaming kernel, one persistent launch for all stages */
+} deamoe_schedule_t;
+
+/*
+ * Layer description (Section 3.1 / 3.2; Table 1 uses the same symbols).
+ * Expert i belongs to department i / experts_per_dept.
+ */
+typedef struct {
+  int32_t hidden;           /* h */
+  int32_t n_dept;           /* m */
+  int32_t experts_per_dept; /* g; n = m*g experts */
+  int32_t ffn;              /* f = h_ffn: department (and standard expert) intermediate size */
+  int32_t priv;             /* r: private matrices A_g, A_u, A_d are [r, f].  r == f is the paper's
+                               square form.  0 = no private parameters (A = identity, nothing is
+                               stored or loaded; sigma is still applied as configured). */
+  int32_t top_k;            /* k_expert of Eq. (2) */
+  int32_t k_dept;           /* 0 = flat top-k.  > 0 = group-limited routing (Section 3.3): only the
+                               k_dept departments with the largest best logit stay eligible. */
+  int32_t n_shared;         /* 0 or 1 always-on shared SwiGLU expert (Eq. (1), weight 1) */
+  int32_t shared_ffn;       /* its intermediate size */
+  int32_t sigma;            /* deamoe_sigma_t */
+  int32_t norm_topk;        /* 1: p = softmax over the k selected logits; 0: softmax over all n */
+  int32_t weight_dtype;     /* deamoe_dtype_t of department / private / shared matrices */
+  int32_t act_dtype;        /* deamoe_dtype_t of tokens and out */
+  int32_t residual;         /* 1: out = tokens + layer(tokens) */
+  int32_t max_batch;        /* largest B any later call may pass (1..DEAMOE_MAX_BATCH) */
+  int32_t schedule;         /* deamoe_schedule_t */
+  float route_scale;        /* gate weights are multiplied by this (Eq. (3) "scaling") */
+} deamoe_config_t;
+
+#define DEAMOE_MAX_BATCH 128
+#define DEAMOE_MAX_TOPK 32
+#define DEAMOE_MAX_EXPERTS 2048
+
+/*
+ * Weights in their canonical layouts.  All DEVICE pointers, caller-owned, read only
+ * during create (the library keeps its own re-packed copy, so the caller may free
+ * them as soon as create returns and the stream has been synchronised).
+ *
+ *   router                       [n, h]  fp32 always (Eq. (2))
+ *   dept_gate, dept_up           [m, f, h]   W_g^j, W_u^j
+ *   dept_down                    [m, f, h]   W_d^j, applied transposed: (W_d^j)^T z
+ *   priv_gate, priv_up           [n, r, f]   A_g^i, A_u^i
+ *   priv_down                    [n, r, f]   A_d^i, applied transposed: (A_d^i)^T y
+ *   shared_gate/up/down          [shared_ffn, h]
+ * priv_* must be NULL iff priv == 0; shared_* must be NULL iff n_shared == 0.
+ * For deamoe_vanilla_create the dept_* pointers hold the n standard experts, [n, f, h].
+ */
+typedef struct {
+  const float *router;
+  const void *dept_gate, *dept_up, *dept_down;
+  const void *priv_gate, *priv_up, *priv_down;
+  const void *shared_gate, *shared_up, *shared_down;
+} deamoe_weights_t;
+
+/*
+ * Build a DeaMoE layer (Section 3.1).  Allocates the library's weight copy and all
+ * workspace for max_batch tokens, enqueues the re-packing on `cuda_stream` and
+ * synchronises it before returning.  *out is set only on DEAMOE_OK.
+ * Errors: INVALID_ARG (NULL, sizes <= 0, top_k > n, priv/shared pointers inconsistent with
+ * the sizes), UNSUPPORTED (bf16 streaming schedules need h, f, r, shared_ffn to be multiples
+ * of 16; n > DEAMOE_MAX_EXPERTS; top_k > DEAMOE_MAX_TOPK), BATCH, ALLOC, CUDA.
+ */
+deamoe_status_t deamoe_layer_create(const deamoe_config_t *cfg, const deamoe_weights_t *weights,
+                                    void *cuda_stream, deamoe_layer_t **out);
+
+/* Standard MoE comparator, Eq. (1)-(3): n experts of three [f, h] matrices, same router
+ * semantics, same optional shared expert.  cfg->priv must be 0; sigma is ignored. */
+deamoe_status_t deamoe_vanilla_create(const deamoe_config_t *cfg, const deamoe_weights_t *weights,
+                                      void *cuda_stream, deamoe_layer_t **out);
+
+/* Frees everything the layer owns.  The caller must make sure no work of this layer is
+ * still running.  NULL is accepted. */
+deamoe_status_t deamoe_layer_destroy(deamoe_layer_t *layer);
+
+/*
+ * Routing only (Eq. (2), gate weights of Eq. (3), department sets of Section 3.2).
+ * tokens: DEVICE [B, h] in act_dtype.  Fills the layer's device-side routing state and, where
+ * non-NULL, the caller's DEVICE outputs topk_idx [B, k] (experts in order of decreasing logit,
+ * ties to the lower index) and topk_w [B, k] fp32.  B == 0 is a no-op.
+ */
+deamoe_status_t deamoe_route(deamoe_layer_t *layer, void *cuda_stream, const void *tokens, int32_t B,
+                             int32_t *topk_idx, float *topk_w);
+
+/*
+ * One decode step of the layer: out[B, h] = sum_{i in S(x)} p_i Expert_i(x) (+ shared expert)
+ * (+ x if residual), Eq. (3) with Eq. (4) (DeaMoE layer) or Eq. (1) (vanilla layer), evaluated
+ * with the two-stage schedule of Section 3.2.  tokens, out: DEVICE [B, h] in act_dtype; out must
+ * not alias tokens.  Includes routing.  B == 0 is a no-op.
+ */
+deamoe_status_t deamoe_forward(deamoe_layer_t *layer, void *cuda_stream, const void *tokens, int32_t B,
+                               void *out);
+
+/* The same step for a layer made by deamoe_vanilla_create (INVALID_ARG for a DeaMoE layer). */
+deamoe_status_t deamoe_vanilla_forward(deamoe_layer_t *layer, void *cuda_stream, const void *tokens,
+                                       int32_t B, void *out);
+
+/*
+ * End-to-end step on HOST buffers: copies tokens (HOST [B, h], act_dtype, ideally pinned) to a
+ * device staging buffer owned by the layer, runs deamoe_forward, copies the result to `out`
+ * (HOST [B, h]) and synchronises the stream before returning.
+ */
+deamoe_status_t deamoe_forward_host(deamoe_layer_t *layer, void *cuda_stream, const void *tokens,
+                                    int32_t B, void *out);
+
+/*
+ * Copy the routing state of the LAST route/forward call to HOST buffers (synchronises the
+ * given stream first).  Any pointer may be NULL.  Sizes: topk_idx/topk_w [B*k]; dept_mask
+ * [ceil(m/64)] (bit j of word j/64 = department j active); dept_off [m+1] and dept_tok
+ * [dept_off[m]] = the distinct tokens of each department, ascending (X^j of Section 3.2);
+ * expert_off [n+1] and expert_tok [B*k] likewise per expert.
+ */
+deamoe_status_t deamoe_get_routing(deamoe_layer_t *layer, void *cuda_stream, int32_t *topk_idx,
+                                   float *topk_w, uint64_t *dept_mask, int32_t *dept_off,
+                                   int32_t *dept_tok, int32_t *expert_off, int32_t *expert_tok);
+
+/*
+ * Counters of the LAST route/forward call (synchronises the stream first), HOST outputs, any may
+ * be NULL: active departments |D|, active experts |E|, (token, department) pairs, the unique weight
+ * bytes the step had to load (|D|*3hf*s + |E|*3rf*s + shared + 4nh for DeaMoE; |E|*3hf*s + shared +
+ * 4nh for vanilla), and the device status word (DEAMOE_OK or DEAMOE_ERR_TIMEOUT).
+ */
+deamoe_status_t deamoe_get_stats(deamoe_layer_t *layer, void *cuda_stream, int32_t *n_active_dept,
+                                 int32_t *n_active_expert, int32_t *n_token_dept_pairs,
+                                 uint64_t *unique_weight_bytes, int32_t *device_status);
+
+/* Number of kernels the last forward/route call of this layer launched (host-side count). */
+int32_t deamoe_last_launches(const deamoe_layer_t *layer);
+
+/* Bytes of device memory the layer owns (weights copy + workspace). */
+uint64_t deamoe_device_bytes(const deamoe_layer_t *layer);
+
+/* Static, never NULL. */
+const char *deamoe_status_string(deamoe_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEAMOE_H */

@@ -1,0 +1,199 @@
+"""Thin ctypes binding of libdeamoe.so: argument marshalling only.
+
+Every step of the layer runs in the library's CUDA kernels.  torch is used here for device
+memory (tensors handed in by the caller) and for the current stream, nothing else.  If the
+library has not been built the import of `lib()` raises -- there is no fallback.
+"""
+import ctypes as C
+import os
+
+import torch
+
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdeamoe.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_BATCH, ERR_TIMEOUT = range(7)
+F32, BF16 = 0, 1
+SIGMA_NONE, SIGMA_SILU, SIGMA_GELU = 0, 1, 2
+SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED = 0, 1, 2, 3
+
+# every symbol include/deamoe.h declares
+SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",
+           "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_get_routing",
+           "deamoe_get_stats", "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
+
+
+class Config(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in (
+        "hidden", "n_dept", "experts_per_dept", "ffn", "priv", "top_k", "k_dept", "n_shared",
+        "shared_ffn", "sigma", "norm_topk", "weight_dtype", "act_dtype", "residual", "max_batch",
+        "schedule")] + [("route_scale", C.c_float)]
+
+
+class Weights(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in (
+        "router", "dept_gate", "dept_up", "dept_down", "priv_gate", "priv_up", "priv_down",
+        "shared_gate", "shared_up", "shared_down")]
+
+
+class DeaMoEError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib():
+    """Load libdeamoe.so (built in-tree by build.py); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_14385_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        for name in SYMBOLS:
+            getattr(L, name)
+        L.deamoe_status_string.restype = C.c_char_p
+        L.deamoe_status_string.argtypes = [C.c_int]
+        L.deamoe_last_launches.restype = C.c_int32
+        L.deamoe_last_launches.argtypes = [C.c_void_p]
+        L.deamoe_device_bytes.restype = C.c_uint64
+        L.deamoe_device_bytes.argtypes = [C.c_void_p]
+        for name in ("deamoe_layer_create", "deamoe_vanilla_create"):
+            getattr(L, name).argtypes = [C.POINTER(Config), C.POINTER(Weights), C.c_void_p,
+                                         C.POINTER(C.c_void_p)]
+        L.deamoe_layer_destroy.argtypes = [C.c_void_p]
+        L.deamoe_route.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        for name in ("deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host"):
+            getattr(L, name).argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.deamoe_get_routing.argtypes = [C.c_void_p] * 9
+        L.deamoe_get_stats.argtypes = [C.c_void_p] * 7
+        _lib = L
+    return _lib
+
+
+def status_string(status):
+    return lib().deamoe_status_string(int(status)).decode()
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def make_config(shape, max_batch, schedule=SCHED_AUTO):
+    d = shape.asdict() if hasattr(shape, "asdict") else dict(shape)
+    return Config(d["hidden"], d["n_dept"], d["experts_per_dept"], d["ffn"], d["priv"], d["top_k"],
+                  d.get("k_dept", 0), d.get("n_shared", 0), d.get("shared_ffn", 0), d.get("sigma", 1),
+                  d.get("norm_topk", 1), d.get("weight_dtype", 1), d.get("act_dtype", 1),
+                  d.get("residual", 0), int(max_batch), int(schedule), float(d.get("route_scale", 1.0)))
+
+
+class Layer:
+    """One DeaMoE (or vanilla MoE) layer living on the current CUDA device."""
+
+    def __init__(self, shape, weights, max_batch, schedule=SCHED_AUTO, vanilla=False):
+        """weights: dict of CUDA tensors in the canonical layouts of include/deamoe.h."""
+        self.shape = shape
+        self.vanilla = vanilla
+        self.cfg = make_config(shape, max_batch, schedule)
+        if vanilla:
+            self.cfg.priv = 0
+        w = Weights()
+        for name, _ in Weights._fields_:
+            t = weights.get(name)
+            if vanilla and name.startswith("priv_"):
+                t = None
+            if t is not None:
+                assert t.is_cuda and t.is_contiguous(), name
+            setattr(w, name, t.data_ptr() if t is not None else None)
+        self._h = C.c_void_p()
+        fn = lib().deamoe_vanilla_create if vanilla else lib().deamoe_layer_create
+        st = fn(C.byref(self.cfg), C.byref(w), _stream(), C.byref(self._h))
+        if st != OK:
+            self._h = C.c_void_p()
+            raise DeaMoEError(st, "deamoe_vanilla_create" if vanilla else "deamoe_layer_create")
+        self.act = torch.float32 if self.cfg.act_dtype == F32 else torch.bfloat16
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().deamoe_layer_destroy(self._h)
+            self._h = C.c_void_p()
+
+    __del__ = close
+
+    def _check_tokens(self, tokens):
+        assert tokens.is_cuda and tokens.is_contiguous() and tokens.dtype == self.act
+        assert tokens.dim() == 2 and tokens.shape[1] == self.cfg.hidden
+        return tokens.shape[0]
+
+    def route(self, tokens, want_outputs=True):
+        B = self._check_tokens(tokens)
+        k = self.cfg.top_k
+        idx = torch.empty((B, k), dtype=torch.int32, device=tokens.device) if want_outputs else None
+        w = torch.empty((B, k), dtype=torch.float32, device=tokens.device) if want_outputs else None
+        st = lib().deamoe_route(self._h, _stream(), _dptr(tokens), B, _dptr(idx), _dptr(w))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_route")
+        return idx, w
+
+    def forward(self, tokens, out=None):
+        B = self._check_tokens(tokens)
+        if out is None:
+            out = torch.empty_like(tokens)
+        fn = lib().deamoe_vanilla_forward if self.vanilla else lib().deamoe_forward
+        st = fn(self._h, _stream(), _dptr(tokens), B, _dptr(out))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_forward")
+        return out
+
+    def forward_host(self, tokens, out):
+        """tokens/out: CPU tensors (pinned for speed) [B, h] in the activation dtype."""
+        assert not tokens.is_cuda and not out.is_cuda and tokens.is_contiguous() and out.is_contiguous()
+        st = lib().deamoe_forward_host(self._h, _stream(), C.c_void_p(tokens.data_ptr()), tokens.shape[0],
+                                       C.c_void_p(out.data_ptr()))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_forward_host")
+        return out
+
+    def routing(self, B):
+        """Host copy of the last call's routing state as numpy arrays."""
+        import numpy as np
+        m, n, k = self.cfg.n_dept, self.cfg.n_dept * self.cfg.experts_per_dept, self.cfg.top_k
+        idx = np.zeros((B, k), np.int32)
+        w = np.zeros((B, k), np.float32)
+        mask = np.zeros(((m + 63) // 64,), np.uint64)
+        doff = np.zeros((m + 1,), np.int32)
+        dtok = np.full((max(1, B * min(k, m)),), -1, np.int32)
+        eoff = np.zeros((n + 1,), np.int32)
+        etok = np.full((max(1, B * k),), -1, np.int32)
+        st = lib().deamoe_get_routing(self._h, _stream(), *(C.c_void_p(a.ctypes.data)
+                                                           for a in (idx, w, mask, doff, dtok, eoff, etok)))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_get_routing")
+        return {"idx": idx, "w": w, "dept_mask": mask, "dept_off": doff, "dept_tok": dtok[:doff[m]],
+                "expert_off": eoff, "expert_tok": etok[:eoff[n]]}
+
+    def stats(self):
+        nd, ne, ntd, st_ = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+        ub = C.c_uint64()
+        st = lib().deamoe_get_stats(self._h, _stream(), C.byref(nd), C.byref(ne), C.byref(ntd), C.byref(ub),
+                                    C.byref(st_))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_get_stats")
+        return {"active_dept": nd.value, "active_expert": ne.value, "token_dept_pairs": ntd.value,
+                "unique_weight_bytes": ub.value, "device_status": st_.value}
+
+    @property
+    def last_launches(self):
+        return lib().deamoe_last_launches(self._h)
+
+    @property
+    def device_bytes(self):
+        return lib().deamoe_device_bytes(self._h)

@@ -1,0 +1,363 @@
+// C ABI of libdeamoe.so: argument checking, ownership, and the order in which the stages of
+// one decode step are enqueued.  All arithmetic lives in the kernels of the other files.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "deamoe_internal.cuh"
+#include "stream.cuh"
+
+using namespace deamoe;
+
+struct deamoe_layer {
+  deamoe_config_t cfg;
+  LayerDev dev;                 // device view (weights + workspace)
+  StreamPlan* plan = nullptr;   // packed weights + work-list machinery of the streaming schedules
+  std::vector<void*> owned;     // every device allocation of this layer
+  uint64_t device_bytes = 0;
+  int schedule = DEAMOE_SCHED_PLAIN;
+  int kslices = 1;
+  int last_launches = 0;
+  int last_B = 0;
+  void* stage_tokens = nullptr; // device staging for deamoe_forward_host
+  void* stage_out = nullptr;
+};
+
+namespace {
+
+size_t dtype_size(int dt) { return dt == DEAMOE_F32 ? 4 : 2; }
+
+template <typename T>
+deamoe_status_t dev_alloc(deamoe_layer* L, T** p, size_t count) {
+  void* q = nullptr;
+  const size_t bytes = (count ? count : 1) * sizeof(T);
+  if (cudaMalloc(&q, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return DEAMOE_ERR_ALLOC;
+  }
+  L->owned.push_back(q);
+  L->device_bytes += bytes;
+  *p = reinterpret_cast<T*>(q);
+  return DEAMOE_OK;
+}
+
+deamoe_status_t dev_copy(deamoe_layer* L, const void** dst, const void* src, size_t bytes, cudaStream_t s) {
+  char* q = nullptr;
+  deamoe_status_t st = dev_alloc(L, &q, bytes);
+  if (st != DEAMOE_OK) return st;
+  if (cudaMemcpyAsync(q, src, bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return DEAMOE_ERR_CUDA;
+  *dst = q;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t check_config(const deamoe_config_t* c, const deamoe_weights_t* w, bool vanilla) {
+  if (!c || !w) return DEAMOE_ERR_INVALID_ARG;
+  if (c->hidden <= 0 || c->n_dept <= 0 || c->experts_per_dept <= 0 || c->ffn <= 0 || c->priv < 0 ||
+      c->top_k <= 0 || c->k_dept < 0 || c->n_shared < 0 || c->n_shared > 1)
+    return DEAMOE_ERR_INVALID_ARG;
+  const long long n = (long long)c->n_dept * c->experts_per_dept;
+  if (c->top_k > n) return DEAMOE_ERR_INVALID_ARG;
+  if (c->k_dept > 0 && (long long)c->k_dept * c->experts_per_dept < c->top_k) return DEAMOE_ERR_INVALID_ARG;
+  if (c->n_shared && c->shared_ffn <= 0) return DEAMOE_ERR_INVALID_ARG;
+  if (c->weight_dtype != DEAMOE_F32 && c->weight_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
+  if (c->act_dtype != DEAMOE_F32 && c->act_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
+  if (c->sigma < DEAMOE_SIGMA_NONE || c->sigma > DEAMOE_SIGMA_GELU) return DEAMOE_ERR_INVALID_ARG;
+  if (c->schedule < DEAMOE_SCHED_AUTO || c->schedule > DEAMOE_SCHED_FUSED) return DEAMOE_ERR_INVALID_ARG;
+  if (!(c->route_scale == c->route_scale)) return DEAMOE_ERR_INVALID_ARG;
+  if (c->max_batch < 1 || c->max_batch > DEAMOE_MAX_BATCH) return DEAMOE_ERR_BATCH;
+  if (!w->router || !w->dept_gate || !w->dept_up || !w->dept_down) return DEAMOE_ERR_INVALID_ARG;
+  if (vanilla && c->priv != 0) return DEAMOE_ERR_INVALID_ARG;
+  const bool has_priv = w->priv_gate && w->priv_up && w->priv_down;
+  const bool no_priv = !w->priv_gate && !w->priv_up && !w->priv_down;
+  if (c->priv > 0 ? !has_priv : !no_priv) return DEAMOE_ERR_INVALID_ARG;
+  const bool has_sh = w->shared_gate && w->shared_up && w->shared_down;
+  const bool no_sh = !w->shared_gate && !w->shared_up && !w->shared_down;
+  if (c->n_shared ? !has_sh : !no_sh) return DEAMOE_ERR_INVALID_ARG;
+  if (n > DEAMOE_MAX_EXPERTS || c->top_k > DEAMOE_MAX_TOPK) return DEAMOE_ERR_UNSUPPORTED;
+  if ((c->hidden | c->ffn | c->priv | c->shared_ffn) & 3) return DEAMOE_ERR_UNSUPPORTED;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* w, void* stream,
+                            deamoe_layer_t** out, bool vanilla) {
+  if (!out) return DEAMOE_ERR_INVALID_ARG;
+  deamoe_status_t st = check_config(cfg, w, vanilla);
+  if (st != DEAMOE_OK) return st;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    return DEAMOE_ERR_CUDA;
+  }
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  deamoe_layer* L = new (std::nothrow) deamoe_layer();
+  if (!L) return DEAMOE_ERR_ALLOC;
+  L->cfg = *cfg;
+  LayerDev& d = L->dev;
+  std::memset(&d, 0, sizeof(d));
+  d.h = cfg->hidden; d.m = cfg->n_dept; d.g = cfg->experts_per_dept; d.n = d.m * d.g;
+  d.f = cfg->ffn; d.r = vanilla ? 0 : cfg->priv; d.k = cfg->top_k; d.k_dept = cfg->k_dept;
+  d.n_shared = cfg->n_shared; d.fs = cfg->n_shared ? cfg->shared_ffn : 0;
+  d.sigma = vanilla ? DEAMOE_SIGMA_NONE : cfg->sigma; d.norm_topk = cfg->norm_topk;
+  d.residual = cfg->residual; d.vanilla = vanilla ? 1 : 0;
+  d.wdt = cfg->weight_dtype; d.adt = cfg->act_dtype; d.max_batch = cfg->max_batch;
+  d.rp = d.r > 0 ? d.r : d.f;
+  d.route_scale = cfg->route_scale;
+
+  int sched = cfg->schedule;
+  const bool streamable = cfg->weight_dtype == DEAMOE_BF16 &&
+                          ((cfg->hidden | cfg->ffn | cfg->priv | cfg->shared_ffn) & 15) == 0;
+  if (sched == DEAMOE_SCHED_AUTO) sched = streamable ? stream_default_schedule() : DEAMOE_SCHED_PLAIN;
+  if ((sched == DEAMOE_SCHED_STAGED || sched == DEAMOE_SCHED_FUSED) && !streamable) {
+    delete L;
+    return DEAMOE_ERR_UNSUPPORTED;
+  }
+  L->schedule = sched;
+
+  const int MB = cfg->max_batch, k = d.k;
+  const int tdmax = MB * (k < d.m ? k : d.m);  // (token, department) rows
+  const int pmax = MB * k;                     // (token, expert) pairs
+  // router column slices: enough CTAs to cover the GPU a few times
+  L->kslices = 1;
+  while (L->kslices < 16 && ((d.n + 3) / 4) * L->kslices < 296 && d.h / (L->kslices * 2) >= 512) L->kslices *= 2;
+
+  bool ok = true;
+  auto A = [&](deamoe_status_t r) { if (r != DEAMOE_OK && ok) { ok = false; st = r; } };
+  const size_t ws = dtype_size(d.wdt);
+  const size_t units = vanilla ? (size_t)d.n : (size_t)d.m;
+  A(dev_copy(L, reinterpret_cast<const void**>(&d.router), w->router, (size_t)d.n * d.h * 4, s));
+  if (ok && sched == DEAMOE_SCHED_PLAIN) {
+    A(dev_copy(L, &d.dept_gate, w->dept_gate, units * d.f * d.h * ws, s));
+    A(dev_copy(L, &d.dept_up, w->dept_up, units * d.f * d.h * ws, s));
+    A(dev_copy(L, &d.dept_down, w->dept_down, units * d.f * d.h * ws, s));
+    if (d.r > 0) {
+      A(dev_copy(L, &d.priv_gate, w->priv_gate, (size_t)d.n * d.r * d.f * ws, s));
+      A(dev_copy(L, &d.priv_up, w->priv_up, (size_t)d.n * d.r * d.f * ws, s));
+      A(dev_copy(L, &d.priv_down, w->priv_down, (size_t)d.n * d.r * d.f * ws, s));
+    }
+    if (d.n_shared) {
+      A(dev_copy(L, &d.shared_gate, w->shared_gate, (size_t)d.fs * d.h * ws, s));
+      A(dev_copy(L, &d.shared_up, w->shared_up, (size_t)d.fs * d.h * ws, s));
+      A(dev_copy(L, &d.shared_down, w->shared_down, (size_t)d.fs * d.h * ws, s));
+    }
+  }
+  if (ok) {
+    if (d.adt == DEAMOE_BF16) A(dev_alloc(L, &d.x32, (size_t)MB * d.h));
+    A(dev_alloc(L, &d.logit_part, (size_t)L->kslices * MB * d.n));
+    A(dev_alloc(L, &d.topk_idx, (size_t)pmax));
+    A(dev_alloc(L, &d.topk_w, (size_t)pmax));
+    A(dev_alloc(L, &d.dept_mask, (size_t)(d.m + 63) / 64));
+    A(dev_alloc(L, &d.dept_off, (size_t)d.m + 1));
+    A(dev_alloc(L, &d.dept_tok, (size_t)tdmax));
+    A(dev_alloc(L, &d.expert_off, (size_t)d.n + 1));
+    A(dev_alloc(L, &d.expert_tok, (size_t)pmax));
+    A(dev_alloc(L, &d.pair_slot, (size_t)pmax));
+    A(dev_alloc(L, &d.pair_gurow, (size_t)pmax));
+    A(dev_alloc(L, &d.active_dept, (size_t)d.m));
+    A(dev_alloc(L, &d.active_expert, (size_t)d.n));
+    A(dev_alloc(L, &d.counts, (size_t)CNT_COUNT));
+    if (!vanilla) {
+      A(dev_alloc(L, &d.GU, (size_t)tdmax * 2 * d.f));
+      A(dev_alloc(L, &d.Z, (size_t)pmax * d.f));
+    }
+    A(dev_alloc(L, &d.Y, (size_t)pmax * (vanilla ? d.f : d.rp)));
+    A(dev_alloc(L, &d.O, (size_t)pmax * d.h));
+    if (d.n_shared) {
+      A(dev_alloc(L, &d.Ysh, (size_t)MB * d.fs));
+      A(dev_alloc(L, &d.Osh, (size_t)MB * d.h));
+    }
+    const size_t io = (size_t)MB * d.h * dtype_size(d.adt);
+    A(dev_alloc(L, reinterpret_cast<char**>(&L->stage_tokens), io));
+    A(dev_alloc(L, reinterpret_cast<char**>(&L->stage_out), io));
+  }
+  if (ok && cudaMemsetAsync(d.counts, 0, CNT_COUNT * sizeof(int32_t), s) != cudaSuccess) A(DEAMOE_ERR_CUDA);
+  if (ok && route_configure(d) != cudaSuccess) A(DEAMOE_ERR_CUDA);
+  if (ok && sched != DEAMOE_SCHED_PLAIN) {
+    uint64_t plan_bytes = 0;
+    A(stream_plan_create(d, *w, sched, s, &L->plan, &plan_bytes));
+    L->device_bytes += plan_bytes;
+  }
+  if (ok && cudaStreamSynchronize(s) != cudaSuccess) A(DEAMOE_ERR_CUDA);
+  if (!ok) {
+    cudaGetLastError();
+    deamoe_layer_destroy(L);
+    return st;
+  }
+  *out = L;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t check_call(deamoe_layer_t* L, const void* tokens, int B) {
+  if (!L) return DEAMOE_ERR_INVALID_ARG;
+  if (B < 0 || B > L->cfg.max_batch) return DEAMOE_ERR_BATCH;
+  if (B > 0 && !tokens) return DEAMOE_ERR_INVALID_ARG;
+  return DEAMOE_OK;
+}
+
+LayerDev call_view(deamoe_layer_t* L, const void* tokens) {
+  LayerDev d = L->dev;
+  if (d.adt == DEAMOE_F32) d.x32 = const_cast<float*>(reinterpret_cast<const float*>(tokens));
+  return d;
+}
+
+}  // namespace
+
+extern "C" {
+
+deamoe_status_t deamoe_layer_create(const deamoe_config_t* cfg, const deamoe_weights_t* weights, void* cuda_stream,
+                                    deamoe_layer_t** out) {
+  return create_impl(cfg, weights, cuda_stream, out, false);
+}
+
+deamoe_status_t deamoe_vanilla_create(const deamoe_config_t* cfg, const deamoe_weights_t* weights,
+                                      void* cuda_stream, deamoe_layer_t** out) {
+  return create_impl(cfg, weights, cuda_stream, out, true);
+}
+
+deamoe_status_t deamoe_layer_destroy(deamoe_layer_t* L) {
+  if (!L) return DEAMOE_OK;
+  if (L->plan) stream_plan_destroy(L->plan);
+  for (void* p : L->owned) cudaFree(p);
+  delete L;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t deamoe_route(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B, int32_t* topk_idx,
+                             float* topk_w) {
+  deamoe_status_t st = check_call(L, tokens, B);
+  if (st != DEAMOE_OK) return st;
+  L->last_B = B;
+  L->last_launches = 0;
+  if (B == 0) return DEAMOE_OK;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  LayerDev d = call_view(L, tokens);
+  int nl = launch_route(d, tokens, B, s, L->kslices, topk_idx, topk_w);
+  if (nl < 0) return DEAMOE_ERR_CUDA;
+  if (L->plan) {
+    const int n2 = stream_build_worklist(*L->plan, d, B, s);
+    if (n2 < 0) return DEAMOE_ERR_CUDA;
+    nl += n2;
+  }
+  L->last_launches = nl;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t deamoe_forward(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B, void* out) {
+  deamoe_status_t st = check_call(L, tokens, B);
+  if (st != DEAMOE_OK) return st;
+  if (B > 0 && (!out || out == tokens)) return DEAMOE_ERR_INVALID_ARG;
+  st = deamoe_route(L, cuda_stream, tokens, B, nullptr, nullptr);
+  if (st != DEAMOE_OK || B == 0) return st;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  LayerDev d = call_view(L, tokens);
+  int nl;
+  if (L->schedule == DEAMOE_SCHED_PLAIN) {
+    nl = launch_plain_forward(d, B, s);
+  } else {
+    nl = stream_forward(*L->plan, d, B, s);
+  }
+  if (nl < 0) return DEAMOE_ERR_CUDA;
+  const int nc = launch_combine(d, tokens, B, out, s);
+  if (nc < 0) return DEAMOE_ERR_CUDA;
+  L->last_launches += nl + nc;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t deamoe_vanilla_forward(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B,
+                                       void* out) {
+  if (!L || !L->dev.vanilla) return DEAMOE_ERR_INVALID_ARG;
+  return deamoe_forward(L, cuda_stream, tokens, B, out);
+}
+
+deamoe_status_t deamoe_forward_host(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B, void* out) {
+  deamoe_status_t st = check_call(L, tokens, B);
+  if (st != DEAMOE_OK) return st;
+  if (B == 0) return DEAMOE_OK;
+  if (!out) return DEAMOE_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t bytes = (size_t)B * L->dev.h * dtype_size(L->dev.adt);
+  if (cudaMemcpyAsync(L->stage_tokens, tokens, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return DEAMOE_ERR_CUDA;
+  st = deamoe_forward(L, cuda_stream, L->stage_tokens, B, L->stage_out);
+  if (st != DEAMOE_OK) return st;
+  if (cudaMemcpyAsync(out, L->stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return DEAMOE_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return DEAMOE_ERR_CUDA;
+  return DEAMOE_OK;
+}
+
+deamoe_status_t deamoe_get_routing(deamoe_layer_t* L, void* cuda_stream, int32_t* topk_idx, float* topk_w,
+                                   uint64_t* dept_mask, int32_t* dept_off, int32_t* dept_tok, int32_t* expert_off,
+                                   int32_t* expert_tok) {
+  if (!L) return DEAMOE_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return DEAMOE_ERR_CUDA;
+  const LayerDev& d = L->dev;
+  const int B = L->last_B, k = d.k;
+  bool ok = true;
+  auto G = [&](void* dst, const void* src, size_t bytes) {
+    if (dst && bytes && cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) ok = false;
+  };
+  G(topk_idx, d.topk_idx, (size_t)B * k * 4);
+  G(topk_w, d.topk_w, (size_t)B * k * 4);
+  if (B == 0) {
+    if (dept_mask) std::memset(dept_mask, 0, ((d.m + 63) / 64) * 8);
+    if (dept_off) std::memset(dept_off, 0, (d.m + 1) * 4);
+    if (expert_off) std::memset(expert_off, 0, (d.n + 1) * 4);
+    return DEAMOE_OK;
+  }
+  G(dept_mask, d.dept_mask, (size_t)((d.m + 63) / 64) * 8);
+  std::vector<int32_t> doff(d.m + 1);
+  G(doff.data(), d.dept_off, (size_t)(d.m + 1) * 4);
+  if (dept_off && ok) std::memcpy(dept_off, doff.data(), (size_t)(d.m + 1) * 4);
+  if (ok) G(dept_tok, d.dept_tok, (size_t)doff[d.m] * 4);
+  G(expert_off, d.expert_off, (size_t)(d.n + 1) * 4);
+  G(expert_tok, d.expert_tok, (size_t)B * k * 4);
+  return ok ? DEAMOE_OK : DEAMOE_ERR_CUDA;
+}
+
+deamoe_status_t deamoe_get_stats(deamoe_layer_t* L, void* cuda_stream, int32_t* n_active_dept,
+                                 int32_t* n_active_expert, int32_t* n_token_dept_pairs,
+                                 uint64_t* unique_weight_bytes, int32_t* device_status) {
+  if (!L) return DEAMOE_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return DEAMOE_ERR_CUDA;
+  int32_t c[CNT_COUNT] = {0};
+  if (L->last_B > 0 && cudaMemcpy(c, L->dev.counts, sizeof(c), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return DEAMOE_ERR_CUDA;
+  const LayerDev& d = L->dev;
+  if (n_active_dept) *n_active_dept = c[CNT_ACTIVE_DEPT];
+  if (n_active_expert) *n_active_expert = c[CNT_ACTIVE_EXPERT];
+  if (n_token_dept_pairs) *n_token_dept_pairs = c[CNT_TOKEN_DEPT];
+  if (unique_weight_bytes) {
+    const uint64_t s_w = dtype_size(d.wdt);
+    const uint64_t big = (uint64_t)3 * d.h * d.f * s_w, small = (uint64_t)3 * d.r * d.f * s_w;
+    uint64_t b = (uint64_t)d.n * d.h * 4 + (uint64_t)d.n_shared * 3 * d.h * d.fs * s_w;
+    if (L->last_B > 0) {
+      if (d.vanilla) b += (uint64_t)c[CNT_ACTIVE_EXPERT] * big;
+      else b += (uint64_t)c[CNT_ACTIVE_DEPT] * big + (uint64_t)c[CNT_ACTIVE_EXPERT] * small;
+    }
+    *unique_weight_bytes = b;
+  }
+  if (device_status) *device_status = c[CNT_STATUS];
+  return DEAMOE_OK;
+}
+
+int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launches : 0; }
+
+uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }
+
+const char* deamoe_status_string(deamoe_status_t st) {
+  switch (st) {
+    case DEAMOE_OK: return "ok";
+    case DEAMOE_ERR_INVALID_ARG: return "invalid argument";
+    case DEAMOE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case DEAMOE_ERR_ALLOC: return "allocation failed";
+    case DEAMOE_ERR_CUDA: return "CUDA runtime error";
+    case DEAMOE_ERR_BATCH: return "batch size out of range";
+    case DEAMOE_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

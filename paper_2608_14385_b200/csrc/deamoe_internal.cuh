@@ -1,0 +1,86 @@
+// Internal declarations shared by the translation units of libdeamoe.so.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "deamoe.h"
+
+namespace deamoe {
+
+// Stages of one decode step (Section 3.2 of the paper; SH* = shared expert, V* = vanilla MoE).
+enum Stage : int {
+  ST_S1 = 0,   // department gate/up:  GU = sigma([W_g; W_u] X^j)
+  ST_S2 = 1,   // private gate/up:     Y = SiLU(A_g G) * (A_u U)
+  ST_S3 = 2,   // private down:        Z = sigma(A_d^T Y)
+  ST_S4 = 3,   // department down:     O = W_d^T Z
+  ST_SH1 = 4,  // shared expert gate/up: Ysh = SiLU(W_sg x) * (W_su x)
+  ST_SH2 = 5,  // shared expert down:    Osh = W_sd^T Ysh
+  ST_V1 = 6,   // vanilla expert gate/up: Y = SiLU(W_gate x) * (W_up x)
+  ST_V2 = 7,   // vanilla expert down:    O = W_down^T Y
+  ST_COUNT = 8
+};
+
+enum Counter : int {
+  CNT_ACTIVE_DEPT = 0,
+  CNT_ACTIVE_EXPERT = 1,
+  CNT_TOKEN_DEPT = 2,
+  CNT_PAIRS = 3,
+  CNT_STATUS = 4,
+  CNT_NSEG = 5,
+  CNT_NITEMS = 6,
+  CNT_COUNT = 16
+};
+
+// Everything a kernel needs to know about the layer; passed by value.
+struct LayerDev {
+  // sizes
+  int h, m, g, n, f, r, k, k_dept, n_shared, fs, sigma, norm_topk, residual, vanilla;
+  int wdt, adt, max_batch;
+  int rp;  // rows of Y per pair: r, or f when there are no private parameters
+  float route_scale;
+  // canonical weights (PLAIN schedule and fp32); element type per wdt
+  const float* router;
+  const void *dept_gate, *dept_up, *dept_down;
+  const void *priv_gate, *priv_up, *priv_down;
+  const void *shared_gate, *shared_up, *shared_down;
+  // workspace
+  float* x32;          // [MB, h] tokens widened to fp32 (aliases the caller's tokens when fp32)
+  float* logit_part;   // [KS, MB, n]
+  int32_t* topk_idx;   // [MB, k]
+  float* topk_w;       // [MB, k]
+  uint64_t* dept_mask; // [ceil(m/64)]
+  int32_t* dept_off;   // [m+1]
+  int32_t* dept_tok;   // [MB*min(k,m)]
+  int32_t* expert_off; // [n+1]
+  int32_t* expert_tok; // [MB*k]
+  int32_t* pair_slot;  // [MB, k] slot of (t, q) in expert-major pair order
+  int32_t* pair_gurow; // [MB*k] pair slot -> row of GU (its (token, department) row)
+  int32_t* active_dept;   // [m]
+  int32_t* active_expert; // [n]
+  int32_t* counts;     // [CNT_COUNT]
+  float* GU;           // [MB*min(k,m), 2f]
+  float* Y;            // [MB*k, rp]   (vanilla: [MB*k, f])
+  float* Z;            // [MB*k, f]
+  float* O;            // [MB*k, h]
+  float* Ysh;          // [MB, fs]
+  float* Osh;          // [MB, h]
+};
+
+static __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
+
+static __device__ __forceinline__ float sigma_f(int kind, float v) {
+  if (kind == DEAMOE_SIGMA_SILU) return silu_f(v);
+  if (kind == DEAMOE_SIGMA_GELU) return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f));
+  return v;
+}
+
+// host-side launchers (each returns the number of kernels it launched, or -1 on a launch error)
+int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices, int32_t* user_idx,
+                 float* user_w);
+size_t bucket_smem_bytes(const LayerDev& L, int B);
+cudaError_t route_configure(const LayerDev& L);
+int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s);
+int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s);
+
+}  // namespace deamoe

@@ -1,0 +1,25 @@
+// Weight-streaming schedules (bf16): packed weights, device-built work list, persistent kernel.
+#pragma once
+#include "deamoe_internal.cuh"
+
+namespace deamoe {
+
+struct StreamPlan;
+
+// The schedule DEAMOE_SCHED_AUTO resolves to for streamable bf16 layers.
+int stream_default_schedule();
+
+// Re-pack the canonical weights into the streaming layout (enqueued on `s`) and allocate the
+// work-list buffers.  *bytes receives the device memory taken.
+deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w, int schedule, cudaStream_t s,
+                                   StreamPlan** out, uint64_t* bytes);
+void stream_plan_destroy(StreamPlan* p);
+
+// Enqueue the work-list construction for the routing state already on the device.
+// Returns the number of kernels launched or -1.
+int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
+
+// Enqueue all stages of one step.  Returns the number of kernels launched or -1.
+int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
+
+}  // namespace deamoe

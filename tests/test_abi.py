@@ -1,0 +1,45 @@
+"""The C-ABI library loads and exports every symbol the header declares (no GPU needed)."""
+import ctypes
+import os
+import re
+
+from paper_2608_14385_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "deamoe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(deamoe_[a-z_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    path = build.build()
+    lib = ctypes.CDLL(path)
+    names = _declared()
+    assert len(names) >= 12
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(binding.SYMBOLS) == names
+
+
+def test_status_strings_and_host_side_argument_errors():
+    L = binding.lib()
+    assert binding.status_string(binding.OK) == "ok"
+    for code in range(1, 7):
+        assert binding.status_string(code) not in ("", "ok")
+    # NULL arguments are rejected on the host before any CUDA call
+    out = ctypes.c_void_p()
+    assert L.deamoe_layer_create(None, None, None, ctypes.byref(out)) == binding.ERR_INVALID_ARG
+    assert L.deamoe_forward(None, None, None, 1, None) == binding.ERR_INVALID_ARG
+    assert L.deamoe_layer_destroy(None) == binding.OK
+    cfg = binding.Config(hidden=64, n_dept=2, experts_per_dept=2, ffn=32, priv=16, top_k=5, max_batch=4)
+    w = binding.Weights(router=1, dept_gate=1, dept_up=1, dept_down=1, priv_gate=1, priv_up=1, priv_down=1)
+    assert L.deamoe_layer_create(ctypes.byref(cfg), ctypes.byref(w), None, ctypes.byref(out)) == binding.ERR_INVALID_ARG
+    cfg.top_k = 2
+    cfg.max_batch = 100000
+    assert L.deamoe_layer_create(ctypes.byref(cfg), ctypes.byref(w), None, ctypes.byref(out)) == binding.ERR_BATCH
+    cfg.max_batch = 4
+    w.priv_gate = None
+    assert L.deamoe_layer_create(ctypes.byref(cfg), ctypes.byref(w), None, ctypes.byref(out)) == binding.ERR_INVALID_ARG

@@ -1,0 +1,206 @@
+"""GPU parity: the CUDA library against the fp64 oracle, through the C ABI, on the same seeded inputs.
+
+Routing indices, department sets and token lists must be bit-exact; gate weights within 1e-5;
+outputs within max|diff| <= 1e-2 * max|ref| + 1e-3 (bf16 weights, fp32 accumulation)."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2608_14385_b200 import binding, synth
+from tests.common import oracle_cfg
+from tests.gpu_common import check_routing, run_case
+
+pytestmark = pytest.mark.gpu
+
+SMALL = synth.LayerShape("small", hidden=64, n_dept=3, experts_per_dept=4, ffn=48, priv=32, top_k=3)
+RAGGED = synth.LayerShape("ragged", hidden=208, n_dept=5, experts_per_dept=3, ffn=176, priv=80, top_k=4,
+                          n_shared=1, shared_ffn=112)
+
+ALL_SCHEDULES = [binding.SCHED_PLAIN]
+
+
+def _scaled(shape, seed, scale=12.0, vanilla=False):
+    """Weights of std 0.02*scale: small layers need larger weights for non-trivial outputs."""
+    dev = torch.device("cuda:0")
+    w = (synth.make_vanilla_weights if vanilla else synth.make_deamoe_weights)(shape, seed, dev)
+    for k in w:
+        w[k] = (w[k].float() * scale).to(w[k].dtype) if k != "router" else w[k] * 4.0
+    return w
+
+
+def test_tiny_fp32_config():
+    """Benchmark configuration 1: h 256, 2 x 4 experts, f 512, r 32, top-2, 4 tokens, all fp32."""
+    res = run_case(synth.TINY, 4, seed=0)
+    assert res["err"] <= 1e-4 * np.abs(res["want"]["out"]).max() + 1e-6   # fp32 end to end is far tighter
+
+
+@pytest.mark.parametrize("schedule", ALL_SCHEDULES)
+@pytest.mark.parametrize("B", [1, 3, 8, 17])
+def test_small_bf16_layer_all_schedules(schedule, B):
+    w = _scaled(SMALL, 1)
+    run_case(SMALL, B, seed=1, schedule=schedule, weights=w)
+
+
+@pytest.mark.parametrize("schedule", ALL_SCHEDULES)
+def test_ragged_sizes_with_shared_expert_and_residual(schedule):
+    """Sizes that are not multiples of the kernel tiles (rows 176/80/112, k-extent 208), shared
+    expert, residual add, batch not a multiple of the token tile."""
+    shape = RAGGED.with_(residual=1)
+    run_case(shape, 11, seed=2, schedule=schedule, weights=_scaled(shape, 2))
+
+
+@pytest.mark.parametrize("schedule", ALL_SCHEDULES)
+def test_vanilla_comparator(schedule):
+    shape = RAGGED
+    run_case(shape, 9, seed=3, schedule=schedule, vanilla=True, weights=_scaled(shape, 3, vanilla=True))
+
+
+@pytest.mark.parametrize("schedule", ALL_SCHEDULES)
+@pytest.mark.parametrize("variant", ["no_private", "sigma_none", "gelu", "square_private", "g1", "k_eq_n",
+                                     "norm_all", "group_limited"])
+def test_variants(schedule, variant):
+    shape = {
+        "no_private": SMALL.with_(priv=0),
+        "sigma_none": SMALL.with_(sigma=0),
+        "gelu": SMALL.with_(sigma=2),
+        "square_private": SMALL.with_(priv=48),
+        "g1": SMALL.with_(n_dept=12, experts_per_dept=1),
+        "k_eq_n": SMALL.with_(n_dept=2, experts_per_dept=2, top_k=4),
+        "norm_all": SMALL.with_(norm_topk=0, route_scale=2.5),
+        "group_limited": SMALL.with_(n_dept=4, experts_per_dept=4, top_k=4, k_dept=2),
+    }[variant]
+    run_case(shape, 6, seed=4, schedule=schedule, weights=_scaled(shape, 4))
+
+
+@pytest.mark.parametrize("schedule", ALL_SCHEDULES)
+def test_all_tokens_identical_and_max_batch(schedule):
+    """Degenerate routing: every token picks the same experts (one department bucket holds the
+    whole batch); batch equal to max_batch."""
+    shape = SMALL
+    w = _scaled(shape, 5)
+    one = synth.make_tokens(shape, 1, 5, "cuda:0")
+    tokens = one.expand(32, shape.hidden).contiguous()
+    res = run_case(shape, 32, seed=5, schedule=schedule, weights=w, tokens=tokens, max_batch=32)
+    assert res["stats"]["active_expert"] == shape.top_k
+
+
+def test_exact_ties_break_to_lowest_index():
+    """Integer-valued router and tokens: logits are exact in fp32 whatever the summation order, so
+    equal logits are true ties and the selection must still match the oracle bit for bit."""
+    shape = SMALL.with_(n_dept=4, experts_per_dept=4, top_k=5)
+    dev = torch.device("cuda:0")
+    w = _scaled(shape, 6)
+    ints = torch.tensor(synth.uniform_ints(16 * 64, 3, 6, "ri"), dtype=torch.float32).reshape(16, 64) - 1.0
+    ints[5] = ints[2]
+    ints[9] = ints[2]
+    ints[12] = ints[0]
+    w["router"] = ints.to(dev)
+    tok = torch.tensor(synth.uniform_ints(7 * 64, 5, 6, "ti"), dtype=torch.float32).reshape(7, 64) - 2.0
+    tok[3] = 0.0                                           # all logits equal (zero)
+    tokens = tok.to(torch.bfloat16).to(dev)
+    layer = binding.Layer(shape, w, 8, binding.SCHED_PLAIN)
+    try:
+        layer.forward(tokens)
+        want, _ = check_routing(shape, layer, w, tokens, 7, require_guard=False)
+        assert (want["gap"] == 0).any()
+        assert list(want["idx"][3]) == [0, 1, 2, 3, 4]
+    finally:
+        layer.close()
+
+
+def test_route_entry_point_and_empty_batch():
+    shape = SMALL
+    w = _scaled(shape, 7)
+    layer = binding.Layer(shape, w, 8)
+    try:
+        tokens = synth.make_tokens(shape, 5, 7, "cuda:0")
+        idx, p = layer.route(tokens)
+        torch.cuda.synchronize()
+        want, _ = check_routing(shape, layer, w, tokens, 5)
+        assert (idx.cpu().numpy() == want["idx"]).all()
+        assert np.abs(p.cpu().numpy() - want["w"]).max() <= 1e-5
+        empty = tokens[:0].contiguous()
+        out = layer.forward(empty)
+        assert out.shape == (0, shape.hidden)
+        st = layer.stats()
+        assert st["active_dept"] == 0 and st["active_expert"] == 0 and st["device_status"] == 0
+        r = layer.routing(0)
+        assert (r["dept_off"] == 0).all() and (r["expert_off"] == 0).all() and r["dept_mask"][0] == 0
+        with pytest.raises(binding.DeaMoEError) as e:
+            layer.forward(synth.make_tokens(shape, 9, 7, "cuda:0"))
+        assert e.value.status == binding.ERR_BATCH
+        st_alias = binding.lib().deamoe_forward(layer._h, None, ctypes.c_void_p(tokens.data_ptr()), 5,
+                                                ctypes.c_void_p(tokens.data_ptr()))
+        assert st_alias == binding.ERR_INVALID_ARG
+    finally:
+        layer.close()
+
+
+def test_forward_host_matches_device_forward():
+    shape = RAGGED
+    w = _scaled(shape, 8)
+    layer = binding.Layer(shape, w, 8)
+    try:
+        tokens = synth.make_tokens(shape, 6, 8, "cuda:0")
+        dev_out = layer.forward(tokens).cpu()
+        host_in = tokens.cpu().pin_memory()
+        host_out = torch.empty_like(host_in).pin_memory()
+        layer.forward_host(host_in, host_out)
+        assert torch.equal(host_out, dev_out)
+    finally:
+        layer.close()
+
+
+def test_repeated_calls_are_bit_reproducible_and_state_is_reset():
+    """Two different batches alternately through one layer: each result must be identical every
+    time (no stale routing state, no order-dependent accumulation)."""
+    shape = RAGGED
+    w = _scaled(shape, 9)
+    layer = binding.Layer(shape, w, 16)
+    try:
+        a = synth.make_tokens(shape, 16, 9, "cuda:0")
+        b = synth.make_tokens(shape, 3, 10, "cuda:0")
+        ra, rb = layer.forward(a).clone(), layer.forward(b).clone()
+        for _ in range(3):
+            assert torch.equal(layer.forward(a), ra)
+            assert torch.equal(layer.forward(b), rb)
+    finally:
+        layer.close()
+
+
+@pytest.mark.parametrize("B", [1, 4, 16])
+def test_7b_class_layer(B):
+    """Benchmark configuration 2 at full size, every output element compared."""
+    run_case(synth.MOE7B, B, seed=0)
+
+
+def test_7b_class_vanilla():
+    run_case(synth.MOE7B, 4, seed=0, vanilla=True)
+
+
+@pytest.mark.parametrize("B,rows", [(1, [0]), (8, [0, 7]), (32, [13])])
+def test_dsv3_shape_full_size_sampled_rows(B, rows):
+    """Benchmark configuration 3 at full size (32 x 8 experts, top-8, shared expert): routing and
+    buckets for the whole batch, output values on sampled token rows (the oracle evaluates one
+    token row independently of the others)."""
+    run_case(synth.DSV3, B, seed=0, rows=rows, max_batch=32)
+
+
+def test_dsv3_shape_vanilla_sampled_row():
+    run_case(synth.DSV3, 4, seed=0, vanilla=True, rows=[2], max_batch=32)
+
+
+def test_unsupported_and_invalid_creates_are_reported():
+    dev = torch.device("cuda:0")
+    shape = SMALL.with_(hidden=66)                         # not a multiple of 4
+    w = {k: torch.zeros(1, device=dev) for k in ("router", "dept_gate", "dept_up", "dept_down",
+                                                 "priv_gate", "priv_up", "priv_down")}
+    with pytest.raises(binding.DeaMoEError) as e:
+        binding.Layer(shape, w, 4)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.DeaMoEError) as e:
+        binding.Layer(SMALL.with_(weight_dtype=0), w, 4, binding.SCHED_FUSED)   # fp32 cannot stream
+    assert e.value.status == binding.ERR_UNSUPPORTED
