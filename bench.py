@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the DeaMoE decode layer on B200: us per step and achieved HBM GB/s against the
+weight-streaming roofline (unique weight bytes / peak HBM bandwidth).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--batch B] [--shape dsv3|7b]
+                    [--schedule auto|plain|staged|fused] [--no-sweep] [--impl reference]
+
+One "step" = one forward of one DeaMoE layer (routing, bucketing, department and private stages,
+combine) over one batch of B synthetic tokens.  The headline workload is the DeepSeek-V3-shaped
+layer (h 7168, 32 departments x 8 experts, f 2048, private part 1/8 of an expert, top-8, one shared
+expert, bf16 weights) at B = 16.  Weights stay resident in HBM; every step streams the unique weights
+of its active departments and experts, far more than the L2 holds, and successive steps use
+different token batches (different routings).  A 256 MiB buffer is overwritten between steps to
+flush L2 (untimed).  Prints ONE JSON line.
+
+With N > 1 (torchrun) every rank runs an independent replica of the same layer on its own GPU --
+the path has no collective -- and the line reports the aggregate.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+PAPER_CONTEXT = {
+    "loaded_weights_reduction_max": 0.509,
+    "tpot_speedup_7b_a40": 1.33,
+    "layer_speedup_dsv3_a40": 2.00,
+    "layer_speedup_dsv3_h100": 1.97,
+    "note": "the paper's figures (other hardware, its own DeaMoE configuration); context only",
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy read+write)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            p = [x.strip() for x in ln.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1])); power.append(float(p[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def pct(xs, q):
+    xs = sorted(xs)
+    return xs[min(len(xs) - 1, max(0, int(round(q * (len(xs) - 1)))))]
+
+
+def oracle_sample_seconds(shape, weights_fn, tokens, rows, vanilla=False):
+    """Time the fp64 oracle (as it stands) on `rows` of this batch with all host cores."""
+    import numpy as np
+    from oracle import ref
+    from paper_2608_14385_b200 import synth
+    cores = ref.host_cores()
+    ref.set_threads(cores)
+    cfg = ref.make_config(**shape.asdict())
+    router = synth.to_numpy(weights_fn("router", None))
+    tok = synth.to_numpy(tokens)
+    r = ref.route(cfg, router, tok)
+    sel = r["idx"][rows].reshape(-1)
+    experts = sorted({int(i) for i in sel})
+    depts = sorted({int(i) // shape.experts_per_dept for i in sel})
+    m, n = shape.n_dept, shape.n_expert
+    w = {"router": router}
+    units = experts if vanilla else depts
+    for name in ("gate", "up", "down"):
+        tab = [None] * (n if vanilla else m)
+        for u in units:
+            tab[u] = synth.to_numpy(weights_fn(f"dept_{name}", u))
+        w[f"dept_{name}"] = tab
+        if not vanilla and shape.priv > 0:
+            tab = [None] * n
+            for i in experts:
+                tab[i] = synth.to_numpy(weights_fn(f"priv_{name}", i))
+            w[f"priv_{name}"] = tab
+        if shape.n_shared:
+            w[f"shared_{name}"] = synth.to_numpy(weights_fn(f"shared_{name}", None))
+    fwd = ref.vanilla_forward if vanilla else ref.deamoe_forward
+    t0 = time.perf_counter()
+    fwd(cfg, w, tok, rows=rows)
+    return time.perf_counter() - t0, cores
+
+
+def run_reference(args, shape, rank, world):
+    """--impl reference: the oracle on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    import torch
+    from paper_2608_14385_b200 import synth
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    B = args.batch
+
+    def wfn(name, unit):
+        if name == "router":
+            return synth.make_router(shape, 0, dev)
+        if unit is None:
+            return synth.normal((shape.shared_ffn, shape.hidden), synth.W_STD, 0, f"L0/{name}", dev,
+                                torch.bfloat16 if shape.weight_dtype else torch.float32)
+        return synth.weight_slice(shape, name, unit, 0, dev)
+    rows = [0]
+    times = []
+    for step in range(args.warmup + args.steps):
+        tokens = synth.make_tokens(shape, B, 100 + step % 4, dev)
+        sec, cores = oracle_sample_seconds(shape, wfn, tokens, rows)
+        if step >= args.warmup:
+            times.append(sec * B / len(rows))
+    us = statistics.mean(times) * 1e6
+    line = {
+        "impl": "reference", "metric": "us_per_step_deamoe_layer", "value": us, "unit": "us", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{shape.name}-shape DeaMoE layer, decode batch {B}", "batch": B},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
+                         "sample": f"{len(rows)} of {B} token rows per step, time scaled by {B}/{len(rows)}"},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def time_layer(layer, batches, steps, warmup, flush, torch, barrier):
+    """Per-step CUDA-event times (ms) of layer.forward over rotating token batches."""
+    outs = [torch.empty_like(b) for b in batches]
+    for i in range(warmup):
+        flush.add_(1)
+        layer.forward(batches[i % len(batches)], outs[i % len(batches)])
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    launches = 0
+    torch.cuda.synchronize()
+    barrier()
+    for i in range(steps):
+        flush.add_(1)                      # overwrite 256 MiB: evicts the previous step from L2
+        ev[i][0].record()
+        layer.forward(batches[i % len(batches)], outs[i % len(batches)])
+        ev[i][1].record()
+        launches += layer.last_launches
+    torch.cuda.synchronize()
+    barrier()
+    return [a.elapsed_time(b) for a, b in ev], launches
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--shape", default="dsv3")
+    ap.add_argument("--schedule", default="auto", choices=["auto", "plain", "staged", "fused"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true", help="skip the batch sweep and the vanilla comparator")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle")
+    args = ap.parse_args()
+
+    from paper_2608_14385_b200 import synth
+    shape = synth.SHAPES[args.shape]
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, shape, rank, world)
+        return
+
+    import torch
+    from paper_2608_14385_b200 import binding
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    sched = {"auto": binding.SCHED_AUTO, "plain": binding.SCHED_PLAIN, "staged": binding.SCHED_STAGED,
+             "fused": binding.SCHED_FUSED}[args.schedule]
+    peak, peak_src = measured_peaks()
+    B = args.batch
+    max_batch = max(32, B)
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    layer = binding.Layer(shape, w, max_batch, sched)
+    router = w["router"]
+    shared = {k: v for k, v in w.items() if k.startswith("shared_")}
+    del w
+    torch.cuda.empty_cache()
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    NB = 4
+    batches = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(NB)]
+    ubytes = []
+    for b in batches:
+        layer.forward(b)
+        ubytes.append(layer.stats()["unique_weight_bytes"])
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    times_ms, launches = time_layer(layer, batches, args.steps, args.warmup, flush, torch, barrier)
+    clocks = sampler.stop()
+    total_ms = sum(times_ms)
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    # aggregate: layer-steps processed by all ranks per unit time -> us per layer-step
+    us_per_step = total_ms * 1e3 / (args.steps * world)
+    step_bytes = [ubytes[i % NB] for i in range(args.steps)]
+    gbs = [bts / (ms * 1e-3) / 1e9 for bts, ms in zip(step_bytes, times_ms)]
+    mean_bytes = statistics.mean(step_bytes)
+
+    # dominant kernel (weight streaming): events recorded by the library around its launches
+    kern = layer.kernel_times(batches, args.steps, flush) if hasattr(layer, "kernel_times") else None
+    router_bytes = shape.n_expert * shape.hidden * 4
+    if kern:
+        k_ms = statistics.mean(kern)
+        achieved = (mean_bytes - router_bytes) / (k_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "kernel": "k_stream (all weight-streaming launches of one step)",
+                "kernel_ms": k_ms, "peak_source": peak_src,
+                "algorithmic_bytes_per_step": mean_bytes - router_bytes}
+    else:
+        achieved = mean_bytes / (statistics.mean(times_ms) * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "kernel": "whole step (plain schedule has no single dominant kernel)",
+                "peak_source": peak_src, "algorithmic_bytes_per_step": mean_bytes}
+
+    # end to end through the public host-buffer entry point
+    host_in = [b.cpu().pin_memory() for b in batches]
+    host_out = torch.empty_like(host_in[0]).pin_memory()
+    for i in range(3):
+        layer.forward_host(host_in[i % NB], host_out)
+    e2e_t = []
+    for i in range(args.steps):
+        flush.add_(1)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        layer.forward_host(host_in[i % NB], host_out)
+        e2e_t.append(time.perf_counter() - t0)
+    io_bytes = B * shape.hidden * (2 if shape.act_dtype else 4)
+    e2e_us = statistics.mean(e2e_t) * 1e6
+    if dist is not None:
+        t = torch.tensor([e2e_us], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_us = float(t.item()) / world
+
+    line = {
+        "metric": "us_per_step_deamoe_layer", "value": us_per_step, "unit": "us", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": us_per_step / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.weight_dtype else "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{shape.name}-shape DeaMoE layer, decode batch {B} (replica per GPU)",
+                   "batch": B, "hidden": shape.hidden, "n_dept": shape.n_dept, "experts_per_dept": shape.experts_per_dept,
+                   "ffn": shape.ffn, "priv": shape.priv, "top_k": shape.top_k, "n_shared": shape.n_shared,
+                   "schedule": args.schedule, "l2": "256 MiB buffer overwritten between steps (untimed); "
+                   "4 rotating token batches", "accumulate": "fp32"},
+        "us_per_step_p10_p50_p90": [pct(times_ms, 0.1) * 1e3, pct(times_ms, 0.5) * 1e3, pct(times_ms, 0.9) * 1e3],
+        "hbm_gbs_on_unique_bytes": {"mean": statistics.mean(gbs), "p50": pct(gbs, 0.5),
+                                    "frac_of_measured_peak": statistics.mean(gbs) / peak,
+                                    "frac_of_nominal_8TBs": statistics.mean(gbs) / 8000.0},
+        "unique_weight_mb_per_step": mean_bytes / 1e6,
+        "clocks": clocks,
+        "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": io_bytes, "d2h_bytes_per_step": io_bytes},
+        "gpu_launches": launches,
+        "roofline": roof,
+        "paper_context": PAPER_CONTEXT,
+    }
+
+    if rank == 0 and not args.no_sweep:
+        line["sweep"] = sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev)
+    if rank == 0 and not args.no_cpu:
+        def wfn(name, unit):
+            if name == "router":
+                return router
+            if unit is None:
+                return shared[name]
+            return synth.weight_slice(shape, name, unit, 0, dev)
+        sec, cores = oracle_sample_seconds(shape, wfn, batches[0], [0])
+        line["cpu_baseline"] = {"value": sec * B * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+                                "sample": f"1 of {B} token rows of one step, time scaled by {B}"}
+    layer.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev):
+    """DeaMoE layer and the in-library vanilla MoE at the same shape over the batch range."""
+    from paper_2608_14385_b200 import binding, synth
+    out = []
+    batches_list = [1, 2, 4, 8, 16, 32] if shape.name == "dsv3" else [1, 4, 16]
+    steps = max(10, args.steps // 2)
+    res = {}
+    for B in batches_list:
+        bs = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(4)]
+        ub = []
+        for b in bs:
+            layer.forward(b)
+            ub.append(layer.stats()["unique_weight_bytes"])
+        t, _ = time_layer(layer, bs, steps, 3, flush, torch, lambda: None)
+        res[B] = {"batch": B, "deamoe_us": pct(t, 0.5) * 1e3, "deamoe_mb": statistics.mean(ub) / 1e6}
+    vw = synth.make_vanilla_weights(shape, 0, dev, router=router)
+    vl = binding.Layer(shape, vw, 32, sched, vanilla=True)
+    del vw
+    torch.cuda.empty_cache()
+    for B in batches_list:
+        bs = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(4)]
+        ub = []
+        for b in bs:
+            vl.forward(b)
+            ub.append(vl.stats()["unique_weight_bytes"])
+        t, _ = time_layer(vl, bs, steps, 3, flush, torch, lambda: None)
+        r = res[B]
+        r["vanilla_us"] = pct(t, 0.5) * 1e3
+        r["vanilla_mb"] = statistics.mean(ub) / 1e6
+        r["deamoe_gbs"] = r["deamoe_mb"] / r["deamoe_us"] * 1e3
+        r["vanilla_gbs"] = r["vanilla_mb"] / r["vanilla_us"] * 1e3
+        r["deamoe_frac_of_measured_peak"] = r["deamoe_gbs"] / peak
+        r["speedup_vs_vanilla"] = r["vanilla_us"] / r["deamoe_us"]
+        r["byte_ratio_vanilla_over_deamoe"] = r["vanilla_mb"] / r["deamoe_mb"]
+        out.append(r)
+    vl.close()
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -242,6 +242,7 @@ __global__ void __launch_bounds__(BUCKET_THREADS) k_bucket(LayerDev L, int B) {
   for (int i = tid; i <= n; i += BUCKET_THREADS) L.expert_off[i] = s_eoff[i];
   for (int j = tid; j <= m; j += BUCKET_THREADS) L.dept_off[j] = s_doff[j];
   if (tid == 0) {
+    L.counts[CNT_STATUS] = 0;
     L.counts[CNT_TOKEN_DEPT] = s_doff[m];
     L.counts[CNT_PAIRS] = s_eoff[n];
   }

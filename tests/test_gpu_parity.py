@@ -19,7 +19,7 @@ SMALL = synth.LayerShape("small", hidden=64, n_dept=3, experts_per_dept=4, ffn=4
 RAGGED = synth.LayerShape("ragged", hidden=208, n_dept=5, experts_per_dept=3, ffn=176, priv=80, top_k=4,
                           n_shared=1, shared_ffn=112)
 
-ALL_SCHEDULES = [binding.SCHED_PLAIN]
+ALL_SCHEDULES = [binding.SCHED_PLAIN, binding.SCHED_STAGED]
 
 
 def _scaled(shape, seed, scale=12.0, vanilla=False):
