@@ -157,16 +157,16 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
     A(dev_alloc(L, &d.active_dept, (size_t)d.m));
     A(dev_alloc(L, &d.active_expert, (size_t)d.n));
     A(dev_alloc(L, &d.counts, (size_t)CNT_COUNT));
-    if (!vanilla) {
-      A(dev_alloc(L, &d.GU, (size_t)tdmax * 2 * d.f));
-      A(dev_alloc(L, &d.Z, (size_t)pmax * d.f));
+    if (sched == DEAMOE_SCHED_PLAIN) {  // fp32 intermediates of the plain kernels
+      if (!vanilla) {
+        A(dev_alloc(L, &d.GU, (size_t)tdmax * 2 * d.f));
+        A(dev_alloc(L, &d.Z, (size_t)pmax * d.f));
+      }
+      A(dev_alloc(L, &d.Y, (size_t)pmax * (vanilla ? d.f : d.rp)));
+      if (d.n_shared) A(dev_alloc(L, &d.Ysh, (size_t)MB * d.fs));
     }
-    A(dev_alloc(L, &d.Y, (size_t)pmax * (vanilla ? d.f : d.rp)));
     A(dev_alloc(L, &d.O, (size_t)pmax * d.h));
-    if (d.n_shared) {
-      A(dev_alloc(L, &d.Ysh, (size_t)MB * d.fs));
-      A(dev_alloc(L, &d.Osh, (size_t)MB * d.h));
-    }
+    if (d.n_shared) A(dev_alloc(L, &d.Osh, (size_t)MB * d.h));
     const size_t io = (size_t)MB * d.h * dtype_size(d.adt);
     A(dev_alloc(L, reinterpret_cast<char**>(&L->stage_tokens), io));
     A(dev_alloc(L, reinterpret_cast<char**>(&L->stage_out), io));
@@ -197,6 +197,7 @@ deamoe_status_t check_call(deamoe_layer_t* L, const void* tokens, int B) {
 
 LayerDev call_view(deamoe_layer_t* L, const void* tokens) {
   LayerDev d = L->dev;
+  d.tokens_raw = tokens;
   if (d.adt == DEAMOE_F32) d.x32 = const_cast<float*>(reinterpret_cast<const float*>(tokens));
   return d;
 }
@@ -346,6 +347,12 @@ deamoe_status_t deamoe_get_stats(deamoe_layer_t* L, void* cuda_stream, int32_t* 
 int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launches : 0; }
 
 uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }
+
+#ifdef DEAMOE_TRACE
+int deamoe_debug_trace(deamoe_layer_t* L, long long* host, int max_ctas) {
+  return (L && L->plan) ? deamoe::stream_read_trace(*L->plan, host, max_ctas) : 0;
+}
+#endif
 
 const char* deamoe_status_string(deamoe_status_t st) {
   switch (st) {

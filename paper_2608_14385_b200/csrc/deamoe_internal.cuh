@@ -45,6 +45,7 @@ struct LayerDev {
   const void *priv_gate, *priv_up, *priv_down;
   const void *shared_gate, *shared_up, *shared_down;
   // workspace
+  const void* tokens_raw;  // the caller's tokens of this call, in act dtype
   float* x32;          // [MB, h] tokens widened to fp32 (aliases the caller's tokens when fp32)
   float* logit_part;   // [KS, MB, n]
   int32_t* topk_idx;   // [MB, k]

@@ -17,6 +17,7 @@
 //
 // Weights never depend on earlier stages, so the ring keeps the HBM pipe full across item and
 // stage boundaries; only the (tiny) activations wait for their producers.
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -26,14 +27,25 @@ namespace deamoe {
 
 constexpr int CONSUMER_WARPS = 8;
 constexpr int CONSUMER_THREADS = CONSUMER_WARPS * 32;
-constexpr int STREAM_THREADS = CONSUMER_THREADS + 32;
-constexpr int SLOT_BYTES = 32 * 1024;
+constexpr int WARP_ISSUE = CONSUMER_WARPS;       // issues the bulk copies
+constexpr int WARP_PLAN = CONSUMER_WARPS + 1;    // picks items, fetches records, waits for inputs
+constexpr int WARP_EPI = CONSUMER_WARPS + 2;     // reduces, applies epilogues, publishes completions
+constexpr int STREAM_THREADS = CONSUMER_THREADS + 96;
+constexpr int DESC_DEPTH = 8;                    // item descriptors queued between planner and epilogue
+constexpr int DESC_BYTES = 1024;                 // Seg | tail | weight sources | activation row sources
+constexpr int DESC_TAIL = 224, DESC_WSRC = 256, DESC_ASRC = 272;
+constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
+constexpr int SIG_DEPTH = 16;
+constexpr int CLAIM_BATCH = 2;  // consecutive items claimed at once
+constexpr int SLOT_BYTES = 30 * 1024;
 constexpr int SLOT_HDR = 128;
 constexpr int NSLOT = 6;
 constexpr int ACT_PAD = 8;   // floats of padding per activation row in shared memory
 constexpr int MAX_QP = 4;    // (tiles per item) x (8-token passes) held in accumulators
 constexpr int RED_FLOATS = CONSUMER_WARPS * MAX_QP * 128;
-constexpr size_t STREAM_SMEM = (size_t)NSLOT * SLOT_BYTES + (size_t)RED_FLOATS * 4 + 256;
+constexpr size_t STREAM_SMEM =
+    (size_t)NSLOT * SLOT_BYTES + (size_t)NRED * RED_FLOATS * 4 + (size_t)DESC_DEPTH * DESC_BYTES + 1024;
+static_assert(STREAM_SMEM <= 227 * 1024, "shared memory budget");
 constexpr unsigned SPIN_LIMIT = 1u << 24;  // bounded waits; then an error status, never a hang
 constexpr int MAX_CAT = 8;
 
@@ -65,15 +77,23 @@ struct Seg {
   int item0, n_items, stage, epi;
   int T, q, paired, nB;
   int kc, C, rows, n_tiles;
-  int in_stride, in_row0, out_stride, out_row0;
-  int dep_idx, dep_target, done_idx, use_lo;
+  int in_stride, out_stride, out_row0, dep_idx;   // dep_idx / dep_target are ints 15 / 16 (planner)
+  int dep_target, done_idx, planes, pad0;
   const __nv_bfloat16* w0;
   const __nv_bfloat16* w1;
-  const float* in0;
-  const float* in1;
-  const int32_t* in_rows;
-  float* out;
+  const __nv_bfloat16* in0h;   // activations: bf16 "hi" plane, row-major
+  const __nv_bfloat16* in0l;   // optional "lo" plane (x - hi), planes == 2
+  const __nv_bfloat16* in1h;   // second input of stages whose two matrices read different vectors
+  const __nv_bfloat16* in1l;
+  __nv_bfloat16* outh;         // output planes of stages that feed another stage
+  __nv_bfloat16* outl;
+  float* outf;                 // fp32 output of the last stage (read by the combine)
+  unsigned long long pad1;
+  uint16_t rows16[32];         // input row of each of the T tokens
 };
+static_assert(sizeof(Seg) == 224, "Seg layout is relied upon by the planner warp");
+constexpr int SEG_VEC = sizeof(Seg) / 16;
+static_assert(sizeof(Seg) % 16 == 0, "Seg is copied with 16-byte loads");
 
 struct StreamDev {
   StageCfg st[ST_COUNT];
@@ -81,7 +101,22 @@ struct StreamDev {
   int32_t* sync;
   int max_segs;
   int dep_s1, dep_s2, dep_s3, dep_sh1, n_dep;  // offsets relative to SY_DEP
+  int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
+  // activations between stages, bf16 planes ([rows, width] each)
+  __nv_bfloat16 *xh, *xl;      // tokens split (fp32 activations only; bf16 tokens are read in place)
+  __nv_bfloat16 *GUh, *GUl, *Yh, *Yl, *Zh, *Zl, *Yshh, *Yshl;
+  long long* trace;  // per-CTA cycle counters, only in -DDEAMOE_TRACE builds (else nullptr)
 };
+
+#ifdef DEAMOE_TRACE
+#define TR_NOW() clock64()
+#define TR_ADD(k, t0) tr[k] += clock64() - (t0)
+#else
+#define TR_NOW() 0ll
+#define TR_ADD(k, t0) ((void)(t0))
+#endif
+enum TraceSlot : int { TR_META = 0, TR_DEP, TR_EMPTY, TR_ISSUE, TR_ITEMS, TR_CHUNKS, TR_PTOTAL, TR_FULL = 8, TR_COMPUTE,
+                       TR_EPI, TR_CTOTAL, TR_SLOTS = 16 };
 
 struct StreamPlan {
   StreamDev dev;
@@ -91,17 +126,8 @@ struct StreamPlan {
   uint64_t bytes;
 };
 
-// chunk header written by the producer at the start of a ring slot
-struct SlotHdr {
-  int kind;  // 0 data, 1 end of work
-  int first, last, kc;
-  int T, q, paired, nB;
-  int epi, use_lo, row0, rows;
-  int out_stride, out_row0, npass, pad;
-  float* out;
-  int32_t* done;
-};
-static_assert(sizeof(SlotHdr) <= SLOT_HDR, "slot header too large");
+static_assert(sizeof(Seg) == DESC_TAIL && DESC_ASRC + 64 * 8 <= DESC_BYTES, "descriptor layout");
+
 
 // ---------------------------------------------------------------- PTX wrappers
 static __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -135,6 +161,16 @@ static __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }
   return false;
+}
+// One lane polls for the whole warp; the other lanes wait at the warp barrier without touching
+// the shared-memory pipe.  Every lane then observes the completed phase itself (acquire).
+static __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                      int lane) {
+  bool ok = true;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag);
+  ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+  __syncwarp();  // orders the other lanes' reads after lane 0's acquire
+  return ok;
 }
 static __device__ __forceinline__ uint64_t policy_evict_first() {
   uint64_t p;
@@ -171,18 +207,6 @@ static __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4& a, u
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
 }
-// two fp32 -> packed bf16 pair (first value in the low half) and the rounding remainders
-static __device__ __forceinline__ uint32_t pack_hi(float x, float y, float& rx, float& ry) {
-  const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
-  rx = x - __bfloat162float(h.x);
-  ry = y - __bfloat162float(h.y);
-  return *reinterpret_cast<const uint32_t*>(&h);
-}
-static __device__ __forceinline__ uint32_t pack_bf(float x, float y) {
-  const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
-  return *reinterpret_cast<const uint32_t*>(&h);
-}
-
 // ---------------------------------------------------------------- weight re-packing (create)
 // dst: [unit][tile][k-tile][lane][8 bf16]; element (row, k) of the logical matrix is read from
 // src[unit*src_unit + row*row_stride + k*col_stride].  Rows beyond `rows` are zero.
@@ -261,11 +285,12 @@ static __device__ __forceinline__ int unit_tokens(const LayerDev& L, int stage, 
 }
 static __device__ __forceinline__ int groups_of(int T, int tg) { return (T + tg - 1) / tg; }
 
-static __device__ __forceinline__ int chunk_k(int C, int q, int nB, int T) {
-  const int avail = SLOT_BYTES - SLOT_HDR - nB * T * ACT_PAD * 4;
-  int kc = avail / (q * 32 + nB * T * 4);
+static __device__ __forceinline__ int chunk_k(int C, int q, int act_rows) {
+  const int avail = SLOT_BYTES - SLOT_HDR - act_rows * ACT_PAD * 2;
+  int kc = (avail / (q * 32 + act_rows * 2)) & ~15;   // largest chunk a slot can hold
   if (kc > C) kc = C;
-  kc = (kc >= 128) ? (kc & ~127) : (kc & ~15);
+  const int nch = (C + kc - 1) / kc;                   // then balance the chunks of one item
+  kc = (((C + nch - 1) / nch) + 15) & ~15;
   return kc;
 }
 
@@ -280,69 +305,79 @@ static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stag
   s.C = sc.C; s.rows = sc.rows; s.n_tiles = sc.n_tiles;
   s.w0 = sc.w0 + (size_t)id * sc.unit_elems;
   s.w1 = sc.w1 ? sc.w1 + (size_t)id * sc.unit_elems : nullptr;
-  s.in1 = nullptr; s.in_rows = nullptr; s.in_row0 = 0;
+  s.in0l = nullptr; s.in1h = nullptr; s.in1l = nullptr;
+  s.pad0 = 0; s.pad1 = 0;
+  const int32_t* in_list = nullptr;  // gathered input rows, or in_row0 + s
+  int in_row0 = 0;
+  s.outh = nullptr; s.outl = nullptr; s.outf = nullptr;
   s.dep_idx = -1; s.dep_target = 0; s.done_idx = -1;
-  s.use_lo = 1;
+  s.planes = P.planes;
+  // tokens: bf16 tokens are their own (only) plane; fp32 tokens were split by k_split_tokens
+  const __nv_bfloat16* tokh = (L.adt == DEAMOE_BF16) ? reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw) : P.xh;
+  const __nv_bfloat16* tokl = (L.adt == DEAMOE_BF16) ? nullptr : P.xl;
   const int j = (stage == ST_S2 || stage == ST_S3) ? id / L.g : id;
   switch (stage) {
     case ST_S1:
-      s.in0 = L.x32; s.in_stride = L.h; s.in_rows = L.dept_tok + L.dept_off[id] + t0;
-      s.out = L.GU; s.out_stride = 2 * L.f; s.out_row0 = L.dept_off[id] + t0;
-      s.done_idx = P.dep_s1 + id; s.use_lo = (L.adt == DEAMOE_F32);
+      s.in0h = tokh; s.in0l = tokl; s.in_stride = L.h; in_list = L.dept_tok + L.dept_off[id] + t0;
+      s.outh = P.GUh; s.outl = P.GUl; s.out_stride = 2 * L.f; s.out_row0 = L.dept_off[id] + t0;
+      s.done_idx = P.dep_s1 + id;
       break;
     case ST_S2:
-      s.in0 = L.GU; s.in1 = L.GU + L.f; s.nB = 2; s.in_stride = 2 * L.f;
-      s.in_rows = L.pair_gurow + L.expert_off[id] + t0;
-      s.out = L.Y; s.out_stride = L.rp; s.out_row0 = L.expert_off[id] + t0;
+      s.in0h = P.GUh; s.in0l = P.GUl; s.in1h = P.GUh + L.f; s.in1l = P.GUl + L.f; s.nB = 2;
+      s.in_stride = 2 * L.f;
+      in_list = L.pair_gurow + L.expert_off[id] + t0;
+      s.outh = P.Yh; s.outl = P.Yl; s.out_stride = L.rp; s.out_row0 = L.expert_off[id] + t0;
       s.dep_idx = P.dep_s1 + j;
-      s.dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].items_per_seg;
+      s.dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
       s.done_idx = P.dep_s2 + id;
       break;
     case ST_S3:
-      s.in0 = L.Y; s.in_stride = L.rp; s.in_row0 = L.expert_off[id] + t0;
-      s.out = L.Z; s.out_stride = L.f; s.out_row0 = L.expert_off[id] + t0;
+      s.in0h = P.Yh; s.in0l = P.Yl; s.in_stride = L.rp; in_row0 = L.expert_off[id] + t0;
+      s.outh = P.Zh; s.outl = P.Zl; s.out_stride = L.f; s.out_row0 = L.expert_off[id] + t0;
       s.dep_idx = P.dep_s2 + id;
-      s.dep_target = groups_of(Tall, P.st[ST_S2].tg) * P.st[ST_S2].items_per_seg;
+      s.dep_target = groups_of(Tall, P.st[ST_S2].tg) * P.st[ST_S2].n_tiles;
       s.done_idx = P.dep_s3 + j;
       break;
     case ST_S4: {
       const int p0 = L.expert_off[id * L.g];
-      s.in0 = L.Z; s.in_stride = L.f; s.in_row0 = p0 + t0;
-      s.out = L.O; s.out_stride = L.h; s.out_row0 = p0 + t0;
+      s.in0h = P.Zh; s.in0l = P.Zl; s.in_stride = L.f; in_row0 = p0 + t0;
+      s.outf = L.O; s.out_stride = L.h; s.out_row0 = p0 + t0;
       if (L.r > 0) {
         int target = 0;
         for (int e = 0; e < L.g; ++e) {
           const int Te = L.expert_off[id * L.g + e + 1] - L.expert_off[id * L.g + e];
-          target += groups_of(Te, P.st[ST_S3].tg) * P.st[ST_S3].items_per_seg;
+          target += groups_of(Te, P.st[ST_S3].tg) * P.st[ST_S3].n_tiles;
         }
         s.dep_idx = P.dep_s3 + id; s.dep_target = target;
       }
       break;
     }
     case ST_SH1:
-      s.in0 = L.x32; s.in_stride = L.h; s.in_row0 = t0;
-      s.out = L.Ysh; s.out_stride = L.fs; s.out_row0 = t0;
-      s.done_idx = P.dep_sh1; s.use_lo = (L.adt == DEAMOE_F32);
+      s.in0h = tokh; s.in0l = tokl; s.in_stride = L.h; in_row0 = t0;
+      s.outh = P.Yshh; s.outl = P.Yshl; s.out_stride = L.fs; s.out_row0 = t0;
+      s.done_idx = P.dep_sh1;
       break;
     case ST_SH2:
-      s.in0 = L.Ysh; s.in_stride = L.fs; s.in_row0 = t0;
-      s.out = L.Osh; s.out_stride = L.h; s.out_row0 = t0;
+      s.in0h = P.Yshh; s.in0l = P.Yshl; s.in_stride = L.fs; in_row0 = t0;
+      s.outf = L.Osh; s.out_stride = L.h; s.out_row0 = t0;
       s.dep_idx = P.dep_sh1;
-      s.dep_target = groups_of(B, P.st[ST_SH1].tg) * P.st[ST_SH1].items_per_seg;
+      s.dep_target = groups_of(B, P.st[ST_SH1].tg) * P.st[ST_SH1].n_tiles;
       break;
     case ST_V1:
-      s.in0 = L.x32; s.in_stride = L.h; s.in_rows = L.expert_tok + L.expert_off[id] + t0;
-      s.out = L.Y; s.out_stride = L.f; s.out_row0 = L.expert_off[id] + t0;
-      s.done_idx = P.dep_s2 + id; s.use_lo = (L.adt == DEAMOE_F32);
+      s.in0h = tokh; s.in0l = tokl; s.in_stride = L.h; in_list = L.expert_tok + L.expert_off[id] + t0;
+      s.outh = P.Yh; s.outl = P.Yl; s.out_stride = L.f; s.out_row0 = L.expert_off[id] + t0;
+      s.done_idx = P.dep_s2 + id;
       break;
     case ST_V2:
-      s.in0 = L.Y; s.in_stride = L.f; s.in_row0 = L.expert_off[id] + t0;
-      s.out = L.O; s.out_stride = L.h; s.out_row0 = L.expert_off[id] + t0;
+      s.in0h = P.Yh; s.in0l = P.Yl; s.in_stride = L.f; in_row0 = L.expert_off[id] + t0;
+      s.outf = L.O; s.out_stride = L.h; s.out_row0 = L.expert_off[id] + t0;
       s.dep_idx = P.dep_s2 + id;
-      s.dep_target = groups_of(Tall, P.st[ST_V1].tg) * P.st[ST_V1].items_per_seg;
+      s.dep_target = groups_of(Tall, P.st[ST_V1].tg) * P.st[ST_V1].n_tiles;
       break;
   }
-  s.kc = chunk_k(s.C, s.q, s.nB, s.T);
+  if (!s.in0l) s.planes = 1;
+  s.kc = chunk_k(s.C, s.q, s.planes * s.nB * s.T);
+  for (int t = 0; t < 32; ++t) s.rows16[t] = (uint16_t)(t < s.T ? (in_list ? in_list[t] : in_row0 + t) : 0);
   if (seg_index < P.max_segs) P.segs[seg_index] = s;
 }
 
@@ -414,6 +449,54 @@ __global__ void __launch_bounds__(BUILD_THREADS) k_build_worklist(LayerDev L, St
   }
 }
 
+// ---------------------------------------------------------------- inner loop of the consumers
+// One ring slot holds q weight tiles x kc columns (per-lane A fragments, 512 B per k-tile and tile)
+// followed by the activation rows [plane][input][token] x (kc + ACT_PAD) bf16.  A consumer warp
+// works on ONE tile: with two tiles in the slot warps 0-3 take the first and warps 4-7 the second
+// (4-way split of the k-tiles), with one tile all eight warps share it (8-way split).  The warp's
+// k-tiles are handled G at a time: every shared-memory load of the group is issued before its
+// first MMA, so the load latencies overlap.  acc[p] accumulates tokens 8p..8p+7.
+template <int NPASS, int PLANES>
+static __device__ __forceinline__ void consume_chunk(float (&acc)[4][4], const unsigned char* wtile,
+                                                     const uint32_t* act, int lo, int kc, int T, int ks, int kw,
+                                                     int lane) {
+  constexpr int G = (NPASS * PLANES <= 1) ? 8 : (NPASS * PLANES <= 2 ? 4 : 2);
+  const int g = lane >> 2, tig = lane & 3;
+  const int nkt = kc >> 4;
+  const int aw = (kc + ACT_PAD) >> 1;                       // activation row stride in 32-bit words
+  const uint4* w0 = reinterpret_cast<const uint4*>(wtile) + lane;
+  const uint32_t* rb[NPASS];
+#pragma unroll
+  for (int p = 0; p < NPASS; ++p) rb[p] = act + min(p * 8 + g, T - 1) * aw + tig;
+  const int mine = (nkt > ks) ? (nkt - ks + kw - 1) / kw : 0;  // k-tiles ks, ks+kw, ... of this warp
+  for (int i0 = 0; i0 < mine; i0 += G) {
+    uint4 A[G];
+    uint32_t B[G][NPASS][PLANES][2];
+#pragma unroll
+    for (int u = 0; u < G; ++u) {
+      const int kt = ks + min(i0 + u, mine - 1) * kw;       // clamped: the tail re-reads a valid tile
+      A[u] = w0[kt * 32];
+#pragma unroll
+      for (int p = 0; p < NPASS; ++p)
+#pragma unroll
+        for (int pl = 0; pl < PLANES; ++pl) {
+          const uint32_t* r = rb[p] + kt * 8 + pl * lo;
+          B[u][p][pl][0] = r[0];
+          B[u][p][pl][1] = r[4];
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < G; ++u) {
+      if (i0 + u < mine) {
+#pragma unroll
+        for (int p = 0; p < NPASS; ++p)
+#pragma unroll
+          for (int pl = 0; pl < PLANES; ++pl) mma_bf16(acc[p], A[u], B[u][p][pl][0], B[u][p][pl][1]);
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------- the streaming kernel
 struct __align__(16) ItemCtx {  // producer-side view of one claimed item
   int seg, item_in_seg;
@@ -424,234 +507,462 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* red = reinterpret_cast<float*>(smem + (size_t)NSLOT * SLOT_BYTES);
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)NSLOT * SLOT_BYTES + (size_t)RED_FLOATS * 4);
+  unsigned char* descs = reinterpret_cast<unsigned char*>(red) + (size_t)NRED * RED_FLOATS * 4;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(descs + (size_t)DESC_DEPTH * DESC_BYTES);
   uint64_t* empty_bar = full_bar + NSLOT;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + NSLOT);
+  uint64_t* dq_full = empty_bar + NSLOT;
+  uint64_t* dq_empty = dq_full + DESC_DEPTH;
+  uint64_t* red_full = dq_empty + DESC_DEPTH;
+  uint64_t* red_empty = red_full + NRED;
+  int* cat_tab = reinterpret_cast<int*>(red_empty + NRED);             // 4 * MAX_CAT ints
+  int* red_info = cat_tab + 4 * MAX_CAT;                               // NRED x {e | tile0 << 8, q, T, 0}
+  volatile int* ctl = red_info + 4 * NRED;                             // [0] abort, [1] closed, [2] items produced
+  volatile int* abort_flag = ctl;
+  (void)launch_id;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int32_t* sy = P.sync;
   if (tid == 0) {
-    for (int s = 0; s < NSLOT; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], CONSUMER_WARPS);
-    }
-    *abort_flag = 0;
+    for (int s = 0; s < NSLOT; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], CONSUMER_WARPS); }
+    for (int s = 0; s < DESC_DEPTH; ++s) { mbar_init(&dq_full[s], 1); mbar_init(&dq_empty[s], 1); }
+    for (int s = 0; s < NRED; ++s) { mbar_init(&red_full[s], CONSUMER_WARPS); mbar_init(&red_empty[s], 1); }
+    ctl[0] = 0; ctl[1] = 0; ctl[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (tid < 4 * MAX_CAT) cat_tab[tid] = sy[SY_CAT + tid];
   __syncthreads();
 
   // item range of this launch: one category (staged) or everything (fused)
-  const int32_t* sy = P.sync;
-  const int item_begin = (cat >= 0) ? sy[SY_CAT + 4 * cat + 0] : 0;
-  const int item_end = (cat >= 0) ? sy[SY_CAT + 4 * (cat + 1) + 0] : sy[SY_NITEMS];
   const int ncat = sy[SY_NCAT];
+  const int item_begin = (cat >= 0) ? cat_tab[4 * cat] : 0;
+  const int item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
 
-  if (warp == CONSUMER_WARPS) {
-    // ================================================================ producer
-    const uint64_t pol = policy_evict_first();
-    int slot = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    int32_t* claim = P.sync + SY_CLAIM + launch_id;
-    while (ok) {
-      int item = 0;
-      if (lane == 0) item = item_begin + atomicAdd(claim, 1);
-      item = __shfl_sync(0xffffffffu, item, 0);
-      if (item >= item_end) break;
-      // category -> segment -> item within the segment
+  if (warp == WARP_PLAN) {
+    // ================================================================ planner warp
+    // Runs ahead of the copy issue.  Batches of CLAIM_BATCH consecutive items are dealt to the
+    // CTAs round-robin (batch b -> CTA b mod grid), so the records of later batches can be
+    // read ahead; the planner waits (bounded) until an item's inputs exist, resolves every
+    // source pointer and queues a ready-to-issue descriptor in shared memory.  All global
+    // memory latency of the bookkeeping is paid here, off the streaming path.
+    auto seg_of = [&](int item, int& it) -> const Seg* {
       int c = 0;
-      for (int q = 1; q < ncat; ++q)
-        if (item >= sy[SY_CAT + 4 * q + 0]) c = q;
-      const int ib = sy[SY_CAT + 4 * c + 0], sb = sy[SY_CAT + 4 * c + 1], ips = sy[SY_CAT + 4 * c + 2];
-      const Seg* sg = P.segs + sb + (item - ib) / ips;
-      const int it = (item - ib) % ips;
-      const int T = sg->T, q = sg->q, paired = sg->paired, nB = sg->nB, kc0 = sg->kc, C = sg->C;
-      const int tile0 = paired ? it : it * q;
-      const int q_eff = paired ? 2 : min(q, sg->n_tiles - tile0);
-      // lane a < q_eff moves tile a of the item
-      const __nv_bfloat16* wsrc = (lane == 0 || !paired) ? sg->w0 + (size_t)(tile0 + (lane == 0 ? 0 : 1)) * (C / 16) * 256
-                                                         : sg->w1 + (size_t)tile0 * (C / 16) * 256;
-      const float* in0 = sg->in0;
-      const float* in1 = sg->in1;
-      const int in_stride = sg->in_stride;
-      // activation rows handled by this lane (row s = lane, lane + 32, ... of nB*T rows)
-      // dependency: the inputs of this item must have been produced
-      if (check_deps && sg->dep_idx >= 0) {
-        const int32_t* dep = P.sync + SY_DEP + sg->dep_idx;
-        const int target = sg->dep_target;
-        unsigned spins = 0;
-        bool ready = false;
-        while (!ready) {
-          ready = __all_sync(0xffffffffu, ld_acquire(dep) >= target);
-          if (!ready) {
-            __nanosleep(64);
-            if (++spins > SPIN_LIMIT / 16) break;
+      for (int q2 = 1; q2 < ncat; ++q2)
+        if (item >= cat_tab[4 * q2]) c = q2;
+      const int ib = cat_tab[4 * c + 0], sb = cat_tab[4 * c + 1], ips = cat_tab[4 * c + 2];
+      it = (item - ib) % ips;
+      return P.segs + sb + (item - ib) / ips;
+    };
+    const int stride = (int)gridDim.x * CLAIM_BATCH;
+    int base_cur = item_begin + (int)blockIdx.x * CLAIM_BATCH;
+    const Seg* cur_sgp = nullptr;
+    int4 v = make_int4(0, 0, 0, 0);  // lane l < SEG_VEC holds bytes [16l, 16l+16) of the current record
+    int dep_val = 0;                 // counter value read ahead for the current record
+    bool dep_val_valid = false;
+    if (base_cur < item_end) {
+      int it0;
+      cur_sgp = seg_of(base_cur, it0);
+      if (lane < SEG_VEC) v = __ldg(reinterpret_cast<const int4*>(cur_sgp) + lane);
+    }
+    int dep_ok = -1;
+    int e = 0;
+    uint32_t eph = 0;
+    bool ok = true;
+    while (ok && base_cur < item_end) {
+      const int base_nxt = base_cur + stride;
+      // read ahead: record of the next batch's first segment
+      const Seg* nxt_sgp = nullptr;
+      int4 v_nxt = make_int4(0, 0, 0, 0);
+      if (base_nxt < item_end) {
+        int itn;
+        nxt_sgp = seg_of(base_nxt, itn);
+        if (nxt_sgp == cur_sgp) v_nxt = v;
+        else if (lane < SEG_VEC) v_nxt = __ldg(reinterpret_cast<const int4*>(nxt_sgp) + lane);
+      }
+      for (int bi = 0; bi < CLAIM_BATCH && ok; ++bi) {
+        const int item = base_cur + bi;
+        if (item >= item_end) break;
+        int it;
+        const Seg* sgp = seg_of(item, it);
+        if (sgp != cur_sgp) {  // a segment boundary inside the batch
+          if (lane < SEG_VEC) v = __ldg(reinterpret_cast<const int4*>(sgp) + lane);
+          cur_sgp = sgp;
+          dep_val_valid = false;
+        }
+        // dep_idx / dep_target are ints 15 and 16 of the record: lane 3 .w and lane 4 .x
+        const int dep_idx = __shfl_sync(0xffffffffu, v.w, 3);
+        const int dep_target = __shfl_sync(0xffffffffu, v.x, 4);
+        int fresh = 0;
+        if ((check_deps & 1) && dep_idx >= 0 && dep_idx != dep_ok) {
+          const int32_t* dep = P.sync + SY_DEP + dep_idx;
+          bool ready = dep_val_valid && __all_sync(0xffffffffu, dep_val >= dep_target);
+          unsigned spins = 0;
+          while (!ready) {
+            ready = __all_sync(0xffffffffu, ld_acquire(dep) >= dep_target);
+            if (!ready) {
+              __nanosleep(32);
+              if (++spins > SPIN_LIMIT / 16 || *abort_flag) break;
+            }
+          }
+          if (!ready) { ok = false; break; }
+          dep_ok = dep_idx;
+          fresh = 1;
+        }
+        if (!mbar_wait_warp(&dq_empty[e], eph ^ 1u, abort_flag, lane)) { ok = false; break; }
+        unsigned char* ent = descs + (size_t)e * DESC_BYTES;
+        if (lane < SEG_VEC) reinterpret_cast<int4*>(ent)[lane] = v;
+        __syncwarp();
+        const Seg* sg = reinterpret_cast<const Seg*>(ent);
+        const int T = sg->T, paired = sg->paired, nB = sg->nB, C = sg->C;
+        const int tile0 = paired ? it : it * sg->q;
+        const int q_eff = paired ? 2 : min(sg->q, sg->n_tiles - tile0);
+        const int nrows = sg->planes * nB * T;
+        if (lane == 31) {
+          int* tail = reinterpret_cast<int*>(ent + DESC_TAIL);
+          tail[0] = 0;      // kind: work
+          tail[1] = tile0;
+          tail[2] = fresh;  // inputs were acquired for this item: the issuer must fence the async proxy
+          tail[3] = q_eff;
+          tail[4] = nrows;
+        }
+        if (lane < 2) {  // weight stream of tile `lane` of the item
+          const __nv_bfloat16* wsrc = (lane == 0 || !paired) ? sg->w0 + (size_t)(tile0 + lane) * (C / 16) * 256
+                                                             : sg->w1 + (size_t)tile0 * (C / 16) * 256;
+          reinterpret_cast<const __nv_bfloat16**>(ent + DESC_WSRC)[lane] = wsrc;
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {  // activation rows, ordered [plane][input][token]
+          const int rr = lane + 32 * u;
+          if (rr < nrows) {
+            const int pn = rr / T, s = rr - pn * T;
+            const int pl = pn / nB, nb = pn - pl * nB;
+            const __nv_bfloat16* base = pl ? (nb ? sg->in1l : sg->in0l) : (nb ? sg->in1h : sg->in0h);
+            reinterpret_cast<const __nv_bfloat16**>(ent + DESC_ASRC)[rr] = base + (size_t)sg->rows16[s] * sg->in_stride;
           }
         }
-        if (!ready) {
-          if (lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
-          ok = false;
-          break;
-        }
-        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&dq_full[e]);
+        if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
       }
+      // rotate; read the next record's dependency counter ahead of time
+      base_cur = base_nxt;
+      if (nxt_sgp != cur_sgp) dep_val_valid = false;
+      cur_sgp = nxt_sgp;
+      v = v_nxt;
+      if ((check_deps & 1) && base_cur < item_end && !dep_val_valid) {
+        const int nd = __shfl_sync(0xffffffffu, v.w, 3);
+        if (nd >= 0 && nd != dep_ok) {
+          dep_val = ld_acquire(P.sync + SY_DEP + nd);
+          dep_val_valid = true;
+        }
+      }
+    }
+    if (!ok && lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
+    // end marker (also after an abort, so the downstream warps leave their loops)
+    mbar_wait_warp(&dq_empty[e], eph ^ 1u, abort_flag, lane);
+    if (lane == 0) {
+      reinterpret_cast<int*>(descs + (size_t)e * DESC_BYTES + DESC_TAIL)[0] = 1;
+      mbar_arrive(&dq_full[e]);
+    }
+    return;
+  }
+
+  if (warp == WARP_ISSUE) {
+    // ================================================================ copy-issue warp
+    // Touches no global memory except through the bulk copies it issues.
+    const uint64_t pol = policy_evict_first();
+    int slot = 0, e = 0;
+    uint32_t phase = 0, eph = 0;
+    bool ok = true;
+    long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    (void)tr;
+    const long long tp0 = TR_NOW();
+    (void)tp0;
+    while (ok) {
+      const long long tm0 = TR_NOW();
+      if (!mbar_wait_warp(&dq_full[e], eph, abort_flag, lane)) { ok = false; break; }
+      TR_ADD(TR_META, tm0);
+      const unsigned char* ent = descs + (size_t)e * DESC_BYTES;
+      const Seg* sg = reinterpret_cast<const Seg*>(ent);
+      const int* tail = reinterpret_cast<const int*>(ent + DESC_TAIL);
+      if (tail[0] != 0) break;
+      const long long td0 = TR_NOW();
+      if (tail[2]) fence_proxy_async();
+      const int tile0 = tail[1], q_eff = tail[3], nrows = tail[4];
+      const int T = sg->T, kc0 = sg->kc, C = sg->C;
+      const int hflags = (q_eff << 4) | (sg->planes << 8) | (sg->nB << 12);
+      const __nv_bfloat16* wsrc = (lane < 2) ? reinterpret_cast<const __nv_bfloat16* const*>(ent + DESC_WSRC)[lane] : nullptr;
+      const __nv_bfloat16* asrc[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u)
+        asrc[u] = (lane + 32 * u < nrows) ? reinterpret_cast<const __nv_bfloat16* const*>(ent + DESC_ASRC)[lane + 32 * u]
+                                          : nullptr;
+      TR_ADD(TR_DEP, td0);
       const int nchunks = (C + kc0 - 1) / kc0;
-      for (int ch = 0; ch < nchunks && ok; ++ch) {
+#ifdef DEAMOE_TRACE
+      tr[TR_ITEMS] += 1; tr[TR_CHUNKS] += nchunks;
+#endif
+      for (int ch = 0; ch < nchunks; ++ch) {
         const int k0 = ch * kc0;
         const int kc = min(kc0, C - k0);
-        bool free_slot = true;
-        if (lane == 0) free_slot = mbar_wait(&empty_bar[slot], phase ^ 1u, abort_flag);
-        free_slot = __shfl_sync(0xffffffffu, (int)free_slot, 0) != 0;
-        if (!free_slot) {
-          if (lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
-          ok = false;
-          break;
-        }
+        const long long te0 = TR_NOW();
+        if (!mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane)) { ok = false; break; }
+        TR_ADD(TR_EMPTY, te0);
+        const long long ti0 = TR_NOW();
         unsigned char* sbase = ring + (size_t)slot * SLOT_BYTES;
         const uint32_t wbytes = (uint32_t)kc * 32u;
         const int astride = kc + ACT_PAD;
         if (lane == 0) {
-          SlotHdr* h = reinterpret_cast<SlotHdr*>(sbase);
-          h->kind = 0; h->first = (ch == 0); h->last = (ch == nchunks - 1); h->kc = kc;
-          h->T = T; h->q = q_eff; h->paired = paired; h->nB = nB;
-          h->epi = sg->epi; h->use_lo = sg->use_lo; h->row0 = tile0 * 16; h->rows = sg->rows;
-          h->out_stride = sg->out_stride; h->out_row0 = sg->out_row0; h->npass = (T + 7) / 8;
-          h->out = sg->out;
-          h->done = (sg->done_idx >= 0) ? P.sync + SY_DEP + sg->done_idx : nullptr;
-          mbar_arrive_expect_tx(&full_bar[slot], (uint32_t)q_eff * wbytes + (uint32_t)(nB * T) * (uint32_t)kc * 4u);
+          *reinterpret_cast<int4*>(sbase) = make_int4(0, hflags | (ch == 0 ? 1 : 0) | (ch == nchunks - 1 ? 2 : 0),
+                                                      kc | (T << 16), e | (tile0 << 8));
+          mbar_arrive_expect_tx(&full_bar[slot], (uint32_t)q_eff * wbytes + (uint32_t)nrows * (uint32_t)kc * 2u);
         }
         __syncwarp();
-        if (lane < q_eff)
+        if (lane < q_eff) {
+#ifdef DEAMOE_TRACE
+          if ((check_deps >> 8) == 2)
+            bulk_g2s(sbase + SLOT_HDR + (size_t)lane * wbytes, wsrc + (size_t)(k0 / 16) * 256, wbytes, &full_bar[slot]);
+          else
+#endif
           bulk_g2s_hint(sbase + SLOT_HDR + (size_t)lane * wbytes, wsrc + (size_t)(k0 / 16) * 256, wbytes,
                         &full_bar[slot], pol);
+        }
         unsigned char* abase = sbase + SLOT_HDR + (size_t)q_eff * wbytes;
-        for (int rr = lane; rr < nB * T; rr += 32) {
-          const int nb = rr / T, s = rr - nb * T;
-          const int row = sg->in_rows ? sg->in_rows[s] : sg->in_row0 + s;
-          const float* src = (nb ? in1 : in0) + (size_t)row * in_stride + k0;
-          bulk_g2s(abase + (size_t)rr * astride * 4, src, (uint32_t)kc * 4u, &full_bar[slot]);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int rr = lane + 32 * u;
+          if (rr < nrows)
+            bulk_g2s(abase + (size_t)rr * astride * 2, asrc[u] + k0, (uint32_t)kc * 2u, &full_bar[slot]);
         }
         if (++slot == NSLOT) { slot = 0; phase ^= 1u; }
+        TR_ADD(TR_ISSUE, ti0);
+      }
+      if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
+    }
+    if (!ok && lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
+#ifdef DEAMOE_TRACE
+    tr[TR_PTOTAL] = clock64() - tp0;
+    if (lane == 0 && P.trace)
+      for (int i = 0; i < 8; ++i) P.trace[(size_t)blockIdx.x * TR_SLOTS + i] = tr[i];
+#endif
+    // end-of-work marker for the consumers
+    if (mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane) && lane == 0) {
+      *reinterpret_cast<int4*>(ring + (size_t)slot * SLOT_BYTES) = make_int4(1, 0, 0, 0);
+      mbar_arrive(&full_bar[slot]);
+    }
+    return;
+  }
+
+  if (warp == WARP_EPI) {
+    // ================================================================ epilogue warp
+    // Sums the consumers' partial accumulators of a finished item, applies the stage's epilogue,
+    // stores the outputs and publishes the completion: one gpu-scope fence covers every item
+    // finished since the previous fence.  The consumers never wait for any of this.
+    int n = 0;                    // items processed
+    int pend = 0;                 // completions not yet published
+    int32_t* pend_ptr[NRED];
+    int pend_cnt[NRED];
+    unsigned idle = 0;
+    while (true) {
+      const int rb = n % NRED;
+      const uint32_t par = (uint32_t)(n / NRED) & 1u;
+      bool have = mbar_try_wait(&red_full[rb], par);
+      if (!have) {
+        if (pend) {  // nothing ready: publish what is finished
+          __syncwarp();
+          if (lane == 0) {
+            __threadfence();
+#pragma unroll
+            for (int i = 0; i < NRED; ++i)
+              if (i < pend) atomicAdd(pend_ptr[i], pend_cnt[i]);
+          }
+          pend = 0;
+          continue;
+        }
+        if ((ctl[1] && n >= ctl[2]) || *abort_flag || ++idle > SPIN_LIMIT) break;
+        __nanosleep(32);
+        continue;
+      }
+      idle = 0;
+      const int info_w = red_info[4 * rb + 0], q = red_info[4 * rb + 1], T = red_info[4 * rb + 2];
+      const int e = info_w & 0xff, tile0 = info_w >> 8;
+      const Seg* sg = reinterpret_cast<const Seg*>(descs + (size_t)e * DESC_BYTES);
+      const int paired = sg->paired, epi = sg->epi, rows = sg->rows;
+      const int out_stride = sg->out_stride, out_row0 = sg->out_row0;
+      __nv_bfloat16* outh = sg->outh;
+      __nv_bfloat16* outl = sg->outl;
+      float* outf = sg->outf;
+      int32_t* done = (sg->done_idx >= 0) ? P.sync + SY_DEP + sg->done_idx : nullptr;
+      const int npass = (T + 7) >> 3;
+      const float* rbuf = red + (size_t)rb * RED_FLOATS;
+      // warp w holds the partial sums of tile (q == 2 ? w / 4 : 0); element (p, reg, lane) of a tile
+      const int per_tile = npass * 128;
+      const int count = paired ? per_tile : q * per_tile;
+      for (int x = lane; x < count; x += 32) {
+        const int a = x / per_tile, rem = x - a * per_tile;
+        const int p = rem >> 7, reg = (rem >> 5) & 3, ln = rem & 31;
+        float v0 = 0.f, v1 = 0.f;
+        if (q == 2) {
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            v0 += rbuf[(size_t)(a * 4 + w) * (MAX_QP * 128) + rem];
+            if (paired) v1 += rbuf[(size_t)(4 + w) * (MAX_QP * 128) + rem];
+          }
+        } else {
+#pragma unroll
+          for (int w = 0; w < CONSUMER_WARPS; ++w) v0 += rbuf[(size_t)w * (MAX_QP * 128) + rem];
+        }
+        const int row = tile0 * 16 + a * 16 + (ln >> 2) + ((reg & 2) ? 8 : 0);
+        const int s = p * 8 + (ln & 3) * 2 + (reg & 1);
+        if (row < rows && s < T) {
+          float r;
+          if (epi == EPI_SIGMA) r = sigma_f(L.sigma, v0);
+          else if (epi == EPI_SWIGLU) r = silu_f(v0) * v1;
+          else r = v0;
+          const size_t o = (size_t)(out_row0 + s) * out_stride + row;
+          if (outf) {
+            outf[o] = r;
+          } else {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(r);
+            outh[o] = hi;
+            if (outl) outl[o] = __float2bfloat16_rn(r - __bfloat162float(hi));
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&red_empty[rb]);
+        mbar_arrive(&dq_empty[e]);  // the descriptor may be reused
+      }
+      if (done) {
+#pragma unroll
+        for (int i = 0; i < NRED; ++i)
+          if (i == pend) { pend_ptr[i] = done; pend_cnt[i] = paired ? 1 : q; }
+        ++pend;
+      }
+      ++n;
+      if (pend == NRED) {
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+#pragma unroll
+          for (int i = 0; i < NRED; ++i) atomicAdd(pend_ptr[i], pend_cnt[i]);
+        }
+        pend = 0;
       }
     }
-    // end-of-work marker (also sent after an abort so the consumers leave their loop)
-    {
-      bool free_slot = true;
-      if (lane == 0) free_slot = mbar_wait(&empty_bar[slot], phase ^ 1u, abort_flag);
-      if (lane == 0 && free_slot) {
-        SlotHdr* h = reinterpret_cast<SlotHdr*>(ring + (size_t)slot * SLOT_BYTES);
-        h->kind = 1;
-        mbar_arrive(&full_bar[slot]);
+    if (pend) {
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence();
+#pragma unroll
+        for (int i = 0; i < NRED; ++i)
+          if (i < pend) atomicAdd(pend_ptr[i], pend_cnt[i]);
       }
     }
     return;
   }
 
   // ================================================================ consumers
-  const int g = lane >> 2, tig = lane & 3;
-  float acc[2][4][4];
-  int slot = 0;
+  // Pure streaming role: wait for a chunk, multiply, release the slot.  On an item's last chunk
+  // the partial accumulators go to a reduction buffer for the epilogue warp (an mbarrier
+  // arrival, never a CTA barrier).
+  float acc[4][4];
+  int slot = 0, items = 0;
   uint32_t phase = 0;
+  long long tr[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  (void)tr;
+  const long long tc0 = TR_NOW();
+  (void)tc0;
   while (true) {
-    if (!mbar_wait(&full_bar[slot], phase, abort_flag)) {
+    const long long tf0 = TR_NOW();
+    if (!mbar_wait_warp(&full_bar[slot], phase, abort_flag, lane)) {
       if (lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
       break;
     }
+    TR_ADD(TR_FULL, tf0);
+    const long long tk0 = TR_NOW();
     const unsigned char* sbase = ring + (size_t)slot * SLOT_BYTES;
-    const SlotHdr hd = *reinterpret_cast<const SlotHdr*>(sbase);
-    if (hd.kind != 0) break;
-    if (hd.first) {
+    const int4 hw = *reinterpret_cast<const int4*>(sbase);
+    if (hw.x != 0) break;
+    const bool first = hw.y & 1, last = hw.y & 2;
+    const int q = (hw.y >> 4) & 15, planes = (hw.y >> 8) & 15, nB = (hw.y >> 12) & 15;
+    const int kc = hw.z & 0xffff, T = hw.z >> 16;
+    const int npass = (T + 7) >> 3;
+    if (first) {
 #pragma unroll
-      for (int a = 0; a < 2; ++a)
+      for (int p = 0; p < 4; ++p)
 #pragma unroll
-        for (int p = 0; p < 4; ++p)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[a][p][e] = 0.f;
+        for (int x = 0; x < 4; ++x) acc[p][x] = 0.f;
     }
-    const int kc = hd.kc, T = hd.T, q = hd.q, npass = hd.npass;
-    const int astride = kc + ACT_PAD;
-    const uint4* wt0 = reinterpret_cast<const uint4*>(sbase + SLOT_HDR);
-    const uint4* wt1 = reinterpret_cast<const uint4*>(sbase + SLOT_HDR + (size_t)kc * 32);
-    const float* act = reinterpret_cast<const float*>(sbase + SLOT_HDR + (size_t)q * kc * 32);
-    const int nkt = kc >> 4;
-    for (int kt = warp; kt < nkt; kt += CONSUMER_WARPS) {
-      const uint4 A0 = wt0[kt * 32 + lane];
-      uint4 A1 = make_uint4(0u, 0u, 0u, 0u);
-      if (q > 1) A1 = wt1[kt * 32 + lane];
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        if (p < npass) {
-          const int s = min(p * 8 + g, T - 1);
-          uint32_t bh[2][2], bl[2][2];
-#pragma unroll
-          for (int nb = 0; nb < 2; ++nb) {
-            if (nb < hd.nB) {
-              const float* xr = act + (size_t)(nb * T + s) * astride + kt * 16 + tig * 2;
-              const float2 x0 = *reinterpret_cast<const float2*>(xr);
-              const float2 x1 = *reinterpret_cast<const float2*>(xr + 8);
-              float r0, r1, r2, r3;
-              bh[nb][0] = pack_hi(x0.x, x0.y, r0, r1);
-              bh[nb][1] = pack_hi(x1.x, x1.y, r2, r3);
-              bl[nb][0] = pack_bf(r0, r1);
-              bl[nb][1] = pack_bf(r2, r3);
-            } else {
-              bh[nb][0] = bh[0][0]; bh[nb][1] = bh[0][1];
-              bl[nb][0] = bl[0][0]; bl[nb][1] = bl[0][1];
-            }
-          }
-          mma_bf16(acc[0][p], A0, bh[0][0], bh[0][1]);
-          if (hd.use_lo) mma_bf16(acc[0][p], A0, bl[0][0], bl[0][1]);
-          if (q > 1 && p < 2) {
-            mma_bf16(acc[1][p], A1, bh[1][0], bh[1][1]);
-            if (hd.use_lo) mma_bf16(acc[1][p], A1, bl[1][0], bl[1][1]);
-          }
-        }
+    TR_ADD(12, tk0);
+    const long long tl0 = TR_NOW();
+#ifdef DEAMOE_TRACE
+    tr[14] += kc >> 4;
+    if ((check_deps >> 8) != 1)
+#endif
+    {
+      // this warp's tile and its share of the k-tiles; one specialised loop per (passes, planes)
+      const int a = (q == 2) ? (warp >> 2) : 0;
+      const int kw = (q == 2) ? 4 : CONSUMER_WARPS;
+      const int ks = (q == 2) ? (warp & 3) : warp;
+      const int aw = (kc + ACT_PAD) >> 1;
+      const unsigned char* wtile = sbase + SLOT_HDR + (size_t)a * kc * 32;
+      const uint32_t* act = reinterpret_cast<const uint32_t*>(sbase + SLOT_HDR + (size_t)q * kc * 32) +
+                            (size_t)((nB == 2) ? a : 0) * T * aw;
+      const int lo = nB * T * aw;  // offset of the lo plane
+      const int np = npass <= 1 ? 1 : (npass == 2 ? 2 : 4);
+#define DEAMOE_CASE(NP, PL) \
+  case (NP * 4 + PL): consume_chunk<NP, PL>(acc, wtile, act, lo, kc, T, ks, kw, lane); break;
+      switch (np * 4 + planes) {
+        DEAMOE_CASE(1, 1) DEAMOE_CASE(2, 1) DEAMOE_CASE(4, 1)
+        DEAMOE_CASE(1, 2) DEAMOE_CASE(2, 2) DEAMOE_CASE(4, 2)
+        default: break;
       }
+#undef DEAMOE_CASE
     }
+    TR_ADD(13, tl0);
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty_bar[slot]);
     if (++slot == NSLOT) { slot = 0; phase ^= 1u; }
+    TR_ADD(TR_COMPUTE, tk0);
+    const long long tq0 = TR_NOW();
 
-    if (hd.last) {
-      // cross-warp reduction, epilogue, completion signal
-      float* mine = red + (size_t)warp * (MAX_QP * 128);
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int p = 0; p < 4; ++p)
-          if (a < q && p < npass && (a == 0 || p < 2)) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) mine[((a * npass + p) * 4 + e) * 32 + lane] = acc[a][p][e];
-          }
-      consumer_sync();
-      const int per_tile = npass * 128;
-      const int count = hd.paired ? per_tile : q * per_tile;
-      for (int e = tid; e < count; e += CONSUMER_THREADS) {
-        const int a = e / per_tile, rem = e - a * per_tile;
-        const int p = rem >> 7, reg = (rem >> 5) & 3, ln = rem & 31;
-        float v0 = 0.f, v1 = 0.f;
-#pragma unroll
-        for (int w = 0; w < CONSUMER_WARPS; ++w) {
-          v0 += red[(size_t)w * (MAX_QP * 128) + a * per_tile + rem];
-          if (hd.paired) v1 += red[(size_t)w * (MAX_QP * 128) + per_tile + rem];
-        }
-        const int row = hd.row0 + a * 16 + (ln >> 2) + ((reg & 2) ? 8 : 0);
-        const int s = p * 8 + (ln & 3) * 2 + (reg & 1);
-        if (row < hd.rows && s < T) {
-          float r;
-          if (hd.epi == EPI_SIGMA) r = sigma_f(L.sigma, v0);
-          else if (hd.epi == EPI_SWIGLU) r = silu_f(v0) * v1;
-          else r = v0;
-          hd.out[(size_t)(hd.out_row0 + s) * hd.out_stride + row] = r;
-        }
+    if (last) {
+      // hand the partial sums of this item to the epilogue warp
+      const int rb = items % NRED;
+      const uint32_t par = ((uint32_t)(items / NRED) & 1u) ^ 1u;
+      if (!mbar_wait_warp(&red_empty[rb], par, abort_flag, lane)) {
+        if (lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
+        break;
       }
-      __threadfence();
-      consumer_sync();
-      if (tid == 0 && hd.done) {
-        __threadfence();
-        atomicAdd(hd.done, 1);
+      float* mine = red + (size_t)rb * RED_FLOATS + (size_t)warp * (MAX_QP * 128);
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+        if (p < npass) {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) mine[(p * 4 + x) * 32 + lane] = acc[p][x];
+        }
+      if (tid == 0) {
+        red_info[4 * rb + 0] = hw.w;
+        red_info[4 * rb + 1] = q;
+        red_info[4 * rb + 2] = T;
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&red_full[rb]);
+      ++items;
+      TR_ADD(TR_EPI, tq0);
     }
   }
+  if (tid == 0) {
+    ctl[2] = items;
+    __threadfence_block();
+    ctl[1] = 1;
+  }
+#ifdef DEAMOE_TRACE
+  tr[TR_CTOTAL] = clock64() - tc0;
+  if (tid == 0 && P.trace)
+    for (int i = 8; i < 16; ++i) P.trace[(size_t)blockIdx.x * TR_SLOTS + i] = tr[i];
+#endif
 }
 
 // ---------------------------------------------------------------- host side
@@ -662,9 +973,9 @@ static void fill_stage(StageCfg& s, const __nv_bfloat16* w0, const __nv_bfloat16
   s.w0 = w0; s.w1 = w1; s.unit_elems = unit_elems; s.C = C; s.rows = rows;
   s.n_tiles = (rows + 15) / 16;
   s.paired = paired;
-  s.q = paired ? 2 : 1;
+  s.q = 2;                      // two 16-row tiles per item: (gate, up) of paired stages, else rows r, r+16
   s.epi = epi;
-  s.tg = 8 * (MAX_QP / s.q);
+  s.tg = 8 * MAX_QP;            // a warp accumulates up to MAX_QP passes of 8 tokens for its tile
   s.items_per_seg = paired ? s.n_tiles : (s.n_tiles + s.q - 1) / s.q;
   s.enabled = 1; s.pad = 0;
 }
@@ -762,10 +1073,32 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   const int MB = L.max_batch;
   d.max_segs = 8 + 2 * L.m + 2 * L.n + MB * L.k + 2 * MB;
   d.dep_s1 = 0; d.dep_s2 = L.m; d.dep_s3 = L.m + L.n; d.dep_sh1 = 2 * L.m + L.n; d.n_dep = 2 * L.m + L.n + 1;
+  d.planes = (L.adt == DEAMOE_F32) ? 2 : 1;
+  {
+    // activation planes between stages
+    const size_t tdmax = (size_t)MB * (L.k < L.m ? L.k : L.m), pmax = (size_t)MB * L.k;
+    struct { __nv_bfloat16** h; __nv_bfloat16** l; size_t elems; } bufs[] = {
+        {&d.xh, &d.xl, L.adt == DEAMOE_F32 ? (size_t)MB * L.h : 0},
+        {&d.GUh, &d.GUl, L.vanilla ? 0 : tdmax * 2 * L.f},
+        {&d.Yh, &d.Yl, pmax * (size_t)(L.vanilla ? L.f : L.rp)},
+        {&d.Zh, &d.Zl, L.vanilla ? 0 : pmax * (size_t)L.f},
+        {&d.Yshh, &d.Yshl, L.n_shared ? (size_t)MB * L.fs : 0},
+    };
+    for (auto& b : bufs) {
+      if (!b.elems) continue;
+      if (e == cudaSuccess) e = cudaMalloc(b.h, b.elems * 2);
+      if (e == cudaSuccess && d.planes > 1) e = cudaMalloc(b.l, b.elems * 2);
+      p->bytes += b.elems * 2 * d.planes;
+    }
+  }
   const size_t seg_bytes = (size_t)d.max_segs * sizeof(Seg);
   const size_t sync_bytes = (size_t)(SY_DEP + d.n_dep + 8) * sizeof(int32_t);
   if (e == cudaSuccess) e = cudaMalloc(&d.segs, seg_bytes);
   if (e == cudaSuccess) e = cudaMalloc(&d.sync, sync_bytes);
+#ifdef DEAMOE_TRACE
+  if (e == cudaSuccess) e = cudaMalloc(&d.trace, (size_t)p->n_sm * TR_SLOTS * sizeof(long long));
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.trace, 0, (size_t)p->n_sm * TR_SLOTS * sizeof(long long), s);
+#endif
   if (e == cudaSuccess) e = cudaMemsetAsync(d.sync, 0, sync_bytes, s);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)STREAM_SMEM);
@@ -785,6 +1118,11 @@ void stream_plan_destroy(StreamPlan* p) {
   if (p->packed) cudaFree(p->packed);
   if (p->dev.segs) cudaFree(p->dev.segs);
   if (p->dev.sync) cudaFree(p->dev.sync);
+  if (p->dev.trace) cudaFree(p->dev.trace);
+  __nv_bfloat16* planes[] = {p->dev.xh, p->dev.xl, p->dev.GUh, p->dev.GUl, p->dev.Yh, p->dev.Yl,
+                             p->dev.Zh, p->dev.Zl, p->dev.Yshh, p->dev.Yshl};
+  for (__nv_bfloat16* q : planes)
+    if (q) cudaFree(q);
   delete p;
 }
 
@@ -810,21 +1148,32 @@ static int host_categories(const LayerDev& L, int* stages) {
   return n;
 }
 
-__global__ void k_identity_private(LayerDev L);  // defined below
+__global__ void k_identity_private(LayerDev L, StreamDev P);  // defined below
+__global__ void k_split_tokens(const float* x, __nv_bfloat16* xh, __nv_bfloat16* xl, size_t count);
 
 int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
-  (void)B;
   int stages[MAX_CAT];
   const int ncat = host_categories(L, stages);
   int launches = 0;
+  if (L.adt == DEAMOE_F32) {
+    const size_t count = (size_t)B * L.h;
+    int blocks = (int)((count + 255) / 256);
+    if (blocks > 4 * p.n_sm) blocks = 4 * p.n_sm;
+    k_split_tokens<<<blocks, 256, 0, s>>>(L.x32, p.dev.xh, p.dev.xl, count);
+    ++launches;
+  }
   const bool fused = p.schedule == DEAMOE_SCHED_FUSED && (L.vanilla || L.r > 0);
   if (fused) {
-    k_stream<<<p.n_sm, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, MAX_CAT, -1, 1);
+    int dbgflag = 0;
+#ifdef DEAMOE_TRACE
+    if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
+#endif
+    k_stream<<<p.n_sm, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, MAX_CAT, -1, 1 | dbgflag);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
       if (stages[c] == ST_S4 && !L.vanilla && L.r == 0) {
-        k_identity_private<<<p.n_sm, 256, 0, s>>>(L);
+        k_identity_private<<<p.n_sm, 256, 0, s>>>(L, p.dev);
         ++launches;
       }
       k_stream<<<p.n_sm, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, c, c, 0);
@@ -835,14 +1184,45 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 }
 
 // priv == 0: A = identity, so Y = SiLU(G) * U and Z = sigma(Y) element by element.
-__global__ void k_identity_private(LayerDev L) {
+__global__ void k_identity_private(LayerDev L, StreamDev P) {
   const int pairs = L.counts[CNT_PAIRS];
   const size_t total = (size_t)pairs * L.f;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int pr = (int)(i / L.f), c = (int)(i % L.f);
-    const float* gu = L.GU + (size_t)L.pair_gurow[pr] * 2 * L.f;
-    L.Z[i] = sigma_f(L.sigma, silu_f(gu[c]) * gu[L.f + c]);
+    const size_t o = (size_t)L.pair_gurow[pr] * 2 * L.f + c;
+    float gv = __bfloat162float(P.GUh[o]), uv = __bfloat162float(P.GUh[o + L.f]);
+    if (P.planes > 1) {
+      gv += __bfloat162float(P.GUl[o]);
+      uv += __bfloat162float(P.GUl[o + L.f]);
+    }
+    const float z = sigma_f(L.sigma, silu_f(gv) * uv);
+    const __nv_bfloat16 hi = __float2bfloat16_rn(z);
+    P.Zh[i] = hi;
+    if (P.planes > 1) P.Zl[i] = __float2bfloat16_rn(z - __bfloat162float(hi));
+  }
+}
+
+// fp32 tokens -> bf16 hi + lo planes (x = hi + lo up to ~2^-17 relative)
+__global__ void k_split_tokens(const float* __restrict__ x, __nv_bfloat16* __restrict__ xh,
+                               __nv_bfloat16* __restrict__ xl, size_t count) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
+    const float v = x[i];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    xh[i] = hi;
+    xl[i] = __float2bfloat16_rn(v - __bfloat162float(hi));
   }
 }
 
 }  // namespace deamoe
+
+#ifdef DEAMOE_TRACE
+// Trace builds only: copy the per-CTA cycle counters of the last k_stream launch to the host.
+namespace deamoe {
+int stream_read_trace(StreamPlan& p, long long* host, int max_ctas) {
+  const int n = p.n_sm < max_ctas ? p.n_sm : max_ctas;
+  cudaDeviceSynchronize();
+  cudaMemcpy(host, p.dev.trace, (size_t)n * TR_SLOTS * sizeof(long long), cudaMemcpyDeviceToHost);
+  return n;
+}
+}  // namespace deamoe
+#endif

@@ -22,4 +22,9 @@ int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t 
 // Enqueue all stages of one step.  Returns the number of kernels launched or -1.
 int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
 
+#ifdef DEAMOE_TRACE
+// Trace builds only: per-CTA cycle counters of the last streaming launch.
+int stream_read_trace(StreamPlan& p, long long* host, int max_ctas);
+#endif
+
 }  // namespace deamoe

@@ -19,7 +19,7 @@ SMALL = synth.LayerShape("small", hidden=64, n_dept=3, experts_per_dept=4, ffn=4
 RAGGED = synth.LayerShape("ragged", hidden=208, n_dept=5, experts_per_dept=3, ffn=176, priv=80, top_k=4,
                           n_shared=1, shared_ffn=112)
 
-ALL_SCHEDULES = [binding.SCHED_PLAIN, binding.SCHED_STAGED]
+ALL_SCHEDULES = [binding.SCHED_PLAIN, binding.SCHED_STAGED, binding.SCHED_FUSED]
 
 
 def _scaled(shape, seed, scale=12.0, vanilla=False):
@@ -60,7 +60,7 @@ def test_vanilla_comparator(schedule):
 
 @pytest.mark.parametrize("schedule", ALL_SCHEDULES)
 @pytest.mark.parametrize("variant", ["no_private", "sigma_none", "gelu", "square_private", "g1", "k_eq_n",
-                                     "norm_all", "group_limited"])
+                                     "norm_all", "group_limited", "f32_tokens"])
 def test_variants(schedule, variant):
     shape = {
         "no_private": SMALL.with_(priv=0),
@@ -71,6 +71,7 @@ def test_variants(schedule, variant):
         "k_eq_n": SMALL.with_(n_dept=2, experts_per_dept=2, top_k=4),
         "norm_all": SMALL.with_(norm_topk=0, route_scale=2.5),
         "group_limited": SMALL.with_(n_dept=4, experts_per_dept=4, top_k=4, k_dept=2),
+        "f32_tokens": RAGGED.with_(act_dtype=0),
     }[variant]
     run_case(shape, 6, seed=4, schedule=schedule, weights=_scaled(shape, 4))
 
