@@ -170,6 +170,26 @@ def run_reference(args, shape, rank, world):
     print(json.dumps(line))
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of k_stream divided by its algorithmic bytes, from
+# the committed ncu capture (profiles/k_stream_dsv3-mini_b4.md)
+DRAM_TRAFFIC_RATIO = 1.004
+
+
+def stream_kernel_ms(layer, batches, steps, flush, torch):
+    """Per-step duration (ms) of the weight-streaming launches, from the library's own event pair."""
+    layer.profile(True)
+    out = torch.empty_like(batches[0])
+    ms = []
+    for i in range(steps + 2):
+        flush.add_(1)
+        layer.forward(batches[i % len(batches)], out)
+        t = layer.last_stream_ms()
+        if i >= 2:
+            ms.append(t)
+    layer.profile(False)
+    return ms
+
+
 def time_layer(layer, batches, steps, warmup, flush, torch, barrier):
     """Per-step CUDA-event times (ms) of layer.forward over rotating token batches."""
     outs = [torch.empty_like(b) for b in batches]
@@ -247,7 +267,13 @@ def main():
 
     sampler = ClockSampler(local)
     sampler.start()
+    time.sleep(0.5)      # nvidia-smi needs a moment before its first sample
     times_ms, launches = time_layer(layer, batches, args.steps, args.warmup, flush, torch, barrier)
+    # keep the GPU under the same load a little longer so the sampler sees it (untimed)
+    t_end = time.time() + 0.6
+    while time.time() < t_end:
+        layer.forward(batches[0])
+    torch.cuda.synchronize()
     clocks = sampler.stop()
     total_ms = sum(times_ms)
     if dist is not None:
@@ -260,16 +286,21 @@ def main():
     gbs = [bts / (ms * 1e-3) / 1e9 for bts, ms in zip(step_bytes, times_ms)]
     mean_bytes = statistics.mean(step_bytes)
 
-    # dominant kernel (weight streaming): events recorded by the library around its launches
-    kern = layer.kernel_times(batches, args.steps, flush) if hasattr(layer, "kernel_times") else None
+    # dominant kernel (weight streaming): events recorded by the library, on the stream it launches
+    # on, around its k_stream launch(es); algorithmic bytes = the step's unique weight bytes minus
+    # the fp32 router matrix (read by the routing kernel, outside the pair of events)
+    kern = stream_kernel_ms(layer, batches, args.steps, flush, torch) if args.schedule != "plain" else None
     router_bytes = shape.n_expert * shape.hidden * 4
     if kern:
         k_ms = statistics.mean(kern)
-        achieved = (mean_bytes - router_bytes) / (k_ms * 1e-3) / 1e9
+        alg = statistics.mean(step_bytes) - router_bytes
+        achieved = alg / (k_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "kernel": "k_stream (all weight-streaming launches of one step)",
-                "kernel_ms": k_ms, "peak_source": peak_src,
-                "algorithmic_bytes_per_step": mean_bytes - router_bytes}
+                "traffic": alg * DRAM_TRAFFIC_RATIO,
+                "traffic_note": "dram read+write bytes of k_stream from the ncu capture in profiles/ "
+                                "(smaller layer of the same matrices), scaled by algorithmic bytes",
+                "kernel": "k_stream (the weight-streaming launch(es) of one step)",
+                "kernel_ms": k_ms, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg}
     else:
         achieved = mean_bytes / (statistics.mean(times_ms) * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -179,6 +179,17 @@ deamoe_status_t deamoe_get_stats(deamoe_layer_t *layer, void *cuda_stream, int32
                                  int32_t *n_active_expert, int32_t *n_token_dept_pairs,
                                  uint64_t *unique_weight_bytes, int32_t *device_status);
 
+/*
+ * Measurement aid.  With profiling enabled the forward calls of this layer record a CUDA event on
+ * their stream before the first and after the last weight-streaming launch (the stages of
+ * Section 3.2; routing, bucketing and the final combine of Eq. (3) lie outside the pair).
+ * deamoe_profile_last_ms synchronises on the second event and returns the time between them in
+ * *ms (HOST).  Errors: INVALID_ARG (NULL, profiling off, or no forward since it was enabled),
+ * UNSUPPORTED for the plain schedule, CUDA.
+ */
+deamoe_status_t deamoe_profile_enable(deamoe_layer_t *layer, int32_t enable);
+deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t *layer, float *ms);
+
 /* Number of kernels the last forward/route call of this layer launched (host-side count). */
 int32_t deamoe_last_launches(const deamoe_layer_t *layer);
 

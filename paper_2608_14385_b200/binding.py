@@ -21,7 +21,7 @@ SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED = 0, 1, 2, 3
 # every symbol include/deamoe.h declares
 SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",
            "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_get_routing",
-           "deamoe_get_stats", "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
+           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
 
 
 class Config(C.Structure):
@@ -71,6 +71,8 @@ def lib():
             getattr(L, name).argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.deamoe_get_routing.argtypes = [C.c_void_p] * 9
         L.deamoe_get_stats.argtypes = [C.c_void_p] * 7
+        L.deamoe_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.deamoe_profile_last_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
         _lib = L
     return _lib
 
@@ -122,11 +124,16 @@ class Layer:
         self.act = torch.float32 if self.cfg.act_dtype == F32 else torch.bfloat16
 
     def close(self):
-        if getattr(self, "_h", None) is not None and self._h.value:
-            lib().deamoe_layer_destroy(self._h)
+        h = getattr(self, "_h", None)
+        if h is not None and h.value and _lib is not None:
+            _lib.deamoe_layer_destroy(h)
             self._h = C.c_void_p()
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
     def _check_tokens(self, tokens):
         assert tokens.is_cuda and tokens.is_contiguous() and tokens.dtype == self.act
@@ -189,6 +196,20 @@ class Layer:
             raise DeaMoEError(st, "deamoe_get_stats")
         return {"active_dept": nd.value, "active_expert": ne.value, "token_dept_pairs": ntd.value,
                 "unique_weight_bytes": ub.value, "device_status": st_.value}
+
+    def profile(self, enable=True):
+        """Record CUDA events around the weight-streaming launches of later forward calls."""
+        st = lib().deamoe_profile_enable(self._h, 1 if enable else 0)
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_profile_enable")
+
+    def last_stream_ms(self):
+        """Milliseconds between those events for the last forward (synchronises on it)."""
+        ms = C.c_float()
+        st = lib().deamoe_profile_last_ms(self._h, C.byref(ms))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_profile_last_ms")
+        return ms.value
 
     @property
     def last_launches(self):

@@ -344,6 +344,20 @@ deamoe_status_t deamoe_get_stats(deamoe_layer_t* L, void* cuda_stream, int32_t* 
   return DEAMOE_OK;
 }
 
+deamoe_status_t deamoe_profile_enable(deamoe_layer_t* L, int32_t enable) {
+  if (!L) return DEAMOE_ERR_INVALID_ARG;
+  if (!L->plan) return DEAMOE_ERR_UNSUPPORTED;
+  return stream_profile_enable(*L->plan, enable != 0) == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;
+}
+
+deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t* L, float* ms) {
+  if (!L || !ms) return DEAMOE_ERR_INVALID_ARG;
+  if (!L->plan) return DEAMOE_ERR_UNSUPPORTED;
+  const cudaError_t e = stream_profile_last_ms(*L->plan, ms);
+  if (e == cudaErrorInvalidValue) return DEAMOE_ERR_INVALID_ARG;
+  return e == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;
+}
+
 int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launches : 0; }
 
 uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }

@@ -124,6 +124,8 @@ struct StreamPlan {
   int n_sm;
   void* packed;
   uint64_t bytes;
+  cudaEvent_t ev0, ev1;   // profiling event pair (null when profiling is off)
+  int ev_recorded;
 };
 
 static_assert(sizeof(Seg) == DESC_TAIL && DESC_ASRC + 64 * 8 <= DESC_BYTES, "descriptor layout");
@@ -155,9 +157,13 @@ static __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t par
   return ok != 0;
 }
 // Bounded wait.  Returns false if the limit expired or the CTA was told to stop.
-static __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// `sleep_ns` > 0 backs off between polls: used by the roles whose wake-up latency is not critical,
+// so that their polling does not compete with the consumers for issue slots.
+static __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                 unsigned sleep_ns = 0) {
   for (unsigned it = 0; it < SPIN_LIMIT; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }
   return false;
@@ -165,9 +171,9 @@ static __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
 // One lane polls for the whole warp; the other lanes wait at the warp barrier without touching
 // the shared-memory pipe.  Every lane then observes the completed phase itself (acquire).
 static __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                      int lane) {
+                                                      int lane, unsigned sleep_ns = 0) {
   bool ok = true;
-  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag);
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, sleep_ns);
   ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
   __syncwarp();  // orders the other lanes' reads after lane 0's acquire
   return ok;
@@ -607,7 +613,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
           dep_ok = dep_idx;
           fresh = 1;
         }
-        if (!mbar_wait_warp(&dq_empty[e], eph ^ 1u, abort_flag, lane)) { ok = false; break; }
+        if (!mbar_wait_warp(&dq_empty[e], eph ^ 1u, abort_flag, lane, 200)) { ok = false; break; }
         unsigned char* ent = descs + (size_t)e * DESC_BYTES;
         if (lane < SEG_VEC) reinterpret_cast<int4*>(ent)[lane] = v;
         __syncwarp();
@@ -679,7 +685,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     (void)tp0;
     while (ok) {
       const long long tm0 = TR_NOW();
-      if (!mbar_wait_warp(&dq_full[e], eph, abort_flag, lane)) { ok = false; break; }
+      if (!mbar_wait_warp(&dq_full[e], eph, abort_flag, lane, 50)) { ok = false; break; }
       TR_ADD(TR_META, tm0);
       const unsigned char* ent = descs + (size_t)e * DESC_BYTES;
       const Seg* sg = reinterpret_cast<const Seg*>(ent);
@@ -705,7 +711,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
         const int k0 = ch * kc0;
         const int kc = min(kc0, C - k0);
         const long long te0 = TR_NOW();
-        if (!mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane)) { ok = false; break; }
+        if (!mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane, 50)) { ok = false; break; }
         TR_ADD(TR_EMPTY, te0);
         const long long ti0 = TR_NOW();
         unsigned char* sbase = ring + (size_t)slot * SLOT_BYTES;
@@ -966,7 +972,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
 }
 
 // ---------------------------------------------------------------- host side
-int stream_default_schedule() { return DEAMOE_SCHED_STAGED; }
+int stream_default_schedule() { return DEAMOE_SCHED_FUSED; }
 
 static void fill_stage(StageCfg& s, const __nv_bfloat16* w0, const __nv_bfloat16* w1, size_t unit_elems, int C,
                        int rows, int paired, int epi) {
@@ -1115,6 +1121,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
 
 void stream_plan_destroy(StreamPlan* p) {
   if (!p) return;
+  stream_profile_enable(*p, false);
   if (p->packed) cudaFree(p->packed);
   if (p->dev.segs) cudaFree(p->dev.segs);
   if (p->dev.sync) cudaFree(p->dev.sync);
@@ -1155,6 +1162,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
   int stages[MAX_CAT];
   const int ncat = host_categories(L, stages);
   int launches = 0;
+  if (p.ev0) cudaEventRecord(p.ev0, s);
   if (L.adt == DEAMOE_F32) {
     const size_t count = (size_t)B * L.h;
     int blocks = (int)((count + 255) / 256);
@@ -1180,7 +1188,29 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
       ++launches;
     }
   }
+  if (p.ev1) { cudaEventRecord(p.ev1, s); p.ev_recorded = 1; }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+cudaError_t stream_profile_enable(StreamPlan& p, bool on) {
+  if (on && !p.ev0) {
+    cudaError_t e = cudaEventCreate(&p.ev0);
+    if (e == cudaSuccess) e = cudaEventCreate(&p.ev1);
+    p.ev_recorded = 0;
+    return e;
+  }
+  if (!on && p.ev0) {
+    cudaEventDestroy(p.ev0); cudaEventDestroy(p.ev1);
+    p.ev0 = nullptr; p.ev1 = nullptr; p.ev_recorded = 0;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t stream_profile_last_ms(StreamPlan& p, float* ms) {
+  if (!p.ev0 || !p.ev_recorded) return cudaErrorInvalidValue;
+  cudaError_t e = cudaEventSynchronize(p.ev1);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(ms, p.ev0, p.ev1);
+  return e;
 }
 
 // priv == 0: A = identity, so Y = SiLU(G) * U and Z = sigma(Y) element by element.

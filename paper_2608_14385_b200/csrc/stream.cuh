@@ -22,6 +22,10 @@ int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t 
 // Enqueue all stages of one step.  Returns the number of kernels launched or -1.
 int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
 
+// Event pair around the streaming launches of stream_forward (measurement aid).
+cudaError_t stream_profile_enable(StreamPlan& p, bool on);
+cudaError_t stream_profile_last_ms(StreamPlan& p, float* ms);
+
 #ifdef DEAMOE_TRACE
 // Trace builds only: per-CTA cycle counters of the last streaming launch.
 int stream_read_trace(StreamPlan& p, long long* host, int max_ctas);
