@@ -94,6 +94,21 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value, dist=None, device=None):
+    """The slowest rank's value (all ranks get it); identity without a process group."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def us_per_layer_step(total_ms_max, steps, world):
+    """Whole-job figure: every rank ran `steps` layer-steps of its own replica in total_ms_max."""
+    return total_ms_max * 1e3 / (steps * world)
+
+
 def pct(xs, q):
     xs = sorted(xs)
     return xs[min(len(xs) - 1, max(0, int(round(q * (len(xs) - 1)))))]
@@ -275,13 +290,9 @@ def main():
         layer.forward(batches[0])
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    total_ms = sum(times_ms)
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(sum(times_ms), dist, dev)
     # aggregate: layer-steps processed by all ranks per unit time -> us per layer-step
-    us_per_step = total_ms * 1e3 / (args.steps * world)
+    us_per_step = us_per_layer_step(total_ms, args.steps, world)
     step_bytes = [ubytes[i % NB] for i in range(args.steps)]
     gbs = [bts / (ms * 1e-3) / 1e9 for bts, ms in zip(step_bytes, times_ms)]
     mean_bytes = statistics.mean(step_bytes)
@@ -320,11 +331,7 @@ def main():
         layer.forward_host(host_in[i % NB], host_out)
         e2e_t.append(time.perf_counter() - t0)
     io_bytes = B * shape.hidden * (2 if shape.act_dtype else 4)
-    e2e_us = statistics.mean(e2e_t) * 1e6
-    if dist is not None:
-        t = torch.tensor([e2e_us], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_us = float(t.item()) / world
+    e2e_us = max_over_ranks(statistics.mean(e2e_t) * 1e6, dist, dev) / world
 
     line = {
         "metric": "us_per_step_deamoe_layer", "value": us_per_step, "unit": "us", "n_gpus": world,

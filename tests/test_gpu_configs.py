@@ -1,0 +1,76 @@
+"""GPU parity for the benchmark's structured workloads: routing-locality sweep (configuration 4) and a
+stack of consecutive layers with a residual add (configuration 5)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import accounting, ref
+from paper_2608_14385_b200 import binding, synth
+from tests.common import oracle_cfg, within_tolerance
+from tests.gpu_common import check_routing, lazy_oracle_weights, run_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("c", [1, 2, 4])
+def test_locality_sweep_planted_routing(c):
+    """Tokens whose top-k picks are planted in exactly c departments (through the real router): the
+    oracle must confirm the planted selection, the GPU routing must match it bit for bit, the unique
+    weight bytes must equal the closed form on the counted sets, and outputs must be in tolerance."""
+    shape = synth.DSV3_MINI
+    dev = torch.device("cuda:0")
+    B = 8
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    tokens, chosen = synth.plant_locality(shape, w["router"], synth.make_tokens(shape, B, 1, dev), c, seed=c)
+    want = ref.route(oracle_cfg(shape), synth.to_numpy(w["router"]), synth.to_numpy(tokens))
+    for t in range(B):
+        assert sorted(int(i) for i in want["idx"][t]) == chosen[t]
+        assert len({i // shape.experts_per_dept for i in chosen[t]}) == c
+    res = run_case(shape, B, weights=w, tokens=tokens, rows=[0, B - 1], max_batch=8)
+    nd, ne, _ = accounting.count_active(chosen, shape.experts_per_dept)
+    assert res["stats"]["active_dept"] == nd and res["stats"]["active_expert"] == ne
+    assert res["stats"]["unique_weight_bytes"] == accounting.unique_bytes_deamoe(
+        nd, ne, shape.hidden, shape.ffn, shape.priv, shape.n_expert, 2, shape.n_shared, shape.shared_ffn)
+
+
+@pytest.mark.parametrize("B", [1, 8])
+def test_stack_of_layers_teacher_forced_and_free_running(B):
+    """x_{l+1} = x_l + Layer_l(x_l), every layer with its own seeded weights.  Teacher forced: GPU layer l
+    is fed the oracle's x_l (rounded to the activation dtype) and must match routing bit-exactly and
+    the output in tolerance.  Free running: the GPU feeds its own outputs forward; the final rows are
+    compared only for tokens whose routing agreed in every layer."""
+    n_layers = 8
+    shape = synth.MOE7B.with_(residual=1)
+    dev = torch.device("cuda:0")
+    cfg = oracle_cfg(shape)
+    layers, hostw = [], []
+    for l in range(n_layers):
+        w = synth.make_deamoe_weights(shape, 0, dev, layer=l)
+        layers.append(binding.Layer(shape, w, 8))
+        hostw.append({k: synth.to_numpy(v) for k, v in w.items()})
+        del w
+    try:
+        x_forced = synth.make_tokens(shape, B, 3, dev)
+        x_free = x_forced.clone()
+        agree = np.ones(B, bool)
+        for l in range(n_layers):
+            want = ref.deamoe_forward(cfg, hostw[l], synth.to_numpy(x_forced))
+            got = layers[l].forward(x_forced)
+            torch.cuda.synchronize()
+            r = layers[l].routing(B)
+            assert (r["idx"] == want["idx"]).all(), f"layer {l}"
+            ok, err, bound = within_tolerance(got.float().cpu().numpy(), want["out"])
+            assert ok, (l, err, bound)
+            free_out = layers[l].forward(x_free)
+            torch.cuda.synchronize()
+            agree &= (layers[l].routing(B)["idx"] == want["idx"]).all(axis=1)
+            x_free = free_out
+            x_forced = torch.from_numpy(want["out"]).to(torch.bfloat16).to(dev)
+        assert agree.any()
+        a = x_free.float().cpu().numpy()[agree]
+        b = x_forced.float().cpu().numpy()[agree]
+        ok, err, bound = within_tolerance(a, b, rel=3e-2, abs_=1e-2)   # rounding accumulates over the stack
+        assert ok, (err, bound, int(agree.sum()))
+    finally:
+        for layer in layers:
+            layer.close()
