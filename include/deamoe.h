@@ -190,6 +190,43 @@ deamoe_status_t deamoe_get_stats(deamoe_layer_t *layer, void *cuda_stream, int32
 deamoe_status_t deamoe_profile_enable(deamoe_layer_t *layer, int32_t enable);
 deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t *layer, float *ms);
 
+/*
+ * Routing for callers that must not allocate.  (The paper has no counterpart: this is an
+ * integration convenience of the library, not part of the method.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they need a routing
+ * decision: code that runs while a stream is being captured into a CUDA graph, a latency-critical
+ * serving loop in which an allocation would synchronise the whole device, or a plug-in that is
+ * handed a stream and pre-allocated buffers by a framework that owns all device memory.  A layer
+ * object (deamoe_layer_create) is out of reach for them because it allocates its workspace.  This
+ * entry point computes the same routing -- Eq. (2) top-k, ties to the lower index, and the gate
+ * weights of Eq. (3), flat top-k only -- without creating anything: the partial logits, the one
+ * piece of scratch the two routing kernels need, live in a fixed array of
+ * DEAMOE_STATIC_ROUTE_SCRATCH_BYTES inside the library image (every GPU that loads the library
+ * holds those bytes until the process exits).
+ *
+ *   router   DEVICE [n, hidden] fp32,  n = n_dept * experts_per_dept
+ *   tokens   DEVICE [B, hidden] fp32 (16-byte aligned)
+ *   topk_idx DEVICE [B, top_k] out, topk_w DEVICE [B, top_k] out (fp32)
+ *
+ * Limits: slices * B * n * 4 bytes must fit the fixed array, where slices (1..16) is the number of
+ * column slices the logits kernel uses for this n and hidden; a larger request returns
+ * DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout, n = 256, hidden = 7168: 4 slices,
+ * B up to 1024; n = 2048: B up to 128.)  Other errors as for deamoe_route.
+ *
+ * The first call on each device resolves the array's device address and sets one kernel
+ * attribute (the device must be current); make that first call before any stream capture begins.
+ * Later calls only enqueue two kernels on `cuda_stream`.  All calls share the one array and it
+ * keeps the previous call's contents: nothing has to be cleared, because every entry a call reads
+ * it has first written itself, but two calls that overlap on the GPU (different streams, or the
+ * same array used from two threads) race on it -- serialise them.
+ */
+#define DEAMOE_STATIC_ROUTE_SCRATCH_BYTES (4u << 20)
+deamoe_status_t deamoe_route_static(void *cuda_stream, const float *router, const float *tokens,
+                                    int32_t n_dept, int32_t experts_per_dept, int32_t hidden, int32_t top_k,
+                                    int32_t norm_topk, float route_scale, int32_t B, int32_t *topk_idx,
+                                    float *topk_w);
+
 /* Number of kernels the last forward/route call of this layer launched (host-side count). */
 int32_t deamoe_last_launches(const deamoe_layer_t *layer);
 

@@ -21,7 +21,7 @@ SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED = 0, 1, 2, 3
 # every symbol include/deamoe.h declares
 SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",
            "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_get_routing",
-           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
+           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_route_static", "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
 
 
 class Config(C.Structure):
@@ -71,6 +71,8 @@ def lib():
             getattr(L, name).argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.deamoe_get_routing.argtypes = [C.c_void_p] * 9
         L.deamoe_get_stats.argtypes = [C.c_void_p] * 7
+        L.deamoe_route_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
         L.deamoe_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.deamoe_profile_last_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
         _lib = L
@@ -95,6 +97,29 @@ def make_config(shape, max_batch, schedule=SCHED_AUTO):
                   d.get("k_dept", 0), d.get("n_shared", 0), d.get("shared_ffn", 0), d.get("sigma", 1),
                   d.get("norm_topk", 1), d.get("weight_dtype", 1), d.get("act_dtype", 1),
                   d.get("residual", 0), int(max_batch), int(schedule), float(d.get("route_scale", 1.0)))
+
+
+STATIC_ROUTE_SCRATCH_BYTES = 4 << 20
+
+
+def route_static(router, tokens, n_dept, experts_per_dept, top_k, norm_topk=1, route_scale=1.0, idx=None, w=None):
+    """Allocation-free routing (deamoe_route_static): for hosts that cannot create a layer object
+    because they may not allocate device memory (graph capture, latency-critical loops, plug-ins
+    working inside someone else's memory pool).  router [n, h] and tokens [B, h] are fp32 CUDA
+    tensors; idx [B, k] int32 and w [B, k] fp32 are caller-provided outputs (made here only when
+    omitted, for convenience in tests).  All calls share one fixed scratch array inside the library:
+    do not overlap two calls on the GPU."""
+    assert router.is_cuda and tokens.is_cuda and router.dtype == torch.float32 and tokens.dtype == torch.float32
+    B, h = tokens.shape
+    if idx is None:
+        idx = torch.empty((B, top_k), dtype=torch.int32, device=tokens.device)
+    if w is None:
+        w = torch.empty((B, top_k), dtype=torch.float32, device=tokens.device)
+    st = lib().deamoe_route_static(_stream(), _dptr(router), _dptr(tokens), n_dept, experts_per_dept, h, top_k,
+                                   norm_topk, float(route_scale), B, _dptr(idx), _dptr(w))
+    if st != OK:
+        raise DeaMoEError(st, "deamoe_route_static")
+    return idx, w
 
 
 class Layer:

@@ -1,5 +1,7 @@
 // Router (Eq. (2)), gate weights (Eq. (3)) and the department / expert token lists of
 // Section 3.2, all on the device with no host round trip.
+#include <cstring>
+
 #include "deamoe_internal.cuh"
 
 namespace deamoe {
@@ -324,3 +326,74 @@ int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, i
 }
 
 }  // namespace deamoe
+
+// ---------------------------------------------------------------- routing without any allocation
+// deamoe_route_static: the router logits + top-k pair for callers that may not allocate.  The
+// partial logits, which the layer object normally keeps in cudaMalloc'ed workspace, live in a
+// fixed array inside the library image instead.
+namespace {
+
+constexpr size_t STATIC_SCRATCH_FLOATS = DEAMOE_STATIC_ROUTE_SCRATCH_BYTES / sizeof(float);
+static __device__ __align__(256) float g_route_scratch[STATIC_SCRATCH_FLOATS];
+
+constexpr int MAX_DEVICES = 64;
+float* g_route_scratch_ptr[MAX_DEVICES];  // device address of the array, per device, after set-up
+bool g_route_ready[MAX_DEVICES];
+
+// Once per device, with that device current: resolve the array's device address (in host code the
+// symbol is only a handle) and let the top-k kernel use its full dynamic shared memory.
+deamoe_status_t static_route_setup(int dev) {
+  if (g_route_ready[dev]) return DEAMOE_OK;
+  float* p = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_route_scratch) != cudaSuccess || !p) {
+    cudaGetLastError();
+    return DEAMOE_ERR_CUDA;
+  }
+  if (cudaFuncSetAttribute(deamoe::k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess) {
+    cudaGetLastError();
+    return DEAMOE_ERR_CUDA;
+  }
+  g_route_scratch_ptr[dev] = p;
+  g_route_ready[dev] = true;
+  return DEAMOE_OK;
+}
+
+}  // namespace
+
+extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* router, const float* tokens,
+                                               int32_t n_dept, int32_t experts_per_dept, int32_t hidden,
+                                               int32_t top_k, int32_t norm_topk, float route_scale, int32_t B,
+                                               int32_t* topk_idx, float* topk_w) {
+  using namespace deamoe;
+  if (n_dept <= 0 || experts_per_dept <= 0 || hidden <= 0 || top_k <= 0 || B < 0) return DEAMOE_ERR_INVALID_ARG;
+  const long long n = (long long)n_dept * experts_per_dept;
+  if (top_k > n || !(route_scale == route_scale)) return DEAMOE_ERR_INVALID_ARG;
+  if (n > DEAMOE_MAX_EXPERTS || top_k > DEAMOE_MAX_TOPK || (hidden & 3)) return DEAMOE_ERR_UNSUPPORTED;
+  if (B == 0) return DEAMOE_OK;
+  if (!router || !tokens || !topk_idx || !topk_w) return DEAMOE_ERR_INVALID_ARG;
+  // column slices of the logits kernel, chosen as the layer object does
+  int kslices = 1;
+  while (kslices < 16 && ((n + 3) / 4) * kslices < 296 && hidden / (kslices * 2) >= 512) kslices *= 2;
+  const int kslice = (((hidden + kslices - 1) / kslices) + 3) & ~3;
+  const int ny = (hidden + kslice - 1) / kslice;
+  if ((size_t)ny * (size_t)B * (size_t)n > STATIC_SCRATCH_FLOATS) return DEAMOE_ERR_BATCH;  // beyond the fixed scratch
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+    cudaGetLastError();
+    return DEAMOE_ERR_CUDA;
+  }
+  const deamoe_status_t st = static_route_setup(dev);
+  if (st != DEAMOE_OK) return st;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  LayerDev L;
+  memset(&L, 0, sizeof(L));
+  L.h = hidden; L.m = n_dept; L.g = experts_per_dept; L.n = (int)n; L.k = top_k; L.k_dept = 0;
+  L.norm_topk = norm_topk; L.route_scale = route_scale;
+  L.logit_part = g_route_scratch_ptr[dev];   // every (slice, token, expert) entry used below is overwritten
+  L.topk_idx = topk_idx; L.topk_w = topk_w;  // results go straight to the caller's buffers
+  dim3 grid((L.n + RG - 1) / RG, ny);
+  k_router_logits<<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice);
+  const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
+  k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, ny, nullptr, nullptr);
+  return cudaGetLastError() == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;
+}
