@@ -211,8 +211,8 @@ deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t *layer, float *ms);
  *
  * Limits: slices * B * n * 4 bytes must fit the fixed array, where slices (1..16) is the number of
  * column slices the logits kernel uses for this n and hidden; a larger request returns
- * DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout, n = 256, hidden = 7168: 4 slices,
- * B up to 1024; n = 2048: B up to 128.)  Other errors as for deamoe_route.
+ * DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout, n = 256, hidden = 7168: 16 slices,
+ * B up to 256; hidden <= 512: 1 slice.)  Other errors as for deamoe_route.
  *
  * The first call on each device resolves the array's device address and sets one kernel
  * attribute (the device must be current); make that first call before any stream capture begins.

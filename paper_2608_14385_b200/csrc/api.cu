@@ -120,7 +120,7 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   const int pmax = MB * k;                     // (token, expert) pairs
   // router column slices: enough CTAs to cover the GPU a few times
   L->kslices = 1;
-  while (L->kslices < 16 && ((d.n + 3) / 4) * L->kslices < 296 && d.h / (L->kslices * 2) >= 512) L->kslices *= 2;
+  while (L->kslices < 16 && d.h / L->kslices > 512) L->kslices *= 2;  // one 512-column pass per thread block
 
   bool ok = true;
   auto A = [&](deamoe_status_t r) { if (r != DEAMOE_OK && ok) { ok = false; st = r; } };
@@ -233,13 +233,9 @@ deamoe_status_t deamoe_route(deamoe_layer_t* L, void* cuda_stream, const void* t
   if (B == 0) return DEAMOE_OK;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
   LayerDev d = call_view(L, tokens);
-  int nl = launch_route(d, tokens, B, s, L->kslices, topk_idx, topk_w);
+  const int nl = L->plan ? stream_route(*L->plan, d, tokens, B, s, L->kslices, topk_idx, topk_w)
+                         : launch_route(d, tokens, B, s, L->kslices, topk_idx, topk_w);
   if (nl < 0) return DEAMOE_ERR_CUDA;
-  if (L->plan) {
-    const int n2 = stream_build_worklist(*L->plan, d, B, s);
-    if (n2 < 0) return DEAMOE_ERR_CUDA;
-    nl += n2;
-  }
   L->last_launches = nl;
   return DEAMOE_OK;
 }
@@ -363,6 +359,11 @@ int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launc
 uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }
 
 #ifdef DEAMOE_TRACE
+int deamoe_debug_counts(deamoe_layer_t* L, int* host) {
+  cudaDeviceSynchronize();
+  cudaMemcpy(host, L->dev.counts, CNT_COUNT * sizeof(int), cudaMemcpyDeviceToHost);
+  return 0;
+}
 int deamoe_debug_trace(deamoe_layer_t* L, long long* host, int max_ctas) {
   return (L && L->plan) ? deamoe::stream_read_trace(*L->plan, host, max_ctas) : 0;
 }

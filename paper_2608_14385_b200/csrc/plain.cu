@@ -236,7 +236,9 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
     for (int q = 0; q < L.k; ++q)
       acc = fmaf(L.topk_w[t * L.k + q], L.O[(size_t)L.pair_slot[t * L.k + q] * L.h + c], acc);
     if (L.n_shared) acc += L.Osh[i];
-    if (L.residual) acc += x32[i];
+    if (L.residual)
+      acc += (L.adt == DEAMOE_F32) ? reinterpret_cast<const float*>(L.tokens_raw)[i]
+                                   : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw)[i]);
     if (L.adt == DEAMOE_F32) reinterpret_cast<float*>(out)[i] = acc;
     else reinterpret_cast<__nv_bfloat16*>(out)[i] = __float2bfloat16_rn(acc);
   }

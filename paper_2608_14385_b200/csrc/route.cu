@@ -3,6 +3,7 @@
 #include <cstring>
 
 #include "deamoe_internal.cuh"
+#include "route_device.cuh"
 
 namespace deamoe {
 
@@ -20,8 +21,18 @@ constexpr int RG = 4;   // router rows per CTA
 constexpr int TG = 8;   // tokens per register tile
 constexpr int ROUTER_THREADS = 128;
 
+static __device__ __forceinline__ float4 load_x4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+static __device__ __forceinline__ float4 load_x4(const __nv_bfloat16* p) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+  return make_float4(__bfloat162float(a.x), __bfloat162float(a.y), __bfloat162float(b.x), __bfloat162float(b.y));
+}
+
+// XT = float: tokens already fp32; XT = bf16: tokens widened on the fly (exact).
+template <typename XT>
 __global__ void __launch_bounds__(ROUTER_THREADS)
-k_router_logits(const float* __restrict__ Wr, const float* __restrict__ x32, float* __restrict__ part,
+k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float* __restrict__ part,
                 int n, int h, int B, int kslice) {
   const int row0 = blockIdx.x * RG;
   const int c0 = blockIdx.y * kslice;
@@ -44,7 +55,7 @@ k_router_logits(const float* __restrict__ Wr, const float* __restrict__ x32, flo
 #pragma unroll
       for (int b = 0; b < TG; ++b) {
         const int t = min(t0 + b, B - 1);
-        const float4 x = *reinterpret_cast<const float4*>(x32 + (size_t)t * h + c);
+        const float4 x = load_x4(x32 + (size_t)t * h + c);
 #pragma unroll
         for (int a = 0; a < RG; ++a) {
           acc[a][b] = fmaf(w[a].x, x.x, acc[a][b]);
@@ -76,218 +87,21 @@ k_router_logits(const float* __restrict__ Wr, const float* __restrict__ x32, flo
   }
 }
 
-// ---------------------------------------------------------------- top-k + gate weights
-// One warp per token.  Order: logit descending, ties to the lower expert index.
-constexpr int TOPK_WARPS = 4;
-
-static __device__ __forceinline__ bool better(float v, int i, float bv, int bi) {
-  return (v > bv) || (v == bv && i < bi);
-}
-
+// ---------------------------------------------------------------- top-k, gate weights, bucketing
 __global__ void __launch_bounds__(TOPK_WARPS * 32)
 k_topk(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   extern __shared__ float s_log[];  // [TOPK_WARPS][n] logits, then [TOPK_WARPS][n] bytes "dead"
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x * TOPK_WARPS + warp;
-  const int n = L.n, g = L.g, m = L.m, k = L.k;
-  float* lg = s_log + (size_t)warp * n;
-  unsigned char* dead = reinterpret_cast<unsigned char*>(s_log + (size_t)TOPK_WARPS * n) + (size_t)warp * n;
   if (t >= B) return;
-  float mx_all = -INFINITY;
-  for (int i = lane; i < n; i += 32) {
-    float v = 0.f;
-    for (int s = 0; s < kslices; ++s) v += L.logit_part[((size_t)s * B + t) * n + i];
-    lg[i] = v;
-    dead[i] = 0;
-    mx_all = fmaxf(mx_all, v);
-  }
-  __syncwarp();
-  if (L.k_dept > 0 && L.k_dept < m) {
-    // group limit: only the k_dept departments with the largest best logit stay eligible.
-    // A department is eliminated if at least k_dept departments rank ahead of it.
-    for (int j = lane; j < m; j += 32) {
-      float best = lg[(size_t)j * g];
-      for (int e = 1; e < g; ++e) best = fmaxf(best, lg[(size_t)j * g + e]);
-      int ahead = 0;
-      for (int j2 = 0; j2 < m; ++j2) {
-        float b2 = lg[(size_t)j2 * g];
-        for (int e = 1; e < g; ++e) b2 = fmaxf(b2, lg[(size_t)j2 * g + e]);
-        ahead += better(b2, j2, best, j) ? 1 : 0;
-      }
-      if (ahead >= L.k_dept)
-        for (int e = 0; e < g; ++e) dead[(size_t)j * g + e] = 1;
-    }
-    __syncwarp();
-  }
-  float den_all = 0.f;
-  if (!L.norm_topk) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx_all = fmaxf(mx_all, __shfl_xor_sync(0xffffffffu, mx_all, o));
-    for (int i = lane; i < n; i += 32) den_all += expf(lg[i] - mx_all);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) den_all += __shfl_xor_sync(0xffffffffu, den_all, o);
-  }
-  float my_v = 0.f;  // lane q keeps the q-th selected logit (k <= 32)
-  int my_i = 0;
-  for (int q = 0; q < k; ++q) {
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
-    for (int i = lane; i < n; i += 32)
-      if (!dead[i] && better(lg[i], i, bv, bi)) { bv = lg[i]; bi = i; }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
-    if (lane == q) { my_v = bv; my_i = bi; }
-    if (lane == 0 && bi < n) dead[bi] = 1;
-    __syncwarp();
-  }
-  // gate weights
-  const float top = __shfl_sync(0xffffffffu, my_v, 0);
-  float e, den;
-  if (L.norm_topk) {
-    e = (lane < k) ? expf(my_v - top) : 0.f;
-    den = e;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-  } else {
-    e = (lane < k) ? expf(my_v - mx_all) : 0.f;
-    den = den_all;
-  }
-  if (lane < k) {
-    const float p = L.route_scale * e / den;
-    L.topk_idx[(size_t)t * k + lane] = my_i;
-    L.topk_w[(size_t)t * k + lane] = p;
-    if (user_idx) user_idx[(size_t)t * k + lane] = my_i;
-    if (user_w) user_w[(size_t)t * k + lane] = p;
-  }
-}
-
-// ---------------------------------------------------------------- department bucketing
-// One CTA.  Token-membership bitmasks per department and per expert are built with shared
-// atomics, then counts, offsets (warp ballot/popc scans), ascending token lists, the pair
-// order (expert-major) and the (token, department) row of every pair.
-constexpr int BUCKET_THREADS = 512;
-
-static __device__ __forceinline__ int warp_exclusive_offsets(const int* cnt, int count, int32_t* off,
-                                                             int32_t* active, int lane, int* n_active) {
-  // exclusive prefix sum of cnt[0..count) into off[0..count], compaction of the non-empty
-  // indices into active[]; executed by one warp.
-  int run = 0, nact = 0;
-  for (int base = 0; base < count; base += 32) {
-    const int i = base + lane;
-    const int c = (i < count) ? cnt[i] : 0;
-    int incl = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
-    }
-    if (i < count) off[i] = run + incl - c;
-    const unsigned live = __ballot_sync(0xffffffffu, c > 0);
-    if (c > 0) active[nact + __popc(live & ((1u << lane) - 1u))] = i;
-    nact += __popc(live);
-    run += __shfl_sync(0xffffffffu, incl, 31);
-  }
-  if (lane == 0) { off[count] = run; *n_active = nact; }
-  return run;
+  topk_one_token(L, t, B, kslices, s_log + (size_t)warp * L.n,
+                 reinterpret_cast<unsigned char*>(s_log + (size_t)TOPK_WARPS * L.n) + (size_t)warp * L.n, lane, user_idx,
+                 user_w);
 }
 
 __global__ void __launch_bounds__(BUCKET_THREADS) k_bucket(LayerDev L, int B) {
-  extern __shared__ uint32_t s_u32[];
-  const int n = L.n, m = L.m, g = L.g, k = L.k;
-  const int W = (B + 31) / 32;
-  uint32_t* emask = s_u32;                    // [n][W]
-  uint32_t* dmask = emask + (size_t)n * W;    // [m][W]
-  int* ecnt = reinterpret_cast<int*>(dmask + (size_t)m * W);  // [n]
-  int* dcnt = ecnt + n;                                        // [m]
-  int* s_eoff = dcnt + m;                                      // [n+1]
-  int* s_doff = s_eoff + n + 1;                                // [m+1]
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int i = tid; i < (n + m) * W; i += BUCKET_THREADS) s_u32[i] = 0u;
-  __syncthreads();
-  for (int p = tid; p < B * k; p += BUCKET_THREADS) {
-    const int t = p / k;
-    const int i = L.topk_idx[p];
-    atomicOr(&emask[(size_t)i * W + (t >> 5)], 1u << (t & 31));
-    atomicOr(&dmask[(size_t)(i / g) * W + (t >> 5)], 1u << (t & 31));
-  }
-  __syncthreads();
-  for (int i = tid; i < n; i += BUCKET_THREADS) {
-    int c = 0;
-    for (int w = 0; w < W; ++w) c += __popc(emask[(size_t)i * W + w]);
-    ecnt[i] = c;
-  }
-  for (int j = tid; j < m; j += BUCKET_THREADS) {
-    int c = 0;
-    for (int w = 0; w < W; ++w) c += __popc(dmask[(size_t)j * W + w]);
-    dcnt[j] = c;
-  }
-  for (int w = tid; w < (m + 63) / 64; w += BUCKET_THREADS) {
-    uint64_t bits = 0;
-    for (int b = 0; b < 64 && w * 64 + b < m; ++b) {
-      bool any = false;
-      for (int q = 0; q < W; ++q) any |= dmask[(size_t)(w * 64 + b) * W + q] != 0u;
-      if (any) bits |= (uint64_t)1 << b;
-    }
-    L.dept_mask[w] = bits;
-  }
-  __syncthreads();
-  if (warp == 0) {
-    warp_exclusive_offsets(dcnt, m, s_doff, L.active_dept, lane, &L.counts[CNT_ACTIVE_DEPT]);
-  } else if (warp == 1) {
-    warp_exclusive_offsets(ecnt, n, s_eoff, L.active_expert, lane, &L.counts[CNT_ACTIVE_EXPERT]);
-  }
-  __syncthreads();
-  for (int i = tid; i <= n; i += BUCKET_THREADS) L.expert_off[i] = s_eoff[i];
-  for (int j = tid; j <= m; j += BUCKET_THREADS) L.dept_off[j] = s_doff[j];
-  if (tid == 0) {
-    L.counts[CNT_STATUS] = 0;
-    L.counts[CNT_TOKEN_DEPT] = s_doff[m];
-    L.counts[CNT_PAIRS] = s_eoff[n];
-  }
-  // ascending token lists
-  for (int i = tid; i < n; i += BUCKET_THREADS) {
-    int pos = s_eoff[i];
-    for (int w = 0; w < W; ++w) {
-      uint32_t bits = emask[(size_t)i * W + w];
-      while (bits) {
-        const int b = __ffs(bits) - 1;
-        bits &= bits - 1;
-        L.expert_tok[pos++] = w * 32 + b;
-      }
-    }
-  }
-  for (int j = tid; j < m; j += BUCKET_THREADS) {
-    int pos = s_doff[j];
-    for (int w = 0; w < W; ++w) {
-      uint32_t bits = dmask[(size_t)j * W + w];
-      while (bits) {
-        const int b = __ffs(bits) - 1;
-        bits &= bits - 1;
-        L.dept_tok[pos++] = w * 32 + b;
-      }
-    }
-  }
-  // pair order and the GU row of every pair
-  for (int p = tid; p < B * k; p += BUCKET_THREADS) {
-    const int t = p / k;
-    const int i = L.topk_idx[p];
-    const int j = i / g;
-    int re = 0, rd = 0;
-    for (int w = 0; w < (t >> 5); ++w) {
-      re += __popc(emask[(size_t)i * W + w]);
-      rd += __popc(dmask[(size_t)j * W + w]);
-    }
-    const uint32_t below = (1u << (t & 31)) - 1u;
-    re += __popc(emask[(size_t)i * W + (t >> 5)] & below);
-    rd += __popc(dmask[(size_t)j * W + (t >> 5)] & below);
-    const int slot = s_eoff[i] + re;
-    L.pair_slot[p] = slot;
-    L.pair_gurow[slot] = s_doff[j] + rd;
-  }
+  extern __shared__ uint32_t s_bucket[];
+  bucket_block(L, B, s_bucket, BUCKET_THREADS);
 }
 
 size_t bucket_smem_bytes(const LayerDev& L, int B) {
@@ -304,6 +118,20 @@ cudaError_t route_configure(const LayerDev& L) {
   return cudaFuncSetAttribute(k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
 }
 
+// Router logits straight from the caller's tokens (no fp32 copy): used by the streaming schedules.
+// Returns the number of column slices written (the second grid dimension), or -1.
+int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices) {
+  const int kslice = (((L.h + kslices - 1) / kslices) + 3) & ~3;
+  dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
+  if (L.adt == DEAMOE_BF16)
+    k_router_logits<__nv_bfloat16><<<grid, ROUTER_THREADS, 0, s>>>(L.router, reinterpret_cast<const __nv_bfloat16*>(tokens),
+                                                                  L.logit_part, L.n, L.h, B, kslice);
+  else
+    k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, reinterpret_cast<const float*>(tokens), L.logit_part,
+                                                          L.n, L.h, B, kslice);
+  return cudaGetLastError() == cudaSuccess ? (int)grid.y : -1;
+}
+
 int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices, int32_t* user_idx,
                  float* user_w) {
   int launches = 0;
@@ -315,7 +143,7 @@ int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, i
   }
   const int kslice = (((L.h + kslices - 1) / kslices) + 3) & ~3;
   dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
-  k_router_logits<<<grid, ROUTER_THREADS, 0, s>>>(L.router, L.x32, L.logit_part, L.n, L.h, B, kslice);
+  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, L.x32, L.logit_part, L.n, L.h, B, kslice);
   ++launches;
   const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
   k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, (int)grid.y, user_idx, user_w);
@@ -373,7 +201,7 @@ extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* r
   if (!router || !tokens || !topk_idx || !topk_w) return DEAMOE_ERR_INVALID_ARG;
   // column slices of the logits kernel, chosen as the layer object does
   int kslices = 1;
-  while (kslices < 16 && ((n + 3) / 4) * kslices < 296 && hidden / (kslices * 2) >= 512) kslices *= 2;
+  while (kslices < 16 && hidden / kslices > 512) kslices *= 2;
   const int kslice = (((hidden + kslices - 1) / kslices) + 3) & ~3;
   const int ny = (hidden + kslice - 1) / kslice;
   if ((size_t)ny * (size_t)B * (size_t)n > STATIC_SCRATCH_FLOATS) return DEAMOE_ERR_BATCH;  // beyond the fixed scratch
@@ -392,7 +220,7 @@ extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* r
   L.logit_part = g_route_scratch_ptr[dev];   // every (slice, token, expert) entry used below is overwritten
   L.topk_idx = topk_idx; L.topk_w = topk_w;  // results go straight to the caller's buffers
   dim3 grid((L.n + RG - 1) / RG, ny);
-  k_router_logits<<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice);
+  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice);
   const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
   k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, ny, nullptr, nullptr);
   return cudaGetLastError() == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;

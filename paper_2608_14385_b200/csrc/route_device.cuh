@@ -1,0 +1,301 @@
+// Device-side pieces of the routing step shared by the stand-alone kernels (route.cu) and the
+// fused routing kernel of the streaming schedules (stream.cu).
+#pragma once
+#include "deamoe_internal.cuh"
+
+namespace deamoe {
+
+// ---------------------------------------------------------------- top-k + gate weights
+// One warp per token.  Order: logit descending, ties to the lower expert index.
+constexpr int TOPK_WARPS = 4;
+
+static __device__ __forceinline__ bool better(float v, int i, float bv, int bi) {
+  return (v > bv) || (v == bv && i < bi);
+}
+
+// Top-k and gate weights of token t by one warp.  lg: n floats, dead: n bytes of shared memory.
+static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslices, float* lg, unsigned char* dead,
+                                      int lane, int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
+  const int n = L.n, g = L.g, m = L.m, k = L.k;
+  float mx_all = -INFINITY;
+  for (int i = lane; i < n; i += 32) {
+    float v = 0.f;
+    for (int s = 0; s < kslices; ++s) v += L.logit_part[((size_t)s * B + t) * n + i];
+    lg[i] = v;
+    dead[i] = 0;
+    mx_all = fmaxf(mx_all, v);
+  }
+  __syncwarp();
+  if (L.k_dept > 0 && L.k_dept < m) {
+    // group limit: only the k_dept departments with the largest best logit stay eligible.
+    // A department is eliminated if at least k_dept departments rank ahead of it.
+    for (int j = lane; j < m; j += 32) {
+      float best = lg[(size_t)j * g];
+      for (int e = 1; e < g; ++e) best = fmaxf(best, lg[(size_t)j * g + e]);
+      int ahead = 0;
+      for (int j2 = 0; j2 < m; ++j2) {
+        float b2 = lg[(size_t)j2 * g];
+        for (int e = 1; e < g; ++e) b2 = fmaxf(b2, lg[(size_t)j2 * g + e]);
+        ahead += better(b2, j2, best, j) ? 1 : 0;
+      }
+      if (ahead >= L.k_dept)
+        for (int e = 0; e < g; ++e) dead[(size_t)j * g + e] = 1;
+    }
+    __syncwarp();
+  }
+  float den_all = 0.f;
+  if (!L.norm_topk) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx_all = fmaxf(mx_all, __shfl_xor_sync(0xffffffffu, mx_all, o));
+    for (int i = lane; i < n; i += 32) den_all += expf(lg[i] - mx_all);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den_all += __shfl_xor_sync(0xffffffffu, den_all, o);
+  }
+  float my_v = 0.f;  // lane q keeps the q-th selected logit (k <= 32)
+  int my_i = 0;
+  for (int q = 0; q < k; ++q) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int i = lane; i < n; i += 32)
+      if (!dead[i] && better(lg[i], i, bv, bi)) { bv = lg[i]; bi = i; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == q) { my_v = bv; my_i = bi; }
+    if (lane == 0 && bi < n) dead[bi] = 1;
+    __syncwarp();
+  }
+  // gate weights
+  const float top = __shfl_sync(0xffffffffu, my_v, 0);
+  float e, den;
+  if (L.norm_topk) {
+    e = (lane < k) ? expf(my_v - top) : 0.f;
+    den = e;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+  } else {
+    e = (lane < k) ? expf(my_v - mx_all) : 0.f;
+    den = den_all;
+  }
+  if (lane < k) {
+    const float p = L.route_scale * e / den;
+    L.topk_idx[(size_t)t * k + lane] = my_i;
+    L.topk_w[(size_t)t * k + lane] = p;
+    if (user_idx) user_idx[(size_t)t * k + lane] = my_i;
+    if (user_w) user_w[(size_t)t * k + lane] = p;
+  }
+}
+
+
+// Same result with the logits held in registers (n <= 32 * VPL, flat top-k): every partial-logit
+// load is issued before the first use, and the k selection rounds touch no memory at all.
+template <int VPL, int KS>
+static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int lane,
+                                           int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
+  const int n = L.n, k = L.k;
+  float v[VPL];
+  unsigned taken = 0;
+  {
+    // all VPL * KS partial logits are loaded (clamped index, no branches) before the first add
+    float part[VPL][KS];
+    const float* __restrict__ src = L.logit_part + (size_t)t * n;
+    const size_t slice = (size_t)B * n;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j)
+#pragma unroll
+      for (int sl = 0; sl < KS; ++sl) part[j][sl] = __ldg(src + (size_t)sl * slice + min(lane + 32 * j, n - 1));
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      float sum = 0.f;
+#pragma unroll
+      for (int sl = 0; sl < KS; ++sl) sum += part[j][sl];  // fixed order: slice 0, 1, ...
+      if (lane + 32 * j >= n) { sum = -INFINITY; taken |= 1u << j; }
+      v[j] = sum;
+    }
+  }
+#ifdef DEAMOE_TRACE
+  float chk = 0.f;
+#pragma unroll
+  for (int j = 0; j < VPL; ++j) chk += v[j];
+  long long ta = clock64();
+  if (chk == 12345.678f) L.counts[15] = 1;
+#endif
+  float mx_all = -INFINITY, den_all = 0.f;
+  if (!L.norm_topk) {
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) mx_all = fmaxf(mx_all, v[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx_all = fmaxf(mx_all, __shfl_xor_sync(0xffffffffu, mx_all, o));
+#pragma unroll
+    for (int j = 0; j < VPL; ++j)
+      if (!((taken >> j) & 1u)) den_all += expf(v[j] - mx_all);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den_all += __shfl_xor_sync(0xffffffffu, den_all, o);
+  }
+  float my_v = 0.f;  // lane q keeps the q-th selected logit (k <= 32)
+  int my_i = 0;
+  for (int q = 0; q < k; ++q) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j)
+      if (!((taken >> j) & 1u) && better(v[j], lane + 32 * j, bv, bi)) { bv = v[j]; bi = lane + 32 * j; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == q) { my_v = bv; my_i = bi; }
+    if (bi < n && lane == (bi & 31)) taken |= 1u << (bi >> 5);
+  }
+#ifdef DEAMOE_TRACE
+  if (lane == 0 && t == 0) { L.counts[11] = (int)(clock64() - ta); L.counts[12] = (int)(ta & 0x7fffffff); }
+#endif
+  const float top = __shfl_sync(0xffffffffu, my_v, 0);
+  float e, den;
+  if (L.norm_topk) {
+    e = (lane < k) ? expf(my_v - top) : 0.f;
+    den = e;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+  } else {
+    e = (lane < k) ? expf(my_v - mx_all) : 0.f;
+    den = den_all;
+  }
+  if (lane < k) {
+    const float p = L.route_scale * e / den;
+    L.topk_idx[(size_t)t * k + lane] = my_i;
+    L.topk_w[(size_t)t * k + lane] = p;
+    if (user_idx) user_idx[(size_t)t * k + lane] = my_i;
+    if (user_w) user_w[(size_t)t * k + lane] = p;
+  }
+}
+
+// ---------------------------------------------------------------- department bucketing
+// One CTA.  Token-membership bitmasks per department and per expert are built with shared
+// atomics, then counts, offsets (warp ballot/popc scans), ascending token lists, the pair
+// order (expert-major) and the (token, department) row of every pair.
+constexpr int BUCKET_THREADS = 512;
+
+static __device__ __forceinline__ int warp_exclusive_offsets(const int* cnt, int count, int32_t* off,
+                                                             int32_t* active, int lane, int* n_active) {
+  // exclusive prefix sum of cnt[0..count) into off[0..count], compaction of the non-empty
+  // indices into active[]; executed by one warp.
+  int run = 0, nact = 0;
+  for (int base = 0; base < count; base += 32) {
+    const int i = base + lane;
+    const int c = (i < count) ? cnt[i] : 0;
+    int incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (i < count) off[i] = run + incl - c;
+    const unsigned live = __ballot_sync(0xffffffffu, c > 0);
+    if (c > 0) active[nact + __popc(live & ((1u << lane) - 1u))] = i;
+    nact += __popc(live);
+    run += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 0) { off[count] = run; *n_active = nact; }
+  return run;
+}
+
+// Body of the bucketing step for one CTA of `nthr` threads (a multiple of 64); s_u32: bucket_smem_bytes().
+static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, int nthr) {
+  const int n = L.n, m = L.m, g = L.g, k = L.k;
+  const int W = (B + 31) / 32;
+  uint32_t* emask = s_u32;                    // [n][W]
+  uint32_t* dmask = emask + (size_t)n * W;    // [m][W]
+  int* ecnt = reinterpret_cast<int*>(dmask + (size_t)m * W);  // [n]
+  int* dcnt = ecnt + n;                                        // [m]
+  int* s_eoff = dcnt + m;                                      // [n+1]
+  int* s_doff = s_eoff + n + 1;                                // [m+1]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int i = tid; i < (n + m) * W; i += nthr) s_u32[i] = 0u;
+  __syncthreads();
+  for (int p = tid; p < B * k; p += nthr) {
+    const int t = p / k;
+    const int i = L.topk_idx[p];
+    atomicOr(&emask[(size_t)i * W + (t >> 5)], 1u << (t & 31));
+    atomicOr(&dmask[(size_t)(i / g) * W + (t >> 5)], 1u << (t & 31));
+  }
+  __syncthreads();
+  for (int i = tid; i < n; i += nthr) {
+    int c = 0;
+    for (int w = 0; w < W; ++w) c += __popc(emask[(size_t)i * W + w]);
+    ecnt[i] = c;
+  }
+  // department counts; the active-department bitmask falls out of a warp ballot (32 departments
+  // per warp iteration, written as the two 32-bit halves of the 64-bit words)
+  for (int j = tid; j < ((m + 63) & ~63); j += nthr) {
+    int c = 0;
+    if (j < m) {
+      for (int w = 0; w < W; ++w) c += __popc(dmask[(size_t)j * W + w]);
+      dcnt[j] = c;
+    }
+    const unsigned live = __ballot_sync(0xffffffffu, c > 0);
+    if ((tid & 31) == 0) reinterpret_cast<uint32_t*>(L.dept_mask)[j >> 5] = live;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    warp_exclusive_offsets(dcnt, m, s_doff, L.active_dept, lane, &L.counts[CNT_ACTIVE_DEPT]);
+  } else if (warp == 1) {
+    warp_exclusive_offsets(ecnt, n, s_eoff, L.active_expert, lane, &L.counts[CNT_ACTIVE_EXPERT]);
+  }
+  __syncthreads();
+  for (int i = tid; i <= n; i += nthr) L.expert_off[i] = s_eoff[i];
+  for (int j = tid; j <= m; j += nthr) L.dept_off[j] = s_doff[j];
+  if (tid == 0) {
+    L.counts[CNT_STATUS] = 0;
+    L.counts[CNT_TOKEN_DEPT] = s_doff[m];
+    L.counts[CNT_PAIRS] = s_eoff[n];
+  }
+  // ascending token lists
+  for (int i = tid; i < n; i += nthr) {
+    int pos = s_eoff[i];
+    for (int w = 0; w < W; ++w) {
+      uint32_t bits = emask[(size_t)i * W + w];
+      while (bits) {
+        const int b = __ffs(bits) - 1;
+        bits &= bits - 1;
+        L.expert_tok[pos++] = w * 32 + b;
+      }
+    }
+  }
+  for (int j = tid; j < m; j += nthr) {
+    int pos = s_doff[j];
+    for (int w = 0; w < W; ++w) {
+      uint32_t bits = dmask[(size_t)j * W + w];
+      while (bits) {
+        const int b = __ffs(bits) - 1;
+        bits &= bits - 1;
+        L.dept_tok[pos++] = w * 32 + b;
+      }
+    }
+  }
+  // pair order and the GU row of every pair
+  for (int p = tid; p < B * k; p += nthr) {
+    const int t = p / k;
+    const int i = L.topk_idx[p];
+    const int j = i / g;
+    int re = 0, rd = 0;
+    for (int w = 0; w < (t >> 5); ++w) {
+      re += __popc(emask[(size_t)i * W + w]);
+      rd += __popc(dmask[(size_t)j * W + w]);
+    }
+    const uint32_t below = (1u << (t & 31)) - 1u;
+    re += __popc(emask[(size_t)i * W + (t >> 5)] & below);
+    rd += __popc(dmask[(size_t)j * W + (t >> 5)] & below);
+    const int slot = s_eoff[i] + re;
+    L.pair_slot[p] = slot;
+    L.pair_gurow[slot] = s_doff[j] + rd;
+  }
+}
+
+
+}  // namespace deamoe

@@ -21,6 +21,7 @@
 #include <cstring>
 #include <new>
 
+#include "route_device.cuh"
 #include "stream.cuh"
 
 namespace deamoe {
@@ -36,7 +37,7 @@ constexpr int DESC_BYTES = 1024;                 // Seg | tail | weight sources 
 constexpr int DESC_TAIL = 224, DESC_WSRC = 256, DESC_ASRC = 272;
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SIG_DEPTH = 16;
-constexpr int CLAIM_BATCH = 2;  // consecutive items claimed at once
+constexpr int CLAIM_BATCH = 1;  // consecutive items claimed at once
 constexpr int SLOT_BYTES = 30 * 1024;
 constexpr int SLOT_HDR = 128;
 constexpr int NSLOT = 6;
@@ -383,18 +384,19 @@ static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stag
   }
   if (!s.in0l) s.planes = 1;
   s.kc = chunk_k(s.C, s.q, s.planes * s.nB * s.T);
-  for (int t = 0; t < 32; ++t) s.rows16[t] = (uint16_t)(t < s.T ? (in_list ? in_list[t] : in_row0 + t) : 0);
+  for (int t = 0; t < s.T; ++t) s.rows16[t] = (uint16_t)(in_list ? in_list[t] : in_row0 + t);
   if (seg_index < P.max_segs) P.segs[seg_index] = s;
 }
 
 constexpr int BUILD_THREADS = 32 * MAX_CAT;
 
-__global__ void __launch_bounds__(BUILD_THREADS) k_build_worklist(LayerDev L, StreamDev P, int B) {
+// Body of the work-list construction for one CTA of at least BUILD_THREADS threads.
+static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B) {
   __shared__ int s_nseg[MAX_CAT], s_segbase[MAX_CAT + 1], s_itembase[MAX_CAT + 1];
   CatInfo cats[MAX_CAT];
   const int ncat = category_list(L, P, cats);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int i = threadIdx.x; i < P.n_dep + MAX_CAT + 8; i += BUILD_THREADS) P.sync[SY_CLAIM + i] = 0;
+  for (int i = threadIdx.x; i < P.n_dep + MAX_CAT + 8; i += blockDim.x) P.sync[SY_CLAIM + i] = 0;
   if (warp < ncat) {
     const int stage = cats[warp].stage, kind = cats[warp].unit_kind;
     const int U = unit_count(L, kind);
@@ -453,6 +455,110 @@ __global__ void __launch_bounds__(BUILD_THREADS) k_build_worklist(LayerDev L, St
       running += __shfl_sync(0xffffffffu, incl, 31);
     }
   }
+}
+
+__global__ void __launch_bounds__(BUILD_THREADS) k_build_worklist(LayerDev L, StreamDev P, int B) {
+  worklist_block(L, P, B);
+}
+
+// Routing tail in one CTA: top-k + gate weights (warp per token), bucketing, work list.  The
+// routing state (selection, gate weights, offsets, token lists, counters) is built in shared
+// memory -- the three steps read each other's results from there, not through L2 -- and copied
+// to the layer's global arrays at the end for the later kernels and for deamoe_get_routing.
+constexpr int FINISH_THREADS = 512;
+
+struct FinishSmem {  // element counts of the shared-memory copy of the routing state
+  int idx, w, dept_off, dept_tok, expert_off, expert_tok, pair_slot, pair_gurow, active_dept, active_expert, counts,
+      dept_mask, total;
+};
+static __host__ __device__ FinishSmem finish_layout(int n, int m, int k, int B) {
+  FinishSmem f;
+  const int pk = B * k, td = B * (k < m ? k : m);
+  int o = 0;
+  f.idx = o; o += pk; f.w = o; o += pk; f.dept_off = o; o += m + 1; f.dept_tok = o; o += td;
+  f.expert_off = o; o += n + 1; f.expert_tok = o; o += pk; f.pair_slot = o; o += pk; f.pair_gurow = o; o += pk;
+  f.active_dept = o; o += m; f.active_expert = o; o += n; f.counts = o; o += CNT_COUNT;
+  o = (o + 1) & ~1;
+  f.dept_mask = o; o += 2 * ((m + 63) / 64);
+  f.total = (o + 3) & ~3;
+  return f;
+}
+
+__global__ void __launch_bounds__(FINISH_THREADS)
+k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
+               int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
+  extern __shared__ uint32_t s_dyn[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
+  uint32_t* state = s_dyn + scratch_words;  // persistent part, after the scratch of top-k / bucketing
+  // a view of the layer whose routing arrays live in shared memory
+  LayerDev S = L;
+  S.topk_idx = reinterpret_cast<int32_t*>(state + fl.idx);
+  S.topk_w = reinterpret_cast<float*>(state + fl.w);
+  S.dept_off = reinterpret_cast<int32_t*>(state + fl.dept_off);
+  S.dept_tok = reinterpret_cast<int32_t*>(state + fl.dept_tok);
+  S.expert_off = reinterpret_cast<int32_t*>(state + fl.expert_off);
+  S.expert_tok = reinterpret_cast<int32_t*>(state + fl.expert_tok);
+  S.pair_slot = reinterpret_cast<int32_t*>(state + fl.pair_slot);
+  S.pair_gurow = reinterpret_cast<int32_t*>(state + fl.pair_gurow);
+  S.active_dept = reinterpret_cast<int32_t*>(state + fl.active_dept);
+  S.active_expert = reinterpret_cast<int32_t*>(state + fl.active_expert);
+  S.counts = reinterpret_cast<int32_t*>(state + fl.counts);
+  S.dept_mask = reinterpret_cast<uint64_t*>(state + fl.dept_mask);
+#ifdef DEAMOE_TRACE
+  long long tt0 = clock64();
+#endif
+  for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) S.counts[i] = 0;
+  const bool regs_ok = (L.k_dept <= 0 || L.k_dept >= L.m) && L.n <= 512 &&
+                       (kslices == 1 || kslices == 2 || kslices == 4 || kslices == 8 || kslices == 16);
+  if (warp < topk_warps) {
+    const int per_warp = (L.n * 5 + 15) & ~15;  // n fp32 logits + n flag bytes (memory path only)
+    unsigned char* base = reinterpret_cast<unsigned char*>(s_dyn) + (size_t)warp * per_warp;
+    for (int t = warp; t < B; t += topk_warps) {
+#define DEAMOE_TOPK(VPL, KS) topk_one_token_regs<VPL, KS>(S, t, B, lane, user_idx, user_w)
+      if (regs_ok && L.n <= 256) {
+        if (kslices == 16) DEAMOE_TOPK(8, 16); else if (kslices == 8) DEAMOE_TOPK(8, 8); else if (kslices == 4) DEAMOE_TOPK(8, 4);
+        else if (kslices == 2) DEAMOE_TOPK(8, 2); else DEAMOE_TOPK(8, 1);
+      } else if (regs_ok) {
+        if (kslices == 16) DEAMOE_TOPK(16, 16); else if (kslices == 8) DEAMOE_TOPK(16, 8); else if (kslices == 4) DEAMOE_TOPK(16, 4);
+        else if (kslices == 2) DEAMOE_TOPK(16, 2); else DEAMOE_TOPK(16, 1);
+      }
+#undef DEAMOE_TOPK
+      else topk_one_token(S, t, B, kslices, reinterpret_cast<float*>(base), base + (size_t)L.n * 4, lane, user_idx, user_w);
+    }
+  }
+  __syncthreads();
+#ifdef DEAMOE_TRACE
+  long long tt1 = clock64();
+#endif
+  bucket_block(S, B, s_dyn, FINISH_THREADS);
+  __syncthreads();
+#ifdef DEAMOE_TRACE
+  long long tt2 = clock64();
+#endif
+  worklist_block(S, P, B);
+  __syncthreads();
+  // publish the routing state
+  const int pk = B * L.k;
+  for (int i = tid; i < pk; i += FINISH_THREADS) {
+    L.topk_idx[i] = S.topk_idx[i]; L.topk_w[i] = S.topk_w[i];
+    L.expert_tok[i] = S.expert_tok[i]; L.pair_slot[i] = S.pair_slot[i]; L.pair_gurow[i] = S.pair_gurow[i];
+  }
+  const int ntd = S.counts[CNT_TOKEN_DEPT];
+  for (int i = tid; i < ntd; i += FINISH_THREADS) L.dept_tok[i] = S.dept_tok[i];
+  for (int i = tid; i <= L.m; i += FINISH_THREADS) L.dept_off[i] = S.dept_off[i];
+  for (int i = tid; i <= L.n; i += FINISH_THREADS) L.expert_off[i] = S.expert_off[i];
+  for (int i = tid; i < L.m; i += FINISH_THREADS) L.active_dept[i] = S.active_dept[i];
+  for (int i = tid; i < L.n; i += FINISH_THREADS) L.active_expert[i] = S.active_expert[i];
+  for (int i = tid; i < (L.m + 63) / 64; i += FINISH_THREADS) L.dept_mask[i] = S.dept_mask[i];
+  for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) L.counts[i] = S.counts[i];
+#ifdef DEAMOE_TRACE
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    L.counts[8] = (int)(tt1 - tt0); L.counts[9] = (int)(tt2 - tt1); L.counts[10] = (int)(clock64() - tt2);
+    L.counts[11] = S.counts[11]; L.counts[12] = (int)((S.counts[12] - (int)(tt0 & 0x7fffffff)));
+  }
+#endif
 }
 
 // ---------------------------------------------------------------- inner loop of the consumers
@@ -1108,6 +1214,8 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   if (e == cudaSuccess) e = cudaMemsetAsync(d.sync, 0, sync_bytes, s);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)STREAM_SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_route_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   p->bytes += seg_bytes + sync_bytes;
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -1131,6 +1239,26 @@ void stream_plan_destroy(StreamPlan* p) {
   for (__nv_bfloat16* q : planes)
     if (q) cudaFree(q);
   delete p;
+}
+
+int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
+                 int32_t* user_idx, float* user_w) {
+  const int ny = launch_router_logits(L, tokens, B, s, kslices);
+  if (ny < 0) return -1;
+  const int per_warp = (L.n * 5 + 15) & ~15;
+  int topk_warps = (48 * 1024) / per_warp;
+  if (topk_warps > FINISH_THREADS / 32) topk_warps = FINISH_THREADS / 32;
+  if (topk_warps > B) topk_warps = B;
+  if (topk_warps < 1) topk_warps = 1;
+  size_t scratch = (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
+  const size_t bs = bucket_smem_bytes(L, B);
+  if (bs > scratch) scratch = bs;
+  scratch = (scratch + 15) & ~(size_t)15;
+  const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
+  const size_t smem = scratch + (size_t)fl.total * 4;
+  if (smem > 200 * 1024) return -1;
+  k_route_finish<<<1, FINISH_THREADS, smem, s>>>(L, p.dev, B, ny, topk_warps, (int)(scratch / 4), user_idx, user_w);
+  return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {

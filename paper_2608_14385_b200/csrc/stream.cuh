@@ -15,6 +15,11 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
                                    StreamPlan** out, uint64_t* bytes);
 void stream_plan_destroy(StreamPlan* p);
 
+// Routing for the streaming schedules: router logits, then ONE kernel for top-k + gate weights,
+// bucketing and the work list.  Returns the number of kernels launched or -1.
+int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
+                 int32_t* user_idx, float* user_w);
+
 // Enqueue the work-list construction for the routing state already on the device.
 // Returns the number of kernels launched or -1.
 int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
