@@ -26,7 +26,7 @@
 
 namespace deamoe {
 
-constexpr int CONSUMER_WARPS = 8;
+constexpr int CONSUMER_WARPS = 16;
 constexpr int CONSUMER_THREADS = CONSUMER_WARPS * 32;
 constexpr int WARP_ISSUE = CONSUMER_WARPS;       // issues the bulk copies
 constexpr int WARP_PLAN = CONSUMER_WARPS + 1;    // picks items, fetches records, waits for inputs
@@ -42,7 +42,7 @@ constexpr int SLOT_BYTES = 30 * 1024;
 constexpr int SLOT_HDR = 128;
 constexpr int NSLOT = 6;
 constexpr int ACT_PAD = 8;   // floats of padding per activation row in shared memory
-constexpr int MAX_QP = 4;    // (tiles per item) x (8-token passes) held in accumulators
+constexpr int MAX_QP = 2;    // 8-token passes a consumer warp accumulates for its tile (16 tokens per segment)
 constexpr int RED_FLOATS = CONSUMER_WARPS * MAX_QP * 128;
 constexpr size_t STREAM_SMEM =
     (size_t)NSLOT * SLOT_BYTES + (size_t)NRED * RED_FLOATS * 4 + (size_t)DESC_DEPTH * DESC_BYTES + 1024;
@@ -569,10 +569,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
 // k-tiles are handled G at a time: every shared-memory load of the group is issued before its
 // first MMA, so the load latencies overlap.  acc[p] accumulates tokens 8p..8p+7.
 template <int NPASS, int PLANES>
-static __device__ __forceinline__ void consume_chunk(float (&acc)[4][4], const unsigned char* wtile,
+static __device__ __forceinline__ void consume_chunk(float (&acc)[MAX_QP][4], const unsigned char* wtile,
                                                      const uint32_t* act, int lo, int kc, int T, int ks, int kw,
                                                      int lane) {
-  constexpr int G = (NPASS * PLANES <= 1) ? 8 : (NPASS * PLANES <= 2 ? 4 : 2);
+  constexpr int G = (NPASS * PLANES <= 2) ? 4 : 2;
   const int g = lane >> 2, tig = lane & 3;
   const int nkt = kc >> 4;
   const int aw = (kc + ACT_PAD) >> 1;                       // activation row stride in 32-bit words
@@ -906,25 +906,29 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
       int32_t* done = (sg->done_idx >= 0) ? P.sync + SY_DEP + sg->done_idx : nullptr;
       const int npass = (T + 7) >> 3;
       const float* rbuf = red + (size_t)rb * RED_FLOATS;
-      // warp w holds the partial sums of tile (q == 2 ? w / 4 : 0); element (p, reg, lane) of a tile
-      const int per_tile = npass * 128;
-      const int count = paired ? per_tile : q * per_tile;
+      // Only the real outputs are reduced: (tile a, row rr of 16, token s < T).  In the MMA D
+      // fragment that element is register reg = (rr >= 8 ? 2 : 0) + (s & 1) of lane (rr % 8) * 4 +
+      // (s % 8) / 2 in pass s / 8.  Consecutive lanes of this warp take consecutive rows, so the
+      // stores of one token are contiguous.
+      const int ntile = paired ? 1 : q;
+      const int count = ntile * T * 16;
       for (int x = lane; x < count; x += 32) {
-        const int a = x / per_tile, rem = x - a * per_tile;
-        const int p = rem >> 7, reg = (rem >> 5) & 3, ln = rem & 31;
+        const int rr = x & 15, s = (x >> 4) % T, a = x / (16 * T);
+        const int p = s >> 3, reg = ((rr & 8) ? 2 : 0) + (s & 1), ln = (rr & 7) * 4 + ((s & 7) >> 1);
+        const int rem = (p * 4 + reg) * 32 + ln;
         float v0 = 0.f, v1 = 0.f;
         if (q == 2) {
+          constexpr int HW = CONSUMER_WARPS / 2;
 #pragma unroll
-          for (int w = 0; w < 4; ++w) {
-            v0 += rbuf[(size_t)(a * 4 + w) * (MAX_QP * 128) + rem];
-            if (paired) v1 += rbuf[(size_t)(4 + w) * (MAX_QP * 128) + rem];
+          for (int w = 0; w < HW; ++w) {
+            v0 += rbuf[(size_t)(a * HW + w) * (MAX_QP * 128) + rem];
+            if (paired) v1 += rbuf[(size_t)(HW + w) * (MAX_QP * 128) + rem];
           }
         } else {
 #pragma unroll
           for (int w = 0; w < CONSUMER_WARPS; ++w) v0 += rbuf[(size_t)w * (MAX_QP * 128) + rem];
         }
-        const int row = tile0 * 16 + a * 16 + (ln >> 2) + ((reg & 2) ? 8 : 0);
-        const int s = p * 8 + (ln & 3) * 2 + (reg & 1);
+        const int row = tile0 * 16 + a * 16 + rr;
         if (row < rows && s < T) {
           float r;
           if (epi == EPI_SIGMA) r = sigma_f(L.sigma, v0);
@@ -978,7 +982,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
   // Pure streaming role: wait for a chunk, multiply, release the slot.  On an item's last chunk
   // the partial accumulators go to a reduction buffer for the epilogue warp (an mbarrier
   // arrival, never a CTA barrier).
-  float acc[4][4];
+  float acc[MAX_QP][4];
   int slot = 0, items = 0;
   uint32_t phase = 0;
   long long tr[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
@@ -1002,7 +1006,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     const int npass = (T + 7) >> 3;
     if (first) {
 #pragma unroll
-      for (int p = 0; p < 4; ++p)
+      for (int p = 0; p < MAX_QP; ++p)
 #pragma unroll
         for (int x = 0; x < 4; ++x) acc[p][x] = 0.f;
     }
@@ -1014,20 +1018,19 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
 #endif
     {
       // this warp's tile and its share of the k-tiles; one specialised loop per (passes, planes)
-      const int a = (q == 2) ? (warp >> 2) : 0;
-      const int kw = (q == 2) ? 4 : CONSUMER_WARPS;
-      const int ks = (q == 2) ? (warp & 3) : warp;
+      const int a = (q == 2) ? (warp / (CONSUMER_WARPS / 2)) : 0;
+      const int kw = (q == 2) ? CONSUMER_WARPS / 2 : CONSUMER_WARPS;
+      const int ks = (q == 2) ? (warp % (CONSUMER_WARPS / 2)) : warp;
       const int aw = (kc + ACT_PAD) >> 1;
       const unsigned char* wtile = sbase + SLOT_HDR + (size_t)a * kc * 32;
       const uint32_t* act = reinterpret_cast<const uint32_t*>(sbase + SLOT_HDR + (size_t)q * kc * 32) +
                             (size_t)((nB == 2) ? a : 0) * T * aw;
       const int lo = nB * T * aw;  // offset of the lo plane
-      const int np = npass <= 1 ? 1 : (npass == 2 ? 2 : 4);
 #define DEAMOE_CASE(NP, PL) \
   case (NP * 4 + PL): consume_chunk<NP, PL>(acc, wtile, act, lo, kc, T, ks, kw, lane); break;
-      switch (np * 4 + planes) {
-        DEAMOE_CASE(1, 1) DEAMOE_CASE(2, 1) DEAMOE_CASE(4, 1)
-        DEAMOE_CASE(1, 2) DEAMOE_CASE(2, 2) DEAMOE_CASE(4, 2)
+      switch (npass * 4 + planes) {
+        DEAMOE_CASE(1, 1) DEAMOE_CASE(2, 1)
+        DEAMOE_CASE(1, 2) DEAMOE_CASE(2, 2)
         default: break;
       }
 #undef DEAMOE_CASE
@@ -1049,7 +1052,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
       }
       float* mine = red + (size_t)rb * RED_FLOATS + (size_t)warp * (MAX_QP * 128);
 #pragma unroll
-      for (int p = 0; p < 4; ++p)
+      for (int p = 0; p < MAX_QP; ++p)
         if (p < npass) {
 #pragma unroll
           for (int x = 0; x < 4; ++x) mine[(p * 4 + x) * 32 + lane] = acc[p][x];
