@@ -68,6 +68,25 @@ struct LayerDev {
   float* Osh;          // [MB, h]
 };
 
+// Programmatic dependent launch: a kernel launched with launch_pdl() may start while its
+// predecessor in the stream is still running (after the predecessor called pdl_trigger()); it must
+// call pdl_wait() before touching anything the predecessor wrote.  Both are no-ops for a kernel that
+// was launched the ordinary way.
+static __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+static __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 static __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
 
 static __device__ __forceinline__ float sigma_f(int kind, float v) {

@@ -229,6 +229,7 @@ __global__ void k_plain_identity_private(LayerDev L) {
 
 // Eq. (3): out[t] = sum_q p[t,q] * O[slot(t,q)] (+ shared expert) (+ x[t]), written in act dtype.
 __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void* __restrict__ out) {
+  pdl_wait();  // stage outputs of the preceding kernel
   const size_t total = (size_t)B * L.h;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int t = (int)(i / L.h), c = (int)(i % L.h);
@@ -287,8 +288,8 @@ int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cuda
   const size_t total = (size_t)B * L.h;
   int blocks = (int)((total + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  k_combine<<<blocks, 256, 0, s>>>(L, B, L.x32, out);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  const cudaError_t e = launch_pdl(k_combine, dim3(blocks), dim3(256), 0, s, L, B, (const float*)L.x32, out);
+  return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? 1 : -1;
 }
 
 }  // namespace deamoe

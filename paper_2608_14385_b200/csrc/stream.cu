@@ -489,6 +489,8 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   extern __shared__ uint32_t s_dyn[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  pdl_trigger();  // the streaming kernel may be launched now; it waits for this grid before reading
+  pdl_wait();     // the router logits of the preceding kernel
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   uint32_t* state = s_dyn + scratch_words;  // persistent part, after the scratch of top-k / bucketing
   // a view of the layer whose routing arrays live in shared memory
@@ -641,6 +643,8 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     ctl[0] = 0; ctl[1] = 0; ctl[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  pdl_trigger();  // the combine kernel may be launched; it waits for this grid to finish
+  pdl_wait();     // the work list is written by the preceding routing kernel
   if (tid < 4 * MAX_CAT) cat_tab[tid] = sy[SY_CAT + tid];
   __syncthreads();
 
@@ -1260,7 +1264,8 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   const size_t smem = scratch + (size_t)fl.total * 4;
   if (smem > 200 * 1024) return -1;
-  k_route_finish<<<1, FINISH_THREADS, smem, s>>>(L, p.dev, B, ny, topk_warps, (int)(scratch / 4), user_idx, user_w);
+  launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, p.dev, B, ny, topk_warps, (int)(scratch / 4),
+             user_idx, user_w);
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
@@ -1307,7 +1312,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    k_stream<<<p.n_sm, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, MAX_CAT, -1, 1 | dbgflag);
+    launch_pdl(k_stream, dim3(p.n_sm), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, (int)MAX_CAT, -1, 1 | dbgflag);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
