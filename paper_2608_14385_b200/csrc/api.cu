@@ -359,6 +359,13 @@ int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launc
 uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }
 
 #ifdef DEAMOE_TRACE
+cudaEvent_t g_tl[6];
+int g_tl_init = 0;
+int deamoe_debug_timeline(float* ms) {  // gaps between: start, after logits, after finish, after stream, after combine
+  cudaEventSynchronize(g_tl[4]);
+  for (int i = 0; i < 4; ++i) cudaEventElapsedTime(ms + i, g_tl[i], g_tl[i + 1]);
+  return 0;
+}
 int deamoe_debug_counts(deamoe_layer_t* L, int* host) {
   cudaDeviceSynchronize();
   cudaMemcpy(host, L->dev.counts, CNT_COUNT * sizeof(int), cudaMemcpyDeviceToHost);

@@ -6,6 +6,13 @@
 
 #include "deamoe.h"
 
+#ifdef DEAMOE_TRACE
+extern "C" {
+extern cudaEvent_t g_tl[6];  // trace builds only: events between the kernels of one step
+extern int g_tl_init;
+}
+#endif
+
 namespace deamoe {
 
 // Stages of one decode step (Section 3.2 of the paper; SH* = shared expert, V* = vanilla MoE).

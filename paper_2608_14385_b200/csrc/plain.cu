@@ -289,6 +289,9 @@ int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cuda
   int blocks = (int)((total + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
   const cudaError_t e = launch_pdl(k_combine, dim3(blocks), dim3(256), 0, s, L, B, (const float*)L.x32, out);
+#ifdef DEAMOE_TRACE
+  cudaEventRecord(g_tl[4], s);
+#endif
   return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? 1 : -1;
 }
 
