@@ -28,10 +28,11 @@ namespace deamoe {
 
 constexpr int CONSUMER_WARPS = 16;
 constexpr int CONSUMER_THREADS = CONSUMER_WARPS * 32;
-constexpr int WARP_ISSUE = CONSUMER_WARPS;       // issues the bulk copies
-constexpr int WARP_PLAN = CONSUMER_WARPS + 1;    // picks items, fetches records, waits for inputs
-constexpr int WARP_EPI = CONSUMER_WARPS + 2;     // reduces, applies epilogues, publishes completions
-constexpr int STREAM_THREADS = CONSUMER_THREADS + 96;
+constexpr int ISSUE_WARPS = 2;                   // copy-issue warps; warp p fills chunks p, p + ISSUE_WARPS, ...
+constexpr int WARP_ISSUE = CONSUMER_WARPS;       // first of the warps that issue the bulk copies
+constexpr int WARP_PLAN = WARP_ISSUE + ISSUE_WARPS;  // picks items, fetches records, waits for inputs
+constexpr int WARP_EPI = WARP_PLAN + 1;          // reduces, applies epilogues, publishes completions
+constexpr int STREAM_THREADS = (WARP_EPI + 1) * 32;
 constexpr int DESC_DEPTH = 8;                    // item descriptors queued between planner and epilogue
 constexpr int DESC_BYTES = 1024;                 // Seg | tail | weight sources | activation row sources
 constexpr int DESC_TAIL = 224, DESC_WSRC = 256, DESC_ASRC = 272;
@@ -810,12 +811,19 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     return;
   }
 
-  if (warp == WARP_ISSUE) {
-    // ================================================================ copy-issue warp
-    // Touches no global memory except through the bulk copies it issues.
+  if (warp >= WARP_ISSUE && warp < WARP_ISSUE + ISSUE_WARPS) {
+    // ================================================================ copy-issue warps
+    // Touch no global memory except through the bulk copies they issue.  Issuing one chunk's
+    // copies keeps a warp busy for 600-1000 cycles (about 270 for a bulk-copy instruction plus
+    // 55 for every further lane that takes part), close to the ~1150 cycles a chunk may take at
+    // full bandwidth, so the chunks of the CTA's stream alternate between ISSUE_WARPS warps.
+    // Every issue warp walks the whole descriptor queue and skips the chunks that are not its own.
+    static_assert(NSLOT % ISSUE_WARPS == 0, "an issue warp must own fixed ring slots");
+    const int ip = warp - WARP_ISSUE;
     const uint64_t pol = policy_evict_first();
-    int slot = 0, e = 0;
-    uint32_t phase = 0, eph = 0;
+    int e = 0;
+    int cidx = 0;  // index of the item's first chunk in the CTA's chunk stream
+    uint32_t eph = 0;
     bool ok = true;
     long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     (void)tr;
@@ -846,6 +854,9 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
       tr[TR_ITEMS] += 1; tr[TR_CHUNKS] += nchunks;
 #endif
       for (int ch = 0; ch < nchunks; ++ch) {
+        if ((cidx + ch) % ISSUE_WARPS != ip) continue;
+        const int slot = (cidx + ch) % NSLOT;
+        const uint32_t phase = (uint32_t)((cidx + ch) / NSLOT) & 1u;
         const int k0 = ch * kc0;
         const int kc = min(kc0, C - k0);
         const long long te0 = TR_NOW();
@@ -877,19 +888,21 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
           if (rr < nrows)
             bulk_g2s(abase + (size_t)rr * astride * 2, asrc[u] + k0, (uint32_t)kc * 2u, &full_bar[slot]);
         }
-        if (++slot == NSLOT) { slot = 0; phase ^= 1u; }
         TR_ADD(TR_ISSUE, ti0);
       }
+      cidx += nchunks;
       if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
     }
     if (!ok && lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
 #ifdef DEAMOE_TRACE
     tr[TR_PTOTAL] = clock64() - tp0;
-    if (lane == 0 && P.trace)
+    if (lane == 0 && P.trace && ip == 0)
       for (int i = 0; i < 7; ++i) P.trace[(size_t)blockIdx.x * TR_SLOTS + i] = tr[i];
 #endif
-    // end-of-work marker for the consumers
-    if (mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane) && lane == 0) {
+    // end-of-work marker for the consumers, in the slot after the last chunk
+    const int slot = cidx % NSLOT;
+    const uint32_t phase = (uint32_t)(cidx / NSLOT) & 1u;
+    if (cidx % ISSUE_WARPS == ip && mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane) && lane == 0) {
       *reinterpret_cast<int4*>(ring + (size_t)slot * SLOT_BYTES) = make_int4(1, 0, 0, 0);
       mbar_arrive(&full_bar[slot]);
     }
