@@ -4,19 +4,27 @@
 // down, and the shared / vanilla experts of Eq. (1)) is the same operation: a few token rows
 // times a weight matrix that is read exactly once.  At create the matrices are re-packed so
 // that one 16-row tile of a matrix is a contiguous stream whose 512-byte pieces are the
-// per-lane A fragments of mma.sync.m16n8k16.  One persistent kernel then works through a
-// device-built list of items (one or two 16-row tiles x the full contraction length):
+// per-lane A fragments of mma.sync.m16n8k16.  One persistent kernel (CTAS_PER_SM co-resident
+// CTAs on every SM) then works through a device-built list of items (one or two 16-row tiles x
+// the full contraction length), item i going to CTA i mod grid.  Warp roles inside a CTA:
 //
-//   producer warp   : claims items, waits (bounded) until the item's inputs exist, and moves
-//                     weight chunks (HBM) and the matching activation chunks (L2) into a
-//                     shared-memory ring with cp.async.bulk, completion on mbarriers;
-//   8 consumer warps: split each chunk's k-tiles, build bf16 hi/lo B fragments from the fp32
-//                     activations (products keep ~16 mantissa bits), accumulate in fp32 with
-//                     mma.sync, and on the item's last chunk reduce across warps, apply the
-//                     stage's epilogue and signal completion.
+//   planner warp  : reads the records of its items ahead of time, waits (bounded) until an
+//                   item's inputs exist, resolves all source pointers and queues a descriptor
+//                   in shared memory;
+//   issue warp(s) : move weight chunks (HBM, evict-first) and the matching activation rows
+//                   (L2) into a shared-memory ring with cp.async.bulk, completion on mbarriers;
+//   consumer warps: split each chunk's k-tiles, accumulate in fp32 with mma.sync on bf16
+//                   activations (one plane, or hi + lo planes for fp32 tokens) and hand their
+//                   partial sums of a finished item to
+//   epilogue warp : sums the partials, applies the stage's epilogue (sigma, SwiGLU), stores the
+//                   result as the next stage's bf16 planes (or fp32 for the last stage) and
+//                   publishes the item's completion with one fence per batch of items.
 //
 // Weights never depend on earlier stages, so the ring keeps the HBM pipe full across item and
-// stage boundaries; only the (tiny) activations wait for their producers.
+// stage boundaries; only the (tiny) activations wait for their producers.  Two small CTAs per SM
+// measured faster than one large one: a CTA's chunks are consumed strictly one after another, so
+// the fixed latency of a chunk (barrier wait, header, fragment loads, dependent MMAs, release)
+// bounds its rate, and two independent streams per SM hide that latency behind one another.
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -26,9 +34,10 @@
 
 namespace deamoe {
 
-constexpr int CONSUMER_WARPS = 16;
+constexpr int CTAS_PER_SM = 2;                   // co-resident CTAs of the streaming kernel per SM
+constexpr int CONSUMER_WARPS = 4;
 constexpr int CONSUMER_THREADS = CONSUMER_WARPS * 32;
-constexpr int ISSUE_WARPS = 2;                   // copy-issue warps; warp p fills chunks p, p + ISSUE_WARPS, ...
+constexpr int ISSUE_WARPS = 1;                   // copy-issue warps; warp p fills chunks p, p + ISSUE_WARPS, ...
 constexpr int WARP_ISSUE = CONSUMER_WARPS;       // first of the warps that issue the bulk copies
 constexpr int WARP_PLAN = WARP_ISSUE + ISSUE_WARPS;  // picks items, fetches records, waits for inputs
 constexpr int WARP_EPI = WARP_PLAN + 1;          // reduces, applies epilogues, publishes completions
@@ -38,15 +47,15 @@ constexpr int DESC_BYTES = 1024;                 // Seg | tail | weight sources 
 constexpr int DESC_TAIL = 224, DESC_WSRC = 256, DESC_ASRC = 272;
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SIG_DEPTH = 16;
-constexpr int SLOT_BYTES = 30 * 1024;
+constexpr int SLOT_BYTES = 32 * 1024;
 constexpr int SLOT_HDR = 128;
-constexpr int NSLOT = 6;
+constexpr int NSLOT = 3;
 constexpr int ACT_PAD = 8;   // floats of padding per activation row in shared memory
 constexpr int MAX_QP = 2;    // 8-token passes a consumer warp accumulates for its tile (16 tokens per segment)
 constexpr int RED_FLOATS = CONSUMER_WARPS * MAX_QP * 128;
 constexpr size_t STREAM_SMEM =
     (size_t)NSLOT * SLOT_BYTES + (size_t)NRED * RED_FLOATS * 4 + (size_t)DESC_DEPTH * DESC_BYTES + 1024;
-static_assert(STREAM_SMEM <= 227 * 1024, "shared memory budget");
+static_assert((STREAM_SMEM + 1024) * CTAS_PER_SM <= 228 * 1024, "shared memory budget");
 constexpr unsigned SPIN_LIMIT = 1u << 24;  // bounded waits; then an error status, never a hang
 constexpr int MAX_CAT = 8;
 
@@ -123,6 +132,7 @@ struct StreamPlan {
   StreamDev dev;
   int schedule;
   int n_sm;
+  int grid;  // CTAs of the streaming kernel: all of them must be resident at once
   void* packed;
   uint64_t bytes;
   cudaEvent_t ev0, ev1;   // profiling event pair (null when profiling is off)
@@ -566,8 +576,9 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
 // ---------------------------------------------------------------- inner loop of the consumers
 // One ring slot holds q weight tiles x kc columns (per-lane A fragments, 512 B per k-tile and tile)
 // followed by the activation rows [plane][input][token] x (kc + ACT_PAD) bf16.  A consumer warp
-// works on ONE tile: with two tiles in the slot warps 0-3 take the first and warps 4-7 the second
-// (4-way split of the k-tiles), with one tile all eight warps share it (8-way split).  The warp's
+// works on ONE tile: with two tiles in the slot the first half of the consumer warps takes the
+// first tile and the second half the second, with one tile all of them share it; the warps on a
+// tile split its k-tiles round-robin.  The warp's
 // k-tiles are handled G at a time: every shared-memory load of the group is issued before its
 // first MMA, so the load latencies overlap.  acc[p] accumulates tokens 8p..8p+7.
 template <int NPASS, int PLANES>
@@ -616,7 +627,7 @@ struct __align__(16) ItemCtx {  // producer-side view of one claimed item
   int seg, item_in_seg;
 };
 
-__global__ void __launch_bounds__(STREAM_THREADS, 1)
+__global__ void __launch_bounds__(STREAM_THREADS, CTAS_PER_SM)
 k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
@@ -1256,12 +1267,20 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   if (e == cudaSuccess) e = cudaMalloc(&d.segs, seg_bytes);
   if (e == cudaSuccess) e = cudaMalloc(&d.sync, sync_bytes);
 #ifdef DEAMOE_TRACE
-  if (e == cudaSuccess) e = cudaMalloc(&d.trace, (size_t)p->n_sm * TR_SLOTS * sizeof(long long));
-  if (e == cudaSuccess) e = cudaMemsetAsync(d.trace, 0, (size_t)p->n_sm * TR_SLOTS * sizeof(long long), s);
+  if (e == cudaSuccess) e = cudaMalloc(&d.trace, (size_t)p->n_sm * CTAS_PER_SM * TR_SLOTS * sizeof(long long));
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.trace, 0, (size_t)p->n_sm * CTAS_PER_SM * TR_SLOTS * sizeof(long long), s);
 #endif
   if (e == cudaSuccess) e = cudaMemsetAsync(d.sync, 0, sync_bytes, s);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)STREAM_SMEM);
+  if (e == cudaSuccess) {
+    // The CTAs wait on one another's results, so the grid may hold only as many as fit on the
+    // device at once: the occupancy the runtime reports, at most CTAS_PER_SM per SM.
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream, STREAM_THREADS, STREAM_SMEM);
+    if (e == cudaSuccess && occ < 1) e = cudaErrorLaunchOutOfResources;
+    p->grid = p->n_sm * (occ < CTAS_PER_SM ? occ : CTAS_PER_SM);
+  }
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_route_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   p->bytes += seg_bytes + sync_bytes;
@@ -1363,7 +1382,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    launch_pdl(k_stream, dim3(p.n_sm), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, (int)MAX_CAT, -1, 1 | dbgflag);
+    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, (int)MAX_CAT, -1, 1 | dbgflag);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
@@ -1371,7 +1390,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
         k_identity_private<<<p.n_sm, 256, 0, s>>>(L, p.dev);
         ++launches;
       }
-      k_stream<<<p.n_sm, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, c, c, 0);
+      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, c, c, 0);
       ++launches;
     }
   }
