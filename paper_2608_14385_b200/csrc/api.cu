@@ -157,6 +157,9 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
     A(dev_alloc(L, &d.active_dept, (size_t)d.m));
     A(dev_alloc(L, &d.active_expert, (size_t)d.n));
     A(dev_alloc(L, &d.counts, (size_t)CNT_COUNT));
+#ifdef DEAMOE_TRACE
+    A(dev_alloc(L, &d.ts, (size_t)16));
+#endif
     if (sched == DEAMOE_SCHED_PLAIN) {  // fp32 intermediates of the plain kernels
       if (!vanilla) {
         A(dev_alloc(L, &d.GU, (size_t)tdmax * 2 * d.f));
@@ -177,6 +180,7 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
     uint64_t plan_bytes = 0;
     A(stream_plan_create(d, *w, sched, s, &L->plan, &plan_bytes));
     L->device_bytes += plan_bytes;
+    if (ok) d.sh_done = stream_shared_counter(*L->plan);
   }
   if (ok && cudaStreamSynchronize(s) != cudaSuccess) A(DEAMOE_ERR_CUDA);
   if (!ok) {
@@ -359,11 +363,12 @@ int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launc
 uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }
 
 #ifdef DEAMOE_TRACE
-cudaEvent_t g_tl[6];
-int g_tl_init = 0;
-int deamoe_debug_timeline(float* ms) {  // gaps between: start, after logits, after finish, after stream, after combine
-  cudaEventSynchronize(g_tl[4]);
-  for (int i = 0; i < 4; ++i) cudaEventElapsedTime(ms + i, g_tl[i], g_tl[i + 1]);
+int deamoe_debug_ts(deamoe_layer_t* L, unsigned long long* host) {  // read and reset the step's stamps
+  cudaDeviceSynchronize();
+  cudaMemcpy(host, L->dev.ts, 16 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+  unsigned long long init[16];
+  for (int i = 0; i < 16; ++i) init[i] = (i == 1 || i == 4 || i == 7 || i == 10) ? 0ull : ~0ull;
+  cudaMemcpy(L->dev.ts, init, sizeof(init), cudaMemcpyHostToDevice);
   return 0;
 }
 int deamoe_debug_counts(deamoe_layer_t* L, int* host) {

@@ -6,14 +6,25 @@
 
 #include "deamoe.h"
 
-#ifdef DEAMOE_TRACE
-extern "C" {
-extern cudaEvent_t g_tl[6];  // trace builds only: events between the kernels of one step
-extern int g_tl_init;
-}
-#endif
 
 namespace deamoe {
+
+#ifdef DEAMOE_TRACE
+static __device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define TS_MIN(L, i) do { if (threadIdx.x == 0 && (L).ts) atomicMin((L).ts + (i), gtime()); } while (0)
+#define TS_MAX(L, i) do { if (threadIdx.x == 0 && (L).ts) atomicMax((L).ts + (i), gtime()); } while (0)
+#define TS_PARAM , unsigned long long* ts
+#define TS_ARG(L) , (L).ts
+#else
+#define TS_PARAM
+#define TS_ARG(L)
+#define TS_MIN(L, i) ((void)0)
+#define TS_MAX(L, i) ((void)0)
+#endif
 
 // Stages of one decode step (Section 3.2 of the paper; SH* = shared expert, V* = vanilla MoE).
 enum Stage : int {
@@ -41,6 +52,9 @@ enum Counter : int {
 
 // Everything a kernel needs to know about the layer; passed by value.
 struct LayerDev {
+#ifdef DEAMOE_TRACE
+  unsigned long long* ts;  // trace builds: globaltimer stamps of the kernels of one step
+#endif
   // sizes
   int h, m, g, n, f, r, k, k_dept, n_shared, fs, sigma, norm_topk, residual, vanilla;
   int wdt, adt, max_batch;
@@ -73,6 +87,7 @@ struct LayerDev {
   float* O;            // [MB*k, h]
   float* Ysh;          // [MB, fs]
   float* Osh;          // [MB, h]
+  int32_t* sh_done;    // counter the combine kernel resets at the end of a step, or null
 };
 
 // Programmatic dependent launch: a kernel launched with launch_pdl() may start while its

@@ -229,7 +229,10 @@ __global__ void k_plain_identity_private(LayerDev L) {
 
 // Eq. (3): out[t] = sum_q p[t,q] * O[slot(t,q)] (+ shared expert) (+ x[t]), written in act dtype.
 __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void* __restrict__ out) {
+  TS_MIN(L, 8);
   pdl_wait();  // stage outputs of the preceding kernel
+  TS_MIN(L, 9);
+  if (L.sh_done && blockIdx.x == 0 && threadIdx.x == 0) *L.sh_done = 0;  // nothing of this step reads it any more
   const size_t total = (size_t)B * L.h;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int t = (int)(i / L.h), c = (int)(i % L.h);
@@ -243,6 +246,7 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
     if (L.adt == DEAMOE_F32) reinterpret_cast<float*>(out)[i] = acc;
     else reinterpret_cast<__nv_bfloat16*>(out)[i] = __float2bfloat16_rn(acc);
   }
+  TS_MAX(L, 10);
 }
 
 template <typename WT>
@@ -289,9 +293,6 @@ int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cuda
   int blocks = (int)((total + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
   const cudaError_t e = launch_pdl(k_combine, dim3(blocks), dim3(256), 0, s, L, B, (const float*)L.x32, out);
-#ifdef DEAMOE_TRACE
-  cudaEventRecord(g_tl[4], s);
-#endif
   return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? 1 : -1;
 }
 

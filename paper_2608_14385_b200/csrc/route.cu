@@ -33,7 +33,10 @@ static __device__ __forceinline__ float4 load_x4(const __nv_bfloat16* p) {
 template <typename XT>
 __global__ void __launch_bounds__(ROUTER_THREADS)
 k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float* __restrict__ part,
-                int n, int h, int B, int kslice) {
+                int n, int h, int B, int kslice TS_PARAM) {
+#ifdef DEAMOE_TRACE
+  if (threadIdx.x == 0 && ts) atomicMin(ts + 0, gtime());
+#endif
   const int row0 = blockIdx.x * RG;
   const int c0 = blockIdx.y * kslice;
   const int c1 = min(h, c0 + kslice);
@@ -85,6 +88,9 @@ k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float*
     }
     __syncthreads();
   }
+#ifdef DEAMOE_TRACE
+  if (threadIdx.x == 0 && ts) atomicMax(ts + 1, gtime());
+#endif
 }
 
 // ---------------------------------------------------------------- top-k, gate weights, bucketing
@@ -125,10 +131,10 @@ int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStrea
   dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
   if (L.adt == DEAMOE_BF16)
     k_router_logits<__nv_bfloat16><<<grid, ROUTER_THREADS, 0, s>>>(L.router, reinterpret_cast<const __nv_bfloat16*>(tokens),
-                                                                  L.logit_part, L.n, L.h, B, kslice);
+                                                                  L.logit_part, L.n, L.h, B, kslice TS_ARG(L));
   else
     k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, reinterpret_cast<const float*>(tokens), L.logit_part,
-                                                          L.n, L.h, B, kslice);
+                                                          L.n, L.h, B, kslice TS_ARG(L));
   return cudaGetLastError() == cudaSuccess ? (int)grid.y : -1;
 }
 
@@ -143,7 +149,7 @@ int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, i
   }
   const int kslice = (((L.h + kslices - 1) / kslices) + 3) & ~3;
   dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
-  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, L.x32, L.logit_part, L.n, L.h, B, kslice);
+  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, L.x32, L.logit_part, L.n, L.h, B, kslice TS_ARG(L));
   ++launches;
   const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
   k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, (int)grid.y, user_idx, user_w);
@@ -220,7 +226,7 @@ extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* r
   L.logit_part = g_route_scratch_ptr[dev];   // every (slice, token, expert) entry used below is overwritten
   L.topk_idx = topk_idx; L.topk_w = topk_w;  // results go straight to the caller's buffers
   dim3 grid((L.n + RG - 1) / RG, ny);
-  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice);
+  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice TS_ARG(L));
   const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
   k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, ny, nullptr, nullptr);
   return cudaGetLastError() == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;

@@ -45,6 +45,7 @@ constexpr int STREAM_THREADS = (WARP_EPI + 1) * 32;
 constexpr int DESC_DEPTH = 8;                    // item descriptors queued between planner and epilogue
 constexpr int DESC_BYTES = 1024;                 // Seg | tail | weight sources | activation row sources
 constexpr int DESC_TAIL = 224, DESC_WSRC = 256, DESC_ASRC = 272;
+constexpr int MAX_CAT_INTS_PAD = 8;             // cat_tab: 4 ints for each of 8 categories = 16 B x 8
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SIG_DEPTH = 16;
 constexpr int SLOT_BYTES = 32 * 1024;
@@ -56,6 +57,7 @@ constexpr int RED_FLOATS = CONSUMER_WARPS * MAX_QP * 128;
 constexpr size_t STREAM_SMEM =
     (size_t)NSLOT * SLOT_BYTES + (size_t)NRED * RED_FLOATS * 4 + (size_t)DESC_DEPTH * DESC_BYTES + 1024;
 static_assert((STREAM_SMEM + 1024) * CTAS_PER_SM <= 228 * 1024, "shared memory budget");
+static_assert((2 * NSLOT + 2 * DESC_DEPTH + 2 * NRED) * 8 + 16 * MAX_CAT_INTS_PAD + 16 * NRED + 16 + 224 <= 1024, "control region");
 constexpr unsigned SPIN_LIMIT = 1u << 24;  // bounded waits; then an error status, never a hang
 constexpr int MAX_CAT = 8;
 
@@ -111,6 +113,7 @@ struct StreamDev {
   int32_t* sync;
   int max_segs;
   int dep_s1, dep_s2, dep_s3, dep_sh1, n_dep;  // offsets relative to SY_DEP
+  int sh_prefix;  // fused schedule with a shared expert: its items are not in the work list
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
   // activations between stages, bf16 planes ([rows, width] each)
   __nv_bfloat16 *xh, *xl;      // tokens split (fp32 activations only; bf16 tokens are read in place)
@@ -266,21 +269,21 @@ struct CatInfo {
 
 static __device__ __forceinline__ int category_list(const LayerDev& L, const StreamDev& P, CatInfo* cats) {
   int n = 0;
-  if (L.n_shared) cats[n++] = {ST_SH1, 0};
+  const bool sh = L.n_shared && !P.sh_prefix;  // else the streaming kernel generates the shared expert's items
+  if (sh) cats[n++] = {ST_SH1, 0};
   if (L.vanilla) {
     cats[n++] = {ST_V1, 2};
-    if (L.n_shared) cats[n++] = {ST_SH2, 0};
+    if (sh) cats[n++] = {ST_SH2, 0};
     cats[n++] = {ST_V2, 2};
   } else {
     cats[n++] = {ST_S1, 1};
-    if (L.n_shared) cats[n++] = {ST_SH2, 0};
+    if (sh) cats[n++] = {ST_SH2, 0};
     if (L.r > 0) {
       cats[n++] = {ST_S2, 2};
       cats[n++] = {ST_S3, 2};
     }
     cats[n++] = {ST_S4, 1};
   }
-  (void)P;
   return n;
 }
 
@@ -311,12 +314,11 @@ static __device__ __forceinline__ int chunk_k(int C, int q, int act_rows) {
   return kc;
 }
 
-static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stage, int id, int gi, int B,
-                                 int seg_index, int item0) {
+static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stage, int id, int gi, int B, int item0,
+                                 Seg& s) {
   const StageCfg& sc = P.st[stage];
   const int Tall = unit_tokens(L, stage, id, B);
   const int t0 = gi * sc.tg;
-  Seg s;
   s.item0 = item0; s.n_items = sc.items_per_seg; s.stage = stage; s.epi = sc.epi;
   s.T = min(sc.tg, Tall - t0); s.q = sc.q; s.paired = sc.paired; s.nB = 1;
   s.C = sc.C; s.rows = sc.rows; s.n_tiles = sc.n_tiles;
@@ -395,6 +397,12 @@ static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stag
   if (!s.in0l) s.planes = 1;
   s.kc = chunk_k(s.C, s.q, s.planes * s.nB * s.T);
   for (int t = 0; t < s.T; ++t) s.rows16[t] = (uint16_t)(in_list ? in_list[t] : in_row0 + t);
+}
+
+static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stage, int id, int gi, int B,
+                                 int seg_index, int item0) {
+  Seg s;
+  build_seg(L, P, stage, id, gi, B, item0, s);
   if (seg_index < P.max_segs) P.segs[seg_index] = s;
 }
 
@@ -499,8 +507,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   extern __shared__ uint32_t s_dyn[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  TS_MIN(L, 2);
   pdl_trigger();  // the streaming kernel may be launched now; it waits for this grid before reading
   pdl_wait();     // the router logits of the preceding kernel
+  TS_MIN(L, 3);
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   uint32_t* state = s_dyn + scratch_words;  // persistent part, after the scratch of top-k / bucketing
   // a view of the layer whose routing arrays live in shared memory
@@ -519,6 +529,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   S.dept_mask = reinterpret_cast<uint64_t*>(state + fl.dept_mask);
 #ifdef DEAMOE_TRACE
   long long tt0 = clock64();
+  TS_MIN(L, 11);
 #endif
   for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) S.counts[i] = 0;
   const bool regs_ok = (L.k_dept <= 0 || L.k_dept >= L.m) && L.n <= 512 &&
@@ -542,11 +553,13 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   __syncthreads();
 #ifdef DEAMOE_TRACE
   long long tt1 = clock64();
+  TS_MIN(L, 12);
 #endif
   bucket_block(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
 #ifdef DEAMOE_TRACE
   long long tt2 = clock64();
+  TS_MIN(L, 13);
 #endif
   worklist_block(S, P, B);
   __syncthreads();
@@ -566,6 +579,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) L.counts[i] = S.counts[i];
 #ifdef DEAMOE_TRACE
   __syncthreads();
+  TS_MAX(L, 4);
   if (threadIdx.x == 0) {
     L.counts[8] = (int)(tt1 - tt0); L.counts[9] = (int)(tt2 - tt1); L.counts[10] = (int)(clock64() - tt2);
     L.counts[11] = S.counts[11]; L.counts[12] = (int)((S.counts[12] - (int)(tt0 & 0x7fffffff)));
@@ -628,7 +642,7 @@ struct __align__(16) ItemCtx {  // producer-side view of one claimed item
 };
 
 __global__ void __launch_bounds__(STREAM_THREADS, CTAS_PER_SM)
-k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
+k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* red = reinterpret_cast<float*>(smem + (size_t)NSLOT * SLOT_BYTES);
@@ -643,7 +657,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
   int* red_info = cat_tab + 4 * MAX_CAT;                               // NRED x {e | tile0 << 8, q, T, 0}
   volatile int* ctl = red_info + 4 * NRED;                             // [0] abort, [1] closed, [2] items produced
   volatile int* abort_flag = ctl;
-  (void)launch_id;
+  unsigned char* seg_stage = reinterpret_cast<unsigned char*>(red_info + 4 * NRED + 4);  // one Seg, planner only
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int32_t* sy = P.sync;
@@ -654,22 +668,132 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     ctl[0] = 0; ctl[1] = 0; ctl[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  pdl_trigger();  // the combine kernel may be launched; it waits for this grid to finish
-  pdl_wait();     // the work list is written by the preceding routing kernel
-  if (tid < 4 * MAX_CAT) cat_tab[tid] = sy[SY_CAT + tid];
   __syncthreads();
-
-  // item range of this launch: one category (staged) or everything (fused)
-  const int ncat = sy[SY_NCAT];
-  const int item_begin = (cat >= 0) ? cat_tab[4 * cat] : 0;
-  const int item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
+  TS_MIN(L, 5);
+  pdl_trigger();  // the combine kernel may be launched; it waits for this grid to finish
 
   if (warp == WARP_PLAN) {
     // ================================================================ planner warp
     // Runs ahead of the copy issue.  The items of a CTA are fixed by its index, so their records
     // can be read ahead; the planner waits (bounded) until an item's inputs exist, resolves every
     // source pointer and queues a ready-to-issue descriptor in shared memory.  All global
-    // memory latency of the bookkeeping is paid here, off the streaming path.
+    // memory latency of the bookkeeping is paid here, off the streaming path.  It is the only
+    // warp that reads what the routing kernel wrote, so it alone waits for that kernel.
+#ifdef DEAMOE_TRACE
+    long long ptr_dep = 0, ptr_q = 0;
+#endif
+    const int G = (int)gridDim.x;
+    int dep_ok = -1;
+    int e = 0;
+    uint32_t eph = 0;
+    bool ok = true;
+    // Queue the item `it` of the segment record held as one int4 per lane (lane l < SEG_VEC holds
+    // bytes [16 l, 16 l + 16)).  dv is a value of the item's dependency counter read earlier.
+    auto emit = [&](const int4 v, const int it, const bool dv_valid, const int dv) -> bool {
+      // dep_idx / dep_target are ints 15 and 16 of the record: lane 3 .w and lane 4 .x
+      const int dep_idx = __shfl_sync(0xffffffffu, v.w, 3);
+      const int dep_target = __shfl_sync(0xffffffffu, v.x, 4);
+      int fresh = 0;
+      if ((check_deps & 1) && dep_idx >= 0 && dep_idx != dep_ok) {
+        const int32_t* dep = P.sync + SY_DEP + dep_idx;
+        bool ready = dv_valid && __all_sync(0xffffffffu, dv >= dep_target);
+        unsigned spins = 0;
+#ifdef DEAMOE_TRACE
+        const long long tpd0 = clock64();
+#endif
+        while (!ready) {
+          ready = __all_sync(0xffffffffu, ld_acquire(dep) >= dep_target);
+          if (!ready) {
+            __nanosleep(32);
+            if (++spins > SPIN_LIMIT / 16 || *abort_flag) break;
+          }
+        }
+#ifdef DEAMOE_TRACE
+        ptr_dep += clock64() - tpd0;
+#endif
+        if (!ready) return false;
+        dep_ok = dep_idx;
+        fresh = 1;
+      }
+#ifdef DEAMOE_TRACE
+      const long long tpq0 = clock64();
+#endif
+      if (!mbar_wait_warp(&dq_empty[e], eph ^ 1u, abort_flag, lane, 200)) return false;
+#ifdef DEAMOE_TRACE
+      ptr_q += clock64() - tpq0;
+#endif
+      unsigned char* ent = descs + (size_t)e * DESC_BYTES;
+      if (lane < SEG_VEC) reinterpret_cast<int4*>(ent)[lane] = v;
+      __syncwarp();
+      const Seg* sg = reinterpret_cast<const Seg*>(ent);
+      const int T = sg->T, paired = sg->paired, nB = sg->nB, C = sg->C;
+      const int tile0 = paired ? it : it * sg->q;
+      const int q_eff = paired ? 2 : min(sg->q, sg->n_tiles - tile0);
+      const int nrows = sg->planes * nB * T;
+      if (lane == 31) {
+        int* tail = reinterpret_cast<int*>(ent + DESC_TAIL);
+        tail[0] = 0;      // kind: work
+        tail[1] = tile0;
+        tail[2] = fresh;  // inputs were acquired for this item: the issuer must fence the async proxy
+        tail[3] = q_eff;
+        tail[4] = nrows;
+      }
+      if (lane < 2) {  // weight stream of tile `lane` of the item
+        const __nv_bfloat16* wsrc = (lane == 0 || !paired) ? sg->w0 + (size_t)(tile0 + lane) * (C / 16) * 256
+                                                           : sg->w1 + (size_t)tile0 * (C / 16) * 256;
+        reinterpret_cast<const __nv_bfloat16**>(ent + DESC_WSRC)[lane] = wsrc;
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {  // activation rows, ordered [plane][input][token]
+        const int rr = lane + 32 * u;
+        if (rr < nrows) {
+          const int pn = rr / T, s = rr - pn * T;
+          const int pl = pn / nB, nb = pn - pl * nB;
+          const __nv_bfloat16* base = pl ? (nb ? sg->in1l : sg->in0l) : (nb ? sg->in1h : sg->in0h);
+          reinterpret_cast<const __nv_bfloat16**>(ent + DESC_ASRC)[rr] = base + (size_t)sg->rows16[s] * sg->in_stride;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&dq_full[e]);
+      if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
+      return true;
+    };
+
+    // The shared expert (Eq. (1)) does not depend on the routing: in the fused schedule its items
+    // are generated here, from the batch size alone, and stream while the routing kernel that
+    // precedes this grid is still running.
+    if (P.sh_prefix && cat < 0) {
+      Seg* stage_seg = reinterpret_cast<Seg*>(seg_stage);
+      int first_cta = 0;  // the CTA that takes the stage's first item
+      for (int st = ST_SH1; ok && st <= ST_SH2; ++st) {
+        const int ips = P.st[st].items_per_seg;
+        const int n_items = groups_of(B, P.st[st].tg) * ips;
+        int have_seg = -1;
+        int4 v = make_int4(0, 0, 0, 0);
+        for (int x = ((int)blockIdx.x - first_cta + G) % G; ok && x < n_items; x += G) {
+          const int gi = x / ips;
+          if (gi != have_seg) {
+            __syncwarp();
+            if (lane == 0) build_seg(L, P, st, 0, gi, B, 0, *stage_seg);
+            __syncwarp();
+            if (lane < SEG_VEC) v = reinterpret_cast<const int4*>(stage_seg)[lane];
+            have_seg = gi;
+          }
+          ok = emit(v, x - gi * ips, false, 0);
+        }
+        first_cta = (first_cta + n_items) % G;
+      }
+    }
+
+    pdl_wait();  // the work list is written by the preceding routing kernel
+    TS_MIN(L, 6);
+    cat_tab[lane] = sy[SY_CAT + lane];  // 4 * MAX_CAT == 32 entries
+    __syncwarp();
+    // item range of this launch: one category (staged) or everything (fused)
+    const int ncat = sy[SY_NCAT];
+    const int item_begin = (cat >= 0) ? cat_tab[4 * cat] : 0;
+    const int item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
+    if (*abort_flag && lane == 0) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;  // set before the routing kernel reset it
     auto seg_of = [&](int k, int item, int& it) -> const Seg* {
       const int ib = cat_tab[4 * k + 0], sb = cat_tab[4 * k + 1], ips = cat_tab[4 * k + 2];
       it = (item - ib) % ips;
@@ -679,7 +803,6 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     // the items out (rather than giving a CTA one contiguous stretch per category) completes
     // the units one after another, so dependent items of later categories become ready early;
     // contiguous stretches were measured 25-35 % slower for that reason.
-    const int G = (int)gridDim.x;
     int cur_i = item_begin + (int)blockIdx.x;
     auto next_item = [&](int& k) -> int {  // next item of this CTA, -1 at the end
       if (cur_i >= item_end) return -1;
@@ -708,15 +831,8 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
     fetch(sp0, it0, v0);
     fetch(sp1, it1, v1);
     fetch(sp2, it2, v2);
-#ifdef DEAMOE_TRACE
-    long long ptr_dep = 0, ptr_q = 0;
-#endif
     int dv0 = 0;            // counter value read ahead for record 0
     bool dv0_valid = false;
-    int dep_ok = -1;
-    int e = 0;
-    uint32_t eph = 0;
-    bool ok = true;
     while (ok && sp0) {
       // read ahead: dependency counter of the next item, record of the item three ahead
       int dv1 = 0;
@@ -730,76 +846,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
       }
       const Seg* sp3; int it3 = 0; int4 v3 = make_int4(0, 0, 0, 0);
       fetch(sp3, it3, v3);
-      {
-        const int it = it0;
-        const int4 v = v0;
-        // dep_idx / dep_target are ints 15 and 16 of the record: lane 3 .w and lane 4 .x
-        const int dep_idx = __shfl_sync(0xffffffffu, v.w, 3);
-        const int dep_target = __shfl_sync(0xffffffffu, v.x, 4);
-        int fresh = 0;
-        if ((check_deps & 1) && dep_idx >= 0 && dep_idx != dep_ok) {
-          const int32_t* dep = P.sync + SY_DEP + dep_idx;
-          bool ready = dv0_valid && __all_sync(0xffffffffu, dv0 >= dep_target);
-          unsigned spins = 0;
-#ifdef DEAMOE_TRACE
-          const long long tpd0 = clock64();
-#endif
-          while (!ready) {
-            ready = __all_sync(0xffffffffu, ld_acquire(dep) >= dep_target);
-            if (!ready) {
-              __nanosleep(32);
-              if (++spins > SPIN_LIMIT / 16 || *abort_flag) break;
-            }
-          }
-#ifdef DEAMOE_TRACE
-          ptr_dep += clock64() - tpd0;
-#endif
-          if (!ready) { ok = false; break; }
-          dep_ok = dep_idx;
-          fresh = 1;
-        }
-#ifdef DEAMOE_TRACE
-        const long long tpq0 = clock64();
-#endif
-        if (!mbar_wait_warp(&dq_empty[e], eph ^ 1u, abort_flag, lane, 200)) { ok = false; break; }
-#ifdef DEAMOE_TRACE
-        ptr_q += clock64() - tpq0;
-#endif
-        unsigned char* ent = descs + (size_t)e * DESC_BYTES;
-        if (lane < SEG_VEC) reinterpret_cast<int4*>(ent)[lane] = v;
-        __syncwarp();
-        const Seg* sg = reinterpret_cast<const Seg*>(ent);
-        const int T = sg->T, paired = sg->paired, nB = sg->nB, C = sg->C;
-        const int tile0 = paired ? it : it * sg->q;
-        const int q_eff = paired ? 2 : min(sg->q, sg->n_tiles - tile0);
-        const int nrows = sg->planes * nB * T;
-        if (lane == 31) {
-          int* tail = reinterpret_cast<int*>(ent + DESC_TAIL);
-          tail[0] = 0;      // kind: work
-          tail[1] = tile0;
-          tail[2] = fresh;  // inputs were acquired for this item: the issuer must fence the async proxy
-          tail[3] = q_eff;
-          tail[4] = nrows;
-        }
-        if (lane < 2) {  // weight stream of tile `lane` of the item
-          const __nv_bfloat16* wsrc = (lane == 0 || !paired) ? sg->w0 + (size_t)(tile0 + lane) * (C / 16) * 256
-                                                             : sg->w1 + (size_t)tile0 * (C / 16) * 256;
-          reinterpret_cast<const __nv_bfloat16**>(ent + DESC_WSRC)[lane] = wsrc;
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {  // activation rows, ordered [plane][input][token]
-          const int rr = lane + 32 * u;
-          if (rr < nrows) {
-            const int pn = rr / T, s = rr - pn * T;
-            const int pl = pn / nB, nb = pn - pl * nB;
-            const __nv_bfloat16* base = pl ? (nb ? sg->in1l : sg->in0l) : (nb ? sg->in1h : sg->in0h);
-            reinterpret_cast<const __nv_bfloat16**>(ent + DESC_ASRC)[rr] = base + (size_t)sg->rows16[s] * sg->in_stride;
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&dq_full[e]);
-        if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
-      }
+      ok = emit(v0, it0, dv0_valid, dv0);
       // rotate the record pipeline
       sp0 = sp1; it0 = it1; v0 = v1; dv0 = dv1; dv0_valid = dv1_valid;
       sp1 = sp2; it1 = it2; v1 = v2;
@@ -1131,6 +1178,7 @@ k_stream(LayerDev L, StreamDev P, int launch_id, int cat, int check_deps) {
   }
 #ifdef DEAMOE_TRACE
   tr[TR_CTOTAL] = clock64() - tc0;
+  TS_MAX(L, 7);
   if (tid == 0 && P.trace)
     for (int i = 8; i < 15; ++i) P.trace[(size_t)blockIdx.x * TR_SLOTS + i] = tr[i];
 #endif
@@ -1244,6 +1292,11 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   const int MB = L.max_batch;
   d.max_segs = 8 + 2 * L.m + 2 * L.n + MB * L.k + 2 * MB;
   d.dep_s1 = 0; d.dep_s2 = L.m; d.dep_s3 = L.m + L.n; d.dep_sh1 = 2 * L.m + L.n; d.n_dep = 2 * L.m + L.n + 1;
+  // Fused schedule: the shared expert's items run before the routing kernel has finished, which
+  // zeroes counters [0, n_dep); theirs is the first counter after that range, and the combine
+  // kernel, the last of a step, resets it.
+  d.sh_prefix = (schedule == DEAMOE_SCHED_FUSED && L.n_shared && (L.vanilla || L.r > 0)) ? 1 : 0;
+  if (d.sh_prefix) d.dep_sh1 = d.n_dep;
   d.planes = (L.adt == DEAMOE_F32) ? 2 : 1;
   {
     // activation planes between stages
@@ -1308,17 +1361,14 @@ void stream_plan_destroy(StreamPlan* p) {
   delete p;
 }
 
+int32_t* stream_shared_counter(StreamPlan& p) {
+  return p.dev.sh_prefix ? p.dev.sync + SY_DEP + p.dev.dep_sh1 : nullptr;
+}
+
 int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
                  int32_t* user_idx, float* user_w) {
-#ifdef DEAMOE_TRACE
-  if (!g_tl_init) { for (int i = 0; i < 6; ++i) cudaEventCreate(&g_tl[i]); g_tl_init = 1; }
-  cudaEventRecord(g_tl[0], s);
-#endif
   const int ny = launch_router_logits(L, tokens, B, s, kslices);
   if (ny < 0) return -1;
-#ifdef DEAMOE_TRACE
-  cudaEventRecord(g_tl[1], s);
-#endif
   const int per_warp = (L.n * 5 + 15) & ~15;
   int topk_warps = (48 * 1024) / per_warp;
   if (topk_warps > FINISH_THREADS / 32) topk_warps = FINISH_THREADS / 32;
@@ -1333,9 +1383,6 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (smem > 200 * 1024) return -1;
   launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, p.dev, B, ny, topk_warps, (int)(scratch / 4),
              user_idx, user_w);
-#ifdef DEAMOE_TRACE
-  cudaEventRecord(g_tl[2], s);
-#endif
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
@@ -1382,7 +1429,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, (int)MAX_CAT, -1, 1 | dbgflag);
+    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | dbgflag);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
@@ -1390,14 +1437,11 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
         k_identity_private<<<p.n_sm, 256, 0, s>>>(L, p.dev);
         ++launches;
       }
-      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, c, c, 0);
+      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, B, c, 0);
       ++launches;
     }
   }
   if (p.ev1) { cudaEventRecord(p.ev1, s); p.ev_recorded = 1; }
-#ifdef DEAMOE_TRACE
-  cudaEventRecord(g_tl[3], s);
-#endif
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 

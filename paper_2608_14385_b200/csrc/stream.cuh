@@ -17,6 +17,10 @@ void stream_plan_destroy(StreamPlan* p);
 
 // Routing for the streaming schedules: router logits, then ONE kernel for top-k + gate weights,
 // bucketing and the work list.  Returns the number of kernels launched or -1.
+// The completion counter of the shared expert's first stage when the fused schedule runs the
+// shared expert ahead of the routing (else null).  The last kernel of a step must zero it.
+int32_t* stream_shared_counter(StreamPlan& p);
+
 int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
                  int32_t* user_idx, float* user_w);
 
