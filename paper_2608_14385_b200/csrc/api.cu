@@ -158,7 +158,7 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
     A(dev_alloc(L, &d.active_expert, (size_t)d.n));
     A(dev_alloc(L, &d.counts, (size_t)CNT_COUNT));
 #ifdef DEAMOE_TRACE
-    A(dev_alloc(L, &d.ts, (size_t)16));
+    A(dev_alloc(L, &d.ts, (size_t)24));
 #endif
     if (sched == DEAMOE_SCHED_PLAIN) {  // fp32 intermediates of the plain kernels
       if (!vanilla) {
@@ -365,9 +365,9 @@ uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_byt
 #ifdef DEAMOE_TRACE
 int deamoe_debug_ts(deamoe_layer_t* L, unsigned long long* host) {  // read and reset the step's stamps
   cudaDeviceSynchronize();
-  cudaMemcpy(host, L->dev.ts, 16 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
-  unsigned long long init[16];
-  for (int i = 0; i < 16; ++i) init[i] = (i == 1 || i == 4 || i == 7 || i == 10) ? 0ull : ~0ull;
+  cudaMemcpy(host, L->dev.ts, 24 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+  unsigned long long init[24];
+  for (int i = 0; i < 24; ++i) init[i] = (i == 1 || i == 4 || i == 7 || i == 10 || i == 16) ? 0ull : ~0ull;
   cudaMemcpy(L->dev.ts, init, sizeof(init), cudaMemcpyHostToDevice);
   return 0;
 }

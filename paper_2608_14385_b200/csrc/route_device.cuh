@@ -92,29 +92,29 @@ static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslic
 
 // Same result with the logits held in registers (n <= 32 * VPL, flat top-k): every partial-logit
 // load is issued before the first use, and the k selection rounds touch no memory at all.
-template <int VPL, int KS>
-static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int lane,
+template <int VPL>
+static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int kslices, int lane,
                                            int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   const int n = L.n, k = L.k;
   float v[VPL];
   unsigned taken = 0;
   {
-    // all VPL * KS partial logits are loaded (clamped index, no branches) before the first add
-    float part[VPL][KS];
+    // Slices are added in the fixed order 0, 1, ...; four slices (4 * VPL loads per lane) are in
+    // flight at a time.  The loop stays rolled: this runs once per step from a cold instruction
+    // cache, where a short loop beats a long unrolled run of loads.
+    int col[VPL];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) { col[j] = min(lane + 32 * j, n - 1); v[j] = 0.f; }
     const float* __restrict__ src = L.logit_part + (size_t)t * n;
     const size_t slice = (size_t)B * n;
+#pragma unroll 4
+    for (int sl = 0; sl < kslices; ++sl, src += slice) {
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) v[j] += __ldg(src + col[j]);
+    }
 #pragma unroll
     for (int j = 0; j < VPL; ++j)
-#pragma unroll
-      for (int sl = 0; sl < KS; ++sl) part[j][sl] = __ldg(src + (size_t)sl * slice + min(lane + 32 * j, n - 1));
-#pragma unroll
-    for (int j = 0; j < VPL; ++j) {
-      float sum = 0.f;
-#pragma unroll
-      for (int sl = 0; sl < KS; ++sl) sum += part[j][sl];  // fixed order: slice 0, 1, ...
-      if (lane + 32 * j >= n) { sum = -INFINITY; taken |= 1u << j; }
-      v[j] = sum;
-    }
+      if (lane + 32 * j >= n) { v[j] = -INFINITY; taken |= 1u << j; }
   }
 #ifdef DEAMOE_TRACE
   float chk = 0.f;
@@ -206,6 +206,8 @@ static __device__ __forceinline__ int warp_exclusive_offsets(const int* cnt, int
 }
 
 // Body of the bucketing step for one CTA of `nthr` threads (a multiple of 64); s_u32: bucket_smem_bytes().
+// Executed once per step by one CTA, usually with a cold instruction cache: the loops are kept
+// rolled so that the code stays small.
 static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, int nthr) {
   const int n = L.n, m = L.m, g = L.g, k = L.k;
   const int W = (B + 31) / 32;
@@ -216,8 +218,10 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
   int* s_eoff = dcnt + m;                                      // [n+1]
   int* s_doff = s_eoff + n + 1;                                // [m+1]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll 1
   for (int i = tid; i < (n + m) * W; i += nthr) s_u32[i] = 0u;
   __syncthreads();
+#pragma unroll 1
   for (int p = tid; p < B * k; p += nthr) {
     const int t = p / k;
     const int i = L.topk_idx[p];
@@ -225,16 +229,20 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
     atomicOr(&dmask[(size_t)(i / g) * W + (t >> 5)], 1u << (t & 31));
   }
   __syncthreads();
+#pragma unroll 1
   for (int i = tid; i < n; i += nthr) {
     int c = 0;
+#pragma unroll 1
     for (int w = 0; w < W; ++w) c += __popc(emask[(size_t)i * W + w]);
     ecnt[i] = c;
   }
   // department counts; the active-department bitmask falls out of a warp ballot (32 departments
   // per warp iteration, written as the two 32-bit halves of the 64-bit words)
+#pragma unroll 1
   for (int j = tid; j < ((m + 63) & ~63); j += nthr) {
     int c = 0;
     if (j < m) {
+#pragma unroll 1
       for (int w = 0; w < W; ++w) c += __popc(dmask[(size_t)j * W + w]);
       dcnt[j] = c;
     }
@@ -248,7 +256,9 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
     warp_exclusive_offsets(ecnt, n, s_eoff, L.active_expert, lane, &L.counts[CNT_ACTIVE_EXPERT]);
   }
   __syncthreads();
+#pragma unroll 1
   for (int i = tid; i <= n; i += nthr) L.expert_off[i] = s_eoff[i];
+#pragma unroll 1
   for (int j = tid; j <= m; j += nthr) L.dept_off[j] = s_doff[j];
   if (tid == 0) {
     L.counts[CNT_STATUS] = 0;
@@ -256,10 +266,13 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
     L.counts[CNT_PAIRS] = s_eoff[n];
   }
   // ascending token lists
+#pragma unroll 1
   for (int i = tid; i < n; i += nthr) {
     int pos = s_eoff[i];
+#pragma unroll 1
     for (int w = 0; w < W; ++w) {
       uint32_t bits = emask[(size_t)i * W + w];
+#pragma unroll 1
       while (bits) {
         const int b = __ffs(bits) - 1;
         bits &= bits - 1;
@@ -267,10 +280,13 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
       }
     }
   }
+#pragma unroll 1
   for (int j = tid; j < m; j += nthr) {
     int pos = s_doff[j];
+#pragma unroll 1
     for (int w = 0; w < W; ++w) {
       uint32_t bits = dmask[(size_t)j * W + w];
+#pragma unroll 1
       while (bits) {
         const int b = __ffs(bits) - 1;
         bits &= bits - 1;
@@ -279,11 +295,13 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
     }
   }
   // pair order and the GU row of every pair
+#pragma unroll 1
   for (int p = tid; p < B * k; p += nthr) {
     const int t = p / k;
     const int i = L.topk_idx[p];
     const int j = i / g;
     int re = 0, rd = 0;
+#pragma unroll 1
     for (int w = 0; w < (t >> 5); ++w) {
       re += __popc(emask[(size_t)i * W + w]);
       rd += __popc(dmask[(size_t)j * W + w]);

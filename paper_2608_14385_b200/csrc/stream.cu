@@ -25,6 +25,7 @@
 // measured faster than one large one: a CTA's chunks are consumed strictly one after another, so
 // the fixed latency of a chunk (barrier wait, header, fragment loads, dependent MMAs, release)
 // bounds its rate, and two independent streams per SM hide that latency behind one another.
+#include <cstddef>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -314,169 +315,229 @@ static __device__ __forceinline__ int chunk_k(int C, int q, int act_rows) {
   return kc;
 }
 
+// Fills the record of (stage, unit id, token group gi).  Everything is computed in registers and
+// stored as fourteen 16-byte words, so that `dst` may be global or shared memory and nothing
+// passes through per-thread local memory (that cost microseconds per record: this code runs once
+// per step, with cold caches).
+static_assert(offsetof(Seg, w0) == 80 && offsetof(Seg, outf) == 144 && offsetof(Seg, rows16) == 160, "Seg layout");
+static_assert(MAX_QP * 8 <= 16, "build_seg writes at most 16 token rows");
 static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stage, int id, int gi, int B, int item0,
-                                 Seg& s) {
+                                 Seg& dst) {
   const StageCfg& sc = P.st[stage];
   const int Tall = unit_tokens(L, stage, id, B);
   const int t0 = gi * sc.tg;
-  s.item0 = item0; s.n_items = sc.items_per_seg; s.stage = stage; s.epi = sc.epi;
-  s.T = min(sc.tg, Tall - t0); s.q = sc.q; s.paired = sc.paired; s.nB = 1;
-  s.C = sc.C; s.rows = sc.rows; s.n_tiles = sc.n_tiles;
-  s.w0 = sc.w0 + (size_t)id * sc.unit_elems;
-  s.w1 = sc.w1 ? sc.w1 + (size_t)id * sc.unit_elems : nullptr;
-  s.in0l = nullptr; s.in1h = nullptr; s.in1l = nullptr;
-  s.pad0 = 0; s.pad1 = 0;
-  const int32_t* in_list = nullptr;  // gathered input rows, or in_row0 + s
-  int in_row0 = 0;
-  s.outh = nullptr; s.outl = nullptr; s.outf = nullptr;
-  s.dep_idx = -1; s.dep_target = 0; s.done_idx = -1;
-  s.planes = P.planes;
+  const int T = min(sc.tg, Tall - t0);
+  int nB = 1, in_stride = 0, out_stride = 0, out_row0 = 0, dep_idx = -1, dep_target = 0, done_idx = -1, in_row0 = 0;
+  const __nv_bfloat16* in0h = nullptr; const __nv_bfloat16* in0l = nullptr;
+  const __nv_bfloat16* in1h = nullptr; const __nv_bfloat16* in1l = nullptr;
+  __nv_bfloat16* outh = nullptr; __nv_bfloat16* outl = nullptr;
+  float* outf = nullptr;
+  const int32_t* in_list = nullptr;  // gathered input rows, or in_row0 + token
   // tokens: bf16 tokens are their own (only) plane; fp32 tokens were split by k_split_tokens
   const __nv_bfloat16* tokh = (L.adt == DEAMOE_BF16) ? reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw) : P.xh;
   const __nv_bfloat16* tokl = (L.adt == DEAMOE_BF16) ? nullptr : P.xl;
   const int j = (stage == ST_S2 || stage == ST_S3) ? id / L.g : id;
   switch (stage) {
     case ST_S1:
-      s.in0h = tokh; s.in0l = tokl; s.in_stride = L.h; in_list = L.dept_tok + L.dept_off[id] + t0;
-      s.outh = P.GUh; s.outl = P.GUl; s.out_stride = 2 * L.f; s.out_row0 = L.dept_off[id] + t0;
-      s.done_idx = P.dep_s1 + id;
+      in0h = tokh; in0l = tokl; in_stride = L.h; in_list = L.dept_tok + L.dept_off[id] + t0;
+      outh = P.GUh; outl = P.GUl; out_stride = 2 * L.f; out_row0 = L.dept_off[id] + t0;
+      done_idx = P.dep_s1 + id;
       break;
     case ST_S2:
-      s.in0h = P.GUh; s.in0l = P.GUl; s.in1h = P.GUh + L.f; s.in1l = P.GUl + L.f; s.nB = 2;
-      s.in_stride = 2 * L.f;
+      in0h = P.GUh; in0l = P.GUl; in1h = P.GUh + L.f; in1l = P.GUl + L.f; nB = 2;
+      in_stride = 2 * L.f;
       in_list = L.pair_gurow + L.expert_off[id] + t0;
-      s.outh = P.Yh; s.outl = P.Yl; s.out_stride = L.rp; s.out_row0 = L.expert_off[id] + t0;
-      s.dep_idx = P.dep_s1 + j;
-      s.dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
-      s.done_idx = P.dep_s2 + id;
+      outh = P.Yh; outl = P.Yl; out_stride = L.rp; out_row0 = L.expert_off[id] + t0;
+      dep_idx = P.dep_s1 + j;
+      dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
+      done_idx = P.dep_s2 + id;
       break;
     case ST_S3:
-      s.in0h = P.Yh; s.in0l = P.Yl; s.in_stride = L.rp; in_row0 = L.expert_off[id] + t0;
-      s.outh = P.Zh; s.outl = P.Zl; s.out_stride = L.f; s.out_row0 = L.expert_off[id] + t0;
-      s.dep_idx = P.dep_s2 + id;
-      s.dep_target = groups_of(Tall, P.st[ST_S2].tg) * P.st[ST_S2].n_tiles;
-      s.done_idx = P.dep_s3 + j;
+      in0h = P.Yh; in0l = P.Yl; in_stride = L.rp; in_row0 = L.expert_off[id] + t0;
+      outh = P.Zh; outl = P.Zl; out_stride = L.f; out_row0 = in_row0;
+      dep_idx = P.dep_s2 + id;
+      dep_target = groups_of(Tall, P.st[ST_S2].tg) * P.st[ST_S2].n_tiles;
+      done_idx = P.dep_s3 + j;
       break;
     case ST_S4: {
       const int p0 = L.expert_off[id * L.g];
-      s.in0h = P.Zh; s.in0l = P.Zl; s.in_stride = L.f; in_row0 = p0 + t0;
-      s.outf = L.O; s.out_stride = L.h; s.out_row0 = p0 + t0;
+      in0h = P.Zh; in0l = P.Zl; in_stride = L.f; in_row0 = p0 + t0;
+      outf = L.O; out_stride = L.h; out_row0 = p0 + t0;
       if (L.r > 0) {
-        int target = 0;
+#pragma unroll 1
         for (int e = 0; e < L.g; ++e) {
           const int Te = L.expert_off[id * L.g + e + 1] - L.expert_off[id * L.g + e];
-          target += groups_of(Te, P.st[ST_S3].tg) * P.st[ST_S3].n_tiles;
+          dep_target += groups_of(Te, P.st[ST_S3].tg) * P.st[ST_S3].n_tiles;
         }
-        s.dep_idx = P.dep_s3 + id; s.dep_target = target;
+        dep_idx = P.dep_s3 + id;
       }
       break;
     }
     case ST_SH1:
-      s.in0h = tokh; s.in0l = tokl; s.in_stride = L.h; in_row0 = t0;
-      s.outh = P.Yshh; s.outl = P.Yshl; s.out_stride = L.fs; s.out_row0 = t0;
-      s.done_idx = P.dep_sh1;
+      in0h = tokh; in0l = tokl; in_stride = L.h; in_row0 = t0;
+      outh = P.Yshh; outl = P.Yshl; out_stride = L.fs; out_row0 = t0;
+      done_idx = P.dep_sh1;
       break;
     case ST_SH2:
-      s.in0h = P.Yshh; s.in0l = P.Yshl; s.in_stride = L.fs; in_row0 = t0;
-      s.outf = L.Osh; s.out_stride = L.h; s.out_row0 = t0;
-      s.dep_idx = P.dep_sh1;
-      s.dep_target = groups_of(B, P.st[ST_SH1].tg) * P.st[ST_SH1].n_tiles;
+      in0h = P.Yshh; in0l = P.Yshl; in_stride = L.fs; in_row0 = t0;
+      outf = L.Osh; out_stride = L.h; out_row0 = t0;
+      dep_idx = P.dep_sh1;
+      dep_target = groups_of(B, P.st[ST_SH1].tg) * P.st[ST_SH1].n_tiles;
       break;
     case ST_V1:
-      s.in0h = tokh; s.in0l = tokl; s.in_stride = L.h; in_list = L.expert_tok + L.expert_off[id] + t0;
-      s.outh = P.Yh; s.outl = P.Yl; s.out_stride = L.f; s.out_row0 = L.expert_off[id] + t0;
-      s.done_idx = P.dep_s2 + id;
+      in0h = tokh; in0l = tokl; in_stride = L.h; in_list = L.expert_tok + L.expert_off[id] + t0;
+      outh = P.Yh; outl = P.Yl; out_stride = L.f; out_row0 = L.expert_off[id] + t0;
+      done_idx = P.dep_s2 + id;
       break;
     case ST_V2:
-      s.in0h = P.Yh; s.in0l = P.Yl; s.in_stride = L.f; in_row0 = L.expert_off[id] + t0;
-      s.outf = L.O; s.out_stride = L.h; s.out_row0 = L.expert_off[id] + t0;
-      s.dep_idx = P.dep_s2 + id;
-      s.dep_target = groups_of(Tall, P.st[ST_V1].tg) * P.st[ST_V1].n_tiles;
+      in0h = P.Yh; in0l = P.Yl; in_stride = L.f; in_row0 = L.expert_off[id] + t0;
+      outf = L.O; out_stride = L.h; out_row0 = in_row0;
+      dep_idx = P.dep_s2 + id;
+      dep_target = groups_of(Tall, P.st[ST_V1].tg) * P.st[ST_V1].n_tiles;
       break;
   }
-  if (!s.in0l) s.planes = 1;
-  s.kc = chunk_k(s.C, s.q, s.planes * s.nB * s.T);
-  for (int t = 0; t < s.T; ++t) s.rows16[t] = (uint16_t)(in_list ? in_list[t] : in_row0 + t);
+  const int planes = in0l ? P.planes : 1;
+  const int kc = chunk_k(sc.C, sc.q, planes * nB * T);
+  uint32_t rw[8];  // rows16[0..15], two per word
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    const int ta = 2 * w, tb = 2 * w + 1;
+    const uint32_t ra = (ta < T) ? (uint32_t)(in_list ? in_list[ta] : in_row0 + ta) : 0u;
+    const uint32_t rb = (tb < T) ? (uint32_t)(in_list ? in_list[tb] : in_row0 + tb) : 0u;
+    rw[w] = (ra & 0xffffu) | (rb << 16);
+  }
+  auto ptr2 = [](const void* a, const void* b) {
+    const unsigned long long x = reinterpret_cast<unsigned long long>(a), y = reinterpret_cast<unsigned long long>(b);
+    return make_int4((int)(x & 0xffffffffull), (int)(x >> 32), (int)(y & 0xffffffffull), (int)(y >> 32));
+  };
+  int4* o = reinterpret_cast<int4*>(&dst);
+  o[0] = make_int4(item0, sc.items_per_seg, stage, sc.epi);
+  o[1] = make_int4(T, sc.q, sc.paired, nB);
+  o[2] = make_int4(kc, sc.C, sc.rows, sc.n_tiles);
+  o[3] = make_int4(in_stride, out_stride, out_row0, dep_idx);
+  o[4] = make_int4(dep_target, done_idx, planes, 0);
+  o[5] = ptr2(sc.w0 + (size_t)id * sc.unit_elems, sc.w1 ? sc.w1 + (size_t)id * sc.unit_elems : nullptr);
+  o[6] = ptr2(in0h, in0l);
+  o[7] = ptr2(in1h, in1l);
+  o[8] = ptr2(outh, outl);
+  o[9] = ptr2(outf, nullptr);
+  o[10] = make_int4((int)rw[0], (int)rw[1], (int)rw[2], (int)rw[3]);
+  o[11] = make_int4((int)rw[4], (int)rw[5], (int)rw[6], (int)rw[7]);
+  o[12] = make_int4(0, 0, 0, 0);
+  o[13] = make_int4(0, 0, 0, 0);
 }
 
 static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stage, int id, int gi, int B,
                                  int seg_index, int item0) {
-  Seg s;
-  build_seg(L, P, stage, id, gi, B, item0, s);
-  if (seg_index < P.max_segs) P.segs[seg_index] = s;
+  if (seg_index < P.max_segs) build_seg(L, P, stage, id, gi, B, item0, P.segs[seg_index]);
 }
 
-constexpr int BUILD_THREADS = 32 * MAX_CAT;
-
-// Body of the work-list construction for one CTA of at least BUILD_THREADS threads.
-static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B) {
-  __shared__ int s_nseg[MAX_CAT], s_segbase[MAX_CAT + 1], s_itembase[MAX_CAT + 1];
+// Work-list construction by one CTA (any multiple of 32 threads, at most 1024).  One thread per
+// unit (department / expert / shared expert) of every category: the units are numbered
+// category after category, a block-wide exclusive scan of their token-group counts gives each
+// unit the index of its first segment record, and the thread writes the unit's records.
+// `s_excl` is shared-memory scratch for one int per unit (at most 2 m + 2 n + 2 of them).
+static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B, int* s_excl) {
+  __shared__ int s_ubase[MAX_CAT + 1], s_segbase[MAX_CAT + 1], s_itembase[MAX_CAT + 1], s_wsum[32], s_carry;
   CatInfo cats[MAX_CAT];
   const int ncat = category_list(L, P, cats);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int i = threadIdx.x; i < P.n_dep + MAX_CAT + 8; i += blockDim.x) P.sync[SY_CLAIM + i] = 0;
-  if (warp < ncat) {
-    const int stage = cats[warp].stage, kind = cats[warp].unit_kind;
-    const int U = unit_count(L, kind);
-    int cnt = 0;
-    for (int u = lane; u < U; u += 32)
-      cnt += groups_of(unit_tokens(L, stage, unit_id(L, kind, u), B), P.st[stage].tg);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    if (lane == 0) s_nseg[warp] = cnt;
+  const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
+#pragma unroll 1
+  for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
+  if (tid == 0) {
+    int ub = 0;
+#pragma unroll 1
+    for (int c = 0; c < ncat; ++c) { s_ubase[c] = ub; ub += unit_count(L, cats[c].unit_kind); }
+    s_ubase[ncat] = ub;
+    s_carry = 0;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int sb = 0, ib = 0;
+  const int total = s_ubase[ncat];
+  auto category_of = [&](int flat) {
+    int c = 0;
+#pragma unroll 1
+    for (int q2 = 1; q2 < ncat; ++q2)
+      if (flat >= s_ubase[q2]) c = q2;
+    return c;
+  };
+  // pass 1: exclusive scan of the group counts over all units
+#pragma unroll 1
+  for (int base = 0; base < total; base += nthr) {
+    const int flat = base + tid;
+    int gc = 0;
+    if (flat < total) {
+      const int c = category_of(flat);
+      const int stage = cats[c].stage;
+      gc = groups_of(unit_tokens(L, stage, unit_id(L, cats[c].unit_kind, flat - s_ubase[c]), B), P.st[stage].tg);
+    }
+    int incl = gc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int w = (lane < nwarp) ? s_wsum[lane] : 0;
+      int wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += v;
+      }
+      s_wsum[lane] = wi - w;  // exclusive offset of warp `lane`
+      if (lane == 31) s_excl[total] = wi;  // chunk total, parked after the units
+    }
+    __syncthreads();
+    const int carry = s_carry;
+    if (flat < total) s_excl[flat] = carry + s_wsum[warp] + incl - gc;
+    __syncthreads();
+    if (tid == 0) s_carry = carry + s_excl[total];
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const int nseg = s_carry;
+    int ib = 0;
+#pragma unroll 1
     for (int c = 0; c < ncat; ++c) {
-      s_segbase[c] = sb; s_itembase[c] = ib;
+      const int sb = (s_ubase[c] < total) ? s_excl[s_ubase[c]] : nseg;
+      const int sb_next = (c + 1 < ncat && s_ubase[c + 1] < total) ? s_excl[s_ubase[c + 1]] : nseg;
       const int ips = P.st[cats[c].stage].items_per_seg;
+      s_segbase[c] = sb; s_itembase[c] = ib;
       P.sync[SY_CAT + 4 * c + 0] = ib;
       P.sync[SY_CAT + 4 * c + 1] = sb;
       P.sync[SY_CAT + 4 * c + 2] = ips;
       P.sync[SY_CAT + 4 * c + 3] = cats[c].stage;
-      sb += s_nseg[c];
-      ib += s_nseg[c] * ips;
+      ib += (sb_next - sb) * ips;
     }
-    s_segbase[ncat] = sb; s_itembase[ncat] = ib;
+#pragma unroll 1
     for (int c = ncat; c < MAX_CAT; ++c) {
       P.sync[SY_CAT + 4 * c + 0] = ib;
-      P.sync[SY_CAT + 4 * c + 1] = sb;
+      P.sync[SY_CAT + 4 * c + 1] = nseg;
       P.sync[SY_CAT + 4 * c + 2] = 1;
       P.sync[SY_CAT + 4 * c + 3] = -1;
     }
-    P.sync[SY_NCAT] = ncat; P.sync[SY_NSEG] = sb; P.sync[SY_NITEMS] = ib;
-    L.counts[CNT_NSEG] = sb; L.counts[CNT_NITEMS] = ib;
-    if (sb > P.max_segs) L.counts[CNT_STATUS] = DEAMOE_ERR_UNSUPPORTED;
+    P.sync[SY_NCAT] = ncat; P.sync[SY_NSEG] = nseg; P.sync[SY_NITEMS] = ib;
+    L.counts[CNT_NSEG] = nseg; L.counts[CNT_NITEMS] = ib;
+    if (nseg > P.max_segs) L.counts[CNT_STATUS] = DEAMOE_ERR_UNSUPPORTED;
   }
   __syncthreads();
-  if (warp < ncat) {
-    const int stage = cats[warp].stage, kind = cats[warp].unit_kind;
-    const int U = unit_count(L, kind);
+  TS_MIN(L, 14);
+  // pass 2: every unit's records
+#pragma unroll 1
+  for (int flat = tid; flat < total; flat += nthr) {
+    const int c = category_of(flat);
+    const int stage = cats[c].stage;
+    const int id = unit_id(L, cats[c].unit_kind, flat - s_ubase[c]);
+    const int gc = groups_of(unit_tokens(L, stage, id, B), P.st[stage].tg);
     const int ips = P.st[stage].items_per_seg;
-    int running = 0;
-    for (int base = 0; base < U; base += 32) {
-      const int u = base + lane;
-      const int id = (u < U) ? unit_id(L, kind, u) : 0;
-      const int gc = (u < U) ? groups_of(unit_tokens(L, stage, id, B), P.st[stage].tg) : 0;
-      int incl = gc;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      const int first = running + incl - gc;
-      for (int gi = 0; gi < gc; ++gi) {
-        const int si = s_segbase[warp] + first + gi;
-        write_seg(L, P, stage, id, gi, B, si, s_itembase[warp] + (first + gi) * ips);
-      }
-      running += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll 1
+    for (int gi = 0; gi < gc; ++gi) {
+      const int si = s_excl[flat] + gi;
+      write_seg(L, P, stage, id, gi, B, si, s_itembase[c] + (si - s_segbase[c]) * ips);
     }
   }
-}
-
-__global__ void __launch_bounds__(BUILD_THREADS) k_build_worklist(LayerDev L, StreamDev P, int B) {
-  worklist_block(L, P, B);
 }
 
 // Routing tail in one CTA: top-k + gate weights (warp per token), bucketing, work list.  The
@@ -532,21 +593,14 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 11);
 #endif
   for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) S.counts[i] = 0;
-  const bool regs_ok = (L.k_dept <= 0 || L.k_dept >= L.m) && L.n <= 512 &&
-                       (kslices == 1 || kslices == 2 || kslices == 4 || kslices == 8 || kslices == 16);
+  const bool regs_ok = (L.k_dept <= 0 || L.k_dept >= L.m) && L.n <= 512;
   if (warp < topk_warps) {
     const int per_warp = (L.n * 5 + 15) & ~15;  // n fp32 logits + n flag bytes (memory path only)
     unsigned char* base = reinterpret_cast<unsigned char*>(s_dyn) + (size_t)warp * per_warp;
+#pragma unroll 1
     for (int t = warp; t < B; t += topk_warps) {
-#define DEAMOE_TOPK(VPL, KS) topk_one_token_regs<VPL, KS>(S, t, B, lane, user_idx, user_w)
-      if (regs_ok && L.n <= 256) {
-        if (kslices == 16) DEAMOE_TOPK(8, 16); else if (kslices == 8) DEAMOE_TOPK(8, 8); else if (kslices == 4) DEAMOE_TOPK(8, 4);
-        else if (kslices == 2) DEAMOE_TOPK(8, 2); else DEAMOE_TOPK(8, 1);
-      } else if (regs_ok) {
-        if (kslices == 16) DEAMOE_TOPK(16, 16); else if (kslices == 8) DEAMOE_TOPK(16, 8); else if (kslices == 4) DEAMOE_TOPK(16, 4);
-        else if (kslices == 2) DEAMOE_TOPK(16, 2); else DEAMOE_TOPK(16, 1);
-      }
-#undef DEAMOE_TOPK
+      if (regs_ok && L.n <= 256) topk_one_token_regs<8>(S, t, B, kslices, lane, user_idx, user_w);
+      else if (regs_ok) topk_one_token_regs<16>(S, t, B, kslices, lane, user_idx, user_w);
       else topk_one_token(S, t, B, kslices, reinterpret_cast<float*>(base), base + (size_t)L.n * 4, lane, user_idx, user_w);
     }
   }
@@ -561,22 +615,39 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   long long tt2 = clock64();
   TS_MIN(L, 13);
 #endif
-  worklist_block(S, P, B);
+  worklist_block(S, P, B, reinterpret_cast<int*>(s_dyn));
   __syncthreads();
-  // publish the routing state
-  const int pk = B * L.k;
-  for (int i = tid; i < pk; i += FINISH_THREADS) {
-    L.topk_idx[i] = S.topk_idx[i]; L.topk_w[i] = S.topk_w[i];
-    L.expert_tok[i] = S.expert_tok[i]; L.pair_slot[i] = S.pair_slot[i]; L.pair_gurow[i] = S.pair_gurow[i];
+  TS_MIN(L, 15);
+  // publish the routing state: every array is a run of 32-bit words in the shared-memory copy.
+  // One rolled loop over a small table, so that this once-per-step code stays short.
+  __shared__ uint32_t* s_dst[12];
+  __shared__ int s_src[12], s_cnt[12];
+  if (tid == 0) {
+    const int pk = B * L.k;
+    int e = 0;
+    auto add = [&](void* dst, int src, int cnt) { s_dst[e] = reinterpret_cast<uint32_t*>(dst); s_src[e] = src; s_cnt[e] = cnt; ++e; };
+    add(L.topk_idx, fl.idx, pk);
+    add(L.topk_w, fl.w, pk);
+    add(L.expert_tok, fl.expert_tok, pk);
+    add(L.pair_slot, fl.pair_slot, pk);
+    add(L.pair_gurow, fl.pair_gurow, pk);
+    add(L.dept_tok, fl.dept_tok, S.counts[CNT_TOKEN_DEPT]);
+    add(L.dept_off, fl.dept_off, L.m + 1);
+    add(L.expert_off, fl.expert_off, L.n + 1);
+    add(L.active_dept, fl.active_dept, L.m);
+    add(L.active_expert, fl.active_expert, L.n);
+    add(L.dept_mask, fl.dept_mask, 2 * ((L.m + 63) / 64));
+    add(L.counts, fl.counts, CNT_COUNT);
   }
-  const int ntd = S.counts[CNT_TOKEN_DEPT];
-  for (int i = tid; i < ntd; i += FINISH_THREADS) L.dept_tok[i] = S.dept_tok[i];
-  for (int i = tid; i <= L.m; i += FINISH_THREADS) L.dept_off[i] = S.dept_off[i];
-  for (int i = tid; i <= L.n; i += FINISH_THREADS) L.expert_off[i] = S.expert_off[i];
-  for (int i = tid; i < L.m; i += FINISH_THREADS) L.active_dept[i] = S.active_dept[i];
-  for (int i = tid; i < L.n; i += FINISH_THREADS) L.active_expert[i] = S.active_expert[i];
-  for (int i = tid; i < (L.m + 63) / 64; i += FINISH_THREADS) L.dept_mask[i] = S.dept_mask[i];
-  for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) L.counts[i] = S.counts[i];
+  __syncthreads();
+#pragma unroll 1
+  for (int e = 0; e < 12; ++e) {
+    uint32_t* dst = s_dst[e];
+    const uint32_t* src = state + s_src[e];
+    const int cnt = s_cnt[e];
+#pragma unroll 1
+    for (int i = tid; i < cnt; i += FINISH_THREADS) dst[i] = src[i];
+  }
 #ifdef DEAMOE_TRACE
   __syncthreads();
   TS_MAX(L, 4);
@@ -786,7 +857,6 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     }
 
     pdl_wait();  // the work list is written by the preceding routing kernel
-    TS_MIN(L, 6);
     cat_tab[lane] = sy[SY_CAT + lane];  // 4 * MAX_CAT == 32 entries
     __syncwarp();
     // item range of this launch: one category (staged) or everything (fused)
@@ -881,6 +951,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     const uint64_t pol = policy_evict_first();
     int e = 0;
     int cidx = 0;  // index of the item's first chunk in the CTA's chunk stream
+#ifdef DEAMOE_TRACE
+    bool routed_seen = false;
+#endif
     uint32_t eph = 0;
     bool ok = true;
     long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -896,6 +969,13 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       const int* tail = reinterpret_cast<const int*>(ent + DESC_TAIL);
       if (tail[0] != 0) break;
       const long long td0 = TR_NOW();
+#ifdef DEAMOE_TRACE
+      if (ip == 0 && lane == 0 && !routed_seen && sg->stage != ST_SH1 && sg->stage != ST_SH2 && L.ts) {
+        routed_seen = true;
+        const unsigned long long g = gtime();
+        atomicMin(L.ts + 6, g); atomicMax(L.ts + 16, g);
+      }
+#endif
       if (tail[2]) fence_proxy_async();
       const int tile0 = tail[1], q_eff = tail[3], nrows = tail[4];
       const int T = sg->T, kc0 = sg->kc, C = sg->C;
@@ -1386,11 +1466,6 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
-int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
-  k_build_worklist<<<1, BUILD_THREADS, 0, s>>>(L, p.dev, B);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
-}
-
 // category order as built by category_list(), host copy
 static int host_categories(const LayerDev& L, int* stages) {
   int n = 0;
@@ -1502,7 +1577,7 @@ __global__ void k_split_tokens(const float* __restrict__ x, __nv_bfloat16* __res
 // Trace builds only: copy the per-CTA cycle counters of the last k_stream launch to the host.
 namespace deamoe {
 int stream_read_trace(StreamPlan& p, long long* host, int max_ctas) {
-  const int n = p.n_sm < max_ctas ? p.n_sm : max_ctas;
+  const int n = p.grid < max_ctas ? p.grid : max_ctas;
   cudaDeviceSynchronize();
   cudaMemcpy(host, p.dev.trace, (size_t)n * TR_SLOTS * sizeof(long long), cudaMemcpyDeviceToHost);
   return n;

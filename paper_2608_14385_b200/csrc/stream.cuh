@@ -24,10 +24,6 @@ int32_t* stream_shared_counter(StreamPlan& p);
 int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
                  int32_t* user_idx, float* user_w);
 
-// Enqueue the work-list construction for the routing state already on the device.
-// Returns the number of kernels launched or -1.
-int stream_build_worklist(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
-
 // Enqueue all stages of one step.  Returns the number of kernels launched or -1.
 int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
 
