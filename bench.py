@@ -187,7 +187,7 @@ def run_reference(args, shape, rank, world):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of k_stream divided by its algorithmic bytes, from
 # the committed ncu capture (profiles/k_stream_dsv3-mini_b4.md)
-DRAM_TRAFFIC_RATIO = 1.004
+DRAM_TRAFFIC_RATIO = 1.001
 
 
 def stream_kernel_ms(layer, batches, steps, flush, torch):
