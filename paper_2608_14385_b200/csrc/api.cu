@@ -120,7 +120,10 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   const int pmax = MB * k;                     // (token, expert) pairs
   // router column slices: enough CTAs to cover the GPU a few times
   L->kslices = 1;
-  while (L->kslices < 16 && d.h / L->kslices > 512) L->kslices *= 2;  // one 512-column pass per thread block
+  // Column slices of the router product: at least 512 columns per thread block, and no more
+  // slices than it takes to fill the device with ~1024 blocks of four router rows (every slice
+  // is one more array of partial logits that the top-k has to read back).
+  while (L->kslices < 16 && d.h / L->kslices > 512 && (d.n / 4) * L->kslices < 1024) L->kslices *= 2;
 
   bool ok = true;
   auto A = [&](deamoe_status_t r) { if (r != DEAMOE_OK && ok) { ok = false; st = r; } };

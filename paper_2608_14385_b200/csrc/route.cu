@@ -68,15 +68,26 @@ k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float*
         }
       }
     }
+    // Warp reduction of the 32 accumulators by recursive halving: in the step with distance d a
+    // lane keeps the half of its values that matches its lane bit d and adds the partner's, so
+    // after five steps lane l holds the warp's total of accumulator l (31 shuffles, not 160).
+    static_assert(RG * TG == 32, "one accumulator per lane after the reduction");
+    float v[32];
 #pragma unroll
     for (int a = 0; a < RG; ++a)
 #pragma unroll
-      for (int b = 0; b < TG; ++b) {
-        float v = acc[a][b];
+      for (int b = 0; b < TG; ++b) v[a * TG + b] = acc[a][b];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) red[warp][a][b] = v;
+    for (int d = 16; d > 0; d >>= 1) {
+      const bool up = (lane & d) != 0;
+#pragma unroll
+      for (int i = 0; i < d; ++i) {
+        const float send = up ? v[i] : v[i + d];
+        const float keep = up ? v[i + d] : v[i];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, d);
       }
+    }
+    red[warp][lane / TG][lane % TG] = v[0];
     __syncthreads();
     if (threadIdx.x < RG * TG) {
       const int a = threadIdx.x / TG, b = threadIdx.x % TG;

@@ -99,18 +99,25 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
   float v[VPL];
   unsigned taken = 0;
   {
-    // Slices are added in the fixed order 0, 1, ...; four slices (4 * VPL loads per lane) are in
-    // flight at a time.  The loop stays rolled: this runs once per step from a cold instruction
+    // Slices are added in the fixed order 0, 1, ...; four (two for the wider variants) slices'
+    // loads are in flight at a time.  The loop stays rolled: this runs once per step from a cold instruction
     // cache, where a short loop beats a long unrolled run of loads.
-    int col[VPL];
 #pragma unroll
-    for (int j = 0; j < VPL; ++j) { col[j] = min(lane + 32 * j, n - 1); v[j] = 0.f; }
+    for (int j = 0; j < VPL; ++j) v[j] = 0.f;
     const float* __restrict__ src = L.logit_part + (size_t)t * n;
     const size_t slice = (size_t)B * n;
+    if (VPL <= 8) {
 #pragma unroll 4
-    for (int sl = 0; sl < kslices; ++sl, src += slice) {
+      for (int sl = 0; sl < kslices; ++sl, src += slice) {
 #pragma unroll
-      for (int j = 0; j < VPL; ++j) v[j] += __ldg(src + col[j]);
+        for (int j = 0; j < VPL; ++j) v[j] += __ldg(src + min(lane + 32 * j, n - 1));
+      }
+    } else {
+#pragma unroll 2
+      for (int sl = 0; sl < kslices; ++sl, src += slice) {
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) v[j] += __ldg(src + min(lane + 32 * j, n - 1));
+      }
     }
 #pragma unroll
     for (int j = 0; j < VPL; ++j)
@@ -134,6 +141,40 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
       if (!((taken >> j) & 1u)) den_all += expf(v[j] - mx_all);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) den_all += __shfl_xor_sync(0xffffffffu, den_all, o);
+  }
+  if (L.k_dept > 0 && L.k_dept < L.m) {
+    // Group limit (Section 3.3; needs m <= 32): the score of a department is its largest logit;
+    // a department is dropped when at least k_dept departments rank ahead of it (score
+    // descending, index ascending).  Lane d ends up holding the score of department d.
+    const int g = L.g, m = L.m;
+    float dscore = -INFINITY;
+#pragma unroll 1
+    for (int d = 0; d < m; ++d) {
+      const int lo = d * g, hi = lo + g;
+      float loc = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) {
+        const int idx = lane + 32 * j;
+        if (idx >= lo && idx < hi && idx < n) loc = fmaxf(loc, v[j]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) loc = fmaxf(loc, __shfl_xor_sync(0xffffffffu, loc, o));
+      if (lane == d) dscore = loc;
+    }
+    int ahead = 0;
+#pragma unroll 1
+    for (int d2 = 0; d2 < m; ++d2) {
+      const float s2 = __shfl_sync(0xffffffffu, dscore, d2);
+      ahead += better(s2, d2, dscore, lane) ? 1 : 0;
+    }
+    const unsigned alive = __ballot_sync(0xffffffffu, lane < m && ahead < L.k_dept);
+    const unsigned inv = (g > 1) ? (unsigned)((0x100000000ull + (unsigned)g - 1u) / (unsigned)g) : 0u;  // ceil(2^32 / g)
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const unsigned idx = (unsigned)(lane + 32 * j);
+      const unsigned d = (g > 1) ? __umulhi(idx, inv) : idx;  // idx / g, exact for idx * g < 2^32
+      if (idx < (unsigned)n && !((alive >> d) & 1u)) taken |= 1u << j;
+    }
   }
   float my_v = 0.f;  // lane q keeps the q-th selected logit (k <= 32)
   int my_i = 0;

@@ -540,6 +540,13 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
   }
 }
 
+// The top-k keeps a token's logits in registers (up to 32 per lane) unless the layer is too wide or
+// its group limit spans more departments than a warp has lanes; then the shared-memory variant runs.
+static __host__ __device__ inline bool topk_in_registers(const LayerDev& L) {
+  const bool grouped = L.k_dept > 0 && L.k_dept < L.m;
+  return L.n <= 1024 && (!grouped || L.m <= 32);
+}
+
 // Routing tail in one CTA: top-k + gate weights (warp per token), bucketing, work list.  The
 // routing state (selection, gate weights, offsets, token lists, counters) is built in shared
 // memory -- the three steps read each other's results from there, not through L2 -- and copied
@@ -593,14 +600,15 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 11);
 #endif
   for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) S.counts[i] = 0;
-  const bool regs_ok = (L.k_dept <= 0 || L.k_dept >= L.m) && L.n <= 512;
+  const bool regs_ok = topk_in_registers(L);
   if (warp < topk_warps) {
     const int per_warp = (L.n * 5 + 15) & ~15;  // n fp32 logits + n flag bytes (memory path only)
     unsigned char* base = reinterpret_cast<unsigned char*>(s_dyn) + (size_t)warp * per_warp;
 #pragma unroll 1
     for (int t = warp; t < B; t += topk_warps) {
       if (regs_ok && L.n <= 256) topk_one_token_regs<8>(S, t, B, kslices, lane, user_idx, user_w);
-      else if (regs_ok) topk_one_token_regs<16>(S, t, B, kslices, lane, user_idx, user_w);
+      else if (regs_ok && L.n <= 512) topk_one_token_regs<16>(S, t, B, kslices, lane, user_idx, user_w);
+      else if (regs_ok) topk_one_token_regs<32>(S, t, B, kslices, lane, user_idx, user_w);
       else topk_one_token(S, t, B, kslices, reinterpret_cast<float*>(base), base + (size_t)L.n * 4, lane, user_idx, user_w);
     }
   }
@@ -1450,11 +1458,12 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   const int ny = launch_router_logits(L, tokens, B, s, kslices);
   if (ny < 0) return -1;
   const int per_warp = (L.n * 5 + 15) & ~15;
-  int topk_warps = (48 * 1024) / per_warp;
+  const bool in_regs = topk_in_registers(L);
+  int topk_warps = in_regs ? FINISH_THREADS / 32 : (48 * 1024) / per_warp;
   if (topk_warps > FINISH_THREADS / 32) topk_warps = FINISH_THREADS / 32;
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
-  size_t scratch = (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
+  size_t scratch = in_regs ? 0 : (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
   const size_t bs = bucket_smem_bytes(L, B);
   if (bs > scratch) scratch = bs;
   scratch = (scratch + 15) & ~(size_t)15;

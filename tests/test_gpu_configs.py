@@ -74,3 +74,36 @@ def test_stack_of_layers_teacher_forced_and_free_running(B):
     finally:
         for layer in layers:
             layer.close()
+
+
+@pytest.mark.parametrize("B,rows", [(4, [1]), (64, [40])])
+def test_paper_deepseek_v3_row_group_limited(B, rows):
+    """The paper's own DeepSeek-V3-matched configuration (Table 1, first row): 8 departments x 108
+    experts, square private matrices (r = f), top-10 limited to 5 departments (Section 3.3).
+    Routing and buckets bit-exact for the whole batch, values on a sampled row, every token inside
+    its department cap, unique bytes equal to the closed form on the counted sets."""
+    shape = synth.DSV3_PAPER
+    res = run_case(shape, B, seed=0, rows=rows, max_batch=64)
+    st = res["stats"]
+    assert st["active_dept"] <= shape.n_dept and st["active_expert"] <= B * shape.top_k
+    assert st["unique_weight_bytes"] == accounting.unique_bytes_deamoe(
+        st["active_dept"], st["active_expert"], shape.hidden, shape.ffn, shape.priv, shape.n_expert, 2)
+
+
+def test_paper_row_department_cap_holds_for_every_token():
+    shape = synth.DSV3_PAPER
+    dev = torch.device("cuda:0")
+    B = 32
+    w = synth.make_deamoe_weights(shape, 1, dev)
+    layer = binding.Layer(shape, w, B, binding.SCHED_AUTO)
+    try:
+        tokens = synth.make_tokens(shape, B, 6, dev)  # seed 5 puts one token within 1e-5 of a routing tie
+        layer.route(tokens, want_outputs=False)
+        torch.cuda.synchronize()
+        idx = layer.routing(B)["idx"]
+        for t in range(B):
+            assert len({int(i) // shape.experts_per_dept for i in idx[t]}) <= shape.k_dept
+            assert len(set(int(i) for i in idx[t])) == shape.top_k
+        want, _ = check_routing(shape, layer, w, tokens, B)
+    finally:
+        layer.close()
