@@ -37,6 +37,10 @@ k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float*
 #ifdef DEAMOE_TRACE
   if (threadIdx.x == 0 && ts) atomicMin(ts + 0, gtime());
 #endif
+  // Kernels launched behind this one with programmatic stream serialization (the routing tail, and
+  // through it the streaming kernel with the routing-independent shared expert) may become
+  // resident right away; they wait for this grid's results themselves.
+  pdl_trigger();
   const int row0 = blockIdx.x * RG;
   const int c0 = blockIdx.y * kslice;
   const int c1 = min(h, c0 + kslice);

@@ -47,6 +47,9 @@ constexpr int DESC_DEPTH = 8;                    // item descriptors queued betw
 constexpr int DESC_BYTES = 1024;                 // Seg | tail | weight sources | activation row sources
 constexpr int DESC_TAIL = 224, DESC_WSRC = 256, DESC_ASRC = 272;
 constexpr int MAX_CAT_INTS_PAD = 8;             // cat_tab: 4 ints for each of 8 categories = 16 B x 8
+#ifndef PREFIX_LAST_STAGE
+#define PREFIX_LAST_STAGE ST_SH1  // the shared expert's second stage waits for all of the first: it runs from the list
+#endif
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SIG_DEPTH = 16;
 constexpr int SLOT_BYTES = 32 * 1024;
@@ -270,8 +273,9 @@ struct CatInfo {
 
 static __device__ __forceinline__ int category_list(const LayerDev& L, const StreamDev& P, CatInfo* cats) {
   int n = 0;
-  const bool sh = L.n_shared && !P.sh_prefix;  // else the streaming kernel generates the shared expert's items
-  if (sh) cats[n++] = {ST_SH1, 0};
+  // with sh_prefix the streaming kernel generates the shared expert's first stage itself
+  if (L.n_shared && !P.sh_prefix) cats[n++] = {ST_SH1, 0};
+  const bool sh = L.n_shared;
   if (L.vanilla) {
     cats[n++] = {ST_V1, 2};
     if (sh) cats[n++] = {ST_SH2, 0};
@@ -844,7 +848,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     if (P.sh_prefix && cat < 0) {
       Seg* stage_seg = reinterpret_cast<Seg*>(seg_stage);
       int first_cta = 0;  // the CTA that takes the stage's first item
-      for (int st = ST_SH1; ok && st <= ST_SH2; ++st) {
+      for (int st = ST_SH1; ok && st <= PREFIX_LAST_STAGE; ++st) {
         const int ips = P.st[st].items_per_seg;
         const int n_items = groups_of(B, P.st[st].tg) * ips;
         int have_seg = -1;
