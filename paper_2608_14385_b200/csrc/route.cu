@@ -125,10 +125,7 @@ __global__ void __launch_bounds__(BUCKET_THREADS) k_bucket(LayerDev L, int B) {
   bucket_block(L, B, s_bucket, BUCKET_THREADS);
 }
 
-size_t bucket_smem_bytes(const LayerDev& L, int B) {
-  const int W = (B + 31) / 32;
-  return ((size_t)(L.n + L.m) * W + (size_t)L.n + L.m + (L.n + 1) + (L.m + 1)) * sizeof(uint32_t);
-}
+size_t bucket_smem_bytes(const LayerDev& L, int B) { return bucket_smem_words(L.n, L.m, B) * sizeof(uint32_t); }
 
 cudaError_t route_configure(const LayerDev& L) {
   // the bucketing kernel may need more than the default 48 KB of dynamic shared memory

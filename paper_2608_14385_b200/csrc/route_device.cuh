@@ -246,18 +246,41 @@ static __device__ __forceinline__ int warp_exclusive_offsets(const int* cnt, int
   return run;
 }
 
-// Body of the bucketing step for one CTA of `nthr` threads (a multiple of 64); s_u32: bucket_smem_bytes().
-// Executed once per step by one CTA, usually with a cold instruction cache: the loops are kept
-// rolled so that the code stays small.
-static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, int nthr) {
-  const int n = L.n, m = L.m, g = L.g, k = L.k;
+// Bucketing for one CTA of `nthr` threads (a multiple of 64); s_u32: bucket_smem_bytes() of shared
+// memory that must stay untouched between the two parts.  Executed once per step by one CTA,
+// usually with a cold instruction cache: the loops are kept rolled so that the code stays small.
+//
+// Part 1, departments: membership bit masks of tokens per expert and per department (atomicOr),
+// department counts, active-department mask (warp ballot) and list, CSR offsets (warp scan) and
+// the ascending token list X^j of every department.  This is all the first stage of the layer
+// needs, so a caller may hand that stage its work before running part 2.
+// 32-bit words of shared memory the bucketing needs
+static __host__ __device__ inline size_t bucket_smem_words(int n, int m, int B) {
   const int W = (B + 31) / 32;
-  uint32_t* emask = s_u32;                    // [n][W]
-  uint32_t* dmask = emask + (size_t)n * W;    // [m][W]
-  int* ecnt = reinterpret_cast<int*>(dmask + (size_t)m * W);  // [n]
-  int* dcnt = ecnt + n;                                        // [m]
-  int* s_eoff = dcnt + m;                                      // [n+1]
-  int* s_doff = s_eoff + n + 1;                                // [m+1]
+  return (size_t)(n + m) * W + (size_t)n + m + (n + 1) + (m + 1);
+}
+
+struct BucketSmem {
+  uint32_t *emask, *dmask;
+  int *ecnt, *dcnt, *eoff, *doff;
+  int W;
+};
+static __device__ __forceinline__ BucketSmem bucket_smem(const LayerDev& L, int B, uint32_t* s_u32) {
+  BucketSmem b;
+  b.W = (B + 31) / 32;
+  b.emask = s_u32;                                            // [n][W]
+  b.dmask = b.emask + (size_t)L.n * b.W;                      // [m][W]
+  b.ecnt = reinterpret_cast<int*>(b.dmask + (size_t)L.m * b.W);  // [n]
+  b.dcnt = b.ecnt + L.n;                                      // [m]
+  b.eoff = b.dcnt + L.m;                                      // [n+1]
+  b.doff = b.eoff + L.n + 1;                                  // [m+1]
+  return b;
+}
+
+static __device__ void bucket_departments(const LayerDev& L, int B, uint32_t* s_u32, int nthr) {
+  const int n = L.n, m = L.m, g = L.g, k = L.k;
+  const BucketSmem b = bucket_smem(L, B, s_u32);
+  const int W = b.W;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 #pragma unroll 1
   for (int i = tid; i < (n + m) * W; i += nthr) s_u32[i] = 0u;
@@ -266,17 +289,10 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
   for (int p = tid; p < B * k; p += nthr) {
     const int t = p / k;
     const int i = L.topk_idx[p];
-    atomicOr(&emask[(size_t)i * W + (t >> 5)], 1u << (t & 31));
-    atomicOr(&dmask[(size_t)(i / g) * W + (t >> 5)], 1u << (t & 31));
+    atomicOr(&b.emask[(size_t)i * W + (t >> 5)], 1u << (t & 31));
+    atomicOr(&b.dmask[(size_t)(i / g) * W + (t >> 5)], 1u << (t & 31));
   }
   __syncthreads();
-#pragma unroll 1
-  for (int i = tid; i < n; i += nthr) {
-    int c = 0;
-#pragma unroll 1
-    for (int w = 0; w < W; ++w) c += __popc(emask[(size_t)i * W + w]);
-    ecnt[i] = c;
-  }
   // department counts; the active-department bitmask falls out of a warp ballot (32 departments
   // per warp iteration, written as the two 32-bit halves of the 64-bit words)
 #pragma unroll 1
@@ -284,54 +300,69 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
     int c = 0;
     if (j < m) {
 #pragma unroll 1
-      for (int w = 0; w < W; ++w) c += __popc(dmask[(size_t)j * W + w]);
-      dcnt[j] = c;
+      for (int w = 0; w < W; ++w) c += __popc(b.dmask[(size_t)j * W + w]);
+      b.dcnt[j] = c;
     }
     const unsigned live = __ballot_sync(0xffffffffu, c > 0);
     if ((tid & 31) == 0) reinterpret_cast<uint32_t*>(L.dept_mask)[j >> 5] = live;
   }
   __syncthreads();
-  if (warp == 0) {
-    warp_exclusive_offsets(dcnt, m, s_doff, L.active_dept, lane, &L.counts[CNT_ACTIVE_DEPT]);
-  } else if (warp == 1) {
-    warp_exclusive_offsets(ecnt, n, s_eoff, L.active_expert, lane, &L.counts[CNT_ACTIVE_EXPERT]);
-  }
+  if (warp == 0) warp_exclusive_offsets(b.dcnt, m, b.doff, L.active_dept, lane, &L.counts[CNT_ACTIVE_DEPT]);
   __syncthreads();
 #pragma unroll 1
-  for (int i = tid; i <= n; i += nthr) L.expert_off[i] = s_eoff[i];
-#pragma unroll 1
-  for (int j = tid; j <= m; j += nthr) L.dept_off[j] = s_doff[j];
+  for (int j = tid; j <= m; j += nthr) L.dept_off[j] = b.doff[j];
   if (tid == 0) {
     L.counts[CNT_STATUS] = 0;
-    L.counts[CNT_TOKEN_DEPT] = s_doff[m];
-    L.counts[CNT_PAIRS] = s_eoff[n];
-  }
-  // ascending token lists
-#pragma unroll 1
-  for (int i = tid; i < n; i += nthr) {
-    int pos = s_eoff[i];
-#pragma unroll 1
-    for (int w = 0; w < W; ++w) {
-      uint32_t bits = emask[(size_t)i * W + w];
-#pragma unroll 1
-      while (bits) {
-        const int b = __ffs(bits) - 1;
-        bits &= bits - 1;
-        L.expert_tok[pos++] = w * 32 + b;
-      }
-    }
+    L.counts[CNT_TOKEN_DEPT] = b.doff[m];
   }
 #pragma unroll 1
   for (int j = tid; j < m; j += nthr) {
-    int pos = s_doff[j];
+    int pos = b.doff[j];
 #pragma unroll 1
     for (int w = 0; w < W; ++w) {
-      uint32_t bits = dmask[(size_t)j * W + w];
+      uint32_t bits = b.dmask[(size_t)j * W + w];
 #pragma unroll 1
       while (bits) {
-        const int b = __ffs(bits) - 1;
+        const int bb = __ffs(bits) - 1;
         bits &= bits - 1;
-        L.dept_tok[pos++] = w * 32 + b;
+        L.dept_tok[pos++] = w * 32 + bb;
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// Part 2, experts: counts, active list, CSR offsets and ascending token lists per expert, the slot
+// of every (token, expert) pair in expert-major order and the department row each pair reads.
+static __device__ void bucket_experts(const LayerDev& L, int B, uint32_t* s_u32, int nthr) {
+  const int n = L.n, g = L.g, k = L.k;
+  const BucketSmem b = bucket_smem(L, B, s_u32);
+  const int W = b.W;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll 1
+  for (int i = tid; i < n; i += nthr) {
+    int c = 0;
+#pragma unroll 1
+    for (int w = 0; w < W; ++w) c += __popc(b.emask[(size_t)i * W + w]);
+    b.ecnt[i] = c;
+  }
+  __syncthreads();
+  if (warp == 0) warp_exclusive_offsets(b.ecnt, n, b.eoff, L.active_expert, lane, &L.counts[CNT_ACTIVE_EXPERT]);
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i <= n; i += nthr) L.expert_off[i] = b.eoff[i];
+  if (tid == 0) L.counts[CNT_PAIRS] = b.eoff[n];
+#pragma unroll 1
+  for (int i = tid; i < n; i += nthr) {
+    int pos = b.eoff[i];
+#pragma unroll 1
+    for (int w = 0; w < W; ++w) {
+      uint32_t bits = b.emask[(size_t)i * W + w];
+#pragma unroll 1
+      while (bits) {
+        const int bb = __ffs(bits) - 1;
+        bits &= bits - 1;
+        L.expert_tok[pos++] = w * 32 + bb;
       }
     }
   }
@@ -344,16 +375,21 @@ static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, i
     int re = 0, rd = 0;
 #pragma unroll 1
     for (int w = 0; w < (t >> 5); ++w) {
-      re += __popc(emask[(size_t)i * W + w]);
-      rd += __popc(dmask[(size_t)j * W + w]);
+      re += __popc(b.emask[(size_t)i * W + w]);
+      rd += __popc(b.dmask[(size_t)j * W + w]);
     }
     const uint32_t below = (1u << (t & 31)) - 1u;
-    re += __popc(emask[(size_t)i * W + (t >> 5)] & below);
-    rd += __popc(dmask[(size_t)j * W + (t >> 5)] & below);
-    const int slot = s_eoff[i] + re;
+    re += __popc(b.emask[(size_t)i * W + (t >> 5)] & below);
+    rd += __popc(b.dmask[(size_t)j * W + (t >> 5)] & below);
+    const int slot = b.eoff[i] + re;
     L.pair_slot[p] = slot;
-    L.pair_gurow[slot] = s_doff[j] + rd;
+    L.pair_gurow[slot] = b.doff[j] + rd;
   }
+}
+
+static __device__ void bucket_block(const LayerDev& L, int B, uint32_t* s_u32, int nthr) {
+  bucket_departments(L, B, s_u32, nthr);
+  bucket_experts(L, B, s_u32, nthr);
 }
 
 

@@ -118,6 +118,8 @@ struct StreamDev {
   int max_segs;
   int dep_s1, dep_s2, dep_s3, dep_sh1, n_dep;  // offsets relative to SY_DEP
   int sh_prefix;  // fused schedule with a shared expert: its items are not in the work list
+  int early;      // fused DeaMoE layers: the first stage's records are handed over ahead of the rest
+  int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): step number, item count
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
   // activations between stages, bf16 planes ([rows, width] each)
   __nv_bfloat16 *xh, *xl;      // tokens split (fp32 activations only; bf16 tokens are read in place)
@@ -140,6 +142,7 @@ struct StreamPlan {
   int schedule;
   int n_sm;
   int grid;  // CTAs of the streaming kernel: all of them must be resident at once
+  int epoch; // number of the last routing call (never 0): tags the early hand-over flag
   void* packed;
   uint64_t bytes;
   cudaEvent_t ev0, ev1;   // profiling event pair (null when profiling is off)
@@ -216,6 +219,9 @@ static __device__ __forceinline__ void bulk_g2s_hint(void* dst, const void* src,
       : "memory");
 }
 static __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+static __device__ __forceinline__ void st_release(int32_t* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 static __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -441,13 +447,14 @@ static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stag
 // category after category, a block-wide exclusive scan of their token-group counts gives each
 // unit the index of its first segment record, and the thread writes the unit's records.
 // `s_excl` is shared-memory scratch for one int per unit (at most 2 m + 2 n + 2 of them).
-static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B, int* s_excl) {
+static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B, int* s_excl, bool early_done) {
   __shared__ int s_ubase[MAX_CAT + 1], s_segbase[MAX_CAT + 1], s_itembase[MAX_CAT + 1], s_wsum[32], s_carry;
   CatInfo cats[MAX_CAT];
   const int ncat = category_list(L, P, cats);
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
 #pragma unroll 1
-  for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
+  if (!early_done)  // else early_first_stage() has zeroed the counters, and the first stage may be running
+    for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
   if (tid == 0) {
     int ub = 0;
 #pragma unroll 1
@@ -532,6 +539,7 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
 #pragma unroll 1
   for (int flat = tid; flat < total; flat += nthr) {
     const int c = category_of(flat);
+    if (early_done && c == 0) continue;  // written, with the same numbering, by early_first_stage()
     const int stage = cats[c].stage;
     const int id = unit_id(L, cats[c].unit_kind, flat - s_ubase[c]);
     const int gc = groups_of(unit_tokens(L, stage, id, B), P.st[stage].tg);
@@ -541,6 +549,64 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
       const int si = s_excl[flat] + gi;
       write_seg(L, P, stage, id, gi, B, si, s_itembase[c] + (si - s_segbase[c]) * ips);
     }
+  }
+}
+
+// Hand the first stage (department gate / up) to the streaming kernel as soon as the department
+// token lists exist: zero the dependency counters, write the stage's segment records (the same
+// numbering worklist_block() gives them: category 0, units in active-department order), publish
+// the item count and raise the flag with this step's number.  scr: A + 1 ints of shared memory.
+static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, int B, int* scr, int epoch) {
+  __shared__ int s_w[33];
+  const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
+#pragma unroll 1
+  for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
+  const int A = L.counts[CNT_ACTIVE_DEPT];
+  const int tg = P.st[ST_S1].tg, ips = P.st[ST_S1].items_per_seg;
+  int carry = 0;  // exclusive scan of the departments' group counts, 'nthr' departments at a time
+#pragma unroll 1
+  for (int base = 0; base < A; base += nthr) {
+    const int a = base + tid;
+    const int gc = (a < A) ? groups_of(unit_tokens(L, ST_S1, L.active_dept[a], B), tg) : 0;
+    int incl = gc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) s_w[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int w = (lane < nwarp) ? s_w[lane] : 0;
+      int wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += y;
+      }
+      s_w[lane] = wi - w;
+      if (lane == 31) s_w[32] = wi;
+    }
+    __syncthreads();
+    if (a < A) scr[a] = carry + s_w[warp] + incl - gc;
+    carry += s_w[32];
+    __syncthreads();
+  }
+  if (tid == 0) scr[A] = carry;
+  __syncthreads();
+#pragma unroll 1
+  for (int a = tid; a < A; a += nthr) {
+    const int id = L.active_dept[a];
+    const int gc = scr[a + 1] - scr[a];
+#pragma unroll 1
+    for (int gi = 0; gi < gc; ++gi) write_seg(L, P, ST_S1, id, gi, B, scr[a] + gi, (scr[a] + gi) * ips);
+  }
+  __threadfence();  // every thread's records and zeroed counters, before the flag
+  __syncthreads();
+  if (tid == 0) {
+    P.sync[SY_DEP + P.early_items] = (carry <= P.max_segs) ? carry * ips : 0;
+    __threadfence();
+    st_release(P.sync + SY_DEP + P.early_flag, epoch);
   }
 }
 
@@ -575,7 +641,7 @@ static __host__ __device__ FinishSmem finish_layout(int n, int m, int k, int B) 
 }
 
 __global__ void __launch_bounds__(FINISH_THREADS)
-k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
+k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words, int epoch,
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   extern __shared__ uint32_t s_dyn[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
@@ -621,13 +687,16 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   long long tt1 = clock64();
   TS_MIN(L, 12);
 #endif
-  bucket_block(S, B, s_dyn, FINISH_THREADS);
+  bucket_departments(S, B, s_dyn, FINISH_THREADS);
+  if (P.early)  // scratch: the words after the bucketing masks and offsets
+    early_first_stage(S, P, B, reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B), epoch);
+  bucket_experts(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
 #ifdef DEAMOE_TRACE
   long long tt2 = clock64();
   TS_MIN(L, 13);
 #endif
-  worklist_block(S, P, B, reinterpret_cast<int*>(s_dyn));
+  worklist_block(S, P, B, reinterpret_cast<int*>(s_dyn), P.early != 0);
   __syncthreads();
   TS_MIN(L, 15);
   // publish the routing state: every array is a run of 32-bit words in the shared-memory copy.
@@ -725,7 +794,7 @@ struct __align__(16) ItemCtx {  // producer-side view of one claimed item
 };
 
 __global__ void __launch_bounds__(STREAM_THREADS, CTAS_PER_SM)
-k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
+k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* red = reinterpret_cast<float*>(smem + (size_t)NSLOT * SLOT_BYTES);
@@ -868,25 +937,22 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       }
     }
 
-    pdl_wait();  // the work list is written by the preceding routing kernel
-    cat_tab[lane] = sy[SY_CAT + lane];  // 4 * MAX_CAT == 32 entries
-    __syncwarp();
-    // item range of this launch: one category (staged) or everything (fused)
-    const int ncat = sy[SY_NCAT];
-    const int item_begin = (cat >= 0) ? cat_tab[4 * cat] : 0;
-    const int item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
-    if (*abort_flag && lane == 0) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;  // set before the routing kernel reset it
+    // The list is walked in up to two phases.  Phase 1 (fused schedule of DeaMoE layers): the
+    // routing kernel publishes the records of the first stage as soon as the department token
+    // lists exist and raises a flag carrying this step's number; the first stage is by far the
+    // longest, so the rest of the routing (expert lists, the other stages' records) hides behind
+    // it.  Phase 2, after the routing kernel has completed: everything else.
+    int ncat = 0, item_end = 0;
+    int cur_i = (int)blockIdx.x;  // item i of the launch's range goes to CTA i mod grid
     auto seg_of = [&](int k, int item, int& it) -> const Seg* {
       const int ib = cat_tab[4 * k + 0], sb = cat_tab[4 * k + 1], ips = cat_tab[4 * k + 2];
       it = (item - ib) % ips;
       return P.segs + sb + (item - ib) / ips;
     };
-    // Assignment of items to CTAs: item i of the launch's range goes to CTA i mod grid.  Dealing
-    // the items out (rather than giving a CTA one contiguous stretch per category) completes
-    // the units one after another, so dependent items of later categories become ready early;
-    // contiguous stretches were measured 25-35 % slower for that reason.
-    int cur_i = item_begin + (int)blockIdx.x;
-    auto next_item = [&](int& k) -> int {  // next item of this CTA, -1 at the end
+    // Dealing the items out (rather than giving a CTA one contiguous stretch per category)
+    // completes the units one after another, so dependent items of later categories become ready
+    // early; contiguous stretches were measured 25-35 % slower for that reason.
+    auto next_item = [&](int& k) -> int {  // next item of this CTA, -1 at the end of the phase
       if (cur_i >= item_end) return -1;
       const int item = cur_i;
       cur_i += G;
@@ -898,43 +964,80 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     // Three segment records are in flight (this item's and the next two), and the dependency
     // counter of the next item is read while this one is queued, so the planner pays one L2
     // latency per three items, not per item.
-    const Seg* sp0 = nullptr; const Seg* sp1 = nullptr; const Seg* sp2 = nullptr;
-    int it0 = 0, it1 = 0, it2 = 0;
-    int4 v0 = make_int4(0, 0, 0, 0), v1 = v0, v2 = v0;  // lane l < SEG_VEC holds bytes [16l, 16l+16) of a record
-    auto fetch = [&](const Seg*& sp, int& it, int4& v) {
-      sp = nullptr;
-      int k = 0;
-      const int item = next_item(k);
-      if (item >= 0) {
-        sp = seg_of(k, item, it);
-        if (lane < SEG_VEC) v = __ldg(reinterpret_cast<const int4*>(sp) + lane);
+    auto walk = [&]() {
+      const Seg* sp0 = nullptr; const Seg* sp1 = nullptr; const Seg* sp2 = nullptr;
+      int it0 = 0, it1 = 0, it2 = 0;
+      int4 v0 = make_int4(0, 0, 0, 0), v1 = v0, v2 = v0;  // lane l < SEG_VEC holds bytes [16l, 16l+16) of a record
+      auto fetch = [&](const Seg*& sp, int& it, int4& v) {
+        sp = nullptr;
+        int k = 0;
+        const int item = next_item(k);
+        if (item >= 0) {
+          sp = seg_of(k, item, it);
+          // L2 load: in phase 1 the records were written while this kernel was already running
+          if (lane < SEG_VEC) v = __ldcg(reinterpret_cast<const int4*>(sp) + lane);
+        }
+      };
+      fetch(sp0, it0, v0);
+      fetch(sp1, it1, v1);
+      fetch(sp2, it2, v2);
+      int dv0 = 0;            // counter value read ahead for record 0
+      bool dv0_valid = false;
+      while (ok && sp0) {
+        // read ahead: dependency counter of the next item, record of the item three ahead
+        int dv1 = 0;
+        bool dv1_valid = false;
+        if ((check_deps & 1) && sp1) {
+          const int nd = __shfl_sync(0xffffffffu, v1.w, 3);
+          if (nd >= 0 && nd != dep_ok) {
+            dv1 = ld_acquire(P.sync + SY_DEP + nd);
+            dv1_valid = true;
+          }
+        }
+        const Seg* sp3; int it3 = 0; int4 v3 = make_int4(0, 0, 0, 0);
+        fetch(sp3, it3, v3);
+        ok = emit(v0, it0, dv0_valid, dv0);
+        // rotate the record pipeline
+        sp0 = sp1; it0 = it1; v0 = v1; dv0 = dv1; dv0_valid = dv1_valid;
+        sp1 = sp2; it1 = it2; v1 = v2;
+        sp2 = sp3; it2 = it3; v2 = v3;
       }
     };
-    fetch(sp0, it0, v0);
-    fetch(sp1, it1, v1);
-    fetch(sp2, it2, v2);
-    int dv0 = 0;            // counter value read ahead for record 0
-    bool dv0_valid = false;
-    while (ok && sp0) {
-      // read ahead: dependency counter of the next item, record of the item three ahead
-      int dv1 = 0;
-      bool dv1_valid = false;
-      if ((check_deps & 1) && sp1) {
-        const int nd = __shfl_sync(0xffffffffu, v1.w, 3);
-        if (nd >= 0 && nd != dep_ok) {
-          dv1 = ld_acquire(P.sync + SY_DEP + nd);
-          dv1_valid = true;
+
+    if (P.early && cat < 0 && ok) {
+      int n1 = 0;
+      if (lane == 0) {
+        const int32_t* flag = P.sync + SY_DEP + P.early_flag;
+        unsigned spins = 0;
+        bool seen = true;
+        while (ld_acquire(flag) != epoch) {
+          __nanosleep(64);
+          if (++spins > SPIN_LIMIT / 16 || *abort_flag) { seen = false; break; }
         }
+        n1 = seen ? __ldcg(P.sync + SY_DEP + P.early_items) : -1;
       }
-      const Seg* sp3; int it3 = 0; int4 v3 = make_int4(0, 0, 0, 0);
-      fetch(sp3, it3, v3);
-      ok = emit(v0, it0, dv0_valid, dv0);
-      // rotate the record pipeline
-      sp0 = sp1; it0 = it1; v0 = v1; dv0 = dv1; dv0_valid = dv1_valid;
-      sp1 = sp2; it1 = it2; v1 = v2;
-      sp2 = sp3; it2 = it3; v2 = v3;
+      n1 = __shfl_sync(0xffffffffu, n1, 0);
+      if (n1 < 0) {
+        ok = false;
+      } else {
+        if (lane == 0) {
+          cat_tab[0] = 0; cat_tab[1] = 0; cat_tab[2] = P.st[ST_S1].items_per_seg; cat_tab[3] = ST_S1;
+        }
+        __syncwarp();
+        ncat = 1; item_end = n1;
+        walk();
+      }
     }
-    (void)sp0;
+
+    pdl_wait();  // the rest of the work list is complete when the routing kernel is
+    cat_tab[lane] = sy[SY_CAT + lane];  // 4 * MAX_CAT == 32 entries
+    __syncwarp();
+    // item range of this launch: one category (staged) or everything (fused)
+    ncat = sy[SY_NCAT];
+    if (cat >= 0) cur_i = cat_tab[4 * cat] + (int)blockIdx.x;
+    item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
+    if (*abort_flag && lane == 0) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;  // set before the routing kernel reset it
+    if (ok) walk();
 #ifdef DEAMOE_TRACE
     if (lane == 0 && P.trace) {
       P.trace[(size_t)blockIdx.x * TR_SLOTS + 7] = ptr_dep;
@@ -1309,6 +1412,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   if (!p) return DEAMOE_ERR_ALLOC;
   std::memset(p, 0, sizeof(*p));
   p->schedule = schedule;
+  p->epoch = 0;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->n_sm, cudaDevAttrMultiProcessorCount, dev);
@@ -1389,6 +1493,8 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   // kernel, the last of a step, resets it.
   d.sh_prefix = (schedule == DEAMOE_SCHED_FUSED && L.n_shared && (L.vanilla || L.r > 0)) ? 1 : 0;
   if (d.sh_prefix) d.dep_sh1 = d.n_dep;
+  d.early = (schedule == DEAMOE_SCHED_FUSED && !L.vanilla && L.r > 0 && (!L.n_shared || d.sh_prefix)) ? 1 : 0;
+  d.early_flag = d.n_dep + 1; d.early_items = d.n_dep + 2;  // the allocation has 8 spare counters
   d.planes = (L.adt == DEAMOE_F32) ? 2 : 1;
   {
     // activation planes between stages
@@ -1468,13 +1574,15 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
   size_t scratch = in_regs ? 0 : (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
-  const size_t bs = bucket_smem_bytes(L, B);
+  const size_t bs = bucket_smem_bytes(L, B) + (size_t)(L.m + 2) * sizeof(int);  // + early_first_stage()'s scan
   if (bs > scratch) scratch = bs;
   scratch = (scratch + 15) & ~(size_t)15;
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   const size_t smem = scratch + (size_t)fl.total * 4;
   if (smem > 200 * 1024) return -1;
+  if (++p.epoch == 0) p.epoch = 1;
   launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, p.dev, B, ny, topk_warps, (int)(scratch / 4),
+             p.epoch,
              user_idx, user_w);
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
@@ -1517,7 +1625,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | dbgflag);
+    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | dbgflag, p.epoch);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
@@ -1525,7 +1633,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
         k_identity_private<<<p.n_sm, 256, 0, s>>>(L, p.dev);
         ++launches;
       }
-      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, B, c, 0);
+      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, B, c, 0, p.epoch);
       ++launches;
     }
   }
