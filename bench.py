@@ -237,6 +237,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the batch sweep and the vanilla comparator")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle")
+    ap.add_argument("--mode", default="layer", choices=["layer", "locality", "stack"],
+                    help="layer: the contract line (default); locality: routing-locality sweep on the DeepSeek-V3 "
+                         "shape; stack: 32 consecutive 7B-class layers with a residual add, DeaMoE vs vanilla")
     args = ap.parse_args()
 
     from paper_2608_14385_b200 import synth
@@ -264,6 +267,14 @@ def main():
     sched = {"auto": binding.SCHED_AUTO, "plain": binding.SCHED_PLAIN, "staged": binding.SCHED_STAGED,
              "fused": binding.SCHED_FUSED}[args.schedule]
     peak, peak_src = measured_peaks()
+    if args.mode != "layer":
+        if rank == 0:
+            fn = locality_sweep if args.mode == "locality" else stack_bench
+            print(json.dumps(fn(args, sched, peak, torch, dev)))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     B = args.batch
     max_batch = max(64 if shape.name == "dsv3-paper" else 32, B)
     w = synth.make_deamoe_weights(shape, 0, dev)
@@ -422,6 +433,122 @@ def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev):
     return {"rows": out,
             "paper_context": "expected loaded-weights ratio 0.491 .. 0.628 over 4 .. 64 tokens (Section 3.3, Fig. 2); "
                              "peak layer speed-up 2.00x (A40) / 1.97x (H100)"}
+
+
+def locality_sweep(args, sched, peak, torch, dev):
+    """Routing-locality sweep on the DeepSeek-V3 shape: every token's top-8 is planted (through the real
+    router) in exactly c departments; c = 8 with random tokens is the uniform case.  Unique bytes are set
+    against the closed form |D| ~ m (1 - (1 - c/m)^B) with 8 B distinct experts at most."""
+    from paper_2608_14385_b200 import binding, synth
+    shape = synth.DSV3
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    layer = binding.Layer(shape, w, 32, sched)
+    router = w["router"]
+    del w
+    torch.cuda.empty_cache()
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    m, g, k = shape.n_dept, shape.experts_per_dept, shape.top_k
+    dept_b = 3 * shape.hidden * shape.ffn * 2
+    exp_b = 3 * shape.priv * shape.ffn * 2
+    fixed_b = shape.n_shared * 3 * shape.hidden * shape.shared_ffn * 2 + shape.n_expert * shape.hidden * 4
+    rows = []
+    for c in (1, 2, 4, 8, 0):                      # 0 = uniform (no planting)
+        for B in (1, 4, 16, 32):
+            bs = []
+            for i in range(4):
+                t = synth.make_tokens(shape, B, 200 + i, dev)
+                if c:
+                    t, _ = synth.plant_locality(shape, router, t, c, seed=10 * c + i)
+                bs.append(t)
+            ub, nd, ne = [], [], []
+            for b in bs:
+                layer.forward(b)
+                st = layer.stats()
+                ub.append(st["unique_weight_bytes"]); nd.append(st["active_dept"]); ne.append(st["active_expert"])
+            t_ms, _ = time_layer(layer, bs, max(10, args.steps // 2), 3, flush, torch, lambda: None)
+            us = pct(t_ms, 0.5) * 1e3
+            mb = statistics.mean(ub) / 1e6
+            row = {"c": c if c else "uniform", "batch": B, "us": us, "unique_mb": mb, "gbs": mb / us * 1e3,
+                   "frac_of_measured_peak": mb / us * 1e3 / peak, "active_dept": statistics.mean(nd),
+                   "active_expert": statistics.mean(ne)}
+            if c:
+                e_d = m * (1.0 - (1.0 - c / m) ** B)
+                e_e = shape.n_expert * (1.0 - (1.0 - k / shape.n_expert) ** B)   # experts uniform over all n
+                row["closed_form_mb"] = (e_d * dept_b + e_e * exp_b + fixed_b) / 1e6
+                row["closed_form_active_dept"] = e_d
+            rows.append(row)
+    layer.close()
+    return {"metric": "routing_locality_sweep", "unit": "us", "shape": shape.name, "data": "synthetic",
+            "config": {"workload": "dsv3-shape DeaMoE layer, top-8 planted in c departments per token",
+                       "l2": "256 MiB buffer overwritten between steps (untimed)"},
+            "rows": rows}
+
+
+def stack_bench(args, sched, peak, torch, dev):
+    """32 consecutive 7B-class layers, x <- x + Layer_l(x), every layer with its own seeded weights;
+    MoE time per decode step of the DeaMoE stack and of the vanilla-MoE stack at B = 1 and 8.  The stacks
+    (6.6 GB and 17.7 GB) are far larger than L2, so no flush is needed between steps.  The layers are
+    run one at a time (stream synchronised after each), the way the parity test of the stack runs them."""
+    import dataclasses
+    from paper_2608_14385_b200 import binding, synth
+    shape = dataclasses.replace(synth.MOE7B, residual=1)
+    n_layers = 32
+    out = {"metric": "us_per_decode_step_moe_stack", "unit": "us", "layers": n_layers, "shape": shape.name,
+           "data": "synthetic", "config": {"workload": "stack of 32 7B-class layers with residual add",
+                                           "l2": "stack larger than L2, no flush"}, "rows": []}
+    res = {}
+    for vanilla in (False, True):
+        layers = []
+        for l in range(n_layers):
+            w = (synth.make_vanilla_weights if vanilla else synth.make_deamoe_weights)(shape, 0, dev, layer=l)
+            layers.append(binding.Layer(shape, w, 8, sched, vanilla=vanilla))
+            del w
+        torch.cuda.empty_cache()
+        for B in (1, 8):
+            # tokens scaled by 1/16: with N(0,1) tokens the vanilla stack (gain ~0.6 per layer, quadratic in |x|)
+            # overflows bf16 within 32 layers without a normalisation; routing (an arg-max) is scale-invariant
+            xs = [(synth.make_tokens(shape, B, 300 + i, dev).float() / 16).to(torch.bfloat16) for i in range(4)]
+            bufs = [torch.empty_like(xs[0]), torch.empty_like(xs[0])]
+
+            # Every layer is timed with its own pair of events and the stream is synchronised after it;
+            # a step's time is the sum of its layers' device times.
+            def step(x, evs=None):
+                cur = x
+                for l, layer in enumerate(layers):
+                    if evs:
+                        evs[l][0].record()
+                    layer.forward(cur, bufs[l & 1])
+                    if evs:
+                        evs[l][1].record()
+                    torch.cuda.synchronize()
+                    cur = bufs[l & 1]
+                return cur
+            for i in range(3):
+                step(xs[i % 4])
+            steps = max(10, args.steps // 2)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(n_layers)]
+            t = []
+            for i in range(steps):
+                step(xs[i % 4], evs)
+                t.append(sum(a.elapsed_time(b) for a, b in evs))
+            ub = 0
+            for layer in layers:
+                ub += layer.stats()["unique_weight_bytes"]
+            finite = bool(torch.isfinite(bufs[(n_layers - 1) & 1].float()).all())
+            res[(vanilla, B)] = (pct(t, 0.5) * 1e3, ub / 1e6, finite)
+        for layer in layers:
+            layer.close()
+        del layers
+        torch.cuda.empty_cache()
+    for B in (1, 8):
+        d_us, d_mb, d_fin = res[(False, B)]
+        v_us, v_mb, v_fin = res[(True, B)]
+        out["rows"].append({"batch": B, "deamoe_us": d_us, "deamoe_mb_last_step": d_mb, "deamoe_gbs": d_mb / d_us * 1e3,
+                            "vanilla_us": v_us, "vanilla_mb_last_step": v_mb, "vanilla_gbs": v_mb / v_us * 1e3,
+                            "speedup_vs_vanilla": v_us / d_us, "byte_ratio_vanilla_over_deamoe": v_mb / d_mb,
+                            "deamoe_us_per_layer": d_us / n_layers, "outputs_finite": d_fin and v_fin})
+    return out
 
 
 def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev):

@@ -40,7 +40,8 @@ typedef enum {
   DEAMOE_ERR_ALLOC = 3,       /* device or host allocation failed */
   DEAMOE_ERR_CUDA = 4,        /* a CUDA runtime call failed (no device, launch error) */
   DEAMOE_ERR_BATCH = 5,       /* B < 0 or B > max_batch */
-  DEAMOE_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by get_stats) */
+  DEAMOE_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (reported by get_stats) */
+  DEAMOE_ERR_INTERNAL = 7     /* a device-side consistency check failed; the access was skipped (get_stats) */
 } deamoe_status_t;
 
 typedef enum { DEAMOE_F32 = 0, DEAMOE_BF16 = 1 } deamoe_dtype_t;
@@ -173,7 +174,7 @@ deamoe_status_t deamoe_get_routing(deamoe_layer_t *layer, void *cuda_stream, int
  * Counters of the LAST route/forward call (synchronises the stream first), HOST outputs, any may
  * be NULL: active departments |D|, active experts |E|, (token, department) pairs, the unique weight
  * bytes the step had to load (|D|*3hf*s + |E|*3rf*s + shared + 4nh for DeaMoE; |E|*3hf*s + shared +
- * 4nh for vanilla), and the device status word (DEAMOE_OK or DEAMOE_ERR_TIMEOUT).
+ * 4nh for vanilla), and the device status word (DEAMOE_OK, DEAMOE_ERR_TIMEOUT or DEAMOE_ERR_INTERNAL).
  */
 deamoe_status_t deamoe_get_stats(deamoe_layer_t *layer, void *cuda_stream, int32_t *n_active_dept,
                                  int32_t *n_active_expert, int32_t *n_token_dept_pairs,

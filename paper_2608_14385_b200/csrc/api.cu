@@ -387,6 +387,7 @@ int deamoe_debug_trace(deamoe_layer_t* L, long long* host, int max_ctas) {
 const char* deamoe_status_string(deamoe_status_t st) {
   switch (st) {
     case DEAMOE_OK: return "ok";
+    case DEAMOE_ERR_INTERNAL: return "device-side consistency check failed";
     case DEAMOE_ERR_INVALID_ARG: return "invalid argument";
     case DEAMOE_ERR_UNSUPPORTED: return "unsupported configuration";
     case DEAMOE_ERR_ALLOC: return "allocation failed";

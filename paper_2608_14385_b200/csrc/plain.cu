@@ -237,8 +237,14 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int t = (int)(i / L.h), c = (int)(i % L.h);
     float acc = 0.f;
-    for (int q = 0; q < L.k; ++q)
-      acc = fmaf(L.topk_w[t * L.k + q], L.O[(size_t)L.pair_slot[t * L.k + q] * L.h + c], acc);
+    for (int q = 0; q < L.k; ++q) {
+      const int slot = L.pair_slot[t * L.k + q];
+      if ((unsigned)slot >= (unsigned)(L.max_batch * L.k)) {  // consistency check: skip the access, report
+        L.counts[CNT_STATUS] = DEAMOE_ERR_INTERNAL;
+        continue;
+      }
+      acc = fmaf(L.topk_w[t * L.k + q], L.O[(size_t)slot * L.h + c], acc);
+    }
     if (L.n_shared) acc += L.Osh[i];
     if (L.residual)
       acc += (L.adt == DEAMOE_F32) ? reinterpret_cast<const float*>(L.tokens_raw)[i]

@@ -21,6 +21,7 @@ static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslic
   for (int i = lane; i < n; i += 32) {
     float v = 0.f;
     for (int s = 0; s < kslices; ++s) v += L.logit_part[((size_t)s * B + t) * n + i];
+    if (!(v == v)) v = -INFINITY;  // a NaN logit (non-finite input) must still yield valid indices
     lg[i] = v;
     dead[i] = 0;
     mx_all = fmaxf(mx_all, v);
@@ -120,8 +121,10 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
       }
     }
 #pragma unroll
-    for (int j = 0; j < VPL; ++j)
+    for (int j = 0; j < VPL; ++j) {
+      if (!(v[j] == v[j])) v[j] = -INFINITY;  // a NaN logit (non-finite input) must still yield valid indices
       if (lane + 32 * j >= n) { v[j] = -INFINITY; taken |= 1u << j; }
+    }
   }
 #ifdef DEAMOE_TRACE
   float chk = 0.f;

@@ -117,6 +117,8 @@ struct StreamDev {
   int32_t* sync;
   int max_segs;
   int dep_s1, dep_s2, dep_s3, dep_sh1, n_dep;  // offsets relative to SY_DEP
+  const __nv_bfloat16* packed_lo;  // packed weights: first element and element count (record checks)
+  size_t packed_elems;
   int sh_prefix;  // fused schedule with a shared expert: its items are not in the work list
   int early;      // fused DeaMoE layers: the first stage's records are handed over ahead of the rest
   int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): step number, item count
@@ -879,6 +881,22 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
       __syncwarp();
       const Seg* sg = reinterpret_cast<const Seg*>(ent);
       const int T = sg->T, paired = sg->paired, nB = sg->nB, C = sg->C;
+      {
+        // consistency check of the record before anything is copied on its behalf
+        const size_t woff = (size_t)(sg->w0 - P.packed_lo);
+        const bool good = (unsigned)sg->stage < 8u && T >= 1 && T <= MAX_QP * 8 && (nB == 1 || nB == 2) &&
+                          (sg->q == 1 || sg->q == 2) && (sg->planes == 1 || sg->planes == 2) && C >= 16 &&
+                          sg->kc >= 16 && (sg->kc & 15) == 0 && sg->kc <= C && sg->n_tiles >= 1 &&
+                          it >= 0 && it < sg->n_items && sg->in0h != nullptr && woff < P.packed_elems;
+        if (!good) {
+          if (lane == 0) {
+            L.counts[CNT_STATUS] = DEAMOE_ERR_INTERNAL;
+            L.counts[8] = sg->stage; L.counts[9] = T; L.counts[10] = sg->kc; L.counts[11] = it; L.counts[12] = C;
+            *abort_flag = 1;
+          }
+          return false;
+        }
+      }
       const int tile0 = paired ? it : it * sg->q;
       const int q_eff = paired ? 2 : min(sg->q, sg->n_tiles - tile0);
       const int nrows = sg->planes * nB * T;
@@ -1450,6 +1468,8 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   }
   p->packed = base;
   p->bytes = total * 2 + 16;
+  p->dev.packed_lo = base;
+  p->dev.packed_elems = total;
   cudaError_t e = cudaSuccess;
   auto P = [&](const void* src, size_t off, int rows, int C, long long rs, long long cs, long long su, long long du,
                int nu) {

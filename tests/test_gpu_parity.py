@@ -10,7 +10,7 @@ import torch
 
 from oracle import ref
 from paper_2608_14385_b200 import binding, synth
-from tests.common import oracle_cfg
+from tests.common import oracle_cfg, within_tolerance
 from tests.gpu_common import check_routing, run_case
 
 pytestmark = pytest.mark.gpu
@@ -205,3 +205,33 @@ def test_unsupported_and_invalid_creates_are_reported():
     with pytest.raises(binding.DeaMoEError) as e:
         binding.Layer(SMALL.with_(weight_dtype=0), w, 4, binding.SCHED_FUSED)   # fp32 cannot stream
     assert e.value.status == binding.ERR_UNSUPPORTED
+
+
+def test_non_finite_tokens_keep_indices_valid():
+    """Inputs must be finite for the results to mean anything, but a NaN / Inf token row must not
+    turn into an invalid expert index (that would be an out-of-range access): the call completes,
+    every index is a valid expert, and the finite rows are unaffected."""
+    shape = RAGGED
+    w = _scaled(shape, 4)
+    layer = binding.Layer(shape, w, 8)
+    try:
+        good = synth.make_tokens(shape, 6, 21, "cuda:0")
+        bad = good.clone()
+        bad[1, :] = float("nan")
+        bad[4, 3] = float("inf")
+        ref_out = layer.forward(good).clone()
+        out = layer.forward(bad)
+        torch.cuda.synchronize()
+        st = layer.stats()
+        assert st["device_status"] == 0
+        idx = layer.routing(6)["idx"]
+        assert idx.min() >= 0 and idx.max() < shape.n_expert
+        for t in range(6):
+            assert len(set(int(i) for i in idx[t])) == shape.top_k
+        keep = [0, 2, 3, 5]
+        a, b = out[keep].float().cpu().numpy(), ref_out[keep].float().cpu().numpy()
+        assert np.isfinite(a).all()
+        ok, err, bound = within_tolerance(a, b)
+        assert ok, (err, bound)
+    finally:
+        layer.close()
