@@ -487,8 +487,8 @@ def locality_sweep(args, sched, peak, torch, dev):
 def stack_bench(args, sched, peak, torch, dev):
     """32 consecutive 7B-class layers, x <- x + Layer_l(x), every layer with its own seeded weights;
     MoE time per decode step of the DeaMoE stack and of the vanilla-MoE stack at B = 1 and 8.  The stacks
-    (6.6 GB and 17.7 GB) are far larger than L2, so no flush is needed between steps.  The layers are
-    run one at a time (stream synchronised after each), the way the parity test of the stack runs them."""
+    (6.6 GB and 17.7 GB) are far larger than L2, so no flush is needed between steps.  The 128
+    kernels of a step are enqueued back to back; a step is timed by one pair of events."""
     import dataclasses
     from paper_2608_14385_b200 import binding, synth
     shape = dataclasses.replace(synth.MOE7B, residual=1)
@@ -510,28 +510,23 @@ def stack_bench(args, sched, peak, torch, dev):
             xs = [(synth.make_tokens(shape, B, 300 + i, dev).float() / 16).to(torch.bfloat16) for i in range(4)]
             bufs = [torch.empty_like(xs[0]), torch.empty_like(xs[0])]
 
-            # Every layer is timed with its own pair of events and the stream is synchronised after it;
-            # a step's time is the sum of its layers' device times.
-            def step(x, evs=None):
+            def step(x):
                 cur = x
-                for l, layer in enumerate(layers):
-                    if evs:
-                        evs[l][0].record()
+                for l, layer in enumerate(layers):      # enqueued back to back, no host synchronisation
                     layer.forward(cur, bufs[l & 1])
-                    if evs:
-                        evs[l][1].record()
-                    torch.cuda.synchronize()
                     cur = bufs[l & 1]
                 return cur
             for i in range(3):
                 step(xs[i % 4])
             steps = max(10, args.steps // 2)
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                   for _ in range(n_layers)]
-            t = []
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            torch.cuda.synchronize()
             for i in range(steps):
-                step(xs[i % 4], evs)
-                t.append(sum(a.elapsed_time(b) for a, b in evs))
+                ev[i][0].record()
+                step(xs[i % 4])
+                ev[i][1].record()
+            torch.cuda.synchronize()
+            t = [a.elapsed_time(b) for a, b in ev]
             ub = 0
             for layer in layers:
                 ub += layer.stats()["unique_weight_bytes"]

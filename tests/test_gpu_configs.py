@@ -107,3 +107,40 @@ def test_paper_row_department_cap_holds_for_every_token():
         want, _ = check_routing(shape, layer, w, tokens, B)
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("vanilla", [False, True])
+def test_layers_enqueued_back_to_back_match_layers_run_one_by_one(vanilla):
+    """A stack is normally enqueued without waiting for each layer: the kernels of consecutive layers
+    then follow each other directly in the stream (programmatic dependent launches inside a layer,
+    ordinary dependencies between layers).  The result must equal, bit for bit, the result of running
+    the layers one at a time."""
+    n_layers, B = 6, 8
+    shape = synth.MOE7B.with_(residual=1)
+    dev = torch.device("cuda:0")
+    layers = []
+    for l in range(n_layers):
+        w = (synth.make_vanilla_weights if vanilla else synth.make_deamoe_weights)(shape, 0, dev, layer=l)
+        layers.append(binding.Layer(shape, w, 8, vanilla=vanilla))
+        del w
+    try:
+        x0 = (synth.make_tokens(shape, B, 11, dev).float() / 16).to(torch.bfloat16)
+        bufs = [torch.empty_like(x0), torch.empty_like(x0)]
+
+        def run(sync):
+            cur = x0
+            for l, layer in enumerate(layers):
+                layer.forward(cur, bufs[l & 1])
+                if sync:
+                    torch.cuda.synchronize()
+                cur = bufs[l & 1]
+            torch.cuda.synchronize()
+            return cur.clone()
+        one_by_one = run(True)
+        for _ in range(3):
+            assert torch.equal(run(False), one_by_one)
+        assert torch.isfinite(one_by_one.float()).all()
+        assert all(layer.stats()["device_status"] == 0 for layer in layers)
+    finally:
+        for layer in layers:
+            layer.close()
