@@ -114,7 +114,7 @@ def pct(xs, q):
     return xs[min(len(xs) - 1, max(0, int(round(q * (len(xs) - 1)))))]
 
 
-def oracle_sample_seconds(shape, weights_fn, tokens, rows, vanilla=False):
+def oracle_sample_seconds(shape, weights_fn, tokens, rows, vanilla=False, one_thread=None):
     """Time the fp64 oracle (as it stands) on `rows` of this batch with all host cores."""
     import numpy as np
     from oracle import ref
@@ -146,7 +146,14 @@ def oracle_sample_seconds(shape, weights_fn, tokens, rows, vanilla=False):
     fwd = ref.vanilla_forward if vanilla else ref.deamoe_forward
     t0 = time.perf_counter()
     fwd(cfg, w, tok, rows=rows)
-    return time.perf_counter() - t0, cores
+    t_all = time.perf_counter() - t0
+    if one_thread is not None:      # the same sample once more on a single core
+        ref.set_threads(1)
+        t0 = time.perf_counter()
+        fwd(cfg, w, tok, rows=rows)
+        one_thread.append(time.perf_counter() - t0)
+        ref.set_threads(cores)
+    return t_all, cores
 
 
 def run_reference(args, shape, rank, world):
@@ -378,9 +385,11 @@ def main():
             if unit is None:
                 return shared[name]
             return synth.weight_slice(shape, name, unit, 0, dev)
-        sec, cores = oracle_sample_seconds(shape, wfn, batches[0], [0])
+        one = []
+        sec, cores = oracle_sample_seconds(shape, wfn, batches[0], [0], one_thread=one)
         line["cpu_baseline"] = {"value": sec * B * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-                                "sample": f"1 of {B} token rows of one step, time scaled by {B}"}
+                                "sample": f"1 of {B} token rows of one step, time scaled by {B}",
+                                "value_one_core": one[0] * B * 1e6}
     layer.close()
     if rank == 0:
         print(json.dumps(line))

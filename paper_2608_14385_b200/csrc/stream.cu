@@ -37,7 +37,6 @@ namespace deamoe {
 
 constexpr int CTAS_PER_SM = 2;                   // co-resident CTAs of the streaming kernel per SM
 constexpr int CONSUMER_WARPS = 4;
-constexpr int CONSUMER_THREADS = CONSUMER_WARPS * 32;
 constexpr int ISSUE_WARPS = 1;                   // copy-issue warps; warp p fills chunks p, p + ISSUE_WARPS, ...
 constexpr int WARP_ISSUE = CONSUMER_WARPS;       // first of the warps that issue the bulk copies
 constexpr int WARP_PLAN = WARP_ISSUE + ISSUE_WARPS;  // picks items, fetches records, waits for inputs
@@ -51,7 +50,6 @@ constexpr int MAX_CAT_INTS_PAD = 8;             // cat_tab: 4 ints for each of 8
 #define PREFIX_LAST_STAGE ST_SH1  // the shared expert's second stage waits for all of the first: it runs from the list
 #endif
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
-constexpr int SIG_DEPTH = 16;
 constexpr int SLOT_BYTES = 32 * 1024;
 constexpr int SLOT_HDR = 128;
 constexpr int NSLOT = 3;
@@ -228,9 +226,6 @@ static __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-static __device__ __forceinline__ void consumer_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(CONSUMER_THREADS) : "memory");
 }
 static __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4& a, uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -454,8 +449,8 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
   CatInfo cats[MAX_CAT];
   const int ncat = category_list(L, P, cats);
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
-#pragma unroll 1
   if (!early_done)  // else early_first_stage() has zeroed the counters, and the first stage may be running
+#pragma unroll 1
     for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
   if (tid == 0) {
     int ub = 0;
@@ -1089,8 +1084,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
 #endif
     uint32_t eph = 0;
     bool ok = true;
+#ifdef DEAMOE_TRACE
     long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    (void)tr;
+#endif
     const long long tp0 = TR_NOW();
     (void)tp0;
     while (ok) {
@@ -1220,7 +1216,6 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
       __nv_bfloat16* outl = sg->outl;
       float* outf = sg->outf;
       int32_t* done = (sg->done_idx >= 0) ? P.sync + SY_DEP + sg->done_idx : nullptr;
-      const int npass = (T + 7) >> 3;
       const float* rbuf = red + (size_t)rb * RED_FLOATS;
       // Only the real outputs are reduced: (tile a, row rr of 16, token s < T).  In the MMA D
       // fragment that element is register reg = (rr >= 8 ? 2 : 0) + (s & 1) of lane (rr % 8) * 4 +
@@ -1301,8 +1296,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
   float acc[MAX_QP][4];
   int slot = 0, items = 0;
   uint32_t phase = 0;
+#ifdef DEAMOE_TRACE
   long long tr[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-  (void)tr;
+#endif
   const long long tc0 = TR_NOW();
   (void)tc0;
   while (true) {
