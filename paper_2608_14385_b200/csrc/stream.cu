@@ -1546,7 +1546,13 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
     int occ = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream, STREAM_THREADS, STREAM_SMEM);
     if (e == cudaSuccess && occ < 1) e = cudaErrorLaunchOutOfResources;
-    p->grid = p->n_sm * (occ < CTAS_PER_SM ? occ : CTAS_PER_SM);
+    const int per_sm = occ < CTAS_PER_SM ? occ : CTAS_PER_SM;
+    p->grid = p->n_sm * per_sm;
+    // Fused schedule: the routing tail (one CTA that fills an SM's register file) is still running
+    // when this grid starts, and the CTAs that would share its SM could only start when it exits,
+    // tens of microseconds after the others, and would finish the step that much later.  The
+    // grid leaves that SM out (the stream is bound by HBM, not by the number of SMs).
+    if (schedule == DEAMOE_SCHED_FUSED && p->n_sm > 1) p->grid -= per_sm;
   }
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_route_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
