@@ -166,6 +166,17 @@ static __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint
 static __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+static __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {  // never blocks
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 static __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -829,41 +840,16 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     // memory latency of the bookkeeping is paid here, off the streaming path.  It is the only
     // warp that reads what the routing kernel wrote, so it alone waits for that kernel.
 #ifdef DEAMOE_TRACE
-    long long ptr_dep = 0, ptr_q = 0;
+    long long ptr_q = 0;
 #endif
     const int G = (int)gridDim.x;
-    int dep_ok = -1;
     int e = 0;
     uint32_t eph = 0;
     bool ok = true;
     // Queue the item `it` of the segment record held as one int4 per lane (lane l < SEG_VEC holds
-    // bytes [16 l, 16 l + 16)).  dv is a value of the item's dependency counter read earlier.
-    auto emit = [&](const int4 v, const int it, const bool dv_valid, const int dv) -> bool {
-      // dep_idx / dep_target are ints 15 and 16 of the record: lane 3 .w and lane 4 .x
-      const int dep_idx = __shfl_sync(0xffffffffu, v.w, 3);
-      const int dep_target = __shfl_sync(0xffffffffu, v.x, 4);
-      int fresh = 0;
-      if ((check_deps & 1) && dep_idx >= 0 && dep_idx != dep_ok) {
-        const int32_t* dep = P.sync + SY_DEP + dep_idx;
-        bool ready = dv_valid && __all_sync(0xffffffffu, dv >= dep_target);
-        unsigned spins = 0;
-#ifdef DEAMOE_TRACE
-        const long long tpd0 = clock64();
-#endif
-        while (!ready) {
-          ready = __all_sync(0xffffffffu, ld_acquire(dep) >= dep_target);
-          if (!ready) {
-            __nanosleep(32);
-            if (++spins > SPIN_LIMIT / 16 || *abort_flag) break;
-          }
-        }
-#ifdef DEAMOE_TRACE
-        ptr_dep += clock64() - tpd0;
-#endif
-        if (!ready) return false;
-        dep_ok = dep_idx;
-        fresh = 1;
-      }
+    // bytes [16 l, 16 l + 16)).  The planner does not wait for the item's inputs: the issue warp
+    // starts the item's weights at once and holds back only its activation rows.
+    auto emit = [&](const int4 v, const int it) -> bool {
 #ifdef DEAMOE_TRACE
       const long long tpq0 = clock64();
 #endif
@@ -899,7 +885,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
         int* tail = reinterpret_cast<int*>(ent + DESC_TAIL);
         tail[0] = 0;      // kind: work
         tail[1] = tile0;
-        tail[2] = fresh;  // inputs were acquired for this item: the issuer must fence the async proxy
+        tail[2] = 0;
         tail[3] = q_eff;
         tail[4] = nrows;
       }
@@ -944,7 +930,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
             if (lane < SEG_VEC) v = reinterpret_cast<const int4*>(stage_seg)[lane];
             have_seg = gi;
           }
-          ok = emit(v, x - gi * ips, false, 0);
+          ok = emit(v, x - gi * ips);
         }
         first_cta = (first_cta + n_items) % G;
       }
@@ -974,9 +960,8 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
         if (item >= cat_tab[4 * q2]) k = q2;
       return item;
     };
-    // Three segment records are in flight (this item's and the next two), and the dependency
-    // counter of the next item is read while this one is queued, so the planner pays one L2
-    // latency per three items, not per item.
+    // Three segment records are in flight (this item's and the next two), so the planner pays one
+    // L2 latency per three items, not per item.
     auto walk = [&]() {
       const Seg* sp0 = nullptr; const Seg* sp1 = nullptr; const Seg* sp2 = nullptr;
       int it0 = 0, it1 = 0, it2 = 0;
@@ -994,24 +979,12 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
       fetch(sp0, it0, v0);
       fetch(sp1, it1, v1);
       fetch(sp2, it2, v2);
-      int dv0 = 0;            // counter value read ahead for record 0
-      bool dv0_valid = false;
       while (ok && sp0) {
-        // read ahead: dependency counter of the next item, record of the item three ahead
-        int dv1 = 0;
-        bool dv1_valid = false;
-        if ((check_deps & 1) && sp1) {
-          const int nd = __shfl_sync(0xffffffffu, v1.w, 3);
-          if (nd >= 0 && nd != dep_ok) {
-            dv1 = ld_acquire(P.sync + SY_DEP + nd);
-            dv1_valid = true;
-          }
-        }
         const Seg* sp3; int it3 = 0; int4 v3 = make_int4(0, 0, 0, 0);
-        fetch(sp3, it3, v3);
-        ok = emit(v0, it0, dv0_valid, dv0);
+        fetch(sp3, it3, v3);  // read ahead: the record of the item three ahead
+        ok = emit(v0, it0);
         // rotate the record pipeline
-        sp0 = sp1; it0 = it1; v0 = v1; dv0 = dv1; dv0_valid = dv1_valid;
+        sp0 = sp1; it0 = it1; v0 = v1;
         sp1 = sp2; it1 = it2; v1 = v2;
         sp2 = sp3; it2 = it3; v2 = v3;
       }
@@ -1053,7 +1026,6 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     if (ok) walk();
 #ifdef DEAMOE_TRACE
     if (lane == 0 && P.trace) {
-      P.trace[(size_t)blockIdx.x * TR_SLOTS + 7] = ptr_dep;
       P.trace[(size_t)blockIdx.x * TR_SLOTS + 15] = ptr_q;
     }
 #endif
@@ -1067,109 +1039,167 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     return;
   }
 
-  if (warp >= WARP_ISSUE && warp < WARP_ISSUE + ISSUE_WARPS) {
-    // ================================================================ copy-issue warps
-    // Touch no global memory except through the bulk copies they issue.  Issuing one chunk's
-    // copies keeps a warp busy for 600-1000 cycles (about 270 for a bulk-copy instruction plus
-    // 55 for every further lane that takes part), close to the ~1150 cycles a chunk may take at
-    // full bandwidth, so the chunks of the CTA's stream alternate between ISSUE_WARPS warps.
-    // Every issue warp walks the whole descriptor queue and skips the chunks that are not its own.
-    static_assert(NSLOT % ISSUE_WARPS == 0, "an issue warp must own fixed ring slots");
-    const int ip = warp - WARP_ISSUE;
+  if (warp == WARP_ISSUE) {
+    // ================================================================ copy-issue warp
+    // Two cursors walk the CTA's chunk stream.  The WEIGHT cursor runs ahead: weights depend on
+    // nothing, so a chunk's header and weight tiles are issued as soon as a ring slot is free,
+    // also while the item's inputs do not exist yet.  The ACTIVATION cursor follows: the (tiny)
+    // activation rows of a chunk are copied once the dependency counter of its item has reached
+    // its target (one acquire load per poll; then a proxy fence, because the rows were written
+    // with ordinary stores by other CTAs).  So at a stage boundary the HBM pipe keeps running and
+    // a waiting item costs only the latency of its activation rows, not of its weights.
+    // Issuing a chunk's copies keeps the warp busy for 600-1000 cycles (about 270 for a bulk-copy
+    // instruction plus 55 for every further lane that takes part).
+    static_assert(ISSUE_WARPS == 1, "the two-cursor issue loop is written for one issue warp per CTA");
     const uint64_t pol = policy_evict_first();
-    int e = 0;
-    int cidx = 0;  // index of the item's first chunk in the CTA's chunk stream
-#ifdef DEAMOE_TRACE
-    bool routed_seen = false;
-#endif
-    uint32_t eph = 0;
+    // weight cursor
+    int e_w = 0, cw = 0, ch_w = 0, nch_w = 0, kc0_w = 0, C_w = 0, T_w = 0, tile0_w = 0, qeff_w = 0, nrows_w = 0, hflags_w = 0;
+    uint32_t eph_w = 0;
+    bool w_loaded = false, end_seen = false;
+    const __nv_bfloat16* wsrc_w = nullptr;
+    // activation cursor
+    int e_a = 0, ca = 0, ch_a = 0, nch_a = 0, kc0_a = 0, C_a = 0, qeff_a = 0, nrows_a = 0, dep_idx_a = -1, dep_tgt_a = 0;
+    bool a_loaded = false, a_ready = false;
+    const __nv_bfloat16* asrc_a[2] = {nullptr, nullptr};
+    int dep_ok = -1;  // dependency counter last seen at its target
+    unsigned idle = 0;
     bool ok = true;
 #ifdef DEAMOE_TRACE
+    bool routed_seen = false;
     long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const long long tp0 = clock64();
 #endif
-    const long long tp0 = TR_NOW();
-    (void)tp0;
     while (ok) {
-      const long long tm0 = TR_NOW();
-      if (!mbar_wait_warp(&dq_full[e], eph, abort_flag, lane, 50)) { ok = false; break; }
-      TR_ADD(TR_META, tm0);
-      const unsigned char* ent = descs + (size_t)e * DESC_BYTES;
-      const Seg* sg = reinterpret_cast<const Seg*>(ent);
-      const int* tail = reinterpret_cast<const int*>(ent + DESC_TAIL);
-      if (tail[0] != 0) break;
-      const long long td0 = TR_NOW();
+      bool progressed = false;
+      // ---- weights of chunk cw
+      if (!end_seen && !w_loaded) {
+        const bool have = __shfl_sync(0xffffffffu, (lane == 0) ? (int)mbar_test_wait(&dq_full[e_w], eph_w) : 0, 0) != 0;
+        if (have) {
+          __syncwarp();
+          const unsigned char* ent = descs + (size_t)e_w * DESC_BYTES;
+          const Seg* sg = reinterpret_cast<const Seg*>(ent);
+          const int* tail = reinterpret_cast<const int*>(ent + DESC_TAIL);
+          if (tail[0] != 0) {
+            end_seen = true;
+          } else {
+            tile0_w = tail[1]; qeff_w = tail[3]; nrows_w = tail[4];
+            T_w = sg->T; kc0_w = sg->kc; C_w = sg->C;
+            hflags_w = (qeff_w << 4) | (sg->planes << 8) | (sg->nB << 12);
+            wsrc_w = (lane < 2) ? reinterpret_cast<const __nv_bfloat16* const*>(ent + DESC_WSRC)[lane] : nullptr;
+            nch_w = (C_w + kc0_w - 1) / kc0_w;
+            ch_w = 0;
+            w_loaded = true;
 #ifdef DEAMOE_TRACE
-      if (ip == 0 && lane == 0 && !routed_seen && sg->stage != ST_SH1 && sg->stage != ST_SH2 && L.ts) {
-        routed_seen = true;
-        const unsigned long long g = gtime();
-        atomicMin(L.ts + 6, g); atomicMax(L.ts + 16, g);
+            tr[TR_ITEMS] += 1; tr[TR_CHUNKS] += nch_w;
+#endif
+          }
+        }
       }
-#endif
-      if (tail[2]) fence_proxy_async();
-      const int tile0 = tail[1], q_eff = tail[3], nrows = tail[4];
-      const int T = sg->T, kc0 = sg->kc, C = sg->C;
-      const int hflags = (q_eff << 4) | (sg->planes << 8) | (sg->nB << 12);
-      const __nv_bfloat16* wsrc = (lane < 2) ? reinterpret_cast<const __nv_bfloat16* const*>(ent + DESC_WSRC)[lane] : nullptr;
-      const __nv_bfloat16* asrc[2];
-#pragma unroll
-      for (int u = 0; u < 2; ++u)
-        asrc[u] = (lane + 32 * u < nrows) ? reinterpret_cast<const __nv_bfloat16* const*>(ent + DESC_ASRC)[lane + 32 * u]
-                                          : nullptr;
-      TR_ADD(TR_DEP, td0);
-      const int nchunks = (C + kc0 - 1) / kc0;
-#ifdef DEAMOE_TRACE
-      tr[TR_ITEMS] += 1; tr[TR_CHUNKS] += nchunks;
-#endif
-      for (int ch = 0; ch < nchunks; ++ch) {
-        if ((cidx + ch) % ISSUE_WARPS != ip) continue;
-        const int slot = (cidx + ch) % NSLOT;
-        const uint32_t phase = (uint32_t)((cidx + ch) / NSLOT) & 1u;
-        const int k0 = ch * kc0;
-        const int kc = min(kc0, C - k0);
-        const long long te0 = TR_NOW();
-        if (!mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane, 50)) { ok = false; break; }
-        TR_ADD(TR_EMPTY, te0);
-        const long long ti0 = TR_NOW();
-        unsigned char* sbase = ring + (size_t)slot * SLOT_BYTES;
-        const uint32_t wbytes = (uint32_t)kc * 32u;
-        const int astride = kc + ACT_PAD;
-        if (lane == 0) {
-          *reinterpret_cast<int4*>(sbase) = make_int4(0, hflags | (ch == 0 ? 1 : 0) | (ch == nchunks - 1 ? 2 : 0),
-                                                      kc | (T << 16), e | (tile0 << 8));
-          mbar_arrive_expect_tx(&full_bar[slot], (uint32_t)q_eff * wbytes + (uint32_t)nrows * (uint32_t)kc * 2u);
+      if (w_loaded) {
+        const int slot = cw % NSLOT;
+        const uint32_t phase = (uint32_t)(cw / NSLOT) & 1u;
+        const bool free_slot =
+            __shfl_sync(0xffffffffu, (lane == 0) ? (int)mbar_test_wait(&empty_bar[slot], phase ^ 1u) : 0, 0) != 0;
+        if (free_slot) {
+          __syncwarp();
+          const int k0 = ch_w * kc0_w;
+          const int kc = min(kc0_w, C_w - k0);
+          unsigned char* sbase = ring + (size_t)slot * SLOT_BYTES;
+          const uint32_t wbytes = (uint32_t)kc * 32u;
+          if (lane == 0) {
+            *reinterpret_cast<int4*>(sbase) = make_int4(0, hflags_w | (ch_w == 0 ? 1 : 0) | (ch_w == nch_w - 1 ? 2 : 0),
+                                                        kc | (T_w << 16), e_w | (tile0_w << 8));
+            mbar_arrive_expect_tx(&full_bar[slot], (uint32_t)qeff_w * wbytes + (uint32_t)nrows_w * (uint32_t)kc * 2u);
+          }
+          __syncwarp();
+          if (lane < qeff_w)
+            bulk_g2s_hint(sbase + SLOT_HDR + (size_t)lane * wbytes, wsrc_w + (size_t)(k0 / 16) * 256, wbytes,
+                          &full_bar[slot], pol);
+          ++cw;
+          progressed = true;
+          if (++ch_w == nch_w) {
+            w_loaded = false;
+            if (++e_w == DESC_DEPTH) { e_w = 0; eph_w ^= 1u; }
+          }
         }
-        __syncwarp();
-        if (lane < q_eff) {
-#ifdef DEAMOE_TRACE
-          if ((check_deps >> 8) == 2)
-            bulk_g2s(sbase + SLOT_HDR + (size_t)lane * wbytes, wsrc + (size_t)(k0 / 16) * 256, wbytes, &full_bar[slot]);
-          else
-#endif
-          bulk_g2s_hint(sbase + SLOT_HDR + (size_t)lane * wbytes, wsrc + (size_t)(k0 / 16) * 256, wbytes,
-                        &full_bar[slot], pol);
-        }
-        unsigned char* abase = sbase + SLOT_HDR + (size_t)q_eff * wbytes;
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int rr = lane + 32 * u;
-          if (rr < nrows)
-            bulk_g2s(abase + (size_t)rr * astride * 2, asrc[u] + k0, (uint32_t)kc * 2u, &full_bar[slot]);
-        }
-        TR_ADD(TR_ISSUE, ti0);
       }
-      cidx += nchunks;
-      if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
+      // ---- activation rows of chunk ca (its weights have been issued)
+      if (ca < cw) {
+        if (!a_loaded) {
+          const unsigned char* ent = descs + (size_t)e_a * DESC_BYTES;
+          const Seg* sg = reinterpret_cast<const Seg*>(ent);
+          const int* tail = reinterpret_cast<const int*>(ent + DESC_TAIL);
+          qeff_a = tail[3]; nrows_a = tail[4];
+          kc0_a = sg->kc; C_a = sg->C;
+          dep_idx_a = sg->dep_idx; dep_tgt_a = sg->dep_target;
+#pragma unroll
+          for (int u = 0; u < 2; ++u)
+            asrc_a[u] = (lane + 32 * u < nrows_a)
+                            ? reinterpret_cast<const __nv_bfloat16* const*>(ent + DESC_ASRC)[lane + 32 * u] : nullptr;
+          nch_a = (C_a + kc0_a - 1) / kc0_a;
+          ch_a = 0;
+          a_loaded = true;
+          a_ready = !(check_deps & 1) || dep_idx_a < 0 || dep_idx_a == dep_ok;
+#ifdef DEAMOE_TRACE
+          if (lane == 0 && !routed_seen && sg->stage != ST_SH1 && sg->stage != ST_SH2 && L.ts) {
+            routed_seen = true;
+            const unsigned long long g = gtime();
+            atomicMin(L.ts + 6, g); atomicMax(L.ts + 16, g);
+          }
+#endif
+        }
+        if (!a_ready) {
+#ifdef DEAMOE_TRACE
+          const long long td0 = clock64();
+#endif
+          const int seen = __shfl_sync(0xffffffffu, (lane == 0) ? ld_acquire(P.sync + SY_DEP + dep_idx_a) : 0, 0);
+          if (seen >= dep_tgt_a) {
+            dep_ok = dep_idx_a;
+            fence_proxy_async();  // the rows were written through the generic proxy; the copies read through the async proxy
+            a_ready = true;
+          }
+#ifdef DEAMOE_TRACE
+          tr[TR_DEP] += clock64() - td0;
+#endif
+        }
+        if (a_ready) {
+          const int slot = ca % NSLOT;
+          const int k0 = ch_a * kc0_a;
+          const int kc = min(kc0_a, C_a - k0);
+          unsigned char* abase = ring + (size_t)slot * SLOT_BYTES + SLOT_HDR + (size_t)qeff_a * kc * 32;
+          const int astride = kc + ACT_PAD;
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int rr = lane + 32 * u;
+            if (rr < nrows_a)
+              bulk_g2s(abase + (size_t)rr * astride * 2, asrc_a[u] + k0, (uint32_t)kc * 2u, &full_bar[slot]);
+          }
+          ++ca;
+          progressed = true;
+          if (++ch_a == nch_a) {
+            a_loaded = false;
+            if (++e_a == DESC_DEPTH) e_a = 0;
+          }
+        }
+      }
+      if (end_seen && ca == cw) break;
+      if (progressed) {
+        idle = 0;
+      } else {
+        if (++idle > SPIN_LIMIT || *abort_flag) { ok = false; break; }
+        __nanosleep(20);
+      }
     }
     if (!ok && lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
 #ifdef DEAMOE_TRACE
     tr[TR_PTOTAL] = clock64() - tp0;
-    if (lane == 0 && P.trace && ip == 0)
+    if (lane == 0 && P.trace)
       for (int i = 0; i < 7; ++i) P.trace[(size_t)blockIdx.x * TR_SLOTS + i] = tr[i];
 #endif
     // end-of-work marker for the consumers, in the slot after the last chunk
-    const int slot = cidx % NSLOT;
-    const uint32_t phase = (uint32_t)(cidx / NSLOT) & 1u;
-    if (cidx % ISSUE_WARPS == ip && mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane) && lane == 0) {
+    const int slot = cw % NSLOT;
+    const uint32_t phase = (uint32_t)(cw / NSLOT) & 1u;
+    if (mbar_wait_warp(&empty_bar[slot], phase ^ 1u, abort_flag, lane) && lane == 0) {
       *reinterpret_cast<int4*>(ring + (size_t)slot * SLOT_BYTES) = make_int4(1, 0, 0, 0);
       mbar_arrive(&full_bar[slot]);
     }
