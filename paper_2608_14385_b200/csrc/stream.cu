@@ -119,6 +119,7 @@ struct StreamDev {
   size_t packed_elems;
   int sh_prefix;  // fused schedule with a shared expert: its items are not in the work list
   int early;      // fused DeaMoE layers: the first stage's records are handed over ahead of the rest
+  int early_stage;              // the stage handed over early (ST_S1 or ST_V1)
   int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): step number, item count
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
   // activations between stages, bf16 planes ([rows, width] each)
@@ -560,22 +561,28 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
   }
 }
 
-// Hand the first stage (department gate / up) to the streaming kernel as soon as the department
-// token lists exist: zero the dependency counters, write the stage's segment records (the same
+static __device__ __forceinline__ int stage_kind(int stage) {  // 0 single unit, 1 departments, 2 experts
+  return (stage == ST_SH1 || stage == ST_SH2) ? 0 : ((stage == ST_S1 || stage == ST_S4) ? 1 : 2);
+}
+
+// Hand the first stage (department gate / up; for the vanilla layer the experts' gate / up) to the
+// streaming kernel as soon as its token lists exist: zero the dependency counters, write the stage's segment records (the same
 // numbering worklist_block() gives them: category 0, units in active-department order), publish
 // the item count and raise the flag with this step's number.  scr: A + 1 ints of shared memory.
 static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, int B, int* scr, int epoch) {
+  const int stage = P.early_stage;  // department gate / up, or the vanilla experts' gate / up
+  const int kind = stage_kind(stage);
   __shared__ int s_w[33];
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
 #pragma unroll 1
   for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
-  const int A = L.counts[CNT_ACTIVE_DEPT];
-  const int tg = P.st[ST_S1].tg, ips = P.st[ST_S1].items_per_seg;
+  const int A = unit_count(L, kind);
+  const int tg = P.st[stage].tg, ips = P.st[stage].items_per_seg;
   int carry = 0;  // exclusive scan of the departments' group counts, 'nthr' departments at a time
 #pragma unroll 1
   for (int base = 0; base < A; base += nthr) {
     const int a = base + tid;
-    const int gc = (a < A) ? groups_of(unit_tokens(L, ST_S1, L.active_dept[a], B), tg) : 0;
+    const int gc = (a < A) ? groups_of(unit_tokens(L, stage, unit_id(L, kind, a), B), tg) : 0;
     int incl = gc;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -604,10 +611,10 @@ static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, 
   __syncthreads();
 #pragma unroll 1
   for (int a = tid; a < A; a += nthr) {
-    const int id = L.active_dept[a];
+    const int id = unit_id(L, kind, a);
     const int gc = scr[a + 1] - scr[a];
 #pragma unroll 1
-    for (int gi = 0; gi < gc; ++gi) write_seg(L, P, ST_S1, id, gi, B, scr[a] + gi, (scr[a] + gi) * ips);
+    for (int gi = 0; gi < gc; ++gi) write_seg(L, P, stage, id, gi, B, scr[a] + gi, (scr[a] + gi) * ips);
   }
   __threadfence();  // every thread's records and zeroed counters, before the flag
   __syncthreads();
@@ -696,10 +703,11 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 12);
 #endif
   bucket_departments(S, B, s_dyn, FINISH_THREADS);
-  if (P.early)  // scratch: the words after the bucketing masks and offsets
-    early_first_stage(S, P, B, reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B), epoch);
+  int* early_scr = reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B);  // after the masks and offsets
+  if (P.early && P.early_stage == ST_S1) early_first_stage(S, P, B, early_scr, epoch);
   bucket_experts(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
+  if (P.early && P.early_stage != ST_S1) early_first_stage(S, P, B, early_scr, epoch);
 #ifdef DEAMOE_TRACE
   long long tt2 = clock64();
   TS_MIN(L, 13);
@@ -1007,7 +1015,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
         ok = false;
       } else {
         if (lane == 0) {
-          cat_tab[0] = 0; cat_tab[1] = 0; cat_tab[2] = P.st[ST_S1].items_per_seg; cat_tab[3] = ST_S1;
+          cat_tab[0] = 0; cat_tab[1] = 0; cat_tab[2] = P.st[P.early_stage].items_per_seg; cat_tab[3] = P.early_stage;
         }
         __syncwarp();
         ncat = 1; item_end = n1;
@@ -1539,7 +1547,8 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   // kernel, the last of a step, resets it.
   d.sh_prefix = (schedule == DEAMOE_SCHED_FUSED && L.n_shared && (L.vanilla || L.r > 0)) ? 1 : 0;
   if (d.sh_prefix) d.dep_sh1 = d.n_dep;
-  d.early = (schedule == DEAMOE_SCHED_FUSED && !L.vanilla && L.r > 0 && (!L.n_shared || d.sh_prefix)) ? 1 : 0;
+  d.early = (schedule == DEAMOE_SCHED_FUSED && (L.vanilla || L.r > 0) && (!L.n_shared || d.sh_prefix)) ? 1 : 0;
+  d.early_stage = L.vanilla ? ST_V1 : ST_S1;
   d.early_flag = d.n_dep + 1; d.early_items = d.n_dep + 2;  // the allocation has 8 spare counters
   d.planes = (L.adt == DEAMOE_F32) ? 2 : 1;
   {
@@ -1626,7 +1635,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
   size_t scratch = in_regs ? 0 : (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
-  const size_t bs = bucket_smem_bytes(L, B) + (size_t)(L.m + 2) * sizeof(int);  // + early_first_stage()'s scan
+  const size_t bs = bucket_smem_bytes(L, B) + (size_t)((L.vanilla ? L.n : L.m) + 2) * sizeof(int);  // + early_first_stage()'s scan
   if (bs > scratch) scratch = bs;
   scratch = (scratch + 15) & ~(size_t)15;
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
