@@ -49,6 +49,7 @@ constexpr int MAX_CAT_INTS_PAD = 8;             // cat_tab: 4 ints for each of 8
 #ifndef PREFIX_LAST_STAGE
 #define PREFIX_LAST_STAGE ST_SH1  // the shared expert's second stage waits for all of the first: it runs from the list
 #endif
+constexpr int CLAIM_AHEAD = 4;                   // unfinished items a CTA may hold while it claims from the last category
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SLOT_BYTES = 32 * 1024;
 constexpr int SLOT_HDR = 128;
@@ -119,6 +120,7 @@ struct StreamDev {
   size_t packed_elems;
   int sh_prefix;  // fused schedule with a shared expert: its items are not in the work list
   int early;      // fused DeaMoE layers: the first stage's records are handed over ahead of the rest
+  int claim_items;              // fused schedule: the items of the list are claimed, not dealt
   int early_stage;              // the stage handed over early (ST_S1 or ST_V1)
   int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): step number, item count
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
@@ -823,7 +825,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
   uint64_t* red_empty = red_full + NRED;
   int* cat_tab = reinterpret_cast<int*>(red_empty + NRED);             // 4 * MAX_CAT ints
   int* red_info = cat_tab + 4 * MAX_CAT;                               // NRED x {e | tile0 << 8, q, T, 0}
-  volatile int* ctl = red_info + 4 * NRED;                             // [0] abort, [1] closed, [2] items produced
+  volatile int* ctl = red_info + 4 * NRED;  // [0] abort, [1] closed, [2] items produced, [3] items completed
   volatile int* abort_flag = ctl;
   unsigned char* seg_stage = reinterpret_cast<unsigned char*>(red_info + 4 * NRED + 4);  // one Seg, planner only
 
@@ -833,7 +835,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     for (int s = 0; s < NSLOT; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], CONSUMER_WARPS); }
     for (int s = 0; s < DESC_DEPTH; ++s) { mbar_init(&dq_full[s], 1); mbar_init(&dq_empty[s], 1); }
     for (int s = 0; s < NRED; ++s) { mbar_init(&red_full[s], CONSUMER_WARPS); mbar_init(&red_empty[s], 1); }
-    ctl[0] = 0; ctl[1] = 0; ctl[2] = 0;
+    ctl[0] = 0; ctl[1] = 0; ctl[2] = 0; ctl[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -857,6 +859,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     // Queue the item `it` of the segment record held as one int4 per lane (lane l < SEG_VEC holds
     // bytes [16 l, 16 l + 16)).  The planner does not wait for the item's inputs: the issue warp
     // starts the item's weights at once and holds back only its activation rows.
+    int queued = 0;  // items this planner has queued
     auto emit = [&](const int4 v, const int it) -> bool {
 #ifdef DEAMOE_TRACE
       const long long tpq0 = clock64();
@@ -915,6 +918,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&dq_full[e]);
       if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
+      ++queued;
       return true;
     };
 
@@ -959,10 +963,37 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     // Dealing the items out (rather than giving a CTA one contiguous stretch per category)
     // completes the units one after another, so dependent items of later categories become ready
     // early; contiguous stretches were measured 25-35 % slower for that reason.
+    // Fused schedule: the items are not dealt out but CLAIMED, one by one and in list order, from a
+    // global counter, and a CTA claims only while fewer than CLAIM_AHEAD of its items are
+    // unfinished.  The CTAs move through the list at different speeds (the shared expert's items,
+    // stalls at stage boundaries, unequal items); claiming lets the fast ones take what the slow
+    // ones would have been left with, and because claims follow the list order an item still
+    // depends only on items claimed before it.  The first stage (phase 1) is dealt out, item i to
+    // CTA i mod grid, like the categories of a staged launch; claiming starts with the second
+    // category.  A single token's list is dealt out entirely: its short middle stages lose more to
+    // the claim's latency than they gain (171 against 164 us).
+    int claim_base = 0x7fffffff;  // first claimed item (set in phase 2 of a fused launch)
+    bool claiming = false;        // the dealt items before claim_base are used up
     auto next_item = [&](int& k) -> int {  // next item of this CTA, -1 at the end of the phase
-      if (cur_i >= item_end) return -1;
-      const int item = cur_i;
-      cur_i += G;
+      int item = -1;
+      if (!claiming) {
+        if (cur_i >= item_end) return -1;
+        item = cur_i;
+        cur_i += G;
+        if (item >= claim_base) { claiming = true; item = -1; }
+      }
+      if (claiming) {
+        if (lane == 0) {
+          unsigned spins = 0;
+          while (queued - ctl[3] >= CLAIM_AHEAD) {  // throttle: stay close to what is actually finished
+            __nanosleep(100);
+            if (++spins > SPIN_LIMIT / 16 || *abort_flag) break;
+          }
+          item = claim_base + atomicAdd(P.sync + SY_CLAIM, 1);
+        }
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item >= item_end) { cur_i = item_end; return -1; }
+      }
       k = 0;
       for (int q2 = 1; q2 < ncat; ++q2)
         if (item >= cat_tab[4 * q2]) k = q2;
@@ -985,16 +1016,17 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
         }
       };
       fetch(sp0, it0, v0);
-      fetch(sp1, it1, v1);
-      fetch(sp2, it2, v2);
+      if (!claiming) fetch(sp1, it1, v1);
+      if (!claiming) fetch(sp2, it2, v2);
       while (ok && sp0) {
-        const Seg* sp3; int it3 = 0; int4 v3 = make_int4(0, 0, 0, 0);
-        fetch(sp3, it3, v3);  // read ahead: the record of the item three ahead
+        const Seg* sp3 = nullptr; int it3 = 0; int4 v3 = make_int4(0, 0, 0, 0);
+        if (!claiming) fetch(sp3, it3, v3);  // read ahead: the record of the item three ahead
         ok = emit(v0, it0);
         // rotate the record pipeline
         sp0 = sp1; it0 = it1; v0 = v1;
         sp1 = sp2; it1 = it2; v1 = v2;
         sp2 = sp3; it2 = it3; v2 = v3;
+        if (ok && !sp0 && claiming) fetch(sp0, it0, v0);  // no read-ahead while claiming: a claimed item is a held item
       }
     };
 
@@ -1031,6 +1063,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     if (cat >= 0) cur_i = cat_tab[4 * cat] + (int)blockIdx.x;
     item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
     if (*abort_flag && lane == 0) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;  // set before the routing kernel reset it
+    if (cat < 0 && P.claim_items && ncat >= 2 && B > 1) claim_base = cat_tab[4];
     if (ok) walk();
 #ifdef DEAMOE_TRACE
     if (lane == 0 && P.trace) {
@@ -1297,6 +1330,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
       if (lane == 0) {
         mbar_arrive(&red_empty[rb]);
         mbar_arrive(&dq_empty[e]);  // the descriptor may be reused
+        ctl[3] = n + 1;             // items completed (read by the planner while it claims items)
       }
       if (done) {
 #pragma unroll
@@ -1549,6 +1583,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   if (d.sh_prefix) d.dep_sh1 = d.n_dep;
   d.early = (schedule == DEAMOE_SCHED_FUSED && (L.vanilla || L.r > 0) && (!L.n_shared || d.sh_prefix)) ? 1 : 0;
   d.early_stage = L.vanilla ? ST_V1 : ST_S1;
+  d.claim_items = (schedule == DEAMOE_SCHED_FUSED && (L.vanilla || L.r > 0)) ? 1 : 0;
   d.early_flag = d.n_dep + 1; d.early_items = d.n_dep + 2;  // the allocation has 8 spare counters
   d.planes = (L.adt == DEAMOE_F32) ? 2 : 1;
   {
