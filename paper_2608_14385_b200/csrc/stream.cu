@@ -49,6 +49,7 @@ constexpr int MAX_CAT_INTS_PAD = 8;             // cat_tab: 4 ints for each of 8
 #ifndef PREFIX_LAST_STAGE
 #define PREFIX_LAST_STAGE ST_SH1  // the shared expert's second stage waits for all of the first: it runs from the list
 #endif
+constexpr int CLAIM_MIN_PER_CTA = 16;            // lists with fewer items per CTA are dealt out, not claimed
 constexpr int CLAIM_AHEAD = 4;                   // unfinished items a CTA may hold while it claims from the last category
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SLOT_BYTES = 32 * 1024;
@@ -970,8 +971,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     // ones would have been left with, and because claims follow the list order an item still
     // depends only on items claimed before it.  The first stage (phase 1) is dealt out, item i to
     // CTA i mod grid, like the categories of a staged launch; claiming starts with the second
-    // category.  A single token's list is dealt out entirely: its short middle stages lose more to
-    // the claim's latency than they gain (171 against 164 us).
+    // category.  A short list (fewer than CLAIM_MIN_PER_CTA items per CTA: a single token, a small
+    // layer) is dealt out entirely: it loses more to the claim's latency than it gains (171 against
+    // 164 us for one token on the DeepSeek-V3 shape).
     int claim_base = 0x7fffffff;  // first claimed item (set in phase 2 of a fused launch)
     bool claiming = false;        // the dealt items before claim_base are used up
     auto next_item = [&](int& k) -> int {  // next item of this CTA, -1 at the end of the phase
@@ -1063,7 +1065,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
     if (cat >= 0) cur_i = cat_tab[4 * cat] + (int)blockIdx.x;
     item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
     if (*abort_flag && lane == 0) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;  // set before the routing kernel reset it
-    if (cat < 0 && P.claim_items && ncat >= 2 && B > 1) claim_base = cat_tab[4];
+    if (cat < 0 && P.claim_items && ncat >= 2 && item_end >= CLAIM_MIN_PER_CTA * G) claim_base = cat_tab[4];
     if (ok) walk();
 #ifdef DEAMOE_TRACE
     if (lane == 0 && P.trace) {
