@@ -6,13 +6,14 @@
 // that one 16-row tile of a matrix is a contiguous stream whose 512-byte pieces are the
 // per-lane A fragments of mma.sync.m16n8k16.  One persistent kernel (CTAS_PER_SM co-resident
 // CTAs on every SM) then works through a device-built list of items (one or two 16-row tiles x
-// the full contraction length), item i going to CTA i mod grid.  Warp roles inside a CTA:
+// the full contraction length).  Warp roles inside a CTA:
 //
-//   planner warp  : reads the records of its items ahead of time, waits (bounded) until an
-//                   item's inputs exist, resolves all source pointers and queues a descriptor
-//                   in shared memory;
-//   issue warp(s) : move weight chunks (HBM, evict-first) and the matching activation rows
-//                   (L2) into a shared-memory ring with cp.async.bulk, completion on mbarriers;
+//   planner warp  : picks the CTA's items (the first stage is dealt out, the rest is claimed in
+//                   list order from a global counter), checks their records, resolves all source
+//                   pointers and queues a descriptor in shared memory;
+//   issue warp    : moves weight chunks (HBM, evict-first) into a shared-memory ring with
+//                   cp.async.bulk as soon as a slot is free, and the matching activation rows
+//                   (L2) once the item's inputs exist; completion on mbarriers;
 //   consumer warps: split each chunk's k-tiles, accumulate in fp32 with mma.sync on bf16
 //                   activations (one plane, or hi + lo planes for fp32 tokens) and hand their
 //                   partial sums of a finished item to
@@ -37,9 +38,9 @@ namespace deamoe {
 
 constexpr int CTAS_PER_SM = 2;                   // co-resident CTAs of the streaming kernel per SM
 constexpr int CONSUMER_WARPS = 4;
-constexpr int ISSUE_WARPS = 1;                   // copy-issue warps; warp p fills chunks p, p + ISSUE_WARPS, ...
+constexpr int ISSUE_WARPS = 1;                   // copy-issue warps per CTA (two CTAs per SM, so two per SM)
 constexpr int WARP_ISSUE = CONSUMER_WARPS;       // first of the warps that issue the bulk copies
-constexpr int WARP_PLAN = WARP_ISSUE + ISSUE_WARPS;  // picks items, fetches records, waits for inputs
+constexpr int WARP_PLAN = WARP_ISSUE + ISSUE_WARPS;  // picks items, fetches records, queues descriptors
 constexpr int WARP_EPI = WARP_PLAN + 1;          // reduces, applies epilogues, publishes completions
 constexpr int STREAM_THREADS = (WARP_EPI + 1) * 32;
 constexpr int DESC_DEPTH = 8;                    // item descriptors queued between planner and epilogue
