@@ -20,8 +20,8 @@
  *  - deamoe_route / deamoe_forward only ENQUEUE work on the given stream; they never
  *    synchronise and never allocate (all workspace is sized at create for max_batch).
  *    Calls on one layer must be enqueued on one stream (or otherwise ordered): a layer has one
- *    workspace.  A step of the FUSED schedule carries its own sequence number as a kernel
- *    argument, so a step captured into a CUDA graph must not be replayed; use the STAGED schedule there.
+ *    workspace.  A step keeps no per-step state on the host, so it may be captured into a CUDA
+ *    graph and replayed (Section 5 of the paper runs its steps that way).
  *  - There is no CPU fallback and no other backend: without a CUDA device the create
  *    calls fail with DEAMOE_ERR_CUDA.
  */

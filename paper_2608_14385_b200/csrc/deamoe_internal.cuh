@@ -121,7 +121,8 @@ static __device__ __forceinline__ float sigma_f(int kind, float v) {
 int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices, int32_t* user_idx,
                  float* user_w);
 size_t bucket_smem_bytes(const LayerDev& L, int B);
-int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices);
+int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
+                         int32_t* step_flag = nullptr);
 cudaError_t route_configure(const LayerDev& L);
 int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s);
 int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s);

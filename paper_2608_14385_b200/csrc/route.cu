@@ -33,10 +33,20 @@ static __device__ __forceinline__ float4 load_x4(const __nv_bfloat16* p) {
 template <typename XT>
 __global__ void __launch_bounds__(ROUTER_THREADS)
 k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float* __restrict__ part,
-                int n, int h, int B, int kslice TS_PARAM) {
+                int n, int h, int B, int kslice, int32_t* __restrict__ step_flag TS_PARAM) {
 #ifdef DEAMOE_TRACE
   if (threadIdx.x == 0 && ts) atomicMin(ts + 0, gtime());
 #endif
+  // step_flag (may be null): the word through which the routing tail tells the streaming kernel
+  // that the first stage's records exist.  It is cleared here, before this grid releases its
+  // dependents, so a streaming kernel can never see the value of the step before.
+  if (step_flag && blockIdx.x == 0 && blockIdx.y == 0) {
+    if (threadIdx.x == 0) {
+      *step_flag = 0;
+      __threadfence();
+    }
+    __syncthreads();
+  }
   // Kernels launched behind this one with programmatic stream serialization (the routing tail, and
   // through it the streaming kernel with the routing-independent shared expert) may become
   // resident right away; they wait for this grid's results themselves.
@@ -138,15 +148,15 @@ cudaError_t route_configure(const LayerDev& L) {
 
 // Router logits straight from the caller's tokens (no fp32 copy): used by the streaming schedules.
 // Returns the number of column slices written (the second grid dimension), or -1.
-int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices) {
+int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices, int32_t* step_flag) {
   const int kslice = (((L.h + kslices - 1) / kslices) + 3) & ~3;
   dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
   if (L.adt == DEAMOE_BF16)
     k_router_logits<__nv_bfloat16><<<grid, ROUTER_THREADS, 0, s>>>(L.router, reinterpret_cast<const __nv_bfloat16*>(tokens),
-                                                                  L.logit_part, L.n, L.h, B, kslice TS_ARG(L));
+                                                                  L.logit_part, L.n, L.h, B, kslice, step_flag TS_ARG(L));
   else
     k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, reinterpret_cast<const float*>(tokens), L.logit_part,
-                                                          L.n, L.h, B, kslice TS_ARG(L));
+                                                          L.n, L.h, B, kslice, step_flag TS_ARG(L));
   return cudaGetLastError() == cudaSuccess ? (int)grid.y : -1;
 }
 
@@ -161,7 +171,7 @@ int launch_route(const LayerDev& L, const void* tokens, int B, cudaStream_t s, i
   }
   const int kslice = (((L.h + kslices - 1) / kslices) + 3) & ~3;
   dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
-  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, L.x32, L.logit_part, L.n, L.h, B, kslice TS_ARG(L));
+  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(L.router, L.x32, L.logit_part, L.n, L.h, B, kslice, nullptr TS_ARG(L));
   ++launches;
   const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
   k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, (int)grid.y, user_idx, user_w);
@@ -238,7 +248,7 @@ extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* r
   L.logit_part = g_route_scratch_ptr[dev];   // every (slice, token, expert) entry used below is overwritten
   L.topk_idx = topk_idx; L.topk_w = topk_w;  // results go straight to the caller's buffers
   dim3 grid((L.n + RG - 1) / RG, ny);
-  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice TS_ARG(L));
+  k_router_logits<float><<<grid, ROUTER_THREADS, 0, s>>>(router, tokens, L.logit_part, L.n, hidden, B, kslice, nullptr TS_ARG(L));
   const size_t topk_smem = (size_t)TOPK_WARPS * L.n * (sizeof(float) + 1);
   k_topk<<<(B + TOPK_WARPS - 1) / TOPK_WARPS, TOPK_WARPS * 32, topk_smem, s>>>(L, B, ny, nullptr, nullptr);
   return cudaGetLastError() == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;

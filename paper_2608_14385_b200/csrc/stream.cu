@@ -147,7 +147,6 @@ struct StreamPlan {
   int schedule;
   int n_sm;
   int grid;  // CTAs of the streaming kernel: all of them must be resident at once
-  int epoch; // number of the last routing call (never 0): tags the early hand-over flag
   void* packed;
   uint64_t bytes;
   cudaEvent_t ev0, ev1;   // profiling event pair (null when profiling is off)
@@ -573,7 +572,7 @@ static __device__ __forceinline__ int stage_kind(int stage) {  // 0 single unit,
 // streaming kernel as soon as its token lists exist: zero the dependency counters, write the stage's segment records (the same
 // numbering worklist_block() gives them: category 0, units in active-department order), publish
 // the item count and raise the flag with this step's number.  scr: A + 1 ints of shared memory.
-static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, int B, int* scr, int epoch) {
+static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, int B, int* scr) {
   const int stage = P.early_stage;  // department gate / up, or the vanilla experts' gate / up
   const int kind = stage_kind(stage);
   __shared__ int s_w[33];
@@ -625,7 +624,7 @@ static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, 
   if (tid == 0) {
     P.sync[SY_DEP + P.early_items] = (carry <= P.max_segs) ? carry * ips : 0;
     __threadfence();
-    st_release(P.sync + SY_DEP + P.early_flag, epoch);
+    st_release(P.sync + SY_DEP + P.early_flag, 1);  // cleared again by the next step's router kernel
   }
 }
 
@@ -660,7 +659,7 @@ static __host__ __device__ FinishSmem finish_layout(int n, int m, int k, int B) 
 }
 
 __global__ void __launch_bounds__(FINISH_THREADS)
-k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words, int epoch,
+k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   extern __shared__ uint32_t s_dyn[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
@@ -708,10 +707,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
 #endif
   bucket_departments(S, B, s_dyn, FINISH_THREADS);
   int* early_scr = reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B);  // after the masks and offsets
-  if (P.early && P.early_stage == ST_S1) early_first_stage(S, P, B, early_scr, epoch);
+  if (P.early && P.early_stage == ST_S1) early_first_stage(S, P, B, early_scr);
   bucket_experts(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
-  if (P.early && P.early_stage != ST_S1) early_first_stage(S, P, B, early_scr, epoch);
+  if (P.early && P.early_stage != ST_S1) early_first_stage(S, P, B, early_scr);
 #ifdef DEAMOE_TRACE
   long long tt2 = clock64();
   TS_MIN(L, 13);
@@ -814,7 +813,7 @@ struct __align__(16) ItemCtx {  // producer-side view of one claimed item
 };
 
 __global__ void __launch_bounds__(STREAM_THREADS, CTAS_PER_SM)
-k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
+k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* red = reinterpret_cast<float*>(smem + (size_t)NSLOT * SLOT_BYTES);
@@ -1039,7 +1038,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps, int epoch) {
         const int32_t* flag = P.sync + SY_DEP + P.early_flag;
         unsigned spins = 0;
         bool seen = true;
-        while (ld_acquire(flag) != epoch) {
+        while (ld_acquire(flag) != 1) {
           __nanosleep(64);
           if (++spins > SPIN_LIMIT / 16 || *abort_flag) { seen = false; break; }
         }
@@ -1501,7 +1500,6 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   if (!p) return DEAMOE_ERR_ALLOC;
   std::memset(p, 0, sizeof(*p));
   p->schedule = schedule;
-  p->epoch = 0;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->n_sm, cudaDevAttrMultiProcessorCount, dev);
@@ -1664,7 +1662,8 @@ int32_t* stream_shared_counter(StreamPlan& p) {
 
 int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
                  int32_t* user_idx, float* user_w) {
-  const int ny = launch_router_logits(L, tokens, B, s, kslices);
+  const int ny = launch_router_logits(L, tokens, B, s, kslices,
+                                      p.dev.early ? p.dev.sync + SY_DEP + p.dev.early_flag : nullptr);
   if (ny < 0) return -1;
   const int per_warp = (L.n * 5 + 15) & ~15;
   const bool in_regs = topk_in_registers(L);
@@ -1679,9 +1678,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   const size_t smem = scratch + (size_t)fl.total * 4;
   if (smem > 200 * 1024) return -1;
-  if (++p.epoch == 0) p.epoch = 1;
   launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, p.dev, B, ny, topk_warps, (int)(scratch / 4),
-             p.epoch,
              user_idx, user_w);
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
@@ -1724,7 +1721,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | dbgflag, p.epoch);
+    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | dbgflag);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
@@ -1732,7 +1729,7 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
         k_identity_private<<<p.n_sm, 256, 0, s>>>(L, p.dev);
         ++launches;
       }
-      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, B, c, 0, p.epoch);
+      k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev, B, c, 0);
       ++launches;
     }
   }

@@ -235,3 +235,33 @@ def test_non_finite_tokens_keep_indices_valid():
         assert ok, (err, bound)
     finally:
         layer.close()
+
+
+def test_fused_step_can_be_captured_in_a_cuda_graph_and_replayed():
+    """A step allocates nothing and keeps no per-step state on the host, so it can be captured once
+    and replayed on new token values in the same buffer; every replay must equal the eager result."""
+    shape = RAGGED
+    w = _scaled(shape, 6)
+    layer = binding.Layer(shape, w, 8, binding.SCHED_FUSED)
+    try:
+        x = synth.make_tokens(shape, 5, 31, "cuda:0")
+        out = torch.empty_like(x)
+        layer.forward(x, out)                      # warm-up outside the capture
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                layer.forward(x, out)
+        torch.cuda.synchronize()
+        for seed in (32, 33, 34):
+            new = synth.make_tokens(shape, 5, seed, "cuda:0")
+            want = layer.forward(new).clone()
+            torch.cuda.synchronize()
+            x.copy_(new)
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(out, want), seed
+        assert layer.stats()["device_status"] == 0
+    finally:
+        layer.close()
