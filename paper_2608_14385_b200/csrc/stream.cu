@@ -572,8 +572,9 @@ static __device__ __forceinline__ int stage_kind(int stage) {  // 0 single unit,
 // streaming kernel as soon as its token lists exist: zero the dependency counters, write the stage's segment records (the same
 // numbering worklist_block() gives them: category 0, units in active-department order), publish
 // the item count and raise the flag with this step's number.  scr: A + 1 ints of shared memory.
+template <int STAGE>  // ST_S1 or ST_V1: a compile-time stage keeps only that stage's record code (this runs cold)
 static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, int B, int* scr) {
-  const int stage = P.early_stage;  // department gate / up, or the vanilla experts' gate / up
+  constexpr int stage = STAGE;
   const int kind = stage_kind(stage);
   __shared__ int s_w[33];
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
@@ -707,10 +708,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
 #endif
   bucket_departments(S, B, s_dyn, FINISH_THREADS);
   int* early_scr = reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B);  // after the masks and offsets
-  if (P.early && P.early_stage == ST_S1) early_first_stage(S, P, B, early_scr);
+  if (P.early && P.early_stage == ST_S1) early_first_stage<ST_S1>(S, P, B, early_scr);
   bucket_experts(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
-  if (P.early && P.early_stage != ST_S1) early_first_stage(S, P, B, early_scr);
+  if (P.early && P.early_stage != ST_S1) early_first_stage<ST_V1>(S, P, B, early_scr);
 #ifdef DEAMOE_TRACE
   long long tt2 = clock64();
   TS_MIN(L, 13);
