@@ -144,3 +144,64 @@ def test_layers_enqueued_back_to_back_match_layers_run_one_by_one(vanilla):
     finally:
         for layer in layers:
             layer.close()
+
+
+WIDE_ROUTERS = [
+    # n_dept, experts_per_dept, top_k, k_dept
+    (6, 16, 6, 0),       # 96 experts: 8 logits per lane
+    (10, 32, 10, 0),     # 320 experts: 16 logits per lane
+    (10, 32, 10, 4),     # group limited
+    (8, 108, 10, 5),     # the paper's DeepSeek-V3 router
+    (32, 32, 32, 0),     # 1024 experts, top-32: the widest the register top-k takes
+    (32, 32, 8, 3),
+    (40, 40, 8, 6),      # 1600 experts, 40 departments: the shared-memory top-k
+]
+
+
+@pytest.mark.parametrize("m,g,k,k_dept", WIDE_ROUTERS)
+def test_routing_of_wide_and_group_limited_routers(m, g, k, k_dept):
+    """Routing only (indices, gate weights, department and expert lists) on layers with tiny experts but
+    wide routers, so that every top-k variant (8 / 16 / 32 logits per lane, group limit in registers,
+    shared-memory fallback) is compared with the oracle, with random logits and with exact ties."""
+    shape = synth.LayerShape(f"wide{m}x{g}", hidden=256, n_dept=m, experts_per_dept=g, ffn=16, priv=16, top_k=k,
+                             k_dept=k_dept)
+    dev = torch.device("cuda:0")
+    w = synth.make_deamoe_weights(shape, 2, dev)
+    layer = binding.Layer(shape, w, 40)
+    try:
+        cfg = oracle_cfg(shape)
+        for B, seed in ((1, 3), (5, 4), (33, 5), (40, 6)):
+            tokens = synth.make_tokens(shape, B, seed, dev)
+            layer.route(tokens, want_outputs=False)
+            torch.cuda.synchronize()
+            want = ref.route(cfg, synth.to_numpy(w["router"]), synth.to_numpy(tokens), want_logits=True)
+            safe = want["gap"] > 1e-5 * np.abs(want["logits"]).max(axis=1)
+            got = layer.routing(B)
+            assert safe.mean() > 0.5
+            assert (got["idx"][safe] == want["idx"][safe]).all()
+            assert np.abs(got["w"][safe].astype(np.float64) - want["w"][safe]).max() <= 1e-5
+            if safe.all():
+                bk = ref.bucket(cfg, want["idx"])
+                for key in ("dept_mask", "dept_off", "dept_tok", "expert_off", "expert_tok"):
+                    assert (got[key] == bk[key]).all(), key
+        # exact ties: small integers in the router and the tokens make every logit an exact integer in
+        # fp32 and fp64 alike, with many equal values; the order must be (logit descending, index ascending)
+        gen = torch.Generator(device="cpu").manual_seed(7)
+        router = torch.randint(-2, 3, (shape.n_expert, shape.hidden), generator=gen).float()
+        w2 = dict(w)
+        w2["router"] = router.to(dev)
+        tied = binding.Layer(shape, w2, 8)
+        try:
+            tokens = torch.randint(-2, 3, (8, shape.hidden), generator=gen).to(torch.bfloat16).to(dev)
+            tied.route(tokens, want_outputs=False)
+            torch.cuda.synchronize()
+            want = ref.route(cfg, synth.to_numpy(w2["router"]), synth.to_numpy(tokens))
+            got = tied.routing(8)
+            assert (got["idx"] == want["idx"]).all()
+            bk = ref.bucket(cfg, want["idx"])
+            for key in ("dept_off", "dept_tok", "expert_off", "expert_tok"):
+                assert (got[key] == bk[key]).all(), key
+        finally:
+            tied.close()
+    finally:
+        layer.close()
