@@ -93,6 +93,23 @@ static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslic
 
 // Same result with the logits held in registers (n <= 32 * VPL, flat top-k): every partial-logit
 // load is issued before the first use, and the k selection rounds touch no memory at all.
+// Largest key of the eight keys of group GI that are not masked by `taken`, and the lowest index
+// that holds it (strict compare).  GI is a template argument so that key[] is only ever indexed
+// with constants and stays in registers.
+template <int GI, int VPL>
+static __device__ __forceinline__ void rescan_group(const unsigned (&key)[VPL], unsigned taken, unsigned& mx_out,
+                                                    int& mj_out) {
+  unsigned mx = 0u;
+  int mj = GI * 8;
+#pragma unroll
+  for (int jj = 0; jj < 8; ++jj) {
+    const unsigned kq = ((taken >> (GI * 8 + jj)) & 1u) ? 0u : key[GI * 8 + jj];
+    if (kq > mx) { mx = kq; mj = GI * 8 + jj; }
+  }
+  mx_out = mx;
+  mj_out = mj;
+}
+
 template <int VPL>
 static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int kslices, int lane,
                                            int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
@@ -179,23 +196,54 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
       if (idx < (unsigned)n && !((alive >> d) & 1u)) taken |= 1u << j;
     }
   }
+  // Selection on order-preserving integer keys (larger logit <=> larger key, equal logits <=> equal
+  // keys; 0 stands for "not a candidate").  A lane keeps the maximum of each group of eight of its
+  // keys, so a round costs a handful of compares, two warp reductions (largest key, then the
+  // lowest index that holds it: ties go to the lower expert index) and, in the winning lane only,
+  // the rescan of one group.  The keys are never modified: selected and excluded elements are
+  // masked through `taken`.
+  static_assert(VPL % 8 == 0 && VPL <= 32, "keys are grouped by eight, at most four groups");
+  constexpr int NG = VPL / 8;
+  unsigned key[VPL];
+#pragma unroll
+  for (int j = 0; j < VPL; ++j) {
+    const unsigned bits = __float_as_uint(v[j] + 0.f);  // + 0.f: -0 and +0 are one value, so they get one key
+    key[j] = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+  }
+  unsigned gmax[NG];
+  int gj[NG];
+#define DEAMOE_EACH_GROUP(OP) \
+  { if (NG > 0) { OP(0) } if (NG > 1) { OP(1) } if (NG > 2) { OP(2) } if (NG > 3) { OP(3) } }
+#define DEAMOE_GI(GI) ((GI) < NG ? (GI) : 0)
+#define DEAMOE_RESCAN(GI) rescan_group<DEAMOE_GI(GI), VPL>(key, taken, gmax[DEAMOE_GI(GI)], gj[DEAMOE_GI(GI)]);
+#define DEAMOE_RESCAN_IF(GI) if ((js >> 3) == (GI)) { DEAMOE_RESCAN(GI) }
+  DEAMOE_EACH_GROUP(DEAMOE_RESCAN)
   float my_v = 0.f;  // lane q keeps the q-th selected logit (k <= 32)
   int my_i = 0;
+#pragma unroll 1
   for (int q = 0; q < k; ++q) {
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
+    unsigned best = gmax[0];
+    int bj = gj[0];
 #pragma unroll
-    for (int j = 0; j < VPL; ++j)
-      if (!((taken >> j) & 1u) && better(v[j], lane + 32 * j, bv, bi)) { bv = v[j]; bi = lane + 32 * j; }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    for (int gi = 1; gi < NG; ++gi)
+      if (gmax[gi] > best) { best = gmax[gi]; bj = gj[gi]; }
+    const unsigned wmax = __reduce_max_sync(0xffffffffu, best);
+    const unsigned cand = (best == wmax && wmax != 0u) ? (unsigned)(lane + 32 * bj) : 0x7fffffffu;
+    const unsigned widx = __reduce_min_sync(0xffffffffu, cand);
+    if (lane == q) {
+      my_i = (int)widx;
+      my_v = __uint_as_float((wmax & 0x80000000u) ? (wmax ^ 0x80000000u) : ~wmax);
     }
-    if (lane == q) { my_v = bv; my_i = bi; }
-    if (bi < n && lane == (bi & 31)) taken |= 1u << (bi >> 5);
+    if (widx != 0x7fffffffu && lane == (int)(widx & 31u)) {  // the owner masks the element and rescans its group
+      const int js = (int)(widx >> 5);
+      taken |= 1u << js;
+      DEAMOE_EACH_GROUP(DEAMOE_RESCAN_IF)
+    }
   }
+#undef DEAMOE_RESCAN_IF
+#undef DEAMOE_RESCAN
+#undef DEAMOE_GI
+#undef DEAMOE_EACH_GROUP
 #ifdef DEAMOE_TRACE
   if (lane == 0 && t == 0) { L.counts[11] = (int)(clock64() - ta); L.counts[12] = (int)(ta & 0x7fffffff); }
 #endif
