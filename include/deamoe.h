@@ -57,7 +57,13 @@ typedef enum {
   DEAMOE_SCHED_AUTO = 0,   /* the library's best schedule for the dtype */
   DEAMOE_SCHED_PLAIN = 1,  /* one simple kernel per stage on the canonical layouts (any dtype) */
   DEAMOE_SCHED_STAGED = 2, /* bf16 weight-streaming kernel, one launch per stage */
-  DEAMOE_SCHED_FUSED = 3   /* bf16 weight-streaming kernel, one persistent launch for all stages */
+  DEAMOE_SCHED_FUSED = 3,  /* bf16 weight-streaming kernel, one persistent launch for all stages */
+  DEAMOE_SCHED_DENSE = 4   /* larger batches, where a department's token bucket X^j (Section 3.2) is a
+                              dense tile: department and shared-expert matrices on the tcgen05 tensor
+                              cores, private matrices in the streaming kernel.  bf16 weights and
+                              tokens, a DeaMoE layer with private matrices, h, f and shared_ffn
+                              multiples of 128; else UNSUPPORTED.  AUTO takes this schedule by
+                              itself for calls of 48 tokens and more on layers that support it. */
 } deamoe_schedule_t;
 
 /*

@@ -64,7 +64,7 @@ deamoe_status_t check_config(const deamoe_config_t* c, const deamoe_weights_t* w
   if (c->weight_dtype != DEAMOE_F32 && c->weight_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
   if (c->act_dtype != DEAMOE_F32 && c->act_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
   if (c->sigma < DEAMOE_SIGMA_NONE || c->sigma > DEAMOE_SIGMA_GELU) return DEAMOE_ERR_INVALID_ARG;
-  if (c->schedule < DEAMOE_SCHED_AUTO || c->schedule > DEAMOE_SCHED_FUSED) return DEAMOE_ERR_INVALID_ARG;
+  if (c->schedule < DEAMOE_SCHED_AUTO || c->schedule > DEAMOE_SCHED_DENSE) return DEAMOE_ERR_INVALID_ARG;
   if (!(c->route_scale == c->route_scale)) return DEAMOE_ERR_INVALID_ARG;
   if (c->max_batch < 1 || c->max_batch > DEAMOE_MAX_BATCH) return DEAMOE_ERR_BATCH;
   if (!w->router || !w->dept_gate || !w->dept_up || !w->dept_down) return DEAMOE_ERR_INVALID_ARG;
@@ -108,6 +108,9 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   int sched = cfg->schedule;
   const bool streamable = cfg->weight_dtype == DEAMOE_BF16 &&
                           ((cfg->hidden | cfg->ffn | cfg->priv | cfg->shared_ffn) & 15) == 0;
+  // the dense schedule rides on a fused plan: AUTO switches to it by batch size, DENSE always takes it
+  const int dense_mode = sched == DEAMOE_SCHED_DENSE ? 2 : (sched == DEAMOE_SCHED_AUTO ? 1 : 0);
+  if (sched == DEAMOE_SCHED_DENSE) sched = DEAMOE_SCHED_FUSED;
   if (sched == DEAMOE_SCHED_AUTO) sched = streamable ? stream_default_schedule() : DEAMOE_SCHED_PLAIN;
   if ((sched == DEAMOE_SCHED_STAGED || sched == DEAMOE_SCHED_FUSED) && !streamable) {
     delete L;
@@ -181,7 +184,7 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   if (ok && route_configure(d) != cudaSuccess) A(DEAMOE_ERR_CUDA);
   if (ok && sched != DEAMOE_SCHED_PLAIN) {
     uint64_t plan_bytes = 0;
-    A(stream_plan_create(d, *w, sched, s, &L->plan, &plan_bytes));
+    A(stream_plan_create(d, *w, sched, dense_mode, s, &L->plan, &plan_bytes));
     L->device_bytes += plan_bytes;
     if (ok) d.sh_done = stream_shared_counter(*L->plan);
   }

@@ -1,0 +1,35 @@
+// Tensor-core (tcgen05 / TMEM) kernels for the stages whose token buckets are dense at larger
+// batches: the department matrices (Section 3.2, first and last step) and the shared expert.
+#pragma once
+#include "deamoe_internal.cuh"
+
+namespace deamoe {
+
+struct DensePlan;
+
+// Batches from this size on take the dense schedule when the layer has one (DEAMOE_SCHED_AUTO).
+constexpr int DENSE_MIN_BATCH = 48;
+
+// True if the layer's shapes and dtypes fit the dense kernels (bf16 weights and activations, a
+// DeaMoE layer with private matrices, h / f / shared_ffn multiples of 128).
+bool dense_supported(const LayerDev& L);
+
+// Copies the department and shared-expert matrices into the tile layout of the dense kernels
+// (enqueued on `s`).  *bytes receives the device memory taken.
+deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, cudaStream_t s, DensePlan** out,
+                                  uint64_t* bytes);
+void dense_plan_destroy(DensePlan* p);
+
+// Enqueue one launch that runs the given stages (at most two, independent of each other) of one
+// step.  in / out planes are the bf16 activation planes of the streaming schedule.  Returns the
+// number of kernels launched or -1.
+struct DenseIO {
+  const __nv_bfloat16* tokens;  // [B, h]
+  __nv_bfloat16* GU;            // [token-departments, 2f]
+  const __nv_bfloat16* Z;       // [pairs, f]
+  __nv_bfloat16* Ysh;           // [B, fs]
+};
+int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* stages, int n_stages, int B,
+                 cudaStream_t s);
+
+}  // namespace deamoe

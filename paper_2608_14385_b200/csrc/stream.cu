@@ -33,6 +33,7 @@
 
 #include "route_device.cuh"
 #include "stream.cuh"
+#include "dense.cuh"
 
 namespace deamoe {
 
@@ -123,6 +124,7 @@ struct StreamDev {
   int sh_prefix;  // fused schedule with a shared expert: its items are not in the work list
   int early;      // fused DeaMoE layers: the first stage's records are handed over ahead of the rest
   int claim_items;              // fused schedule: the items of the list are claimed, not dealt
+  int dense;                    // dense schedule: the list holds the private stages only (the rest runs on tcgen05 kernels)
   int early_stage;              // the stage handed over early (ST_S1 or ST_V1)
   int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): step number, item count
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
@@ -144,6 +146,9 @@ enum TraceSlot : int { TR_META = 0, TR_DEP, TR_EMPTY, TR_ISSUE, TR_ITEMS, TR_CHU
 
 struct StreamPlan {
   StreamDev dev;
+  StreamDev dev_dense;  // the view of `dev` that the dense schedule's routing and streaming launches get
+  DensePlan* dense;     // tcgen05 kernels for the department / shared-expert stages, or null
+  int dense_min;        // batches from this size on take the dense schedule
   int schedule;
   int n_sm;
   int grid;  // CTAs of the streaming kernel: all of them must be resident at once
@@ -291,6 +296,11 @@ struct CatInfo {
 
 static __device__ __forceinline__ int category_list(const LayerDev& L, const StreamDev& P, CatInfo* cats) {
   int n = 0;
+  if (P.dense) {  // department and shared-expert stages run in the dense kernels, between which this list runs
+    cats[n++] = {ST_S2, 2};
+    cats[n++] = {ST_S3, 2};
+    return n;
+  }
   // with sh_prefix the streaming kernel generates the shared expert's first stage itself
   if (L.n_shared && !P.sh_prefix) cats[n++] = {ST_SH1, 0};
   const bool sh = L.n_shared;
@@ -370,8 +380,10 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
       in_stride = 2 * L.f;
       in_list = L.pair_gurow + L.expert_off[id] + t0;
       outh = P.Yh; outl = P.Yl; out_stride = L.rp; out_row0 = L.expert_off[id] + t0;
-      dep_idx = P.dep_s1 + j;
-      dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
+      if (!P.dense) {  // (dense schedule: the first stage ran in an earlier kernel)
+        dep_idx = P.dep_s1 + j;
+        dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
+      }
       done_idx = P.dep_s2 + id;
       break;
     case ST_S3:
@@ -1495,8 +1507,8 @@ static cudaError_t pack(const void* src, __nv_bfloat16* dst, int rows, int C, lo
   return cudaGetLastError();
 }
 
-deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w, int schedule, cudaStream_t s,
-                                   StreamPlan** out, uint64_t* bytes) {
+deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w, int schedule, int dense_mode,
+                                   cudaStream_t s, StreamPlan** out, uint64_t* bytes) {
   StreamPlan* p = new (std::nothrow) StreamPlan();
   if (!p) return DEAMOE_ERR_ALLOC;
   std::memset(p, 0, sizeof(*p));
@@ -1638,6 +1650,22 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
     stream_plan_destroy(p);
     return e == cudaErrorMemoryAllocation ? DEAMOE_ERR_ALLOC : DEAMOE_ERR_CUDA;
   }
+  // Dense schedule: always (dense_mode 2) or from DENSE_MIN_BATCH tokens on (dense_mode 1, layers
+  // that can be called with that many).  Its routing and its streaming launch see the plan with
+  // the fused schedule's hand-overs switched off and the private stages as the whole list.
+  p->dense_min = dense_mode == 2 ? 1 : DENSE_MIN_BATCH;
+  if (dense_mode == 2 || (dense_mode == 1 && dense_supported(L) && L.max_batch >= DENSE_MIN_BATCH)) {
+    uint64_t db = 0;
+    const deamoe_status_t ds = dense_plan_create(L, w, s, &p->dense, &db);
+    if (ds != DEAMOE_OK) {
+      stream_plan_destroy(p);
+      return ds;
+    }
+    p->bytes += db;
+    p->dev_dense = p->dev;
+    p->dev_dense.dense = 1;
+    p->dev_dense.early = 0; p->dev_dense.sh_prefix = 0; p->dev_dense.claim_items = 0;
+  }
   *out = p;
   *bytes = p->bytes;
   return DEAMOE_OK;
@@ -1647,6 +1675,7 @@ void stream_plan_destroy(StreamPlan* p) {
   if (!p) return;
   stream_profile_enable(*p, false);
   if (p->packed) cudaFree(p->packed);
+  if (p->dense) dense_plan_destroy(p->dense);
   if (p->dev.segs) cudaFree(p->dev.segs);
   if (p->dev.sync) cudaFree(p->dev.sync);
   if (p->dev.trace) cudaFree(p->dev.trace);
@@ -1661,10 +1690,13 @@ int32_t* stream_shared_counter(StreamPlan& p) {
   return p.dev.sh_prefix ? p.dev.sync + SY_DEP + p.dev.dep_sh1 : nullptr;
 }
 
+static bool takes_dense(const StreamPlan& p, int B) { return p.dense && B >= p.dense_min; }
+
 int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
                  int32_t* user_idx, float* user_w) {
+  const StreamDev& dv = takes_dense(p, B) ? p.dev_dense : p.dev;
   const int ny = launch_router_logits(L, tokens, B, s, kslices,
-                                      p.dev.early ? p.dev.sync + SY_DEP + p.dev.early_flag : nullptr);
+                                      dv.early ? dv.sync + SY_DEP + dv.early_flag : nullptr);
   if (ny < 0) return -1;
   const int per_warp = (L.n * 5 + 15) & ~15;
   const bool in_regs = topk_in_registers(L);
@@ -1679,7 +1711,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   const size_t smem = scratch + (size_t)fl.total * 4;
   if (smem > 200 * 1024) return -1;
-  launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, p.dev, B, ny, topk_warps, (int)(scratch / 4),
+  launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, dv, B, ny, topk_warps, (int)(scratch / 4),
              user_idx, user_w);
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
@@ -1717,7 +1749,18 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
     ++launches;
   }
   const bool fused = p.schedule == DEAMOE_SCHED_FUSED && (L.vanilla || L.r > 0);
-  if (fused) {
+  if (takes_dense(p, B)) {
+    // department gate / up (+ shared expert gate / up) on the tensor cores; the private stages in
+    // the streaming kernel; department down (+ shared expert down) on the tensor cores
+    DenseIO io;
+    io.tokens = reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw);
+    io.GU = p.dev.GUh; io.Z = p.dev.Zh; io.Ysh = p.dev.Yshh;
+    const int first[2] = {ST_S1, ST_SH1}, last[2] = {ST_S4, ST_SH2};
+    if (dense_launch(*p.dense, L, io, first, L.n_shared ? 2 : 1, B, s) < 0) return -1;
+    k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev_dense, B, -1, 1);
+    if (dense_launch(*p.dense, L, io, last, L.n_shared ? 2 : 1, B, s) < 0) return -1;
+    launches += 3;
+  } else if (fused) {
     int dbgflag = 0;
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;

@@ -11,8 +11,10 @@ int stream_default_schedule();
 
 // Re-pack the canonical weights into the streaming layout (enqueued on `s`) and allocate the
 // work-list buffers.  *bytes receives the device memory taken.
-deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w, int schedule, cudaStream_t s,
-                                   StreamPlan** out, uint64_t* bytes);
+// dense_mode: 0 = never, 1 = from DENSE_MIN_BATCH tokens on (when the layer supports it), 2 = always (the
+// layer must support it) take the dense schedule (tcgen05 kernels for the department and shared-expert stages).
+deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w, int schedule, int dense_mode,
+                                   cudaStream_t s, StreamPlan** out, uint64_t* bytes);
 void stream_plan_destroy(StreamPlan* p);
 
 // Routing for the streaming schedules: router logits, then ONE kernel for top-k + gate weights,

@@ -1,0 +1,91 @@
+"""Dense schedule (tcgen05 kernels for the department and shared-expert matrices, Section 3.2 at
+larger batches): element-by-element parity with the fp64 oracle, and agreement with the streaming
+schedule."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_14385_b200 import binding, synth
+from tests.common import within_tolerance
+from tests.gpu_common import run_case
+
+pytestmark = pytest.mark.gpu
+
+# h, f, shared_ffn multiples of the 128-row tile; three departments, so 100 tokens put more than 64
+# (one accumulator's worth of) rows into a department's bucket and into the shared expert's.
+DENSE_SMALL = synth.LayerShape("dense-small", hidden=256, n_dept=3, experts_per_dept=4, ffn=128, priv=32, top_k=3,
+                               n_shared=1, shared_ffn=256)
+# several row tiles per matrix and a contraction that spans the 8-stage ring more than once
+DENSE_WIDE = synth.LayerShape("dense-wide", hidden=1024, n_dept=4, experts_per_dept=4, ffn=384, priv=64, top_k=4,
+                              n_shared=1, shared_ffn=128)
+
+
+def _scaled(shape, seed, scale=12.0):
+    dev = torch.device("cuda:0")
+    w = synth.make_deamoe_weights(shape, seed, dev)
+    for k in w:
+        w[k] = (w[k].float() * scale).to(w[k].dtype) if k != "router" else w[k] * 4.0
+    return w
+
+
+@pytest.mark.parametrize("B", [1, 7, 16, 17, 48, 64, 65, 100, 128])
+def test_dense_schedule_small_layer(B):
+    """Buckets of 1 to 128 rows: one ragged group, exactly one accumulator, two groups."""
+    run_case(DENSE_SMALL, B, seed=11, schedule=binding.SCHED_DENSE, weights=_scaled(DENSE_SMALL, 11))
+
+
+@pytest.mark.parametrize("B", [5, 40, 96])
+def test_dense_schedule_wide_layer(B):
+    run_case(DENSE_WIDE, B, seed=12, schedule=binding.SCHED_DENSE, weights=_scaled(DENSE_WIDE, 12, scale=6.0))
+
+
+@pytest.mark.parametrize("variant", ["no_shared", "sigma_none", "gelu", "group_limited", "residual"])
+def test_dense_schedule_variants(variant):
+    shape = {
+        "no_shared": DENSE_SMALL.with_(n_shared=0, shared_ffn=0),
+        "sigma_none": DENSE_SMALL.with_(sigma=0),
+        "gelu": DENSE_SMALL.with_(sigma=2),
+        "group_limited": DENSE_SMALL.with_(n_dept=4, top_k=4, k_dept=2),
+        "residual": DENSE_SMALL.with_(residual=1),
+    }[variant]
+    run_case(shape, 50, seed=13, schedule=binding.SCHED_DENSE, weights=_scaled(shape, 13))
+
+
+def test_dense_schedule_is_refused_for_layers_it_cannot_run():
+    dev = torch.device("cuda:0")
+    for shape, vanilla in ((DENSE_SMALL.with_(priv=0), False), (DENSE_SMALL.with_(hidden=192), False),
+                           (DENSE_SMALL.with_(act_dtype=0), False), (DENSE_SMALL.with_(priv=0), True)):
+        w = (synth.make_vanilla_weights if vanilla else synth.make_deamoe_weights)(shape, 1, dev)
+        with pytest.raises(binding.DeaMoEError) as e:
+            binding.Layer(shape, w, 8, binding.SCHED_DENSE, vanilla=vanilla)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+
+
+def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
+    """One AUTO layer sized for 128 tokens: 16 tokens take the streaming schedule, 64 the dense one;
+    each agrees with a layer fixed to that schedule bit for bit, and the two schedules agree within
+    the tolerance (they round intermediates alike but sum in different orders)."""
+    shape = DENSE_WIDE
+    w = _scaled(shape, 14, scale=6.0)
+    auto = binding.Layer(shape, w, 128, binding.SCHED_AUTO)
+    fused = binding.Layer(shape, w, 128, binding.SCHED_FUSED)
+    dense = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
+    try:
+        for B in (16, 64, 128):
+            x = synth.make_tokens(shape, B, 14 + B, torch.device("cuda:0"))
+            oa, of, od = auto.forward(x).float(), fused.forward(x).float(), dense.forward(x).float()
+            torch.cuda.synchronize()
+            for layer in (auto, fused, dense):
+                assert layer.stats()["device_status"] == 0
+            same = of if B < 48 else od
+            assert torch.equal(oa, same)
+            ok, err, bound = within_tolerance(od.cpu().numpy().astype(np.float64), of.cpu().numpy().astype(np.float64))
+            assert ok, f"{err:.3e} > {bound:.3e}"
+    finally:
+        auto.close(); fused.close(); dense.close()
+
+
+def test_dense_schedule_deepseek_v3_cut_sampled_rows():
+    """The benchmark's matrices (h 7168, f 2048, r 896, shared expert; 8 x 4 experts) at 64 tokens,
+    oracle on sampled token rows."""
+    run_case(synth.DSV3_MINI, 64, seed=3, schedule=binding.SCHED_DENSE, rows=[0, 31, 63])
