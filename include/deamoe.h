@@ -61,8 +61,8 @@ typedef enum {
   DEAMOE_SCHED_DENSE = 4   /* larger batches, where a department's token bucket X^j (Section 3.2) is a
                               dense tile: department and shared-expert matrices on the tcgen05 tensor
                               cores, private matrices in the streaming kernel.  bf16 weights and
-                              tokens, a DeaMoE layer with private matrices, h, f and shared_ffn
-                              multiples of 128; else UNSUPPORTED.  AUTO takes this schedule by
+                              tokens, a DeaMoE layer with private matrices, h a multiple of 256,
+                              f and shared_ffn of 128; else UNSUPPORTED.  AUTO takes this schedule by
                               itself for calls of 48 tokens and more on layers that support it. */
 } deamoe_schedule_t;
 

@@ -3,21 +3,36 @@
 //
 // From a few dozen tokens on, a department's token bucket X^j is a dense tile (16 and more rows),
 // and the per-warp mma.sync path of the streaming kernel becomes issue-bound.  Here one
-// tcgen05.mma covers 128 weight rows x all tokens of the bucket (N up to 64) x 16 columns, with the
-// accumulator in tensor memory, so the kernel is again bound by the weight stream:
+// tcgen05.mma covers up to 64 tokens of the bucket x 256 weight rows x 16 columns, with the
+// accumulator in tensor memory:
 //
-//   D[128 weight rows, N tokens] += W_tile[128, K] . X^j[N, K]^T
+//   D[64 tokens, 256 weight rows] += X^j[64, K] . W_tile[256, K]^T
 //
-// Roles of a CTA (one CTA per SM, persistent over a list of (unit, 128-row tile) jobs):
+// The tokens are the M operand and the weights the N operand, with N as large as the instruction
+// allows, because what limits this kernel is the one thread that issues the MMAs: an MMA costs
+// it about 125 cycles whatever its shape, a wait or a commit 60 to 250, and the weight stream
+// leaves about 700 cycles per 16 KB.  One 256-row MMA moves 8 KB of weights; with 128-row MMAs
+// (4 KB each) the issue thread was the bottleneck at half the HBM rate.
+// An M = 64 accumulator lives in lanes 32 (r / 16) + r % 16 of tensor memory (row r), so each of
+// the four epilogue warps owns 16 tokens and a token's outputs are one contiguous run.
+//
+// Roles of a CTA (one CTA per SM, persistent over a list of (unit, 256-row tile) jobs):
 //   warps 0-3   epilogue: tcgen05.ld of the finished accumulator, sigma / SwiGLU, stores
-//   warp  4     one thread issues the bulk copies of the weight chunks (16 KB each) into the ring
+//   warp  4     one thread issues the bulk copies of the weight chunks (32 KB each) into the weight ring
 //   warp  5     one thread issues the MMAs and the commits that free ring stages / publish accumulators
 //   warps 6-13  loaders: copy the tokens' activation rows of a chunk from their row-major planes
-//               into the core-matrix layout the MMA reads (warp w serves ring stage w)
-// Weights are stored at create time in that same layout, tile by tile and chunk by chunk, so a
-// chunk is one contiguous bulk copy.  Layout of an operand chunk (R rows x BK columns, bf16, "K-major,
-// no swizzle"): 8 x 8 core matrices of 128 contiguous bytes; byte offset of element (r, k) =
-// (r / 8) * (BK * 16) + (k / 8) * 128 + (r % 8) * 16 + (k % 8) * 2.
+//               into the core-matrix layout the MMA reads (warp w takes every eighth chunk)
+// Two rings: weights (5 x 32 KB, filled from HBM) and activation rows (8 x 8 KB, filled from L2;
+// loader warp w owns stage w).  While the weights stream at full rate, an ordinary load from this
+// SM waits behind the bulk copies in flight: 2 to 4 us, measured, whether it hits L2 or not.  So a
+// loader fetches its next chunk's rows into registers as soon as it has stored the current one,
+// eight chunks ahead of the stage it will fill and sixteen ahead of the MMA.
+// Weights are stored at create time tile by tile and chunk by chunk in the layout the MMA reads,
+// so a chunk is one contiguous bulk copy.  Layout of an operand chunk (R rows x 64 columns, bf16,
+// "K-major, no swizzle"): 8 x 8 core matrices of 128 contiguous bytes; byte offset of element
+// (r, k) = (r / 8) * 1024 + (k / 8) * 128 + (r % 8) * 16 + (k % 8) * 2.
+// The jobs are dealt round-robin.  Whole tiles fill as many complete rounds as there are; the
+// tiles left over are split into two 128-row halves each, so that the last round is half as long.
 #include "dense.cuh"
 
 #include <cstring>
@@ -27,31 +42,44 @@ namespace deamoe {
 
 namespace {
 
-constexpr int DN_NST = 8;                   // ring stages = loader warps
-constexpr int DN_NMAX = 64;                 // token columns of one accumulator
-constexpr int DN_A_BYTES = 16 * 1024;       // weights per stage: 128 rows x 64 k, or 2 x (128 x 32)
-constexpr int DN_B_BYTES = DN_NMAX * 128;   // activations per stage: 64 tokens x 64 k
-constexpr int DN_STAGE_BYTES = DN_A_BYTES + DN_B_BYTES;
+constexpr int DN_AST = 5;                   // weight ring stages
+constexpr int DN_BST = 8;                   // activation ring stages
+constexpr int DN_LOADERS = DN_BST;          // loader warps: warp w owns activation stage w
+constexpr int DN_NMAX = 64;                 // token rows of one accumulator (the MMA's M)
+constexpr int DN_BK = 64;                   // columns of a chunk
+constexpr int DN_TILE = 256;                // weight rows of a tile (the MMA's N)
+constexpr int DN_A_BYTES = DN_TILE * DN_BK * 2;   // 32 KB
+constexpr int DN_B_BYTES = DN_NMAX * DN_BK * 2;   // 8 KB
+constexpr int DN_PIECES = DN_B_BYTES / 16 / 32;   // 16-byte pieces of a chunk's rows per loader lane
 constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5, DN_WARP_LOAD0 = 6;
-constexpr int DN_THREADS = (DN_WARP_LOAD0 + DN_NST) * 32;
-constexpr int DN_TMEM_COLS = 256;           // 2 accumulator buffers x 2 matrices x 64 columns
-constexpr size_t DN_SMEM = (size_t)DN_NST * DN_STAGE_BYTES + 1024 /* alignment */ + 512 /* barriers, control */;
+constexpr int DN_THREADS = (DN_WARP_LOAD0 + DN_LOADERS) * 32;
+constexpr int DN_TMEM_COLS = 512;           // 2 accumulator buffers x 256 columns (all of it)
+constexpr size_t DN_SMEM = (size_t)DN_AST * DN_A_BYTES + (size_t)DN_BST * DN_B_BYTES + 512 /* barriers, control */;
 constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits; then an error status, never a hang
 static_assert(DN_SMEM <= 227 * 1024, "shared memory budget");
 // More than half of an SM's shared memory: two of these CTAs never share an SM, so the tensor
 // memory allocation below never waits for another CTA.
 static_assert(DN_SMEM > 114 * 1024, "one CTA per SM is relied upon by the tensor-memory allocation");
 
+#ifdef DEAMOE_TRACE
+__device__ long long dn_trace[256 * 16];  // trace builds: per-CTA cycle counters of the last launch
+#define DN_T0() const long long dn_t0 = clock64()
+#define DN_ADD(k) dn_acc[k] += clock64() - dn_t0
+#else
+#define DN_T0() ((void)0)
+#define DN_ADD(k) ((void)0)
+#endif
+
 enum DenseEpi : int { DE_SIGMA = 0, DE_SWIGLU = 1, DE_NONE = 2 };
 
 struct DensePhase {
   int stage;      // ST_S1, ST_S4, ST_SH1 or ST_SH2
-  int K, tiles;   // contraction length; 128-row tiles of a unit
-  int dual;       // a tile is 128 rows of w and the same rows of w1; epilogue SiLU(a) * b; BK = 32
+  int K, tiles;   // contraction length; 256-row tiles of a unit
+  int dual;       // a tile is 128 rows of the gate matrix followed by the same rows of the up matrix;
+                  // epilogue SiLU(a) * b, 128 outputs per tile
   int epi;
   int in_stride, out_stride;
   const __nv_bfloat16* w;
-  const __nv_bfloat16* w1;
   unsigned long long unit_elems;
   const __nv_bfloat16* in;
   __nv_bfloat16* outh;
@@ -134,60 +162,95 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---------------------------------------------------------------- job decoding (all roles alike)
+struct Sched {
+  int jobs0;   // whole-tile jobs of phase 0
+  int jobs;    // whole-tile jobs of both phases
+  int full;    // of which this many, a multiple of the grid, are done as whole tiles
+  int n_idx;   // job indices: full + 2 * (jobs - full)
+};
 struct Job {
-  int phase, tile;
-  int T;          // token rows of the unit
+  int phase;
+  int T;          // token rows of the unit (0: nothing to do)
   int row0;       // first output row of the unit (and first input row when the rows are contiguous)
-  const int32_t* in_list;  // gathered input rows, or null
-  size_t woff;    // element offset of the unit's weights
+  int ncols;      // weight rows of the job = accumulator columns: 256, or 128 for half a tile
+  int col0;       // output column of accumulator column 0
+  const int32_t* in_list;    // gathered input rows, or null
+  const __nv_bfloat16* w;    // the job's part of the tile's first chunk; the next chunk is DN_TILE * DN_BK further
 };
 
 __device__ __forceinline__ int phase_units(const LayerDev& L, const DensePhase& ph) {
   return (ph.stage == ST_S1 || ph.stage == ST_S4) ? L.counts[CNT_ACTIVE_DEPT] : 1;
 }
 
-__device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A, int job, int jobs0, int B) {
+__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int G) {
+  Sched s;
+  s.jobs0 = phase_units(L, A.ph[0]) * A.ph[0].tiles;
+  s.jobs = s.jobs0 + (A.nph > 1 ? phase_units(L, A.ph[1]) * A.ph[1].tiles : 0);
+  s.full = (s.jobs / G) * G;
+  s.n_idx = s.full + 2 * (s.jobs - s.full);
+  return s;
+}
+
+__device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A, const Sched& sc, int idx, int B) {
   Job j;
-  j.phase = (job >= jobs0) ? 1 : 0;
+  int tjob = idx, half = -1;
+  if (idx >= sc.full) { tjob = sc.full + ((idx - sc.full) >> 1); half = (idx - sc.full) & 1; }
+  j.phase = (tjob >= sc.jobs0) ? 1 : 0;
   const DensePhase& ph = A.ph[j.phase];
-  const int local = job - (j.phase ? jobs0 : 0);
-  const int u = local / ph.tiles;
-  j.tile = local - u * ph.tiles;
+  const int local = tjob - (j.phase ? sc.jobs0 : 0);
+  const int u = local / ph.tiles, tile = local - u * ph.tiles;
   j.in_list = nullptr;
-  j.woff = 0;
+  size_t woff = 0;
   if (ph.stage == ST_S1) {
     const int id = L.active_dept[u];
     j.row0 = L.dept_off[id];
     j.T = L.dept_off[id + 1] - j.row0;
     j.in_list = L.dept_tok + j.row0;
-    j.woff = (size_t)id * ph.unit_elems;
+    woff = (size_t)id * ph.unit_elems;
   } else if (ph.stage == ST_S4) {
     const int id = L.active_dept[u];
     j.row0 = L.expert_off[id * L.g];
     j.T = L.expert_off[(id + 1) * L.g] - j.row0;
-    j.woff = (size_t)id * ph.unit_elems;
+    woff = (size_t)id * ph.unit_elems;
   } else {
     j.row0 = 0;
     j.T = B;
+  }
+  j.w = ph.w + woff + (size_t)tile * DN_TILE * ph.K;
+  j.ncols = DN_TILE;
+  j.col0 = ph.dual ? tile * (DN_TILE / 2) : tile * DN_TILE;
+  if (half >= 0) {
+    if (ph.dual) {
+      if (half == 1) j.T = 0;  // a gate / up tile is not split: its first half-job does all of it
+    } else {
+      j.ncols = DN_TILE / 2;
+      j.col0 += half * (DN_TILE / 2);
+      j.w += (size_t)half * (DN_TILE / 2) * DN_BK;  // row groups 16..31 of every chunk
+    }
   }
   return j;
 }
 
 // ---------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A, int B) {
-  extern __shared__ unsigned char dn_smem_raw[];
-  unsigned char* smem =
-      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dn_smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)DN_NST * DN_STAGE_BYTES);
-  uint64_t* empty_bar = full_bar + DN_NST;
-  uint64_t* acc_full = empty_bar + DN_NST;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* ring_a = smem;
+  unsigned char* ring_b = smem + (size_t)DN_AST * DN_A_BYTES;
+  uint64_t* a_full = reinterpret_cast<uint64_t*>(ring_b + (size_t)DN_BST * DN_B_BYTES);
+  uint64_t* a_empty = a_full + DN_AST;
+  uint64_t* b_full = a_empty + DN_AST;
+  uint64_t* b_empty = b_full + DN_BST;
+  uint64_t* acc_full = b_empty + DN_LOADERS;
   uint64_t* acc_empty = acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  static_assert((2 * DN_AST + DN_BST + DN_LOADERS + 4) * 8 + 8 <= 512, "control region");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int s = 0; s < DN_NST; ++s) { bar_init(&full_bar[s], 2); bar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < DN_AST; ++s) { bar_init(&a_full[s], 1); bar_init(&a_empty[s], 1); }
+    for (int s = 0; s < DN_BST; ++s) bar_init(&b_full[s], 1);
+    for (int s = 0; s < DN_LOADERS; ++s) bar_init(&b_empty[s], 1);
     for (int b = 0; b < 2; ++b) { bar_init(&acc_full[b], 1); bar_init(&acc_empty[b], 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -203,137 +266,211 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int jobs0 = phase_units(L, A.ph[0]) * A.ph[0].tiles;
-  const int jobs = jobs0 + (A.nph > 1 ? phase_units(L, A.ph[1]) * A.ph[1].tiles : 0);
   const int G = (int)gridDim.x;
+  const Sched sc = make_sched(L, A, G);
 
   if (warp == DN_WARP_TMA) {
-    // ============================================================ weight chunks -> ring
+    // ============================================================ weight chunks -> weight ring
     if (lane == 0) {
       const uint64_t pol = policy_stream();
       uint32_t g = 0;
       bool ok = true;
-      for (int job = (int)blockIdx.x; ok && job < jobs; job += G) {
-        const Job j = decode_job(L, A, job, jobs0, B);
-        const DensePhase& ph = A.ph[j.phase];
-        const int bk = ph.dual ? 32 : 64, nch = ph.K / bk;
-        const size_t tile_off = j.woff + (size_t)j.tile * 128 * ph.K;
+#ifdef DEAMOE_TRACE
+      long long dn_acc[2] = {0, 0};
+      const long long dn_start = clock64();
+#endif
+      for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
+        const Job j = decode_job(L, A, sc, idx, B);
+        const int nch = A.ph[j.phase].K / DN_BK;
+        const uint32_t bytes = (uint32_t)j.ncols * DN_BK * 2;
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
         for (int gi = 0; ok && gi < groups; ++gi) {
           for (int c = 0; c < nch; ++c, ++g) {
-            const int s = (int)(g % DN_NST);
-            if (!bar_wait(&empty_bar[s], ((g / DN_NST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-            unsigned char* sa = smem + (size_t)s * DN_STAGE_BYTES;
-            bar_arrive_expect_tx(&full_bar[s], DN_A_BYTES);
-            if (ph.dual) {
-              bulk_load(sa, ph.w + tile_off + (size_t)c * 128 * bk, DN_A_BYTES / 2, &full_bar[s], pol);
-              bulk_load(sa + DN_A_BYTES / 2, ph.w1 + tile_off + (size_t)c * 128 * bk, DN_A_BYTES / 2, &full_bar[s], pol);
-            } else {
-              bulk_load(sa, ph.w + tile_off + (size_t)c * 128 * bk, DN_A_BYTES, &full_bar[s], pol);
-            }
+            const int s = (int)(g % DN_AST);
+            { DN_T0();
+            if (!bar_wait(&a_empty[s], ((g / DN_AST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            DN_ADD(0); }
+            bar_arrive_expect_tx(&a_full[s], bytes);
+            bulk_load(ring_a + (size_t)s * DN_A_BYTES, j.w + (size_t)c * DN_TILE * DN_BK, bytes, &a_full[s], pol);
           }
         }
       }
+#ifdef DEAMOE_TRACE
+      dn_trace[blockIdx.x * 16 + 0] = dn_acc[0];
+      dn_trace[blockIdx.x * 16 + 1] = clock64() - dn_start;
+      dn_trace[blockIdx.x * 16 + 7] = g;
+#endif
     }
   } else if (warp == DN_WARP_MMA) {
     // ============================================================ MMA issue
     if (lane == 0) {
       uint32_t g = 0, a = 0;
       bool ok = true;
-      for (int job = (int)blockIdx.x; ok && job < jobs; job += G) {
-        const Job j = decode_job(L, A, job, jobs0, B);
-        const DensePhase& ph = A.ph[j.phase];
-        const int bk = ph.dual ? 32 : 64, nch = ph.K / bk;
-        const uint32_t sbo = (uint32_t)bk * 16u;
+#ifdef DEAMOE_TRACE
+      long long dn_acc[4] = {0, 0, 0, 0};
+      const long long dn_start = clock64();
+#endif
+      // descriptors of stage 0, first k-step; a k-step of 16 columns is two core matrices (256
+      // bytes) further, which adds 16 to the descriptor's address field
+      const uint64_t desc0_w = umma_smem_desc(smem_addr(ring_a), 128, DN_BK * 16);
+      const uint64_t desc0_x = umma_smem_desc(smem_addr(ring_b), 128, DN_BK * 16);
+      for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
+        const Job j = decode_job(L, A, sc, idx, B);
+        const int nch = A.ph[j.phase].K / DN_BK;
+        const uint32_t idesc = umma_instr_desc(DN_NMAX, j.ncols);  // tokens: M operand; weight rows: N operand
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
         for (int gi = 0; ok && gi < groups; ++gi, ++a) {
-          const int Tg = min(DN_NMAX, j.T - gi * DN_NMAX);
-          const int npad = (Tg + 15) & ~15;
-          const uint32_t idesc = umma_instr_desc(128, npad);
           const uint32_t buf = a & 1u;
           if (!bar_wait(&acc_empty[buf], ((a >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t d0 = tmem_base + buf * 128u, d1 = d0 + 64u;
+          const uint32_t d0 = tmem_base + buf * (uint32_t)DN_TILE;
           for (int c = 0; c < nch; ++c, ++g) {
-            const int s = (int)(g % DN_NST);
-            if (!bar_wait(&full_bar[s], (g / DN_NST) & 1u, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t sa = smem_addr(smem + (size_t)s * DN_STAGE_BYTES), sb = sa + DN_A_BYTES;
-            for (int ks = 0; ks < bk / 16; ++ks) {
-              const uint64_t db = umma_smem_desc(sb + ks * 256, 128, sbo);
-              const uint32_t acc = (c | ks) ? 1u : 0u;
-              umma(d0, umma_smem_desc(sa + ks * 256, 128, sbo), db, idesc, acc);
-              if (ph.dual) umma(d1, umma_smem_desc(sa + DN_A_BYTES / 2 + ks * 256, 128, sbo), db, idesc, acc);
-            }
-            umma_commit(&empty_bar[s]);  // the stage is free once these MMAs have read it
+            const int sa_i = (int)(g % DN_AST), sb_i = (int)(g % DN_BST);
+            { DN_T0();
+            if (!bar_wait(&b_full[sb_i], (g / DN_BST) & 1u, abort_flag)) { ok = false; break; }
+            DN_ADD(0); }
+            { DN_T0();
+            if (!bar_wait(&a_full[sa_i], (g / DN_AST) & 1u, abort_flag)) { ok = false; break; }
+            DN_ADD(1); }
+            // (no tcgen05 fence here: the barrier waits order the copies' and the loaders' writes
+            // before the MMAs)
+            DN_T0();
+            const uint64_t dw = desc0_w + (uint64_t)(sa_i * (DN_A_BYTES >> 4));
+            const uint64_t dx = desc0_x + (uint64_t)(sb_i * (DN_B_BYTES >> 4));
+#pragma unroll
+            for (int ks = 0; ks < DN_BK / 16; ++ks) umma(d0, dx + 16 * ks, dw + 16 * ks, idesc, (c | ks) ? 1u : 0u);
+            DN_ADD(2);
+            { DN_T0();
+            umma_commit(&a_empty[sa_i]);  // the stages of chunk g are free once these MMAs have read them
+            umma_commit(&b_empty[g % DN_LOADERS]);
+            DN_ADD(3); }
           }
           if (ok) umma_commit(&acc_full[buf]);
         }
       }
+#ifdef DEAMOE_TRACE
+      dn_trace[blockIdx.x * 16 + 2] = dn_acc[0];
+      dn_trace[blockIdx.x * 16 + 3] = dn_acc[1];
+      dn_trace[blockIdx.x * 16 + 4] = dn_acc[2];
+      dn_trace[blockIdx.x * 16 + 5] = clock64() - dn_start;
+      dn_trace[blockIdx.x * 16 + 6] = dn_acc[3];
+#endif
     }
   } else if (warp >= DN_WARP_LOAD0) {
-    // ============================================================ activation rows -> ring (stage = w)
+    // ============================================================ activation rows -> activation ring
+    // Warp w takes the chunks g = w, w + 8, ... of the CTA's chunk sequence, all of which use
+    // activation stage w.  The rows of the warp's next chunk are fetched into registers right after
+    // the current one has been stored.
     const int w = warp - DN_WARP_LOAD0;
-    uint32_t g0 = 0;  // chunk counter at the start of the current (job, token group)
-    bool ok = true;
-    for (int job = (int)blockIdx.x; ok && job < jobs; job += G) {
-      const Job j = decode_job(L, A, job, jobs0, B);
-      const DensePhase& ph = A.ph[j.phase];
-      const int bk = ph.dual ? 32 : 64, nch = ph.K / bk;
-      const int pr = bk / 8;                      // 16-byte pieces per row and chunk
-      const int pr_shift = ph.dual ? 2 : 3;
-      const uint32_t sbo = (uint32_t)bk * 16u;
-      const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
-      for (int gi = 0; ok && gi < groups; ++gi) {
-        const int n0 = gi * DN_NMAX, Tg = min(DN_NMAX, j.T - n0);
-        // input row of token n0 + lane and n0 + lane + 32, handed around with shuffles below
-        int rowA = 0, rowB = 0;
-        if (lane < Tg) rowA = j.in_list ? j.in_list[n0 + lane] : j.row0 + n0 + lane;
-        if (lane + 32 < Tg) rowB = j.in_list ? j.in_list[n0 + lane + 32] : j.row0 + n0 + lane + 32;
-        const int pieces = Tg * pr;
-        const int first = (int)((w + DN_NST - (g0 % DN_NST)) % DN_NST);
-        for (int c = first; ok && c < nch; c += DN_NST) {
-          const uint32_t g = g0 + (uint32_t)c;
-          if (lane == 0 && !bar_wait(&empty_bar[w], ((g / DN_NST) & 1u) ^ 1u, abort_flag)) ok = false;
-          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-          if (!ok) break;
-          unsigned char* sb = smem + (size_t)w * DN_STAGE_BYTES + DN_A_BYTES;
-          const __nv_bfloat16* src = ph.in + (size_t)c * bk;
-          for (int i0 = 0; i0 < pieces; i0 += 128) {  // four pieces per lane in flight
-            int4 v[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int i = i0 + q * 32 + lane;
-              const int n = i >> pr_shift, kg = i & (pr - 1);
-              const int ra = __shfl_sync(0xffffffffu, rowA, n & 31), rb = __shfl_sync(0xffffffffu, rowB, n & 31);
-              const int rsel = (n & 32) ? rb : ra;
-              v[q] = make_int4(0, 0, 0, 0);
-              if (i < pieces) v[q] = __ldcg(reinterpret_cast<const int4*>(src + (size_t)rsel * ph.in_stride + kg * 8));
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int i = i0 + q * 32 + lane;
-              const int n = i >> pr_shift, kg = i & (pr - 1);
-              if (i < pieces) *reinterpret_cast<int4*>(sb + (n >> 3) * sbo + kg * 128 + (n & 7) * 16) = v[q];
-            }
-          }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores, read by the MMA
-          __syncwarp();
-          if (lane == 0) bar_arrive(&full_bar[w]);
-        }
-        g0 += (uint32_t)nch;
+    int idx = (int)blockIdx.x, gi = 0, groups = 0, nch = 0, Tg = 0;
+    int rem = w;            // chunk index inside the current (job, token group)
+    uint32_t g = (uint32_t)w;
+    int rowA = 0, rowB = 0;
+    Job j{};
+    bool valid = idx < sc.n_idx;
+    auto enter_group = [&]() {  // per-lane input rows of tokens lane and lane + 32 of the group
+      const int n0 = gi * DN_NMAX;
+      Tg = min(DN_NMAX, j.T - n0);
+      rowA = 0; rowB = 0;
+      if (lane < Tg) rowA = j.in_list ? j.in_list[n0 + lane] : j.row0 + n0 + lane;
+      if (lane + 32 < Tg) rowB = j.in_list ? j.in_list[n0 + lane + 32] : j.row0 + n0 + lane + 32;
+    };
+    auto enter_job = [&]() {  // the next job that has work (a job index may decode to an empty job)
+      while (valid) {
+        j = decode_job(L, A, sc, idx, B);
+        nch = A.ph[j.phase].K / DN_BK;
+        groups = (j.T + DN_NMAX - 1) / DN_NMAX;
+        if (groups > 0) break;
+        idx += G;
+        valid = idx < sc.n_idx;
       }
+      gi = 0;
+      if (valid) enter_group();
+    };
+    auto settle = [&]() {  // move (job, gi, rem) forward until rem lies inside a group
+      while (valid && rem >= nch) {
+        rem -= nch;
+        if (++gi >= groups) {
+          idx += G;
+          valid = idx < sc.n_idx;
+          enter_job();
+        } else {
+          enter_group();
+        }
+      }
+    };
+    int4 v[DN_PIECES];
+    auto fetch = [&]() {  // the rows of chunk `rem` of the current group -> registers
+      const DensePhase& ph = A.ph[j.phase];
+      const int pieces = Tg * (DN_BK / 8);
+      const __nv_bfloat16* src = ph.in + (size_t)rem * DN_BK;
+#pragma unroll
+      for (int q = 0; q < DN_PIECES; ++q) {
+        const int i = q * 32 + lane;
+        const int n = i >> 3, kg = i & 7;
+        const int ra = __shfl_sync(0xffffffffu, rowA, n & 31), rb = __shfl_sync(0xffffffffu, rowB, n & 31);
+        const int rsel = (n & 32) ? rb : ra;
+        // (no default value: a select on the loaded value would make the warp wait for the load here)
+        if (i < pieces) v[q] = __ldcg(reinterpret_cast<const int4*>(src + (size_t)rsel * ph.in_stride + kg * 8));
+      }
+    };
+    enter_job();
+    settle();
+    if (valid) fetch();
+    bool ok = true;
+#ifdef DEAMOE_TRACE
+    long long dn_acc[4] = {0, 0, 0, 0};
+#endif
+    while (valid && ok) {
+      { DN_T0();
+      if (lane == 0 && g >= DN_BST &&
+          !bar_wait(&b_empty[(g - DN_BST) % DN_LOADERS], ((g - DN_BST) / DN_LOADERS) & 1u, abort_flag))
+        ok = false;
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      DN_ADD(0); }
+      if (!ok) break;
+      DN_T0();
+      {
+        unsigned char* sb = ring_b + (size_t)(g % DN_BST) * DN_B_BYTES;
+        const int pieces = Tg * (DN_BK / 8);
+#pragma unroll
+        for (int q = 0; q < DN_PIECES; ++q) {
+          const int i = q * 32 + lane;
+          const int n = i >> 3, kg = i & 7;
+          if (i < pieces) *reinterpret_cast<int4*>(sb + (n >> 3) * (DN_BK * 16) + kg * 128 + (n & 7) * 16) = v[q];
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores, read by the MMA
+      __syncwarp();
+      if (lane == 0) bar_arrive(&b_full[g % DN_BST]);
+      DN_ADD(1);
+      { DN_T0();
+      rem += DN_LOADERS; g += DN_LOADERS;
+      settle();
+      DN_ADD(2); }
+      { DN_T0();
+      if (valid) fetch();
+      DN_ADD(3); }
     }
+#ifdef DEAMOE_TRACE
+    if (w == 0 && lane == 0) {
+      dn_trace[blockIdx.x * 16 + 8] = dn_acc[0];
+      dn_trace[blockIdx.x * 16 + 9] = dn_acc[1];
+      dn_trace[blockIdx.x * 16 + 10] = dn_acc[2];
+      dn_trace[blockIdx.x * 16 + 11] = dn_acc[3];
+    }
+#endif
   } else {
-    // ============================================================ epilogue (warp e owns TMEM lanes 32e..32e+31)
+    // ============================================================ epilogue
+    // Warp e reads TMEM lanes 32e..32e+31, of which the first 16 hold tokens 16e..16e+15 of the group.
     const int e = warp;
     uint32_t a = 0;
     bool ok = true;
-    for (int job = (int)blockIdx.x; ok && job < jobs; job += G) {
-      const Job j = decode_job(L, A, job, jobs0, B);
+    for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
+      const Job j = decode_job(L, A, sc, idx, B);
       const DensePhase& ph = A.ph[j.phase];
       const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
-      const int col = j.tile * 128 + e * 32 + lane;  // output column = weight row of the unit
+      const int nout = ph.dual ? DN_TILE / 2 : j.ncols;  // outputs per token
       for (int gi = 0; ok && gi < groups; ++gi, ++a) {
         const int n0 = gi * DN_NMAX, Tg = min(DN_NMAX, j.T - n0);
         const uint32_t buf = a & 1u;
@@ -341,22 +478,39 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         if (!ok) break;
         tc_fence_after();
-        const uint32_t t0 = tmem_base + ((uint32_t)(e * 32) << 16) + buf * 128u;
-        for (int c0 = 0; c0 < Tg; c0 += 16) {
-          uint32_t r0[16], r1[16];
-          tmem_ld16(t0 + c0, r0);
-          if (ph.dual) tmem_ld16(t0 + 64u + c0, r1);
-          tmem_ld_wait();
+        const int n = 16 * e + lane;                      // token of this lane (lanes 16..31: none)
+        const bool mine = lane < 16 && n < Tg;
+        if (16 * e < Tg) {                                // warp-uniform: some lane of the warp has a token
+          const uint32_t t0 = tmem_base + ((uint32_t)(e * 32) << 16) + buf * (uint32_t)DN_TILE;
+          const size_t o0 = (size_t)(j.row0 + n0 + n) * ph.out_stride + (size_t)j.col0;
+          for (int c0 = 0; c0 < nout; c0 += 16) {
+            uint32_t r0[16], r1[16];
+            tmem_ld16(t0 + c0, r0);
+            if (ph.dual) tmem_ld16(t0 + (uint32_t)(DN_TILE / 2) + c0, r1);
+            tmem_ld_wait();
+            if (mine) {
+              float v[16];
 #pragma unroll
-          for (int q = 0; q < 16; ++q) {
-            const int n = c0 + q;
-            if (n < Tg) {
-              float v = __uint_as_float(r0[q]);
-              if (ph.epi == DE_SWIGLU) v = silu_f(v) * __uint_as_float(r1[q]);
-              else if (ph.epi == DE_SIGMA) v = sigma_f(L.sigma, v);
-              const size_t o = (size_t)(j.row0 + n0 + n) * ph.out_stride + col;
-              if (ph.outf) ph.outf[o] = v;
-              else ph.outh[o] = __float2bfloat16_rn(v);
+              for (int q = 0; q < 16; ++q) {
+                v[q] = __uint_as_float(r0[q]);
+                if (ph.epi == DE_SWIGLU) v[q] = silu_f(v[q]) * __uint_as_float(r1[q]);
+                else if (ph.epi == DE_SIGMA) v[q] = sigma_f(L.sigma, v[q]);
+              }
+              if (ph.outf) {
+                float4* dst = reinterpret_cast<float4*>(ph.outf + o0 + c0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+              } else {
+                uint32_t pk[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+                  pk[q] = *reinterpret_cast<const uint32_t*>(&h2);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(ph.outh + o0 + c0);
+                dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+              }
             }
           }
         }
@@ -378,27 +532,27 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
 }
 
 // Copies `units` matrices [rows, K] (element (r, k) of unit u at src[u * src_unit + r * rs + k * cs])
-// into the tile layout: unit u at dst + u * dst_unit; tile t (128 rows) and chunk c (bk columns) at
-// (t * (K / bk) + c) * 128 * bk elements; inside, the core-matrix layout described at the top.
-// One thread per 16-byte piece (8 consecutive k of one row), in destination order.
+// into the tile layout of unit u at dst + u * dst_unit.  Source row r becomes row
+// R = dst_row0 + (r / spt) * tstride + r % spt of the unit's stacked matrix (two matrices can be
+// stacked, or interleaved 128 rows at a time); tile R / 256 and chunk k / 64 start at
+// ((R / 256) * (K / 64) + k / 64) * 256 * 64 elements; inside, the core-matrix layout described at
+// the top.  One thread per 16-byte piece (8 consecutive k of one row).
 __global__ void k_pack_tiles(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows, int K,
-                             long long rs, long long cs, long long src_unit, long long dst_unit, int bk) {
-  const int pr = bk / 8, nch = K / bk;
-  const long long pieces = (long long)rows * (K / 8);
+                             long long rs, long long cs, long long src_unit, long long dst_unit, int dst_row0, int spt,
+                             int tstride) {
+  const int k8n = K / 8, nch = K / DN_BK;
+  const long long pieces = (long long)rows * k8n;
   const __nv_bfloat16* s = src + (long long)blockIdx.y * src_unit;
   __nv_bfloat16* d = dst + (long long)blockIdx.y * dst_unit;
   for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < pieces; p += (long long)gridDim.x * blockDim.x) {
-    long long x = p;
-    const int r8 = (int)(x % 8); x /= 8;
-    const int kg = (int)(x % pr); x /= pr;
-    const int rg = (int)(x % 16); x /= 16;
-    const int c = (int)(x % nch); x /= nch;
-    const int t = (int)x;
-    const long long r = (long long)t * 128 + rg * 8 + r8, k0 = (long long)c * bk + kg * 8;
+    const int r = (int)(p / k8n), k8 = (int)(p % k8n);
+    const int R = dst_row0 + (r / spt) * tstride + r % spt;
+    const int t = R / DN_TILE, rg = (R % DN_TILE) / 8, r8 = R % 8, c = k8 / 8, kg = k8 % 8;
     __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
-    for (int e2 = 0; e2 < 8; ++e2) v[e2] = s[r * rs + (k0 + e2) * cs];
-    *reinterpret_cast<int4*>(d + p * 8) = *reinterpret_cast<const int4*>(v);
+    for (int e2 = 0; e2 < 8; ++e2) v[e2] = s[(long long)r * rs + ((long long)k8 * 8 + e2) * cs];
+    const size_t o = ((((size_t)t * nch + c) * (DN_TILE / 8) + rg) * 8 + kg) * 64 + (size_t)r8 * 8;
+    *reinterpret_cast<int4*>(d + o) = *reinterpret_cast<const int4*>(v);
   }
 }
 
@@ -406,7 +560,7 @@ __global__ void k_pack_tiles(const __nv_bfloat16* __restrict__ src, __nv_bfloat1
 
 struct DensePlan {
   __nv_bfloat16* tiles;    // all matrices in the tile layout
-  size_t o_gu, o_d, o_sg, o_su, o_sd;  // element offsets: stacked gate;up / down^T of the departments, shared expert
+  size_t o_gu, o_d, o_sgu, o_sd;  // element offsets: stacked gate;up / down^T of the departments, shared expert
   size_t e_gu, e_d;        // elements per department
   int n_sm;
 };
@@ -414,7 +568,7 @@ struct DensePlan {
 bool dense_supported(const LayerDev& L) {
   if (L.vanilla || L.r <= 0) return false;
   if (L.wdt != DEAMOE_BF16 || L.adt != DEAMOE_BF16) return false;
-  if (L.h % 128 || L.f % 128) return false;
+  if (L.h % 256 || L.f % 128) return false;   // 256-row tiles of [2f, h] and of [h, f]; 64-column chunks
   if (L.n_shared && (L.fs % 128)) return false;
   return true;
 }
@@ -436,8 +590,7 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   p->o_d = total; total += (size_t)L.m * p->e_d;
   if (L.n_shared) {
     const size_t sh = (size_t)L.fs * L.h;
-    p->o_sg = total; total += sh;
-    p->o_su = total; total += sh;
+    p->o_sgu = total; total += 2 * sh;
     p->o_sd = total; total += sh;
   }
   if (cudaMalloc(&p->tiles, total * 2) != cudaSuccess) {
@@ -445,22 +598,24 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
     delete p;
     return DEAMOE_ERR_ALLOC;
   }
+  const int NOSPLIT = 1 << 30;
   auto pack = [&](const void* src, size_t off, int rows, int K, long long rs, long long cs, long long su, long long du,
-                  int units, int bk) {
+                  int units, int dst_row0, int spt, int tstride) {
     const long long pieces = (long long)rows * (K / 8);
     int bx = (int)((pieces + 255) / 256);
     if (bx > 8192) bx = 8192;
     k_pack_tiles<<<dim3(bx, units), 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(src), p->tiles + off, rows, K, rs,
-                                                 cs, su, du, bk);
+                                                 cs, su, du, dst_row0, spt, tstride);
   };
   // departments: gate rows [0, f) and up rows [f, 2f) of one stacked matrix; down applied as W_d^T
-  pack(w.dept_gate, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, 64);
-  pack(w.dept_up, p->o_gu + fh, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, 64);
-  pack(w.dept_down, p->o_d, L.h, L.f, 1, L.h, (long long)fh, (long long)p->e_d, L.m, 64);
+  pack(w.dept_gate, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, 0, NOSPLIT, 0);
+  pack(w.dept_up, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, L.f, NOSPLIT, 0);
+  pack(w.dept_down, p->o_d, L.h, L.f, 1, L.h, (long long)fh, (long long)p->e_d, L.m, 0, NOSPLIT, 0);
   if (L.n_shared) {
-    pack(w.shared_gate, p->o_sg, L.fs, L.h, L.h, 1, 0, 0, 1, 32);
-    pack(w.shared_up, p->o_su, L.fs, L.h, L.h, 1, 0, 0, 1, 32);
-    pack(w.shared_down, p->o_sd, L.h, L.fs, 1, L.h, 0, 0, 1, 64);
+    // shared expert: tile t = gate rows [128 t, 128 t + 128) followed by the same rows of up
+    pack(w.shared_gate, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 0, 128, DN_TILE);
+    pack(w.shared_up, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 128, 128, DN_TILE);
+    pack(w.shared_down, p->o_sd, L.h, L.fs, 1, L.h, 0, 0, 1, 0, NOSPLIT, 0);
   }
   cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_dense, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DN_SMEM);
@@ -491,22 +646,22 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
     ph.stage = stages[i];
     switch (stages[i]) {
       case ST_S1:
-        ph.K = L.h; ph.tiles = 2 * L.f / 128; ph.dual = 0; ph.epi = DE_SIGMA;
+        ph.K = L.h; ph.tiles = 2 * L.f / DN_TILE; ph.dual = 0; ph.epi = DE_SIGMA;
         ph.w = p.tiles + p.o_gu; ph.unit_elems = p.e_gu;
         ph.in = io.tokens; ph.in_stride = L.h; ph.outh = io.GU; ph.out_stride = 2 * L.f;
         break;
       case ST_S4:
-        ph.K = L.f; ph.tiles = L.h / 128; ph.dual = 0; ph.epi = DE_NONE;
+        ph.K = L.f; ph.tiles = L.h / DN_TILE; ph.dual = 0; ph.epi = DE_NONE;
         ph.w = p.tiles + p.o_d; ph.unit_elems = p.e_d;
         ph.in = io.Z; ph.in_stride = L.f; ph.outf = L.O; ph.out_stride = L.h;
         break;
       case ST_SH1:
-        ph.K = L.h; ph.tiles = L.fs / 128; ph.dual = 1; ph.epi = DE_SWIGLU;
-        ph.w = p.tiles + p.o_sg; ph.w1 = p.tiles + p.o_su;
+        ph.K = L.h; ph.tiles = L.fs / (DN_TILE / 2); ph.dual = 1; ph.epi = DE_SWIGLU;
+        ph.w = p.tiles + p.o_sgu;
         ph.in = io.tokens; ph.in_stride = L.h; ph.outh = io.Ysh; ph.out_stride = L.fs;
         break;
       case ST_SH2:
-        ph.K = L.fs; ph.tiles = L.h / 128; ph.dual = 0; ph.epi = DE_NONE;
+        ph.K = L.fs; ph.tiles = L.h / DN_TILE; ph.dual = 0; ph.epi = DE_NONE;
         ph.w = p.tiles + p.o_sd;
         ph.in = io.Ysh; ph.in_stride = L.fs; ph.outf = L.Osh; ph.out_stride = L.h;
         break;
@@ -519,3 +674,10 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
 }
 
 }  // namespace deamoe
+
+#ifdef DEAMOE_TRACE
+extern "C" int deamoe_debug_dense(long long* host, int n) {  // trace builds: counters of the last dense launch
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpyFromSymbol(host, deamoe::dn_trace, (size_t)n * sizeof(long long));
+}
+#endif

@@ -11,7 +11,7 @@ struct DensePlan;
 constexpr int DENSE_MIN_BATCH = 48;
 
 // True if the layer's shapes and dtypes fit the dense kernels (bf16 weights and activations, a
-// DeaMoE layer with private matrices, h / f / shared_ffn multiples of 128).
+// DeaMoE layer with private matrices, h a multiple of 256, f and shared_ffn of 128).
 bool dense_supported(const LayerDev& L);
 
 // Copies the department and shared-expert matrices into the tile layout of the dense kernels
