@@ -18,15 +18,18 @@
 //
 // Roles of a CTA (one CTA per SM, persistent over a list of (unit, 256-row tile) jobs):
 //   warps 0-3   epilogue: tcgen05.ld of the finished accumulator, sigma / SwiGLU, stores
-//   warp  4     one thread issues the bulk copies of the weight chunks (32 KB each) into the weight ring
+//   warp  4     one thread issues the copies of a chunk into the ring: the weights (one 32 KB bulk
+//               copy) and the bucket's activation rows (one tiled TMA copy, 64 rows x 64 columns)
 //   warp  5     one thread issues the MMAs and the commits that free ring stages / publish accumulators
-//   warps 6-13  loaders: copy the tokens' activation rows of a chunk from their row-major planes
-//               into the core-matrix layout the MMA reads (warp w takes every eighth chunk)
-// Two rings: weights (5 x 32 KB, filled from HBM) and activation rows (8 x 8 KB, filled from L2;
-// loader warp w owns stage w).  While the weights stream at full rate, an ordinary load from this
-// SM waits behind the bulk copies in flight: 2 to 4 us, measured, whether it hits L2 or not.  So a
-// loader fetches its next chunk's rows into registers as soon as it has stored the current one,
-// eight chunks ahead of the stage it will fill and sixteen ahead of the MMA.
+// The ring has 5 stages of 32 KB weights + 8 KB activation rows.  The activation rows are fetched
+// by TMA, not by loads of a warp: while the weights stream at full rate an ordinary load from this
+// SM waits 2 to 4 us behind the bulk copies in flight (measured, L2 hit or not), and a warp that
+// has to wait that long per chunk cannot keep up, however far ahead it fetches.  The rows' tensor
+// map views a row-major [rows, K] plane as [K / 8][rows][8]; a box of 8 x 64 x 8 lands in shared
+// memory as 8 column blocks of 64 rows x 16 bytes, which is the core-matrix layout with 128 bytes
+// between 8-row groups and 1024 bytes between neighbours along K.  The rows of a bucket are
+// contiguous in every input plane (the first stage's tokens are gathered into bucket order by a
+// small kernel first); a box may run past the bucket's end, into rows that no output depends on.
 // Weights are stored at create time tile by tile and chunk by chunk in the layout the MMA reads,
 // so a chunk is one contiguous bulk copy.  Layout of an operand chunk (R rows x 64 columns, bf16,
 // "K-major, no swizzle"): 8 x 8 core matrices of 128 contiguous bytes; byte offset of element
@@ -35,6 +38,8 @@
 // tiles left over are split into two 128-row halves each, so that the last round is half as long.
 #include "dense.cuh"
 
+#include <cuda.h>  // CUtensorMap and the encode function's signature; the entry point is looked up at run time
+
 #include <cstring>
 #include <new>
 
@@ -42,19 +47,17 @@ namespace deamoe {
 
 namespace {
 
-constexpr int DN_AST = 5;                   // weight ring stages
-constexpr int DN_BST = 8;                   // activation ring stages
-constexpr int DN_LOADERS = DN_BST;          // loader warps: warp w owns activation stage w
+constexpr int DN_AST = 5;                   // ring stages
 constexpr int DN_NMAX = 64;                 // token rows of one accumulator (the MMA's M)
 constexpr int DN_BK = 64;                   // columns of a chunk
 constexpr int DN_TILE = 256;                // weight rows of a tile (the MMA's N)
 constexpr int DN_A_BYTES = DN_TILE * DN_BK * 2;   // 32 KB
 constexpr int DN_B_BYTES = DN_NMAX * DN_BK * 2;   // 8 KB
-constexpr int DN_PIECES = DN_B_BYTES / 16 / 32;   // 16-byte pieces of a chunk's rows per loader lane
-constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5, DN_WARP_LOAD0 = 6;
-constexpr int DN_THREADS = (DN_WARP_LOAD0 + DN_LOADERS) * 32;
+constexpr int DN_STAGE_BYTES = DN_A_BYTES + DN_B_BYTES;
+constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5;
+constexpr int DN_THREADS = (DN_WARP_MMA + 1) * 32;
 constexpr int DN_TMEM_COLS = 512;           // 2 accumulator buffers x 256 columns (all of it)
-constexpr size_t DN_SMEM = (size_t)DN_AST * DN_A_BYTES + (size_t)DN_BST * DN_B_BYTES + 512 /* barriers, control */;
+constexpr size_t DN_SMEM = (size_t)DN_AST * DN_STAGE_BYTES + 512 /* barriers, control */;
 constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits; then an error status, never a hang
 static_assert(DN_SMEM <= 227 * 1024, "shared memory budget");
 // More than half of an SM's shared memory: two of these CTAs never share an SM, so the tensor
@@ -78,10 +81,9 @@ struct DensePhase {
   int dual;       // a tile is 128 rows of the gate matrix followed by the same rows of the up matrix;
                   // epilogue SiLU(a) * b, 128 outputs per tile
   int epi;
-  int in_stride, out_stride;
+  int out_stride, pad;
   const __nv_bfloat16* w;
   unsigned long long unit_elems;
-  const __nv_bfloat16* in;
   __nv_bfloat16* outh;
   float* outf;
 };
@@ -122,6 +124,12 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
       ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(pol) : "memory");
+}
+// Tiled TMA load of one box of a 3-D tensor map (no multicast); x is the innermost coordinate.
+__device__ __forceinline__ void tensor_load_3d(void* dst, const CUtensorMap* tm, int x, int y, int z, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_addr(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(smem_addr(bar)) : "memory");
 }
 __device__ __forceinline__ uint64_t policy_stream() {
   uint64_t p;
@@ -171,10 +179,9 @@ struct Sched {
 struct Job {
   int phase;
   int T;          // token rows of the unit (0: nothing to do)
-  int row0;       // first output row of the unit (and first input row when the rows are contiguous)
+  int row0;       // first row of the unit's bucket, in its input plane and in its output
   int ncols;      // weight rows of the job = accumulator columns: 256, or 128 for half a tile
   int col0;       // output column of accumulator column 0
-  const int32_t* in_list;    // gathered input rows, or null
   const __nv_bfloat16* w;    // the job's part of the tile's first chunk; the next chunk is DN_TILE * DN_BK further
 };
 
@@ -199,13 +206,11 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
   const DensePhase& ph = A.ph[j.phase];
   const int local = tjob - (j.phase ? sc.jobs0 : 0);
   const int u = local / ph.tiles, tile = local - u * ph.tiles;
-  j.in_list = nullptr;
   size_t woff = 0;
   if (ph.stage == ST_S1) {
     const int id = L.active_dept[u];
     j.row0 = L.dept_off[id];
     j.T = L.dept_off[id + 1] - j.row0;
-    j.in_list = L.dept_tok + j.row0;
     woff = (size_t)id * ph.unit_elems;
   } else if (ph.stage == ST_S4) {
     const int id = L.active_dept[u];
@@ -232,25 +237,21 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
 }
 
 // ---------------------------------------------------------------- the kernel
-__global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A, int B) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char* ring_a = smem;
-  unsigned char* ring_b = smem + (size_t)DN_AST * DN_A_BYTES;
-  uint64_t* a_full = reinterpret_cast<uint64_t*>(ring_b + (size_t)DN_BST * DN_B_BYTES);
+__global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A, int B, const __grid_constant__ CUtensorMap tm0,
+                                                         const __grid_constant__ CUtensorMap tm1) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* ring = smem;  // stage s: weights at s * DN_STAGE_BYTES, activation rows DN_A_BYTES further
+  uint64_t* a_full = reinterpret_cast<uint64_t*>(ring + (size_t)DN_AST * DN_STAGE_BYTES);
   uint64_t* a_empty = a_full + DN_AST;
-  uint64_t* b_full = a_empty + DN_AST;
-  uint64_t* b_empty = b_full + DN_BST;
-  uint64_t* acc_full = b_empty + DN_LOADERS;
+  uint64_t* acc_full = a_empty + DN_AST;
   uint64_t* acc_empty = acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  static_assert((2 * DN_AST + DN_BST + DN_LOADERS + 4) * 8 + 8 <= 512, "control region");
+  static_assert((2 * DN_AST + 4) * 8 + 8 <= 512, "control region");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < DN_AST; ++s) { bar_init(&a_full[s], 1); bar_init(&a_empty[s], 1); }
-    for (int s = 0; s < DN_BST; ++s) bar_init(&b_full[s], 1);
-    for (int s = 0; s < DN_LOADERS; ++s) bar_init(&b_empty[s], 1);
     for (int b = 0; b < 2; ++b) { bar_init(&acc_full[b], 1); bar_init(&acc_empty[b], 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -283,6 +284,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t bytes = (uint32_t)j.ncols * DN_BK * 2;
+        const CUtensorMap* tm = j.phase ? &tm1 : &tm0;
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
         for (int gi = 0; ok && gi < groups; ++gi) {
           for (int c = 0; c < nch; ++c, ++g) {
@@ -290,8 +292,10 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
             { DN_T0();
             if (!bar_wait(&a_empty[s], ((g / DN_AST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
             DN_ADD(0); }
-            bar_arrive_expect_tx(&a_full[s], bytes);
-            bulk_load(ring_a + (size_t)s * DN_A_BYTES, j.w + (size_t)c * DN_TILE * DN_BK, bytes, &a_full[s], pol);
+            unsigned char* st = ring + (size_t)s * DN_STAGE_BYTES;
+            bar_arrive_expect_tx(&a_full[s], bytes + DN_B_BYTES);
+            bulk_load(st, j.w + (size_t)c * DN_TILE * DN_BK, bytes, &a_full[s], pol);
+            tensor_load_3d(st + DN_A_BYTES, tm, 0, j.row0 + gi * DN_NMAX, c * (DN_BK / 8), &a_full[s]);
           }
         }
       }
@@ -312,8 +316,9 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
 #endif
       // descriptors of stage 0, first k-step; a k-step of 16 columns is two core matrices (256
       // bytes) further, which adds 16 to the descriptor's address field
-      const uint64_t desc0_w = umma_smem_desc(smem_addr(ring_a), 128, DN_BK * 16);
-      const uint64_t desc0_x = umma_smem_desc(smem_addr(ring_b), 128, DN_BK * 16);
+      const uint64_t desc0_w = umma_smem_desc(smem_addr(ring), 128, DN_BK * 16);
+      // activation rows as the TMA box leaves them: 1024 bytes between neighbours along K, 128 between 8-row groups
+      const uint64_t desc0_x = umma_smem_desc(smem_addr(ring + DN_A_BYTES), DN_NMAX * 16, 128);
       for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
@@ -325,24 +330,20 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
           tc_fence_after();
           const uint32_t d0 = tmem_base + buf * (uint32_t)DN_TILE;
           for (int c = 0; c < nch; ++c, ++g) {
-            const int sa_i = (int)(g % DN_AST), sb_i = (int)(g % DN_BST);
-            { DN_T0();
-            if (!bar_wait(&b_full[sb_i], (g / DN_BST) & 1u, abort_flag)) { ok = false; break; }
-            DN_ADD(0); }
+            const int sa_i = (int)(g % DN_AST);
             { DN_T0();
             if (!bar_wait(&a_full[sa_i], (g / DN_AST) & 1u, abort_flag)) { ok = false; break; }
             DN_ADD(1); }
-            // (no tcgen05 fence here: the barrier waits order the copies' and the loaders' writes
-            // before the MMAs)
+            // (no tcgen05 fence here: the barrier wait orders the copies' writes before the MMAs)
             DN_T0();
-            const uint64_t dw = desc0_w + (uint64_t)(sa_i * (DN_A_BYTES >> 4));
-            const uint64_t dx = desc0_x + (uint64_t)(sb_i * (DN_B_BYTES >> 4));
+            const uint64_t dw = desc0_w + (uint64_t)(sa_i * (DN_STAGE_BYTES >> 4));
+            const uint64_t dx = desc0_x + (uint64_t)(sa_i * (DN_STAGE_BYTES >> 4));
+            // a k-step of 16 columns: two core matrices further, 256 bytes in the weights, 2048 in the rows
 #pragma unroll
-            for (int ks = 0; ks < DN_BK / 16; ++ks) umma(d0, dx + 16 * ks, dw + 16 * ks, idesc, (c | ks) ? 1u : 0u);
+            for (int ks = 0; ks < DN_BK / 16; ++ks) umma(d0, dx + 128 * ks, dw + 16 * ks, idesc, (c | ks) ? 1u : 0u);
             DN_ADD(2);
             { DN_T0();
-            umma_commit(&a_empty[sa_i]);  // the stages of chunk g are free once these MMAs have read them
-            umma_commit(&b_empty[g % DN_LOADERS]);
+            umma_commit(&a_empty[sa_i]);  // the stage is free once these MMAs have read it
             DN_ADD(3); }
           }
           if (ok) umma_commit(&acc_full[buf]);
@@ -356,111 +357,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
       dn_trace[blockIdx.x * 16 + 6] = dn_acc[3];
 #endif
     }
-  } else if (warp >= DN_WARP_LOAD0) {
-    // ============================================================ activation rows -> activation ring
-    // Warp w takes the chunks g = w, w + 8, ... of the CTA's chunk sequence, all of which use
-    // activation stage w.  The rows of the warp's next chunk are fetched into registers right after
-    // the current one has been stored.
-    const int w = warp - DN_WARP_LOAD0;
-    int idx = (int)blockIdx.x, gi = 0, groups = 0, nch = 0, Tg = 0;
-    int rem = w;            // chunk index inside the current (job, token group)
-    uint32_t g = (uint32_t)w;
-    int rowA = 0, rowB = 0;
-    Job j{};
-    bool valid = idx < sc.n_idx;
-    auto enter_group = [&]() {  // per-lane input rows of tokens lane and lane + 32 of the group
-      const int n0 = gi * DN_NMAX;
-      Tg = min(DN_NMAX, j.T - n0);
-      rowA = 0; rowB = 0;
-      if (lane < Tg) rowA = j.in_list ? j.in_list[n0 + lane] : j.row0 + n0 + lane;
-      if (lane + 32 < Tg) rowB = j.in_list ? j.in_list[n0 + lane + 32] : j.row0 + n0 + lane + 32;
-    };
-    auto enter_job = [&]() {  // the next job that has work (a job index may decode to an empty job)
-      while (valid) {
-        j = decode_job(L, A, sc, idx, B);
-        nch = A.ph[j.phase].K / DN_BK;
-        groups = (j.T + DN_NMAX - 1) / DN_NMAX;
-        if (groups > 0) break;
-        idx += G;
-        valid = idx < sc.n_idx;
-      }
-      gi = 0;
-      if (valid) enter_group();
-    };
-    auto settle = [&]() {  // move (job, gi, rem) forward until rem lies inside a group
-      while (valid && rem >= nch) {
-        rem -= nch;
-        if (++gi >= groups) {
-          idx += G;
-          valid = idx < sc.n_idx;
-          enter_job();
-        } else {
-          enter_group();
-        }
-      }
-    };
-    int4 v[DN_PIECES];
-    auto fetch = [&]() {  // the rows of chunk `rem` of the current group -> registers
-      const DensePhase& ph = A.ph[j.phase];
-      const int pieces = Tg * (DN_BK / 8);
-      const __nv_bfloat16* src = ph.in + (size_t)rem * DN_BK;
-#pragma unroll
-      for (int q = 0; q < DN_PIECES; ++q) {
-        const int i = q * 32 + lane;
-        const int n = i >> 3, kg = i & 7;
-        const int ra = __shfl_sync(0xffffffffu, rowA, n & 31), rb = __shfl_sync(0xffffffffu, rowB, n & 31);
-        const int rsel = (n & 32) ? rb : ra;
-        // (no default value: a select on the loaded value would make the warp wait for the load here)
-        if (i < pieces) v[q] = __ldcg(reinterpret_cast<const int4*>(src + (size_t)rsel * ph.in_stride + kg * 8));
-      }
-    };
-    enter_job();
-    settle();
-    if (valid) fetch();
-    bool ok = true;
-#ifdef DEAMOE_TRACE
-    long long dn_acc[4] = {0, 0, 0, 0};
-#endif
-    while (valid && ok) {
-      { DN_T0();
-      if (lane == 0 && g >= DN_BST &&
-          !bar_wait(&b_empty[(g - DN_BST) % DN_LOADERS], ((g - DN_BST) / DN_LOADERS) & 1u, abort_flag))
-        ok = false;
-      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-      DN_ADD(0); }
-      if (!ok) break;
-      DN_T0();
-      {
-        unsigned char* sb = ring_b + (size_t)(g % DN_BST) * DN_B_BYTES;
-        const int pieces = Tg * (DN_BK / 8);
-#pragma unroll
-        for (int q = 0; q < DN_PIECES; ++q) {
-          const int i = q * 32 + lane;
-          const int n = i >> 3, kg = i & 7;
-          if (i < pieces) *reinterpret_cast<int4*>(sb + (n >> 3) * (DN_BK * 16) + kg * 128 + (n & 7) * 16) = v[q];
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores, read by the MMA
-      __syncwarp();
-      if (lane == 0) bar_arrive(&b_full[g % DN_BST]);
-      DN_ADD(1);
-      { DN_T0();
-      rem += DN_LOADERS; g += DN_LOADERS;
-      settle();
-      DN_ADD(2); }
-      { DN_T0();
-      if (valid) fetch();
-      DN_ADD(3); }
-    }
-#ifdef DEAMOE_TRACE
-    if (w == 0 && lane == 0) {
-      dn_trace[blockIdx.x * 16 + 8] = dn_acc[0];
-      dn_trace[blockIdx.x * 16 + 9] = dn_acc[1];
-      dn_trace[blockIdx.x * 16 + 10] = dn_acc[2];
-      dn_trace[blockIdx.x * 16 + 11] = dn_acc[3];
-    }
-#endif
-  } else {
+  } else if (warp < 4) {
     // ============================================================ epilogue
     // Warp e reads TMEM lanes 32e..32e+31, of which the first 16 hold tokens 16e..16e+15 of the group.
     const int e = warp;
@@ -556,10 +453,29 @@ __global__ void k_pack_tiles(const __nv_bfloat16* __restrict__ src, __nv_bfloat1
   }
 }
 
+// First stage's input: the tokens of every department's bucket X^j (Section 3.2), in bucket order.
+// Row r of Xg = token dept_tok[r]; one block per row, 16 bytes per thread and step.
+__global__ void k_gather_buckets(LayerDev L, const __nv_bfloat16* __restrict__ tokens, __nv_bfloat16* __restrict__ Xg) {
+  const int rows = L.counts[CNT_TOKEN_DEPT];
+  const int v = L.h / 8;
+  for (int r = (int)blockIdx.x; r < rows; r += (int)gridDim.x) {
+    const int4* src = reinterpret_cast<const int4*>(tokens + (size_t)L.dept_tok[r] * L.h);
+    int4* dst = reinterpret_cast<int4*>(Xg + (size_t)r * L.h);
+    for (int i = (int)threadIdx.x; i < v; i += (int)blockDim.x) dst[i] = src[i];
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
 }  // namespace
 
 struct DensePlan {
   __nv_bfloat16* tiles;    // all matrices in the tile layout
+  __nv_bfloat16* Xg;       // [max_batch * min(k, m), h] tokens in bucket order
+  int xg_rows;
+  EncodeTiledFn encode;    // cuTensorMapEncodeTiled, looked up through the runtime
   size_t o_gu, o_d, o_sgu, o_sd;  // element offsets: stacked gate;up / down^T of the departments, shared expert
   size_t e_gu, e_d;        // elements per department
   int n_sm;
@@ -593,10 +509,23 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
     p->o_sgu = total; total += 2 * sh;
     p->o_sd = total; total += sh;
   }
-  if (cudaMalloc(&p->tiles, total * 2) != cudaSuccess) {
+  p->xg_rows = L.max_batch * (L.k < L.m ? L.k : L.m);
+  if (cudaMalloc(&p->tiles, total * 2) != cudaSuccess ||
+      cudaMalloc(&p->Xg, (size_t)p->xg_rows * L.h * 2) != cudaSuccess) {
     cudaGetLastError();
-    delete p;
+    dense_plan_destroy(p);
     return DEAMOE_ERR_ALLOC;
+  }
+  {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qr = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess ||
+        qr != cudaDriverEntryPointSuccess || !fn) {
+      cudaGetLastError();
+      dense_plan_destroy(p);
+      return DEAMOE_ERR_CUDA;
+    }
+    p->encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
   const int NOSPLIT = 1 << 30;
   auto pack = [&](const void* src, size_t off, int rows, int K, long long rs, long long cs, long long su, long long du,
@@ -625,14 +554,26 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
     return DEAMOE_ERR_CUDA;
   }
   *out = p;
-  *bytes = total * 2;
+  *bytes = total * 2 + (size_t)p->xg_rows * L.h * 2;
   return DEAMOE_OK;
 }
 
 void dense_plan_destroy(DensePlan* p) {
   if (!p) return;
   if (p->tiles) cudaFree(p->tiles);
+  if (p->Xg) cudaFree(p->Xg);
   delete p;
+}
+
+// Tensor map over a row-major bf16 plane [rows, K], viewed as [K / 8][rows][8]; box 8 x 64 x 8.
+static bool encode_rows_map(const DensePlan& p, CUtensorMap* tm, const void* base, int rows, int K) {
+  const cuuint64_t dims[3] = {8, (cuuint64_t)rows, (cuuint64_t)(K / 8)};
+  const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 16};  // bytes between rows, between 8-column groups
+  const cuuint32_t box[3] = {8, DN_NMAX, DN_BK / 8};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return p.encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* stages, int n_stages, int B,
@@ -641,36 +582,46 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
   DenseArgs A;
   std::memset(&A, 0, sizeof(A));
   A.nph = n_stages;
+  CUtensorMap tm[2];
+  std::memset(tm, 0, sizeof(tm));
+  int launches = 0;
   for (int i = 0; i < n_stages; ++i) {
     DensePhase& ph = A.ph[i];
     ph.stage = stages[i];
+    const void* in = nullptr;
+    int in_rows = 0;
     switch (stages[i]) {
       case ST_S1:
         ph.K = L.h; ph.tiles = 2 * L.f / DN_TILE; ph.dual = 0; ph.epi = DE_SIGMA;
         ph.w = p.tiles + p.o_gu; ph.unit_elems = p.e_gu;
-        ph.in = io.tokens; ph.in_stride = L.h; ph.outh = io.GU; ph.out_stride = 2 * L.f;
+        in = p.Xg; in_rows = p.xg_rows; ph.outh = io.GU; ph.out_stride = 2 * L.f;
+        k_gather_buckets<<<2 * p.n_sm, 256, 0, s>>>(L, io.tokens, p.Xg);
+        ++launches;
         break;
       case ST_S4:
         ph.K = L.f; ph.tiles = L.h / DN_TILE; ph.dual = 0; ph.epi = DE_NONE;
         ph.w = p.tiles + p.o_d; ph.unit_elems = p.e_d;
-        ph.in = io.Z; ph.in_stride = L.f; ph.outf = L.O; ph.out_stride = L.h;
+        in = io.Z; in_rows = L.max_batch * L.k; ph.outf = L.O; ph.out_stride = L.h;
         break;
       case ST_SH1:
         ph.K = L.h; ph.tiles = L.fs / (DN_TILE / 2); ph.dual = 1; ph.epi = DE_SWIGLU;
         ph.w = p.tiles + p.o_sgu;
-        ph.in = io.tokens; ph.in_stride = L.h; ph.outh = io.Ysh; ph.out_stride = L.fs;
+        in = io.tokens; in_rows = B; ph.outh = io.Ysh; ph.out_stride = L.fs;
         break;
       case ST_SH2:
         ph.K = L.fs; ph.tiles = L.h / DN_TILE; ph.dual = 0; ph.epi = DE_NONE;
         ph.w = p.tiles + p.o_sd;
-        ph.in = io.Ysh; ph.in_stride = L.fs; ph.outf = L.Osh; ph.out_stride = L.h;
+        in = io.Ysh; in_rows = L.max_batch; ph.outf = L.Osh; ph.out_stride = L.h;
         break;
       default:
         return -1;
     }
+    if (!encode_rows_map(p, &tm[i], in, in_rows, ph.K)) return -1;
   }
-  k_dense<<<p.n_sm, DN_THREADS, DN_SMEM, s>>>(L, A, B);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  if (n_stages == 1) tm[1] = tm[0];
+  k_dense<<<p.n_sm, DN_THREADS, DN_SMEM, s>>>(L, A, B, tm[0], tm[1]);
+  ++launches;
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 }  // namespace deamoe
