@@ -3,7 +3,7 @@
 weight-streaming roofline (unique weight bytes / peak HBM bandwidth).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--batch B] [--shape dsv3|7b]
-                    [--schedule auto|plain|staged|fused] [--no-sweep] [--impl reference]
+                    [--schedule auto|plain|staged|fused|dense] [--mode layer|locality|stack|large] [--no-sweep] [--impl reference]
 
 One "step" = one forward of one DeaMoE layer (routing, bucketing, department and private stages,
 combine) over one batch of B synthetic tokens.  The headline workload is the DeepSeek-V3-shaped
@@ -240,13 +240,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--batch", type=int, default=16)
     ap.add_argument("--shape", default="dsv3")
-    ap.add_argument("--schedule", default="auto", choices=["auto", "plain", "staged", "fused"])
+    ap.add_argument("--schedule", default="auto", choices=["auto", "plain", "staged", "fused", "dense"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the batch sweep and the vanilla comparator")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle")
-    ap.add_argument("--mode", default="layer", choices=["layer", "locality", "stack"],
+    ap.add_argument("--mode", default="layer", choices=["layer", "locality", "stack", "large"],
                     help="layer: the contract line (default); locality: routing-locality sweep on the DeepSeek-V3 "
-                         "shape; stack: 32 consecutive 7B-class layers with a residual add, DeaMoE vs vanilla")
+                         "shape; stack: 32 consecutive 7B-class layers with a residual add, DeaMoE vs vanilla; "
+                         "large: 32-128 tokens on the DeepSeek-V3 shape, streaming vs dense (tcgen05) schedule")
     args = ap.parse_args()
 
     from paper_2608_14385_b200 import synth
@@ -272,11 +273,11 @@ def main():
             dist.barrier()
 
     sched = {"auto": binding.SCHED_AUTO, "plain": binding.SCHED_PLAIN, "staged": binding.SCHED_STAGED,
-             "fused": binding.SCHED_FUSED}[args.schedule]
+             "fused": binding.SCHED_FUSED, "dense": binding.SCHED_DENSE}[args.schedule]
     peak, peak_src = measured_peaks()
     if args.mode != "layer":
         if rank == 0:
-            fn = locality_sweep if args.mode == "locality" else stack_bench
+            fn = {"locality": locality_sweep, "stack": stack_bench, "large": large_batch_sweep}[args.mode]
             print(json.dumps(fn(args, sched, peak, torch, dev)))
         if dist is not None:
             dist.barrier()
@@ -553,6 +554,61 @@ def stack_bench(args, sched, peak, torch, dev):
                             "speedup_vs_vanilla": v_us / d_us, "byte_ratio_vanilla_over_deamoe": v_mb / d_mb,
                             "deamoe_us_per_layer": d_us / n_layers, "outputs_finite": d_fin and v_fin})
     return out
+
+
+def large_batch_sweep(args, sched, peak, torch, dev):
+    """48 to 128 tokens on the DeepSeek-V3 shape (the upper half of the paper's 4-128 token range),
+    where a department's bucket is a dense tile: the streaming schedule (mma.sync), the dense
+    schedule (tcgen05 kernels for the department and shared-expert matrices), what AUTO picks, and the
+    in-library vanilla MoE."""
+    from paper_2608_14385_b200 import binding, synth
+    shape = synth.SHAPES["dsv3"]
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    steps = max(10, args.steps // 2)
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    router = w["router"]
+    layers = {"streaming": binding.Layer(shape, w, 128, binding.SCHED_FUSED),
+              "dense": binding.Layer(shape, w, 128, binding.SCHED_DENSE),
+              "auto": binding.Layer(shape, w, 128, binding.SCHED_AUTO)}
+    del w
+    torch.cuda.empty_cache()
+    rows = []
+    batches_list = [32, 48, 64, 96, 128]
+    for B in batches_list:
+        bs = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(4)]
+        r = {"batch": B}
+        for name, layer in layers.items():
+            ub = []
+            for b in bs:
+                layer.forward(b)
+                ub.append(layer.stats()["unique_weight_bytes"])
+            t, _ = time_layer(layer, bs, steps, 3, flush, torch, lambda: None)
+            r[name + "_us"] = pct(t, 0.5) * 1e3
+            r["deamoe_mb"] = statistics.mean(ub) / 1e6
+        r["auto_gbs"] = r["deamoe_mb"] / r["auto_us"] * 1e3
+        r["auto_frac_of_measured_peak"] = r["auto_gbs"] / peak
+        rows.append(r)
+    for layer in layers.values():
+        layer.close()
+    torch.cuda.empty_cache()
+    vw = synth.make_vanilla_weights(shape, 0, dev, router=router)
+    vl = binding.Layer(shape, vw, 128, binding.SCHED_AUTO, vanilla=True)
+    del vw
+    torch.cuda.empty_cache()
+    for r in rows:
+        bs = [synth.make_tokens(shape, r["batch"], 100 + i, dev) for i in range(4)]
+        ub = []
+        for b in bs:
+            vl.forward(b)
+            ub.append(vl.stats()["unique_weight_bytes"])
+        t, _ = time_layer(vl, bs, steps, 3, flush, torch, lambda: None)
+        r["vanilla_us"] = pct(t, 0.5) * 1e3
+        r["vanilla_mb"] = statistics.mean(ub) / 1e6
+        r["speedup_vs_vanilla"] = r["vanilla_us"] / r["auto_us"]
+        r["byte_ratio_vanilla_over_deamoe"] = r["vanilla_mb"] / r["deamoe_mb"]
+    vl.close()
+    return {"metric": "large_batch_sweep", "unit": "us", "shape": shape.name, "data": "synthetic", "dtype": "bf16",
+            "l2": "256 MiB buffer overwritten between steps", "peak_gbs_measured": peak, "rows": rows}
 
 
 def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev):
