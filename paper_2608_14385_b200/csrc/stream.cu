@@ -1756,10 +1756,12 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
     io.tokens = reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw);
     io.GU = p.dev.GUh; io.Z = p.dev.Zh; io.Ysh = p.dev.Yshh;
     const int first[2] = {ST_S1, ST_SH1}, last[2] = {ST_S4, ST_SH2};
-    if (dense_launch(*p.dense, L, io, first, L.n_shared ? 2 : 1, B, s) < 0) return -1;
+    const int n1 = dense_launch(*p.dense, L, io, first, L.n_shared ? 2 : 1, B, s);
+    if (n1 < 0) return -1;
     k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev_dense, B, -1, 1);
-    if (dense_launch(*p.dense, L, io, last, L.n_shared ? 2 : 1, B, s) < 0) return -1;
-    launches += 3;
+    const int n2 = dense_launch(*p.dense, L, io, last, L.n_shared ? 2 : 1, B, s);
+    if (n2 < 0) return -1;
+    launches += n1 + 1 + n2;
   } else if (fused) {
     int dbgflag = 0;
 #ifdef DEAMOE_TRACE
