@@ -331,6 +331,12 @@ def main():
                                 "(smaller layer of the same matrices), scaled by algorithmic bytes",
                 "kernel": "k_stream (the weight-streaming launch(es) of one step)",
                 "kernel_ms": k_ms, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg}
+        if args.schedule == "dense" or (args.schedule == "auto" and B >= 56):
+            # dense schedule: the pair of events brackets k_dense, k_stream, k_dense (ordinary launches, back to back)
+            roof["kernel"] = "k_dense + k_stream + k_dense (the three weight-streaming launches of a dense step)"
+            roof["traffic_note"] = ("dram read+write bytes from the ncu captures of k_stream (1.001 x algorithmic) and "
+                                    "k_dense (1.02 x) in profiles/, scaled by algorithmic bytes")
+            roof["traffic"] = alg * 1.01
     else:
         achieved = mean_bytes / (statistics.mean(times_ms) * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
