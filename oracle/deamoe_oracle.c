@@ -29,7 +29,9 @@
  *     logit in the department, the k_dept best departments (ties to the lowest
  *     department index) survive, TopK runs over their experts only;
  *   - department of expert i is i div experts_per_dept;
- *   - an optional always-on shared expert is Eq. (1) with weight 1.
+ *   - an optional always-on shared expert is Eq. (1) with weight 1;
+ *   - sigma = RMSNorm (one of the operators of Section 3.4 / Table 4) acts on the whole
+ *     length-f vector: v / sqrt(mean(v^2) + 1e-6), no learned gain.
  *
  * Only tests, the smoke check and the benchmark's cpu_baseline leg may call
  * this file.  It shares no code with the CUDA library.
@@ -47,7 +49,8 @@
 #endif
 
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
-enum { ORACLE_SIGMA_NONE = 0, ORACLE_SIGMA_SILU = 1, ORACLE_SIGMA_GELU = 2 };
+enum { ORACLE_SIGMA_NONE = 0, ORACLE_SIGMA_SILU = 1, ORACLE_SIGMA_GELU = 2, ORACLE_SIGMA_RMSNORM = 3 };
+#define ORACLE_RMS_EPS 1e-6
 
 typedef struct {
   int32_t hidden;           /* h */
@@ -121,6 +124,19 @@ static inline double sigma_fn(int kind, double v) {
   }
 }
 
+/* sigma of Section 3.1 / 3.4 on a whole vector: element-wise for SiLU / GeLU / none,
+ * root-mean-square normalisation over the vector for RMSNorm */
+static void sigma_vec(int kind, double *v, int n) {
+  if (kind == ORACLE_SIGMA_RMSNORM) {
+    double ss = 0.0;
+    for (int q = 0; q < n; ++q) ss += v[q] * v[q];
+    const double d = sqrt(ss / (double)n + ORACLE_RMS_EPS);
+    for (int q = 0; q < n; ++q) v[q] = v[q] / d;
+    return;
+  }
+  for (int q = 0; q < n; ++q) v[q] = sigma_fn(kind, v[q]);
+}
+
 /* y[r] = sum_c W[r, c] x[c],  W is [rows, cols] row-major */
 static void matvec(const void *W, int dtype, int rows, int cols, const double *x, double *y) {
 #pragma omp parallel for schedule(static)
@@ -171,10 +187,8 @@ int oracle_deamoe_expert(const oracle_config_t *c, const void *Wg, const void *W
   double *U = G + f, *Z = U + f, *yg = Z + f, *yu = yg + r, *Y = yu + r;
   matvec(Wg, dt, f, h, x, G);
   matvec(Wu, dt, f, h, x, U);
-  for (int q = 0; q < f; ++q) {
-    G[q] = sigma_fn(c->sigma, G[q]);
-    U[q] = sigma_fn(c->sigma, U[q]);
-  }
+  sigma_vec(c->sigma, G, f);
+  sigma_vec(c->sigma, U, f);
   if (c->priv > 0) {
     matvec(Ag, dt, r, f, G, yg);
     matvec(Au, dt, r, f, U, yu);
@@ -188,7 +202,7 @@ int oracle_deamoe_expert(const oracle_config_t *c, const void *Wg, const void *W
   } else {
     memcpy(Z, Y, sizeof(double) * f);
   }
-  for (int q = 0; q < f; ++q) Z[q] = sigma_fn(c->sigma, Z[q]);
+  sigma_vec(c->sigma, Z, f);
   matvec_t(Wd, dt, f, h, Z, out);
   if (tapG) memcpy(tapG, G, sizeof(double) * f);
   if (tapU) memcpy(tapU, U, sizeof(double) * f);

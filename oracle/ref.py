@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "deamoe_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 F32, BF16 = 0, 1
-SIGMA_NONE, SIGMA_SILU, SIGMA_GELU = 0, 1, 2
+SIGMA_NONE, SIGMA_SILU, SIGMA_GELU, SIGMA_RMSNORM = 0, 1, 2, 3
 
 
 class OracleConfig(C.Structure):

@@ -343,3 +343,48 @@ def test_unique_bytes_closed_form_against_vanilla():
     van = acc.unique_bytes_vanilla(8, h, f, n, 2, 1, 2048)
     assert dea == 7 * 88080384 + 8 * 11010048 + 88080384 + 7340032
     assert van == 8 * 88080384 + 88080384 + 7340032
+
+
+# ---------------------------------------------------------------- sigma = RMSNorm (Section 3.4, Table 4)
+
+def test_rmsnorm_sigma_against_the_library_routine_and_its_invariants():
+    """sigma = RMSNorm normalises the three length-f vectors of Eq. (4).  Pinned by (1) the taps
+    G, U, Z against torch.nn.functional.rms_norm applied to the un-normalised vectors (sigma = none
+    taps, re-built here with dense numpy for Z), (2) unit mean square of each tap, (3) invariance of
+    the expert's output under scaling W_g, W_u or A_d by powers of two (exact in bf16), which
+    element-wise operators do not have."""
+    shape = SMALL.with_(sigma=ref.SIGMA_RMSNORM)
+    cfg = oracle_cfg(shape)
+    wt = _layer(shape, 8, std=0.3)
+    x = widen(synth.make_tokens(shape, 1, 8))[0]
+    j, i = 1, 1 * shape.experts_per_dept + 2
+    Wg, Wu, Wd = (synth.to_numpy(wt[f"dept_{k}"][j]) for k in ("gate", "up", "down"))
+    Ag, Au, Ad = (synth.to_numpy(wt[f"priv_{k}"][i]) for k in ("gate", "up", "down"))
+    out, G, U, Y, Z = ref.deamoe_expert(cfg, Wg, Wu, Wd, Ag, Au, Ad, x, taps=True)
+    raw_cfg = oracle_cfg(shape.with_(sigma=ref.SIGMA_NONE))
+    _, G0, U0, _, _ = ref.deamoe_expert(raw_cfg, Wg, Wu, Wd, Ag, Au, Ad, x, taps=True)
+
+    def lib_rms(v):
+        return torch.nn.functional.rms_norm(torch.from_numpy(v), (v.size,), eps=1e-6).numpy()
+
+    np.testing.assert_allclose(G, lib_rms(G0), rtol=1e-12)
+    np.testing.assert_allclose(U, lib_rms(U0), rtol=1e-12)
+    Z0 = widen(wt["priv_down"][i]).T @ Y          # (A_d)^T Y, before the last sigma
+    np.testing.assert_allclose(Z, lib_rms(Z0), rtol=1e-11)
+    np.testing.assert_allclose(out, widen(wt["dept_down"][j]).T @ Z, rtol=1e-11, atol=1e-14)
+    for v, v0 in ((G, G0), (U, U0), (Z, Z0)):
+        ms0 = np.mean(v0 * v0)
+        assert abs(np.mean(v * v) - ms0 / (ms0 + 1e-6)) < 1e-12
+    # scale invariance (up to the epsilon): doubling W_g, quartering W_u, doubling A_d
+    wt2 = {k: v.clone() for k, v in wt.items()}
+    wt2["dept_gate"] = (wt["dept_gate"].float() * 2).to(torch.bfloat16)
+    wt2["dept_up"] = (wt["dept_up"].float() * 0.25).to(torch.bfloat16)
+    wt2["priv_down"] = (wt["priv_down"].float() * 2).to(torch.bfloat16)
+    out2 = ref.deamoe_expert(cfg, synth.to_numpy(wt2["dept_gate"][j]), synth.to_numpy(wt2["dept_up"][j]), Wd,
+                             Ag, Au, synth.to_numpy(wt2["priv_down"][i]), x)
+    np.testing.assert_allclose(out2, out, rtol=2e-5, atol=1e-9)
+    # ... which SiLU does not have
+    s_cfg = oracle_cfg(shape.with_(sigma=ref.SIGMA_SILU))
+    a = ref.deamoe_expert(s_cfg, Wg, Wu, Wd, Ag, Au, Ad, x)
+    b = ref.deamoe_expert(s_cfg, synth.to_numpy(wt2["dept_gate"][j]), Wu, Wd, Ag, Au, Ad, x)
+    assert np.abs(a - b).max() > 1e-3 * np.abs(a).max()
