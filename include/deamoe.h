@@ -50,7 +50,12 @@ typedef enum {
 typedef enum { DEAMOE_F32 = 0, DEAMOE_BF16 = 1 } deamoe_dtype_t;
 
 /* sigma of Section 3.1: the non-linearity between department and expert projections */
-typedef enum { DEAMOE_SIGMA_NONE = 0, DEAMOE_SIGMA_SILU = 1, DEAMOE_SIGMA_GELU = 2 } deamoe_sigma_t;
+typedef enum {
+  DEAMOE_SIGMA_NONE = 0,
+  DEAMOE_SIGMA_SILU = 1,    /* the paper's choice (Section 3.4) */
+  DEAMOE_SIGMA_GELU = 2,
+  DEAMOE_SIGMA_RMSNORM = 3  /* v / sqrt(mean(v^2) + 1e-6) over the whole length-f vector, no gain; needs priv > 0 */
+} deamoe_sigma_t;
 
 /* how one forward is issued */
 typedef enum {

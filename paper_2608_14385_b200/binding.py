@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libdeamoe.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_BATCH, ERR_TIMEOUT = range(7)
 F32, BF16 = 0, 1
-SIGMA_NONE, SIGMA_SILU, SIGMA_GELU = 0, 1, 2
+SIGMA_NONE, SIGMA_SILU, SIGMA_GELU, SIGMA_RMSNORM = 0, 1, 2, 3
 SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4
 
 # every symbol include/deamoe.h declares

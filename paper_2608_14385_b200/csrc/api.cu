@@ -63,7 +63,8 @@ deamoe_status_t check_config(const deamoe_config_t* c, const deamoe_weights_t* w
   if (c->n_shared && c->shared_ffn <= 0) return DEAMOE_ERR_INVALID_ARG;
   if (c->weight_dtype != DEAMOE_F32 && c->weight_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
   if (c->act_dtype != DEAMOE_F32 && c->act_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
-  if (c->sigma < DEAMOE_SIGMA_NONE || c->sigma > DEAMOE_SIGMA_GELU) return DEAMOE_ERR_INVALID_ARG;
+  if (c->sigma < DEAMOE_SIGMA_NONE || c->sigma > DEAMOE_SIGMA_RMSNORM) return DEAMOE_ERR_INVALID_ARG;
+  if (!vanilla && c->sigma == DEAMOE_SIGMA_RMSNORM && c->priv <= 0) return DEAMOE_ERR_UNSUPPORTED;
   if (c->schedule < DEAMOE_SCHED_AUTO || c->schedule > DEAMOE_SCHED_DENSE) return DEAMOE_ERR_INVALID_ARG;
   if (!(c->route_scale == c->route_scale)) return DEAMOE_ERR_INVALID_ARG;
   if (c->max_batch < 1 || c->max_batch > DEAMOE_MAX_BATCH) return DEAMOE_ERR_BATCH;
@@ -173,6 +174,10 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
       }
       A(dev_alloc(L, &d.Y, (size_t)pmax * (vanilla ? d.f : d.rp)));
       if (d.n_shared) A(dev_alloc(L, &d.Ysh, (size_t)MB * d.fs));
+    }
+    if (d.sigma == DEAMOE_SIGMA_RMSNORM) {
+      A(dev_alloc(L, &d.ss_gu, (size_t)tdmax * 2));
+      A(dev_alloc(L, &d.ss_z, (size_t)pmax));
     }
     A(dev_alloc(L, &d.O, (size_t)pmax * d.h));
     if (d.n_shared) A(dev_alloc(L, &d.Osh, (size_t)MB * d.h));

@@ -88,7 +88,14 @@ struct LayerDev {
   float* Ysh;          // [MB, fs]
   float* Osh;          // [MB, h]
   int32_t* sh_done;    // counter the combine kernel resets at the end of a step, or null
+  // sigma = RMSNorm: sums of squares of the un-normalised vectors, zeroed by the routing tail
+  float* ss_gu;        // [MB*min(k,m), 2]: G and U of every (token, department) row
+  float* ss_z;         // [MB*k]: Z of every pair
 };
+
+constexpr float RMS_EPS = 1e-6f;
+// 1 / sqrt(mean(v^2) + eps) from a sum of squares over `width` elements
+static __device__ __forceinline__ float rms_scale(float ss, int width) { return rsqrtf(ss / (float)width + RMS_EPS); }
 
 // Programmatic dependent launch: a kernel launched with launch_pdl() may start while its
 // predecessor in the stream is still running (after the predecessor called pdl_trigger()); it must
@@ -114,7 +121,7 @@ static __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __e
 static __device__ __forceinline__ float sigma_f(int kind, float v) {
   if (kind == DEAMOE_SIGMA_SILU) return silu_f(v);
   if (kind == DEAMOE_SIGMA_GELU) return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f));
-  return v;
+  return v;  // none; RMSNorm: the vector is stored un-normalised, its consumer applies rms_scale()
 }
 
 // host-side launchers (each returns the number of kernels it launched, or -1 on a launch error)

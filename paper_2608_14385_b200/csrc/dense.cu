@@ -377,6 +377,12 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
         tc_fence_after();
         const int n = 16 * e + lane;                      // token of this lane (lanes 16..31: none)
         const bool mine = lane < 16 && n < Tg;
+        // sigma = RMSNorm: the first stage stores G and U un-normalised and adds their squares to
+        // the row's two sums; the last stage scales its result by the pair's 1 / rms(Z)
+        const bool rms = L.sigma == DEAMOE_SIGMA_RMSNORM;
+        const int grow = j.row0 + n0 + n;                 // row of this lane's token in the stage's planes
+        float zscale = 1.f;
+        if (rms && mine && ph.stage == ST_S4) zscale = rms_scale(__ldcg(L.ss_z + grow), L.f);
         if (16 * e < Tg) {                                // warp-uniform: some lane of the warp has a token
           const uint32_t t0 = tmem_base + ((uint32_t)(e * 32) << 16) + buf * (uint32_t)DN_TILE;
           const size_t o0 = (size_t)(j.row0 + n0 + n) * ph.out_stride + (size_t)j.col0;
@@ -389,9 +395,15 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
               float v[16];
 #pragma unroll
               for (int q = 0; q < 16; ++q) {
-                v[q] = __uint_as_float(r0[q]);
+                v[q] = __uint_as_float(r0[q]) * zscale;
                 if (ph.epi == DE_SWIGLU) v[q] = silu_f(v[q]) * __uint_as_float(r1[q]);
                 else if (ph.epi == DE_SIGMA) v[q] = sigma_f(L.sigma, v[q]);
+              }
+              if (rms && ph.stage == ST_S1) {  // 16 columns of one half (f is a multiple of 128)
+                float sq = 0.f;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) sq = fmaf(v[q], v[q], sq);
+                atomicAdd(L.ss_gu + (size_t)grow * 2 + ((j.col0 + c0) >= L.f ? 1 : 0), sq);
               }
               if (ph.outf) {
                 float4* dst = reinterpret_cast<float4*>(ph.outf + o0 + c0);

@@ -227,6 +227,31 @@ __global__ void k_plain_identity_private(LayerDev L) {
   }
 }
 
+// sigma = RMSNorm (plain schedule): normalise, in place, the `parts` vectors of `width` floats that
+// make up every row of `buf`; the number of rows is counter `count_idx` of the routing state.
+// One block per (row, part).
+__global__ void k_plain_rmsnorm(LayerDev L, float* __restrict__ buf, int count_idx, int parts, int width) {
+  __shared__ float s_part[32];
+  const int rows = L.counts[count_idx];
+  for (int v = (int)blockIdx.x; v < rows * parts; v += (int)gridDim.x) {
+    float* p = buf + (size_t)v * width;
+    float ss = 0.f;
+    for (int i = (int)threadIdx.x; i < width; i += (int)blockDim.x) ss = fmaf(p[i], p[i], ss);
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      float t = (threadIdx.x < (blockDim.x >> 5)) ? s_part[threadIdx.x] : 0.f;
+      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+      if (threadIdx.x == 0) s_part[0] = t;
+    }
+    __syncthreads();
+    const float sc = rms_scale(s_part[0], width);
+    for (int i = (int)threadIdx.x; i < width; i += (int)blockDim.x) p[i] *= sc;
+    __syncthreads();
+  }
+}
+
 // Eq. (3): out[t] = sum_q p[t,q] * O[slot(t,q)] (+ shared expert) (+ x[t]), written in act dtype.
 __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void* __restrict__ out) {
   TS_MIN(L, 8);
@@ -275,10 +300,19 @@ static int plain_forward_t(const LayerDev& L, int B, cudaStream_t s) {
   } else {
     k_plain_rows<WT><<<rows_grid(2 * L.f, max_dept), PLAIN_THREADS, 0, s>>>(L, ST_S1, B);
     ++launches;
+    const bool rms = L.sigma == DEAMOE_SIGMA_RMSNORM;
+    if (rms) {  // G and U of every (token, department) row
+      k_plain_rmsnorm<<<296, 256, 0, s>>>(L, L.GU, CNT_TOKEN_DEPT, 2, L.f);
+      ++launches;
+    }
     if (L.r > 0) {
       k_plain_rows<WT><<<rows_grid(L.r, max_exp), PLAIN_THREADS, 0, s>>>(L, ST_S2, B);
       k_plain_cols<WT><<<cols_grid(L.f, max_exp), PLAIN_THREADS, 0, s>>>(L, ST_S3, B);
       launches += 2;
+      if (rms) {  // Z of every pair
+        k_plain_rmsnorm<<<296, 256, 0, s>>>(L, L.Z, CNT_PAIRS, 1, L.f);
+        ++launches;
+      }
     } else {
       k_plain_identity_private<<<148, 256, 0, s>>>(L);
       ++launches;

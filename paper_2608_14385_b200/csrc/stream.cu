@@ -701,6 +701,11 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 11);
 #endif
   for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) S.counts[i] = 0;
+  if (L.sigma == DEAMOE_SIGMA_RMSNORM) {  // sums of squares of this step's G, U and Z vectors
+    const int ngu = 2 * B * (L.k < L.m ? L.k : L.m), nz = B * L.k;
+#pragma unroll 1
+    for (int i = tid; i < ngu + nz; i += FINISH_THREADS) (i < ngu ? L.ss_gu[i] : L.ss_z[i - ngu]) = 0.f;
+  }
   const bool regs_ok = topk_in_registers(L);
   if (warp < topk_warps) {
     const int per_warp = (L.n * 5 + 15) & ~15;  // n fp32 logits + n flag bytes (memory path only)
@@ -1309,12 +1314,21 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       // stores of one token are contiguous.
       const int ntile = paired ? 1 : q;
       const int count = ntile * T * 16;
-      for (int x = lane; x < count; x += 32) {
+      // sigma = RMSNorm: a stage that ends in sigma stores its vector un-normalised and adds the
+      // squares to the vector's sum; the stage that reads the vector scales its own result (the
+      // matrix product in between is linear).  The sums are complete when the dependency counter
+      // that lets the reader start is: both are published behind the same fence.
+      const bool rms = L.sigma == DEAMOE_SIGMA_RMSNORM;
+      const int stage = sg->stage;
+      for (int x0 = 0; x0 < count; x0 += 32) {
+        const int x = x0 + lane;
         const int rr = x & 15, s = (x >> 4) % T, a = x / (16 * T);
         const int p = s >> 3, reg = ((rr & 8) ? 2 : 0) + (s & 1), ln = (rr & 7) * 4 + ((s & 7) >> 1);
         const int rem = (p * 4 + reg) * 32 + ln;
         float v0 = 0.f, v1 = 0.f;
-        if (q == 2) {
+        if (x >= count) {
+          // (a lane past the end only takes part in the shuffles below)
+        } else if (q == 2) {
           constexpr int HW = CONSUMER_WARPS / 2;
 #pragma unroll
           for (int w = 0; w < HW; ++w) {
@@ -1326,11 +1340,30 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
           for (int w = 0; w < CONSUMER_WARPS; ++w) v0 += rbuf[(size_t)w * (MAX_QP * 128) + rem];
         }
         const int row = tile0 * 16 + a * 16 + rr;
-        if (row < rows && s < T) {
+        const bool live = x < count && row < rows && s < T;
+        if (rms && epi == EPI_SIGMA) {  // 16 consecutive lanes hold 16 rows of one token and tile
+          float sq = live ? v0 * v0 : 0.f;
+#pragma unroll
+          for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          if ((lane & 15) == 0 && x < count && s < T) {
+            if (stage == ST_S1) atomicAdd(L.ss_gu + (size_t)(out_row0 + s) * 2 + (row >= L.f ? 1 : 0), sq);
+            else atomicAdd(L.ss_z + (out_row0 + s), sq);
+          }
+        }
+        if (live) {
           float r;
           if (epi == EPI_SIGMA) r = sigma_f(L.sigma, v0);
-          else if (epi == EPI_SWIGLU) r = silu_f(v0) * v1;
-          else r = v0;
+          else if (epi == EPI_SWIGLU) {
+            if (rms && stage == ST_S2) {  // inputs were the un-normalised G and U of this pair's row
+              const float* ss = L.ss_gu + (size_t)sg->rows16[s] * 2;
+              v0 *= rms_scale(__ldcg(ss), L.f);
+              v1 *= rms_scale(__ldcg(ss + 1), L.f);
+            }
+            r = silu_f(v0) * v1;
+          } else {
+            r = v0;
+            if (rms && stage == ST_S4) r *= rms_scale(__ldcg(L.ss_z + sg->rows16[s]), L.f);
+          }
           const size_t o = (size_t)(out_row0 + s) * out_stride + row;
           if (outf) {
             outf[o] = r;

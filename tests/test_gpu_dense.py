@@ -41,12 +41,13 @@ def test_dense_schedule_wide_layer(B):
     run_case(DENSE_WIDE, B, seed=12, schedule=binding.SCHED_DENSE, weights=_scaled(DENSE_WIDE, 12, scale=6.0))
 
 
-@pytest.mark.parametrize("variant", ["no_shared", "sigma_none", "gelu", "group_limited", "residual"])
+@pytest.mark.parametrize("variant", ["no_shared", "sigma_none", "gelu", "rmsnorm", "group_limited", "residual"])
 def test_dense_schedule_variants(variant):
     shape = {
         "no_shared": DENSE_SMALL.with_(n_shared=0, shared_ffn=0),
         "sigma_none": DENSE_SMALL.with_(sigma=0),
         "gelu": DENSE_SMALL.with_(sigma=2),
+        "rmsnorm": DENSE_SMALL.with_(sigma=3),
         "group_limited": DENSE_SMALL.with_(n_dept=4, top_k=4, k_dept=2),
         "residual": DENSE_SMALL.with_(residual=1),
     }[variant]

@@ -59,13 +59,15 @@ def test_vanilla_comparator(schedule):
 
 
 @pytest.mark.parametrize("schedule", ALL_SCHEDULES)
-@pytest.mark.parametrize("variant", ["no_private", "sigma_none", "gelu", "square_private", "g1", "k_eq_n",
+@pytest.mark.parametrize("variant", ["no_private", "sigma_none", "gelu", "rmsnorm", "rmsnorm_shared_f32", "square_private", "g1", "k_eq_n",
                                      "norm_all", "group_limited", "f32_tokens"])
 def test_variants(schedule, variant):
     shape = {
         "no_private": SMALL.with_(priv=0),
         "sigma_none": SMALL.with_(sigma=0),
         "gelu": SMALL.with_(sigma=2),
+        "rmsnorm": SMALL.with_(sigma=3),
+        "rmsnorm_shared_f32": RAGGED.with_(sigma=3, act_dtype=0),
         "square_private": SMALL.with_(priv=48),
         "g1": SMALL.with_(n_dept=12, experts_per_dept=1),
         "k_eq_n": SMALL.with_(n_dept=2, experts_per_dept=2, top_k=4),
@@ -204,6 +206,9 @@ def test_unsupported_and_invalid_creates_are_reported():
     assert e.value.status == binding.ERR_UNSUPPORTED
     with pytest.raises(binding.DeaMoEError) as e:
         binding.Layer(SMALL.with_(weight_dtype=0), w, 4, binding.SCHED_FUSED)   # fp32 cannot stream
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.DeaMoEError) as e:
+        binding.Layer(SMALL.with_(sigma=3, priv=0), w, 4, binding.SCHED_PLAIN)   # RMSNorm needs private matrices
     assert e.value.status == binding.ERR_UNSUPPORTED
 
 
