@@ -30,6 +30,10 @@
  *     department index) survive, TopK runs over their experts only;
  *   - department of expert i is i div experts_per_dept;
  *   - an optional always-on shared expert is Eq. (1) with weight 1;
+ *   - strict department coverage (the variant Section 3.3 evaluates and rejects): while the
+ *     selection spans fewer than min(k_dept, k) departments, the lowest-ranked selected expert
+ *     whose department holds another selected expert is replaced, in place, by the expert with
+ *     the largest logit (ties: lowest index) among the departments not yet covered;
  *   - sigma = RMSNorm (one of the operators of Section 3.4 / Table 4) acts on the whole
  *     length-f vector: v / sqrt(mean(v^2) + 1e-6), no learned gain.
  *
@@ -67,6 +71,7 @@ typedef struct {
   int32_t weight_dtype;
   int32_t act_dtype;
   int32_t residual;         /* 1: out = x + layer(x) */
+  int32_t strict_dept;      /* 1: strict department coverage (Section 3.3, last paragraph) */
   double route_scale;
 } oracle_config_t;
 
@@ -264,6 +269,36 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
       if (alive[i / g]) { key[cand].v = l[i]; key[cand].i = i; ++cand; }
     if (cand < k) { rc = 1; break; }
     qsort(key, (size_t)cand, sizeof(keyed_t), cmp_desc_then_index);
+    /* strict department coverage: swap duplicates out until min(k_dept, k) departments are covered */
+    if (c->strict_dept && c->k_dept > 0) {
+      const int target = (c->k_dept < k ? c->k_dept : k) < m ? (c->k_dept < k ? c->k_dept : k) : m;
+      for (;;) {
+        int covered = 0;
+        for (int j = 0; j < m; ++j) {
+          int hit = 0;
+          for (int q = 0; q < k; ++q) if (key[q].i / g == j) hit = 1;
+          covered += hit;
+        }
+        if (covered >= target) break;
+        int victim = -1;
+        for (int q = 0; q < k; ++q) {
+          int same = 0;
+          for (int q2 = 0; q2 < k; ++q2) if (q2 != q && key[q2].i / g == key[q].i / g) same = 1;
+          if (same) victim = q; /* the last such q is the lowest-ranked one */
+        }
+        if (victim < 0) break;
+        int best = -1;
+        for (int i = 0; i < n; ++i) {
+          int used = 0;
+          for (int q = 0; q < k; ++q) if (key[q].i / g == i / g) used = 1;
+          if (used) continue;
+          if (best < 0 || l[i] > l[best]) best = i; /* ascending i: ties keep the lowest index */
+        }
+        if (best < 0) break;
+        key[victim].i = best;
+        key[victim].v = l[best];
+      }
+    }
     for (int q = 0; q < k; ++q) topk_idx[(size_t)t * k + q] = key[q].i;
     if (gap) {
       int upto = (k + 1 < cand) ? k + 1 : cand;

@@ -23,7 +23,7 @@ SIGMA_NONE, SIGMA_SILU, SIGMA_GELU, SIGMA_RMSNORM = 0, 1, 2, 3
 class OracleConfig(C.Structure):
     _fields_ = [(k, C.c_int32) for k in (
         "hidden", "n_dept", "experts_per_dept", "ffn", "priv", "top_k", "k_dept", "n_shared",
-        "shared_ffn", "sigma", "norm_topk", "weight_dtype", "act_dtype", "residual")] + [
+        "shared_ffn", "sigma", "norm_topk", "weight_dtype", "act_dtype", "residual", "strict_dept")] + [
         ("route_scale", C.c_double)]
 
 
@@ -64,9 +64,9 @@ def host_cores():
 
 def make_config(hidden, n_dept, experts_per_dept, ffn, priv, top_k, k_dept=0, n_shared=0,
                 shared_ffn=0, sigma=SIGMA_SILU, norm_topk=1, weight_dtype=BF16, act_dtype=BF16,
-                residual=0, route_scale=1.0, **_ignored):
+                residual=0, route_scale=1.0, strict_dept=0, **_ignored):
     return OracleConfig(hidden, n_dept, experts_per_dept, ffn, priv, top_k, k_dept, n_shared,
-                        shared_ffn, sigma, norm_topk, weight_dtype, act_dtype, residual,
+                        shared_ffn, sigma, norm_topk, weight_dtype, act_dtype, residual, strict_dept,
                         float(route_scale))
 
 

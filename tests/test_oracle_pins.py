@@ -106,6 +106,51 @@ def test_group_limited_routing_bruteforce():
         assert len({i // 3 for i in got["idx"][t]}) <= 2
 
 
+def test_strict_department_coverage_properties():
+    """The strict variant of Section 3.3: every token ends up with exactly min(k_dept, k)
+    departments; a token whose soft selection already has that many is untouched; otherwise only
+    lowest-ranked duplicates leave (the highest-ranked expert of every covered department stays, the
+    number of swaps is the number of missing departments), and every newcomer is the best expert of
+    its department, taken from the best-scoring uncovered departments."""
+    shape = synth.LayerShape("t", hidden=16, n_dept=6, experts_per_dept=6, ffn=8, priv=0, top_k=4,
+                             k_dept=4, weight_dtype=0, act_dtype=0)
+    g, m, k, kd = 6, 6, 4, 4
+    router = synth.normal((36, 16), 1.0, 7, "r").numpy()
+    tokens = synth.normal((64, 16), 1.0, 7, "x").numpy()
+    soft = ref.route(oracle_cfg(shape), router, tokens, want_logits=True)
+    strict = ref.route(oracle_cfg(shape.with_(strict_dept=1)), router, tokens)
+    changed_tokens = 0
+    for t in range(64):
+        l = soft["logits"][t]
+        a, b = list(soft["idx"][t]), list(strict["idx"][t])
+        da, db = [i // g for i in a], [i // g for i in b]
+        assert len(set(b)) == k and len(set(db)) == min(kd, k)
+        missing = min(kd, k) - len(set(da))
+        assert sum(x != y for x, y in zip(a, b)) == missing
+        if missing == 0:
+            continue
+        changed_tokens += 1
+        for q, (x, y) in enumerate(zip(a, b)):
+            if x != y:
+                assert da[q] in da[:q]                       # a lower-ranked duplicate left ...
+                assert y == max(range(db[q] * g, db[q] * g + g), key=lambda i: (l[i], -i))   # ... for a department's best
+                assert db[q] not in da
+        # the departments that came in are the best-scoring uncovered ones
+        score = {j: max(l[j * g:(j + 1) * g]) for j in range(m) if j not in da}
+        came = sorted(set(db) - set(da))
+        assert came == sorted(sorted(score, key=lambda j: (-score[j], j))[:missing])
+        # no higher-ranked duplicate stayed while a lower-ranked one of another department left
+        left = [q for q in range(k) if a[q] != b[q]]
+        stay_dups = [q for q in range(k) if a[q] == b[q] and da[q] in da[:q]]
+        assert all(q < min(left) for q in stay_dups)
+    assert changed_tokens >= 5                               # the case is exercised
+    w_sum = strict["w"].sum(axis=1)
+    np.testing.assert_allclose(w_sum, 1.0, rtol=1e-12)
+    off = ref.route(oracle_cfg(shape.with_(strict_dept=1, k_dept=0)), router, tokens)   # no cap: nothing to enforce
+    free = ref.route(oracle_cfg(shape.with_(k_dept=0)), router, tokens)
+    assert (off["idx"] == free["idx"]).all()
+
+
 # ---------------------------------------------------------------- Section 3.2 sets and lists
 
 def test_bucketing_matches_python_sets():
