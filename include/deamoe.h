@@ -96,6 +96,12 @@ typedef struct {
   int32_t max_batch;        /* largest B any later call may pass (1..DEAMOE_MAX_BATCH) */
   int32_t schedule;         /* deamoe_schedule_t */
   float route_scale;        /* gate weights are multiplied by this (Eq. (3) "scaling") */
+  int32_t strict_dept;      /* 1 (with k_dept > 0): strict department coverage, the variant Section 3.3
+                               evaluates and rejects: while a token's selection spans fewer than
+                               min(k_dept, k) departments, its lowest-ranked selected expert whose
+                               department holds another selected expert is replaced, in place, by
+                               the expert with the largest logit (ties: lowest index) of the
+                               departments not yet covered.  Needs n_dept <= 64.  0: the soft cap. */
 } deamoe_config_t;
 
 #define DEAMOE_MAX_BATCH 128

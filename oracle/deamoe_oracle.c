@@ -269,6 +269,15 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
       if (alive[i / g]) { key[cand].v = l[i]; key[cand].i = i; ++cand; }
     if (cand < k) { rc = 1; break; }
     qsort(key, (size_t)cand, sizeof(keyed_t), cmp_desc_then_index);
+    if (gap) { /* smallest difference between neighbours of the sorted order, up to the first expert left out */
+      int upto = (k + 1 < cand) ? k + 1 : cand;
+      double gmin = INFINITY;
+      for (int q = 1; q < upto; ++q) {
+        double d = key[q - 1].v - key[q].v;
+        if (d < gmin) gmin = d;
+      }
+      gap[t] = gmin;
+    }
     /* strict department coverage: swap duplicates out until min(k_dept, k) departments are covered */
     if (c->strict_dept && c->k_dept > 0) {
       const int target = (c->k_dept < k ? c->k_dept : k) < m ? (c->k_dept < k ? c->k_dept : k) : m;
@@ -300,15 +309,6 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
       }
     }
     for (int q = 0; q < k; ++q) topk_idx[(size_t)t * k + q] = key[q].i;
-    if (gap) {
-      int upto = (k + 1 < cand) ? k + 1 : cand;
-      double gmin = INFINITY;
-      for (int q = 1; q < upto; ++q) {
-        double d = key[q - 1].v - key[q].v;
-        if (d < gmin) gmin = d;
-      }
-      gap[t] = gmin;
-    }
     /* softmax (max-subtracted) over the selection, or over all n logits */
     double mx = key[0].v, den = 0.0;
     if (c->norm_topk) {

@@ -28,7 +28,7 @@ class Config(C.Structure):
     _fields_ = [(k, C.c_int32) for k in (
         "hidden", "n_dept", "experts_per_dept", "ffn", "priv", "top_k", "k_dept", "n_shared",
         "shared_ffn", "sigma", "norm_topk", "weight_dtype", "act_dtype", "residual", "max_batch",
-        "schedule")] + [("route_scale", C.c_float)]
+        "schedule")] + [("route_scale", C.c_float), ("strict_dept", C.c_int32)]
 
 
 class Weights(C.Structure):
@@ -96,7 +96,8 @@ def make_config(shape, max_batch, schedule=SCHED_AUTO):
     return Config(d["hidden"], d["n_dept"], d["experts_per_dept"], d["ffn"], d["priv"], d["top_k"],
                   d.get("k_dept", 0), d.get("n_shared", 0), d.get("shared_ffn", 0), d.get("sigma", 1),
                   d.get("norm_topk", 1), d.get("weight_dtype", 1), d.get("act_dtype", 1),
-                  d.get("residual", 0), int(max_batch), int(schedule), float(d.get("route_scale", 1.0)))
+                  d.get("residual", 0), int(max_batch), int(schedule), float(d.get("route_scale", 1.0)),
+                  int(d.get("strict_dept", 0)))
 
 
 STATIC_ROUTE_SCRATCH_BYTES = 4 << 20

@@ -67,6 +67,8 @@ deamoe_status_t check_config(const deamoe_config_t* c, const deamoe_weights_t* w
   if (!vanilla && c->sigma == DEAMOE_SIGMA_RMSNORM && c->priv <= 0) return DEAMOE_ERR_UNSUPPORTED;
   if (c->schedule < DEAMOE_SCHED_AUTO || c->schedule > DEAMOE_SCHED_DENSE) return DEAMOE_ERR_INVALID_ARG;
   if (!(c->route_scale == c->route_scale)) return DEAMOE_ERR_INVALID_ARG;
+  if (c->strict_dept != 0 && c->strict_dept != 1) return DEAMOE_ERR_INVALID_ARG;
+  if (c->strict_dept && c->k_dept > 0 && c->n_dept > 64) return DEAMOE_ERR_UNSUPPORTED;
   if (c->max_batch < 1 || c->max_batch > DEAMOE_MAX_BATCH) return DEAMOE_ERR_BATCH;
   if (!w->router || !w->dept_gate || !w->dept_up || !w->dept_down) return DEAMOE_ERR_INVALID_ARG;
   if (vanilla && c->priv != 0) return DEAMOE_ERR_INVALID_ARG;
@@ -103,6 +105,7 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   d.sigma = vanilla ? DEAMOE_SIGMA_NONE : cfg->sigma; d.norm_topk = cfg->norm_topk;
   d.residual = cfg->residual; d.vanilla = vanilla ? 1 : 0;
   d.wdt = cfg->weight_dtype; d.adt = cfg->act_dtype; d.max_batch = cfg->max_batch;
+  d.strict_dept = cfg->strict_dept;
   d.rp = d.r > 0 ? d.r : d.f;
   d.route_scale = cfg->route_scale;
 

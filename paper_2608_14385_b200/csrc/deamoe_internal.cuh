@@ -58,6 +58,7 @@ struct LayerDev {
   // sizes
   int h, m, g, n, f, r, k, k_dept, n_shared, fs, sigma, norm_topk, residual, vanilla;
   int wdt, adt, max_batch;
+  int strict_dept;  // 1: strict department coverage routing (with k_dept > 0)
   int rp;  // rows of Y per pair: r, or f when there are no private parameters
   float route_scale;
   // canonical weights (PLAIN schedule and fp32); element type per wdt

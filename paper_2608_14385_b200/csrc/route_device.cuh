@@ -13,6 +13,35 @@ static __device__ __forceinline__ bool better(float v, int i, float bv, int bi) 
   return (v > bv) || (v == bv && i < bi);
 }
 
+// Strict department coverage (the variant Section 3.3 evaluates in its last paragraph), applied by
+// one warp to the selection it holds (lane q < k: the q-th selected expert my_i and its logit
+// my_v): while the selection spans fewer than min(k_dept, k) departments, the lowest-ranked
+// selected expert whose department holds another selected expert is replaced, in place, by the
+// expert with the largest logit (ties: lowest index) of the departments not yet covered.
+// find(covered, v, i) returns that expert to every lane (i = 0x7fffffff: none).  m <= 64.
+template <typename Find>
+static __device__ __forceinline__ void strict_coverage(const LayerDev& L, int lane, float& my_v, int& my_i, Find find) {
+  const int k = L.k, g = L.g;
+  const int target = min(min(L.k_dept, k), L.m);
+#pragma unroll 1
+  for (int round = 0; round < target; ++round) {
+    const int md = (lane < k) ? my_i / g : -1 - lane;  // lanes without a selection match nobody
+    const unsigned long long bit = (lane < k) ? (1ull << md) : 0ull;
+    const unsigned long long covered =
+        (unsigned long long)__reduce_or_sync(0xffffffffu, (unsigned)bit) |
+        ((unsigned long long)__reduce_or_sync(0xffffffffu, (unsigned)(bit >> 32)) << 32);
+    if (__popcll(covered) >= target) break;
+    const unsigned same = __match_any_sync(0xffffffffu, md);
+    const int victim = __reduce_max_sync(0xffffffffu, (lane < k && (same & ~(1u << lane))) ? lane : -1);
+    if (victim < 0) break;
+    float cv;
+    int ci;
+    find(covered, cv, ci);
+    if (ci == 0x7fffffff) break;
+    if (lane == victim) { my_v = cv; my_i = ci; }
+  }
+}
+
 // Top-k and gate weights of token t by one warp.  lg: n floats, dead: n bytes of shared memory.
 static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslices, float* lg, unsigned char* dead,
                                       int lane, int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
@@ -69,6 +98,20 @@ static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslic
     if (lane == 0 && bi < n) dead[bi] = 1;
     __syncwarp();
   }
+  if (L.strict_dept && L.k_dept > 0)
+    strict_coverage(L, lane, my_v, my_i, [&](unsigned long long covered, float& cv, int& ci) {
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+      for (int i = lane; i < n; i += 32)
+        if (!((covered >> (i / g)) & 1ull) && better(lg[i], i, bv, bi)) { bv = lg[i]; bi = i; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      }
+      cv = bv; ci = bi;
+    });
   // gate weights
   const float top = __shfl_sync(0xffffffffu, my_v, 0);
   float e, den;
@@ -247,6 +290,23 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
 #ifdef DEAMOE_TRACE
   if (lane == 0 && t == 0) { L.counts[11] = (int)(clock64() - ta); L.counts[12] = (int)(ta & 0x7fffffff); }
 #endif
+  if (L.strict_dept && L.k_dept > 0)
+    strict_coverage(L, lane, my_v, my_i, [&](unsigned long long covered, float& cv, int& ci) {
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) {
+        const int idx = lane + 32 * j;
+        if (idx < n && !((covered >> (idx / L.g)) & 1ull) && better(v[j], idx, bv, bi)) { bv = v[j]; bi = idx; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      }
+      cv = bv; ci = bi;
+    });
   const float top = __shfl_sync(0xffffffffu, my_v, 0);
   float e, den;
   if (L.norm_topk) {

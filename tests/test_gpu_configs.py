@@ -147,24 +147,27 @@ def test_layers_enqueued_back_to_back_match_layers_run_one_by_one(vanilla):
 
 
 WIDE_ROUTERS = [
-    # n_dept, experts_per_dept, top_k, k_dept
-    (6, 16, 6, 0),       # 96 experts: 8 logits per lane
-    (10, 32, 10, 0),     # 320 experts: 16 logits per lane
-    (10, 32, 10, 4),     # group limited
-    (8, 108, 10, 5),     # the paper's DeepSeek-V3 router
-    (32, 32, 32, 0),     # 1024 experts, top-32: the widest the register top-k takes
-    (32, 32, 8, 3),
-    (40, 40, 8, 6),      # 1600 experts, 40 departments: the shared-memory top-k
+    # n_dept, experts_per_dept, top_k, k_dept, strict department coverage
+    (6, 16, 6, 0, 0),       # 96 experts: 8 logits per lane
+    (10, 32, 10, 0, 0),     # 320 experts: 16 logits per lane
+    (10, 32, 10, 4, 0),     # group limited
+    (8, 108, 10, 5, 0),     # the paper's DeepSeek-V3 router
+    (32, 32, 32, 0, 0),     # 1024 experts, top-32: the widest the register top-k takes
+    (32, 32, 8, 3, 0),
+    (40, 40, 8, 6, 0),      # 1600 experts, 40 departments: the shared-memory top-k
+    (6, 16, 6, 4, 1),       # strict department coverage (Section 3.3, last paragraph)
+    (8, 108, 10, 5, 1),     # ... on the paper's DeepSeek-V3 router
+    (40, 40, 8, 6, 1),      # ... in the shared-memory top-k
 ]
 
 
-@pytest.mark.parametrize("m,g,k,k_dept", WIDE_ROUTERS)
-def test_routing_of_wide_and_group_limited_routers(m, g, k, k_dept):
+@pytest.mark.parametrize("m,g,k,k_dept,strict", WIDE_ROUTERS)
+def test_routing_of_wide_and_group_limited_routers(m, g, k, k_dept, strict):
     """Routing only (indices, gate weights, department and expert lists) on layers with tiny experts but
     wide routers, so that every top-k variant (8 / 16 / 32 logits per lane, group limit in registers,
     shared-memory fallback) is compared with the oracle, with random logits and with exact ties."""
     shape = synth.LayerShape(f"wide{m}x{g}", hidden=256, n_dept=m, experts_per_dept=g, ffn=16, priv=16, top_k=k,
-                             k_dept=k_dept)
+                             k_dept=k_dept, strict_dept=strict)
     dev = torch.device("cuda:0")
     w = synth.make_deamoe_weights(shape, 2, dev)
     layer = binding.Layer(shape, w, 40)
