@@ -284,7 +284,7 @@ def main():
             dist.destroy_process_group()
         return
     B = args.batch
-    max_batch = max(64 if shape.name == "dsv3-paper" else 32, B)
+    max_batch = max(64 if shape.name in synth.PAPER_BASELINES else 32, B)
     w = synth.make_deamoe_weights(shape, 0, dev)
     layer = binding.Layer(shape, w, max_batch, sched)
     router = w["router"]
@@ -381,7 +381,7 @@ def main():
     }
 
     if rank == 0 and not args.no_sweep:
-        if shape.name == "dsv3-paper":
+        if shape.name in synth.PAPER_BASELINES:
             line["sweep"] = paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev)
         else:
             line["sweep"] = sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev)
@@ -423,7 +423,7 @@ def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev):
             ub.append(layer.stats()["unique_weight_bytes"])
         t, _ = time_layer(layer, bs, steps, 3, flush, torch, lambda: None)
         res[B] = {"batch": B, "deamoe_us": pct(t, 0.5) * 1e3, "deamoe_mb": statistics.mean(ub) / 1e6}
-    base = dataclasses.replace(synth.DSV3, name="dsv3-no-shared", n_shared=0, shared_ffn=0)
+    base = synth.PAPER_BASELINES[shape.name]
     vw = synth.make_vanilla_weights(base, 0, dev)
     vl = binding.Layer(base, vw, 64, sched, vanilla=True)
     del vw
@@ -446,9 +446,11 @@ def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev):
         r["speedup_vs_baseline_moe"] = r["baseline_moe_us"] / r["deamoe_us"]
         out.append(r)
     vl.close()
-    return {"rows": out,
-            "paper_context": "expected loaded-weights ratio 0.491 .. 0.628 over 4 .. 64 tokens (Section 3.3, Fig. 2); "
-                             "peak layer speed-up 2.00x (A40) / 1.97x (H100)"}
+    ctx = ("expected loaded-weights ratio 0.491 .. 0.628 over 4 .. 64 tokens (Section 3.3, Fig. 2); peak layer "
+           "speed-up 2.00x (A40) / 1.97x (H100)") if shape.name == "dsv3-paper" else \
+          "Fig. 2 shows this model's loaded-weights ratio as a curve only (no printed numbers)"
+    return {"rows": out, "baseline": {"name": base.name, "n_expert": base.n_expert, "top_k": base.top_k},
+            "paper_context": ctx}
 
 
 def locality_sweep(args, sched, peak, torch, dev):

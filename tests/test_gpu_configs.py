@@ -90,6 +90,26 @@ def test_paper_deepseek_v3_row_group_limited(B, rows):
         st["active_dept"], st["active_expert"], shape.hidden, shape.ffn, shape.priv, shape.n_expert, 2)
 
 
+@pytest.mark.parametrize("name,B,rows", [("qwen3-paper", 16, [3, 15]), ("b7-paper", 64, [0, 40, 63]),
+                                         ("dsv2-paper", 8, [5])])
+def test_other_table1_rows(name, B, rows):
+    """Further rows of Table 1 at full size (Qwen3-235B-, Baseline-7B- and DeepSeek-V2-matched DeaMoE
+    configurations): routing and lists for the whole batch, values on sampled rows, unique bytes
+    equal to the closed form on the counted sets."""
+    shape = synth.SHAPES[name]
+    res = run_case(shape, B, seed=1, rows=rows, max_batch=64)
+    st = res["stats"]
+    assert st["unique_weight_bytes"] == accounting.unique_bytes_deamoe(
+        st["active_dept"], st["active_expert"], shape.hidden, shape.ffn, shape.priv, shape.n_expert, 2)
+
+
+def test_table1_baselines_as_vanilla_layers():
+    """The standard MoE layers the Table 1 rows are matched to run as vanilla layers (flat top-k)."""
+    for name, B in (("qwen3-paper", 8), ("b7-paper", 16)):
+        base = synth.PAPER_BASELINES[name]
+        run_case(base, B, seed=2, vanilla=True, rows=[B - 1], max_batch=16)
+
+
 def test_paper_row_department_cap_holds_for_every_token():
     shape = synth.DSV3_PAPER
     dev = torch.device("cuda:0")
@@ -151,7 +171,11 @@ WIDE_ROUTERS = [
     (6, 16, 6, 0, 0),       # 96 experts: 8 logits per lane
     (10, 32, 10, 0, 0),     # 320 experts: 16 logits per lane
     (10, 32, 10, 4, 0),     # group limited
-    (8, 108, 10, 5, 0),     # the paper's DeepSeek-V3 router
+    (8, 108, 10, 5, 0),     # the paper's DeepSeek-V3 router (Table 1)
+    (8, 64, 10, 5, 0),      # ... DeepSeek-V2 router
+    (8, 40, 8, 5, 0),       # ... Qwen3-235B router
+    (16, 80, 10, 5, 0),     # ... Kimi-K2 router: 1280 experts, the shared-memory top-k with a group limit
+    (8, 84, 10, 4, 0),      # ... Baseline-7B router
     (32, 32, 32, 0, 0),     # 1024 experts, top-32: the widest the register top-k takes
     (32, 32, 8, 3, 0),
     (40, 40, 8, 6, 0),      # 1600 experts, 40 departments: the shared-memory top-k
