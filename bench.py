@@ -284,7 +284,8 @@ def main():
             dist.destroy_process_group()
         return
     B = args.batch
-    max_batch = max(64 if shape.name in synth.PAPER_BASELINES else 32, B)
+    # (sized for the largest batch of the sweep; from 56 tokens on AUTO takes the dense schedule)
+    max_batch = max(64 if shape.name in synth.PAPER_BASELINES else (128 if shape.name == "dsv3" and not args.no_sweep else 32), B)
     w = synth.make_deamoe_weights(shape, 0, dev)
     layer = binding.Layer(shape, w, max_batch, sched)
     router = w["router"]
@@ -623,7 +624,7 @@ def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev):
     """DeaMoE layer and the in-library vanilla MoE at the same shape over the batch range."""
     from paper_2608_14385_b200 import binding, synth
     out = []
-    batches_list = [1, 2, 4, 8, 16, 32] if shape.name == "dsv3" else [1, 4, 16]
+    batches_list = [1, 2, 4, 8, 16, 32, 64, 128] if shape.name == "dsv3" else [1, 4, 16]
     steps = max(10, args.steps // 2)
     res = {}
     for B in batches_list:
@@ -635,7 +636,7 @@ def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev):
         t, _ = time_layer(layer, bs, steps, 3, flush, torch, lambda: None)
         res[B] = {"batch": B, "deamoe_us": pct(t, 0.5) * 1e3, "deamoe_mb": statistics.mean(ub) / 1e6}
     vw = synth.make_vanilla_weights(shape, 0, dev, router=router)
-    vl = binding.Layer(shape, vw, 32, sched, vanilla=True)
+    vl = binding.Layer(shape, vw, max(batches_list), sched, vanilla=True)
     del vw
     torch.cuda.empty_cache()
     for B in batches_list:
