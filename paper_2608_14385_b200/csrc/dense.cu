@@ -27,7 +27,11 @@
 // has to wait that long per chunk cannot keep up, however far ahead it fetches.  The rows' tensor
 // map views a row-major [rows, K] plane as [K / 8][rows][8]; a box of 8 x 64 x 8 lands in shared
 // memory as 8 column blocks of 64 rows x 16 bytes, which is the core-matrix layout with 128 bytes
-// between 8-row groups and 1024 bytes between neighbours along K.  The rows of a bucket are
+// between 8-row groups and 1024 bytes between neighbours along K.  The box is 16, 32 or 64 rows
+// high, whichever holds the group's rows (three tensor maps per input plane; the MMA always reads
+// 64 rows: the ones past the box are stale shared memory of the same stage and feed accumulator
+// rows nobody reads).  The rows come through the same per-SM path as the weights, and a 64-row
+// box for a 15-row bucket would take a fifth of that path.  The rows of a bucket are
 // contiguous in every input plane (the first stage's tokens are gathered into bucket order by a
 // small kernel first); a box may run past the bucket's end, into rows that no output depends on.
 // Weights are stored at create time tile by tile and chunk by chunk in the layout the MMA reads,
@@ -91,6 +95,12 @@ struct DenseArgs {
   DensePhase ph[2];
   int nph;
 };
+// tensor maps of the phases' input planes: [phase][box height 16 / 32 / 64 rows]
+struct DenseMaps {
+  CUtensorMap tm[2][3];
+};
+// box height index for a group of Tg rows
+__host__ __device__ __forceinline__ int box_index(int Tg) { return Tg <= 16 ? 0 : (Tg <= 32 ? 1 : 2); }
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -237,8 +247,7 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
 }
 
 // ---------------------------------------------------------------- the kernel
-__global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A, int B, const __grid_constant__ CUtensorMap tm0,
-                                                         const __grid_constant__ CUtensorMap tm1) {
+__global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A, int B, const __grid_constant__ DenseMaps maps) {
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* ring = smem;  // stage s: weights at s * DN_STAGE_BYTES, activation rows DN_A_BYTES further
   uint64_t* a_full = reinterpret_cast<uint64_t*>(ring + (size_t)DN_AST * DN_STAGE_BYTES);
@@ -284,16 +293,18 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t bytes = (uint32_t)j.ncols * DN_BK * 2;
-        const CUtensorMap* tm = j.phase ? &tm1 : &tm0;
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
         for (int gi = 0; ok && gi < groups; ++gi) {
+          const int bi = box_index(min(DN_NMAX, j.T - gi * DN_NMAX));
+          const CUtensorMap* tm = &maps.tm[j.phase][bi];
+          const uint32_t box_bytes = (16u << bi) * DN_BK * 2;
           for (int c = 0; c < nch; ++c, ++g) {
             const int s = (int)(g % DN_AST);
             { DN_T0();
             if (!bar_wait(&a_empty[s], ((g / DN_AST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
             DN_ADD(0); }
             unsigned char* st = ring + (size_t)s * DN_STAGE_BYTES;
-            bar_arrive_expect_tx(&a_full[s], bytes + DN_B_BYTES);
+            bar_arrive_expect_tx(&a_full[s], bytes + box_bytes);
             bulk_load(st, j.w + (size_t)c * DN_TILE * DN_BK, bytes, &a_full[s], pol);
             tensor_load_3d(st + DN_A_BYTES, tm, 0, j.row0 + gi * DN_NMAX, c * (DN_BK / 8), &a_full[s]);
           }
@@ -317,14 +328,17 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
       // descriptors of stage 0, first k-step; a k-step of 16 columns is two core matrices (256
       // bytes) further, which adds 16 to the descriptor's address field
       const uint64_t desc0_w = umma_smem_desc(smem_addr(ring), 128, DN_BK * 16);
-      // activation rows as the TMA box leaves them: 1024 bytes between neighbours along K, 128 between 8-row groups
-      const uint64_t desc0_x = umma_smem_desc(smem_addr(ring + DN_A_BYTES), DN_NMAX * 16, 128);
+      // activation rows as the TMA box leaves them: (box rows x 16) bytes between neighbours along K,
+      // 128 between 8-row groups; built per token group below
       for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t idesc = umma_instr_desc(DN_NMAX, j.ncols);  // tokens: M operand; weight rows: N operand
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
         for (int gi = 0; ok && gi < groups; ++gi, ++a) {
+          const uint32_t box_rows = 16u << box_index(min(DN_NMAX, j.T - gi * DN_NMAX));
+          const uint64_t desc0_x = umma_smem_desc(smem_addr(ring + DN_A_BYTES), box_rows * 16, 128);
+          const uint32_t xstep = (2 * box_rows * 16) >> 4;  // a k-step of 16 columns = two column blocks of the rows
           const uint32_t buf = a & 1u;
           if (!bar_wait(&acc_empty[buf], ((a >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
@@ -338,9 +352,9 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
             DN_T0();
             const uint64_t dw = desc0_w + (uint64_t)(sa_i * (DN_STAGE_BYTES >> 4));
             const uint64_t dx = desc0_x + (uint64_t)(sa_i * (DN_STAGE_BYTES >> 4));
-            // a k-step of 16 columns: two core matrices further, 256 bytes in the weights, 2048 in the rows
+            // a k-step of 16 columns: two core matrices further, 256 bytes in the weights
 #pragma unroll
-            for (int ks = 0; ks < DN_BK / 16; ++ks) umma(d0, dx + 128 * ks, dw + 16 * ks, idesc, (c | ks) ? 1u : 0u);
+            for (int ks = 0; ks < DN_BK / 16; ++ks) umma(d0, dx + xstep * ks, dw + 16 * ks, idesc, (c | ks) ? 1u : 0u);
             DN_ADD(2);
             { DN_T0();
             umma_commit(&a_empty[sa_i]);  // the stage is free once these MMAs have read it
@@ -577,11 +591,11 @@ void dense_plan_destroy(DensePlan* p) {
   delete p;
 }
 
-// Tensor map over a row-major bf16 plane [rows, K], viewed as [K / 8][rows][8]; box 8 x 64 x 8.
-static bool encode_rows_map(const DensePlan& p, CUtensorMap* tm, const void* base, int rows, int K) {
+// Tensor map over a row-major bf16 plane [rows, K], viewed as [K / 8][rows][8]; box 8 x box_rows x 8.
+static bool encode_rows_map(const DensePlan& p, CUtensorMap* tm, const void* base, int rows, int K, int box_rows) {
   const cuuint64_t dims[3] = {8, (cuuint64_t)rows, (cuuint64_t)(K / 8)};
   const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 16};  // bytes between rows, between 8-column groups
-  const cuuint32_t box[3] = {8, DN_NMAX, DN_BK / 8};
+  const cuuint32_t box[3] = {8, (cuuint32_t)box_rows, DN_BK / 8};
   const cuuint32_t estr[3] = {1, 1, 1};
   return p.encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -594,8 +608,8 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
   DenseArgs A;
   std::memset(&A, 0, sizeof(A));
   A.nph = n_stages;
-  CUtensorMap tm[2];
-  std::memset(tm, 0, sizeof(tm));
+  DenseMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
   int launches = 0;
   for (int i = 0; i < n_stages; ++i) {
     DensePhase& ph = A.ph[i];
@@ -628,10 +642,11 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
       default:
         return -1;
     }
-    if (!encode_rows_map(p, &tm[i], in, in_rows, ph.K)) return -1;
+    for (int b = 0; b < 3; ++b)
+      if (!encode_rows_map(p, &maps.tm[i][b], in, in_rows, ph.K, 16 << b)) return -1;
   }
-  if (n_stages == 1) tm[1] = tm[0];
-  k_dense<<<p.n_sm, DN_THREADS, DN_SMEM, s>>>(L, A, B, tm[0], tm[1]);
+  if (n_stages == 1) std::memcpy(maps.tm[1], maps.tm[0], sizeof(maps.tm[0]));
+  k_dense<<<p.n_sm, DN_THREADS, DN_SMEM, s>>>(L, A, B, maps);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
