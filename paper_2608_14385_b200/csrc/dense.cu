@@ -3,25 +3,26 @@
 //
 // From a few dozen tokens on, a department's token bucket X^j is a dense tile (16 and more rows),
 // and the per-warp mma.sync path of the streaming kernel becomes issue-bound.  Here one
-// tcgen05.mma covers up to 64 tokens of the bucket x 256 weight rows x 16 columns, with the
+// tcgen05.mma covers up to 64 tokens of the bucket x 128 weight rows x 16 columns, with the
 // accumulator in tensor memory:
 //
-//   D[64 tokens, 256 weight rows] += X^j[64, K] . W_tile[256, K]^T
+//   D[64 tokens, 128 weight rows] += X^j[64, K] . W_tile[128, K]^T
 //
-// The tokens are the M operand and the weights the N operand, with N as large as the instruction
-// allows, because what limits this kernel is the one thread that issues the MMAs: an MMA costs
-// it about 125 cycles whatever its shape, a wait or a commit 60 to 250, and the weight stream
-// leaves about 700 cycles per 16 KB.  One 256-row MMA moves 8 KB of weights; with 128-row MMAs
-// (4 KB each) the issue thread was the bottleneck at half the HBM rate.
+// The tokens are the M operand and the weights the N operand.  What limits such a kernel first is
+// the one thread that issues the MMAs: an MMA costs it about 125 cycles whatever its shape, a wait
+// or a commit 60 to 250, and the weight stream leaves about 700 cycles per 16 KB and SM.  With one
+// CTA per SM and 128-row MMAs (4 KB of weights each) that thread was the bottleneck at half the HBM
+// rate; either 256-row MMAs or, as here, two CTAs per SM (two issuing threads, each with twice the
+// time per chunk, and two independent copy / MMA chains whose stalls overlap) remove it.
 // An M = 64 accumulator lives in lanes 32 (r / 16) + r % 16 of tensor memory (row r), so each of
 // the four epilogue warps owns 16 tokens and a token's outputs are one contiguous run.
 //
-// Roles of a CTA (one CTA per SM, persistent over a list of (unit, 256-row tile) jobs):
+// Roles of a CTA (two CTAs per SM, persistent over a list of (unit, 128-row tile) jobs):
 //   warps 0-3   epilogue: tcgen05.ld of the finished accumulator, sigma / SwiGLU, stores
-//   warp  4     one thread issues the copies of a chunk into the ring: the weights (one 32 KB bulk
+//   warp  4     one thread issues the copies of a chunk into the ring: the weights (one 16 KB bulk
 //               copy) and the bucket's activation rows (one tiled TMA copy, 64 rows x 64 columns)
 //   warp  5     one thread issues the MMAs and the commits that free ring stages / publish accumulators
-// The ring has 5 stages of 32 KB weights + 8 KB activation rows.  The activation rows are fetched
+// The ring has 4 stages of 16 KB weights + 8 KB activation rows.  The activation rows are fetched
 // by TMA, not by loads of a warp: while the weights stream at full rate an ordinary load from this
 // SM waits 2 to 4 us behind the bulk copies in flight (measured, L2 hit or not), and a warp that
 // has to wait that long per chunk cannot keep up, however far ahead it fetches.  The rows' tensor
@@ -39,7 +40,7 @@
 // "K-major, no swizzle"): 8 x 8 core matrices of 128 contiguous bytes; byte offset of element
 // (r, k) = (r / 8) * 1024 + (k / 8) * 128 + (r % 8) * 16 + (k % 8) * 2.
 // The jobs are dealt round-robin.  Whole tiles fill as many complete rounds as there are; the
-// tiles left over are split into two 128-row halves each, so that the last round is half as long.
+// tiles left over are split into two 64-row halves each, so that the last round is half as long.
 #include "dense.cuh"
 
 #include <cuda.h>  // CUtensorMap and the encode function's signature; the entry point is looked up at run time
@@ -51,25 +52,27 @@ namespace deamoe {
 
 namespace {
 
-constexpr int DN_AST = 5;                   // ring stages
+constexpr int DN_AST = 4;                   // ring stages
+constexpr int DN_CTAS_PER_SM = 2;
 constexpr int DN_NMAX = 64;                 // token rows of one accumulator (the MMA's M)
 constexpr int DN_BK = 64;                   // columns of a chunk
-constexpr int DN_TILE = 256;                // weight rows of a tile (the MMA's N)
+constexpr int DN_TILE = 128;                // weight rows of a tile (the MMA's N)
 constexpr int DN_A_BYTES = DN_TILE * DN_BK * 2;   // 32 KB
 constexpr int DN_B_BYTES = DN_NMAX * DN_BK * 2;   // 8 KB
 constexpr int DN_STAGE_BYTES = DN_A_BYTES + DN_B_BYTES;
 constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5;
 constexpr int DN_THREADS = (DN_WARP_MMA + 1) * 32;
-constexpr int DN_TMEM_COLS = 512;           // 2 accumulator buffers x 256 columns (all of it)
+constexpr int DN_TMEM_COLS = 2 * DN_TILE;   // 2 accumulator buffers; the CTAs of an SM share its 512 columns
 constexpr size_t DN_SMEM = (size_t)DN_AST * DN_STAGE_BYTES + 512 /* barriers, control */;
 constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits; then an error status, never a hang
-static_assert(DN_SMEM <= 227 * 1024, "shared memory budget");
-// More than half of an SM's shared memory: two of these CTAs never share an SM, so the tensor
-// memory allocation below never waits for another CTA.
-static_assert(DN_SMEM > 114 * 1024, "one CTA per SM is relied upon by the tensor-memory allocation");
+static_assert((DN_SMEM + 1024) * DN_CTAS_PER_SM <= 228 * 1024, "shared memory budget");
+// No more than DN_CTAS_PER_SM of these CTAs fit an SM's shared memory, and together they ask for no
+// more tensor memory than an SM has: the allocation below never waits for another CTA.
+static_assert((DN_SMEM + 1024) * (DN_CTAS_PER_SM + 1) > 228 * 1024 && DN_TMEM_COLS * DN_CTAS_PER_SM <= 512,
+              "tensor-memory allocation must never block");
 
 #ifdef DEAMOE_TRACE
-__device__ long long dn_trace[256 * 16];  // trace builds: per-CTA cycle counters of the last launch
+__device__ long long dn_trace[512 * 16];  // trace builds: per-CTA cycle counters of the last launch
 #define DN_T0() const long long dn_t0 = clock64()
 #define DN_ADD(k) dn_acc[k] += clock64() - dn_t0
 #else
@@ -81,7 +84,7 @@ enum DenseEpi : int { DE_SIGMA = 0, DE_SWIGLU = 1, DE_NONE = 2 };
 
 struct DensePhase {
   int stage;      // ST_S1, ST_S4, ST_SH1 or ST_SH2
-  int K, tiles;   // contraction length; 256-row tiles of a unit
+  int K, tiles;   // contraction length; DN_TILE-row tiles of a unit
   int dual;       // a tile is 128 rows of the gate matrix followed by the same rows of the up matrix;
                   // epilogue SiLU(a) * b, 128 outputs per tile
   int epi;
@@ -190,7 +193,7 @@ struct Job {
   int phase;
   int T;          // token rows of the unit (0: nothing to do)
   int row0;       // first row of the unit's bucket, in its input plane and in its output
-  int ncols;      // weight rows of the job = accumulator columns: 256, or 128 for half a tile
+  int ncols;      // weight rows of the job = accumulator columns: DN_TILE, or half of it for half a tile
   int col0;       // output column of accumulator column 0
   const __nv_bfloat16* w;    // the job's part of the tile's first chunk; the next chunk is DN_TILE * DN_BK further
 };
@@ -247,7 +250,7 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
 }
 
 // ---------------------------------------------------------------- the kernel
-__global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A, int B, const __grid_constant__ DenseMaps maps) {
+__global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L, DenseArgs A, int B, const __grid_constant__ DenseMaps maps) {
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* ring = smem;  // stage s: weights at s * DN_STAGE_BYTES, activation rows DN_A_BYTES further
   uint64_t* a_full = reinterpret_cast<uint64_t*>(ring + (size_t)DN_AST * DN_STAGE_BYTES);
@@ -457,8 +460,8 @@ __global__ void __launch_bounds__(DN_THREADS, 1) k_dense(LayerDev L, DenseArgs A
 // Copies `units` matrices [rows, K] (element (r, k) of unit u at src[u * src_unit + r * rs + k * cs])
 // into the tile layout of unit u at dst + u * dst_unit.  Source row r becomes row
 // R = dst_row0 + (r / spt) * tstride + r % spt of the unit's stacked matrix (two matrices can be
-// stacked, or interleaved 128 rows at a time); tile R / 256 and chunk k / 64 start at
-// ((R / 256) * (K / 64) + k / 64) * 256 * 64 elements; inside, the core-matrix layout described at
+// stacked, or interleaved half a tile at a time); tile R / DN_TILE and chunk k / 64 start at
+// ((R / DN_TILE) * (K / 64) + k / 64) * DN_TILE * 64 elements; inside, the core-matrix layout described at
 // the top.  One thread per 16-byte piece (8 consecutive k of one row).
 __global__ void k_pack_tiles(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows, int K,
                              long long rs, long long cs, long long src_unit, long long dst_unit, int dst_row0, int spt,
@@ -510,7 +513,7 @@ struct DensePlan {
 bool dense_supported(const LayerDev& L) {
   if (L.vanilla || L.r <= 0) return false;
   if (L.wdt != DEAMOE_BF16 || L.adt != DEAMOE_BF16) return false;
-  if (L.h % 256 || L.f % 128) return false;   // 256-row tiles of [2f, h] and of [h, f]; 64-column chunks
+  if (L.h % 256 || L.f % 128) return false;   // whole tiles of [2f, h] and of [h, f]; 64-column chunks
   if (L.n_shared && (L.fs % 128)) return false;
   return true;
 }
@@ -568,8 +571,8 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   pack(w.dept_down, p->o_d, L.h, L.f, 1, L.h, (long long)fh, (long long)p->e_d, L.m, 0, NOSPLIT, 0);
   if (L.n_shared) {
     // shared expert: tile t = gate rows [128 t, 128 t + 128) followed by the same rows of up
-    pack(w.shared_gate, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 0, 128, DN_TILE);
-    pack(w.shared_up, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 128, 128, DN_TILE);
+    pack(w.shared_gate, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 0, DN_TILE / 2, DN_TILE);
+    pack(w.shared_up, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, DN_TILE / 2, DN_TILE / 2, DN_TILE);
     pack(w.shared_down, p->o_sd, L.h, L.fs, 1, L.h, 0, 0, 1, 0, NOSPLIT, 0);
   }
   cudaError_t e = cudaGetLastError();
@@ -646,7 +649,7 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
       if (!encode_rows_map(p, &maps.tm[i][b], in, in_rows, ph.K, 16 << b)) return -1;
   }
   if (n_stages == 1) std::memcpy(maps.tm[1], maps.tm[0], sizeof(maps.tm[0]));
-  k_dense<<<p.n_sm, DN_THREADS, DN_SMEM, s>>>(L, A, B, maps);
+  k_dense<<<p.n_sm * DN_CTAS_PER_SM, DN_THREADS, DN_SMEM, s>>>(L, A, B, maps);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
