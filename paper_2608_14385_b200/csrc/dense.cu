@@ -243,7 +243,7 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
     } else {
       j.ncols = DN_TILE / 2;
       j.col0 += half * (DN_TILE / 2);
-      j.w += (size_t)half * (DN_TILE / 2) * DN_BK;  // row groups 16..31 of every chunk
+      j.w += (size_t)half * (DN_TILE / 2) * DN_BK;  // the second half of the row groups of every chunk
     }
   }
   return j;
@@ -570,7 +570,7 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   pack(w.dept_up, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, L.f, NOSPLIT, 0);
   pack(w.dept_down, p->o_d, L.h, L.f, 1, L.h, (long long)fh, (long long)p->e_d, L.m, 0, NOSPLIT, 0);
   if (L.n_shared) {
-    // shared expert: tile t = gate rows [128 t, 128 t + 128) followed by the same rows of up
+    // shared expert: tile t = half a tile of gate rows followed by the same rows of up
     pack(w.shared_gate, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 0, DN_TILE / 2, DN_TILE);
     pack(w.shared_up, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, DN_TILE / 2, DN_TILE / 2, DN_TILE);
     pack(w.shared_down, p->o_sd, L.h, L.fs, 1, L.h, 0, 0, 1, 0, NOSPLIT, 0);
