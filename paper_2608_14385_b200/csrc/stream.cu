@@ -1697,7 +1697,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
     p->bytes += db;
     p->dev_dense = p->dev;
     p->dev_dense.dense = 1;
-    p->dev_dense.early = 0; p->dev_dense.sh_prefix = 0; p->dev_dense.claim_items = 0;
+    p->dev_dense.early = 0; p->dev_dense.sh_prefix = 0;  // (items of the second private stage are still claimed)
   }
   *out = p;
   *bytes = p->bytes;
