@@ -671,6 +671,22 @@ static __host__ __device__ FinishSmem finish_layout(int n, int m, int k, int B) 
   return f;
 }
 
+// Top-k + gate weights for larger batches: one warp per token over as many CTAs as it takes, instead
+// of the routing tail's one CTA ranking its tokens sixteen at a time.  Writes the layer's global
+// selection arrays; the routing tail that follows (topk_warps == 0) reads them from there.
+constexpr int TOPK_CTA_WARPS = 4;
+__global__ void __launch_bounds__(TOPK_CTA_WARPS * 32)
+k_topk_tokens(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
+  pdl_trigger();
+  pdl_wait();  // the router logits of the preceding kernel
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = (int)blockIdx.x * TOPK_CTA_WARPS + warp;
+  if (t >= B) return;
+  if (L.n <= 256) topk_one_token_regs<8>(L, t, B, kslices, lane, user_idx, user_w);
+  else if (L.n <= 512) topk_one_token_regs<16>(L, t, B, kslices, lane, user_idx, user_w);
+  else topk_one_token_regs<32>(L, t, B, kslices, lane, user_idx, user_w);
+}
+
 __global__ void __launch_bounds__(FINISH_THREADS)
 k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
@@ -707,7 +723,13 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     for (int i = tid; i < ngu + nz; i += FINISH_THREADS) (i < ngu ? L.ss_gu[i] : L.ss_z[i - ngu]) = 0.f;
   }
   const bool regs_ok = topk_in_registers(L);
-  if (warp < topk_warps) {
+  if (topk_warps == 0) {  // the selection was made by k_topk_tokens
+#pragma unroll 1
+    for (int i = tid; i < B * L.k; i += FINISH_THREADS) {
+      S.topk_idx[i] = __ldcg(L.topk_idx + i);
+      S.topk_w[i] = __ldcg(L.topk_w + i);
+    }
+  } else if (warp < topk_warps) {
     const int per_warp = (L.n * 5 + 15) & ~15;  // n fp32 logits + n flag bytes (memory path only)
     unsigned char* base = reinterpret_cast<unsigned char*>(s_dyn) + (size_t)warp * per_warp;
 #pragma unroll 1
@@ -1737,6 +1759,13 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (topk_warps > FINISH_THREADS / 32) topk_warps = FINISH_THREADS / 32;
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
+  int extra = 0;
+  if (takes_dense(p, B) && in_regs) {  // larger batches: the selection gets a grid of its own
+    launch_pdl(k_topk_tokens, dim3((B + TOPK_CTA_WARPS - 1) / TOPK_CTA_WARPS), dim3(TOPK_CTA_WARPS * 32), 0, s, L, B, ny,
+               user_idx, user_w);
+    topk_warps = 0;
+    extra = 1;
+  }
   size_t scratch = in_regs ? 0 : (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
   const size_t bs = bucket_smem_bytes(L, B) + (size_t)((L.vanilla ? L.n : L.m) + 2) * sizeof(int);  // + early_first_stage()'s scan
   if (bs > scratch) scratch = bs;
@@ -1746,7 +1775,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (smem > 200 * 1024) return -1;
   launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, dv, B, ny, topk_warps, (int)(scratch / 4),
              user_idx, user_w);
-  return cudaGetLastError() == cudaSuccess ? 2 : -1;
+  return cudaGetLastError() == cudaSuccess ? 2 + extra : -1;
 }
 
 // category order as built by category_list(), host copy
