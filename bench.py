@@ -284,7 +284,7 @@ def main():
             dist.destroy_process_group()
         return
     B = args.batch
-    # (sized for the largest batch of the sweep; from 56 tokens on AUTO takes the dense schedule)
+    # (sized for the largest batch of the sweep; from 48 tokens on AUTO takes the dense schedule)
     max_batch = max(64 if shape.name in synth.PAPER_BASELINES else (128 if shape.name == "dsv3" and not args.no_sweep else 32), B)
     w = synth.make_deamoe_weights(shape, 0, dev)
     layer = binding.Layer(shape, w, max_batch, sched)
@@ -332,7 +332,7 @@ def main():
                                 "(smaller layer of the same matrices), scaled by algorithmic bytes",
                 "kernel": "k_stream (the weight-streaming launch(es) of one step)",
                 "kernel_ms": k_ms, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg}
-        if args.schedule == "dense" or (args.schedule == "auto" and B >= 56):
+        if args.schedule == "dense" or (args.schedule == "auto" and B >= 48):
             # dense schedule: the pair of events brackets k_dense, k_stream, k_dense (ordinary launches, back to back)
             roof["kernel"] = "k_dense + k_stream + k_dense (the three weight-streaming launches of a dense step)"
             roof["traffic_note"] = ("dram read+write bytes from the ncu captures of k_stream (1.001 x algorithmic) and "

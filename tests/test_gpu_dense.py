@@ -80,7 +80,7 @@ def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
             torch.cuda.synchronize()
             for layer in (auto, fused, dense):
                 assert layer.stats()["device_status"] == 0
-            same = of if B < 56 else od
+            same = of if B < 48 else od
             assert torch.equal(oa, same)
             ok, err, bound = within_tolerance(od.cpu().numpy().astype(np.float64), of.cpu().numpy().astype(np.float64))
             assert ok, f"{err:.3e} > {bound:.3e}"
