@@ -31,8 +31,9 @@
 // between 8-row groups and 1024 bytes between neighbours along K.  The box is 16, 32 or 64 rows
 // high, whichever holds the group's rows (three tensor maps per input plane; the MMA always reads
 // 64 rows: the ones past the box are stale shared memory of the same stage and feed accumulator
-// rows nobody reads).  The rows come through the same per-SM path as the weights, and a 64-row
-// box for a 15-row bucket would take a fifth of that path.  The rows of a bucket are
+// rows nobody reads; a box of R rows puts R x 16 bytes between neighbours along K).  The rows
+// come through the same per-SM path as the weights, and a 64-row box for a 15-row bucket would
+// take a third of that path.  The rows of a bucket are
 // contiguous in every input plane (the first stage's tokens are gathered into bucket order by a
 // small kernel first); a box may run past the bucket's end, into rows that no output depends on.
 // Weights are stored at create time tile by tile and chunk by chunk in the layout the MMA reads,
@@ -54,10 +55,10 @@ namespace {
 
 constexpr int DN_AST = 4;                   // ring stages
 constexpr int DN_CTAS_PER_SM = 2;
-constexpr int DN_NMAX = 64;                 // token rows of one accumulator (the MMA's M)
+constexpr int DN_NMAX = 64;                 // token rows of one accumulator (the MMA's M) = rows of a bucket per pass
 constexpr int DN_BK = 64;                   // columns of a chunk
 constexpr int DN_TILE = 128;                // weight rows of a tile (the MMA's N)
-constexpr int DN_A_BYTES = DN_TILE * DN_BK * 2;   // 32 KB
+constexpr int DN_A_BYTES = DN_TILE * DN_BK * 2;   // 16 KB
 constexpr int DN_B_BYTES = DN_NMAX * DN_BK * 2;   // 8 KB
 constexpr int DN_STAGE_BYTES = DN_A_BYTES + DN_B_BYTES;
 constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5;
@@ -85,8 +86,8 @@ enum DenseEpi : int { DE_SIGMA = 0, DE_SWIGLU = 1, DE_NONE = 2 };
 struct DensePhase {
   int stage;      // ST_S1, ST_S4, ST_SH1 or ST_SH2
   int K, tiles;   // contraction length; DN_TILE-row tiles of a unit
-  int dual;       // a tile is 128 rows of the gate matrix followed by the same rows of the up matrix;
-                  // epilogue SiLU(a) * b, 128 outputs per tile
+  int dual;       // a tile is half a tile of gate rows followed by the same rows of the up matrix;
+                  // epilogue SiLU(a) * b, DN_TILE / 2 outputs per tile
   int epi;
   int out_stride, pad;
   const __nv_bfloat16* w;
