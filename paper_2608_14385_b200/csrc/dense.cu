@@ -199,14 +199,18 @@ struct Job {
   const __nv_bfloat16* w;    // the job's part of the tile's first chunk; the next chunk is DN_TILE * DN_BK further
 };
 
-__device__ __forceinline__ int phase_units(const LayerDev& L, const DensePhase& ph) {
-  return (ph.stage == ST_S1 || ph.stage == ST_S4) ? L.counts[CNT_ACTIVE_DEPT] : 1;
+// Units of a phase: the active departments, or, for the shared expert, the groups of DN_NMAX tokens
+// of the batch.  (A department's bucket of more than DN_NMAX rows is rare and stays one job that
+// passes over its tile once per group; the shared expert sees every token, so from 65 tokens on
+// each of its groups is a job of its own: jobs of one length deal out evenly.)
+__device__ __forceinline__ int phase_units(const LayerDev& L, const DensePhase& ph, int B) {
+  return (ph.stage == ST_S1 || ph.stage == ST_S4) ? L.counts[CNT_ACTIVE_DEPT] : (B + DN_NMAX - 1) / DN_NMAX;
 }
 
-__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int G) {
+__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int G, int B) {
   Sched s;
-  s.jobs0 = phase_units(L, A.ph[0]) * A.ph[0].tiles;
-  s.jobs = s.jobs0 + (A.nph > 1 ? phase_units(L, A.ph[1]) * A.ph[1].tiles : 0);
+  s.jobs0 = phase_units(L, A.ph[0], B) * A.ph[0].tiles;
+  s.jobs = s.jobs0 + (A.nph > 1 ? phase_units(L, A.ph[1], B) * A.ph[1].tiles : 0);
   s.full = (s.jobs / G) * G;
   s.n_idx = s.full + 2 * (s.jobs - s.full);
   return s;
@@ -232,8 +236,8 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
     j.T = L.expert_off[(id + 1) * L.g] - j.row0;
     woff = (size_t)id * ph.unit_elems;
   } else {
-    j.row0 = 0;
-    j.T = B;
+    j.row0 = u * DN_NMAX;  // shared expert: unit u = token group u
+    j.T = min(DN_NMAX, B - j.row0);
   }
   j.w = ph.w + woff + (size_t)tile * DN_TILE * ph.K;
   j.ncols = DN_TILE;
@@ -281,7 +285,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   const uint32_t tmem_base = *tmem_slot;
 
   const int G = (int)gridDim.x;
-  const Sched sc = make_sched(L, A, G);
+  const Sched sc = make_sched(L, A, G, B);
 
   if (warp == DN_WARP_TMA) {
     // ============================================================ weight chunks -> weight ring
