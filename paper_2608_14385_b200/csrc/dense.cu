@@ -139,7 +139,7 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
       ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(pol) : "memory");
 }
-// Tiled TMA load of one box of a 3-D tensor map (no multicast); x is the innermost coordinate.
+// Tiled TMA load of one box of a 3-D tensor map into this CTA only; x is the innermost coordinate.
 __device__ __forceinline__ void tensor_load_3d(void* dst, const CUtensorMap* tm, int x, int y, int z, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
