@@ -258,24 +258,47 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
   pdl_wait();  // stage outputs of the preceding kernel
   TS_MIN(L, 9);
   if (L.sh_done && blockIdx.x == 0 && threadIdx.x == 0) *L.sh_done = 0;  // nothing of this step reads it any more
-  const size_t total = (size_t)B * L.h;
+  // four consecutive columns per thread (h is a multiple of 4 in every accepted configuration)
+  const int h4 = L.h >> 2;
+  const size_t total = (size_t)B * h4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const int t = (int)(i / L.h), c = (int)(i % L.h);
-    float acc = 0.f;
+    const int t = (int)(i / h4), c4 = (int)(i % h4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int q = 0; q < L.k; ++q) {
       const int slot = L.pair_slot[t * L.k + q];
       if ((unsigned)slot >= (unsigned)(L.max_batch * L.k)) {  // consistency check: skip the access, report
         L.counts[CNT_STATUS] = DEAMOE_ERR_INTERNAL;
         continue;
       }
-      acc = fmaf(L.topk_w[t * L.k + q], L.O[(size_t)slot * L.h + c], acc);
+      const float p = L.topk_w[t * L.k + q];
+      const float4 o = __ldcg(reinterpret_cast<const float4*>(L.O + (size_t)slot * L.h) + c4);
+      acc.x = fmaf(p, o.x, acc.x); acc.y = fmaf(p, o.y, acc.y); acc.z = fmaf(p, o.z, acc.z); acc.w = fmaf(p, o.w, acc.w);
     }
-    if (L.n_shared) acc += L.Osh[i];
-    if (L.residual)
-      acc += (L.adt == DEAMOE_F32) ? reinterpret_cast<const float*>(L.tokens_raw)[i]
-                                   : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw)[i]);
-    if (L.adt == DEAMOE_F32) reinterpret_cast<float*>(out)[i] = acc;
-    else reinterpret_cast<__nv_bfloat16*>(out)[i] = __float2bfloat16_rn(acc);
+    if (L.n_shared) {
+      const float4 o = __ldcg(reinterpret_cast<const float4*>(L.Osh) + i);
+      acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+    }
+    if (L.residual) {
+      if (L.adt == DEAMOE_F32) {
+        const float4 x = reinterpret_cast<const float4*>(L.tokens_raw)[i];
+        acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+      } else {
+        const uint2 raw = reinterpret_cast<const uint2*>(L.tokens_raw)[i];
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+        acc.x += __bfloat162float(a.x); acc.y += __bfloat162float(a.y);
+        acc.z += __bfloat162float(b.x); acc.w += __bfloat162float(b.y);
+      }
+    }
+    if (L.adt == DEAMOE_F32) {
+      reinterpret_cast<float4*>(out)[i] = acc;
+    } else {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(out)[i] = pk;
+    }
   }
   TS_MAX(L, 10);
 }
@@ -329,7 +352,7 @@ int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s) {
 
 int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s) {
   (void)tokens;
-  const size_t total = (size_t)B * L.h;
+  const size_t total = (size_t)B * (L.h / 4);  // four columns per thread
   int blocks = (int)((total + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
   const cudaError_t e = launch_pdl(k_combine, dim3(blocks), dim3(256), 0, s, L, B, (const float*)L.x32, out);
