@@ -91,7 +91,7 @@ def test_paper_deepseek_v3_row_group_limited(B, rows):
 
 
 @pytest.mark.parametrize("name,B,rows", [("qwen3-paper", 16, [3, 15]), ("b7-paper", 64, [0, 40, 63]),
-                                         ("dsv2-paper", 8, [5])])
+                                         ("dsv2-paper", 8, [5]), ("kimi-k2-paper", 4, [2])])
 def test_other_table1_rows(name, B, rows):
     """Further rows of Table 1 at full size (Qwen3-235B-, Baseline-7B- and DeepSeek-V2-matched DeaMoE
     configurations): routing and lists for the whole batch, values on sampled rows, unique bytes
@@ -179,6 +179,7 @@ WIDE_ROUTERS = [
     (32, 32, 32, 0, 0),     # 1024 experts, top-32: the widest the register top-k takes
     (32, 32, 8, 3, 0),
     (40, 40, 8, 6, 0),      # 1600 experts, 40 departments: the shared-memory top-k
+    (32, 64, 8, 0, 0),      # 2048 experts: the most a layer may have
     (6, 16, 6, 4, 1),       # strict department coverage (Section 3.3, last paragraph)
     (8, 108, 10, 5, 1),     # ... on the paper's DeepSeek-V3 router
     (40, 40, 8, 6, 1),      # ... in the shared-memory top-k
