@@ -1760,7 +1760,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
   int extra = 0;
-  if (takes_dense(p, B) && in_regs) {  // larger batches: the selection gets a grid of its own
+  if ((takes_dense(p, B) || B > FINISH_THREADS / 32) && in_regs) {  // more tokens than the tail has warps: the selection gets a grid of its own
     launch_pdl(k_topk_tokens, dim3((B + TOPK_CTA_WARPS - 1) / TOPK_CTA_WARPS), dim3(TOPK_CTA_WARPS * 32), 0, s, L, B, ny,
                user_idx, user_w);
     topk_warps = 0;
