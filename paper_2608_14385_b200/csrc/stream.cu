@@ -673,9 +673,9 @@ static __host__ __device__ FinishSmem finish_layout(int n, int m, int k, int B) 
 
 // Top-k + gate weights in a grid of their own: one warp per token over as many CTAs as it takes,
 // instead of the routing tail's one CTA ranking its tokens sixteen at a time.  Used when a call has
-// more tokens than the tail has warps, in the dense schedule, and for routers of more than 512
-// experts (32 logits per lane: inside the 512-thread tail that variant is short of registers and
-// measured 4 us slower per token round).  Writes the layer's global selection arrays; the routing
+// more tokens than the tail has warps, in the dense schedule, and for routers of more than 256
+// experts (16 or 32 logits per lane: inside the 512-thread tail those variants are short of
+// registers; the widest measured 4 us slower per token round there).  Writes the layer's global selection arrays; the routing
 // tail that follows (topk_warps == 0) reads them from there.
 constexpr int TOPK_CTA_WARPS = 4;
 __global__ void __launch_bounds__(TOPK_CTA_WARPS * 32)
@@ -1763,7 +1763,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
   int extra = 0;
-  if ((takes_dense(p, B) || B > FINISH_THREADS / 32 || L.n > 512) && in_regs) {  // the selection gets a grid of its own
+  if ((takes_dense(p, B) || B > FINISH_THREADS / 32 || L.n > 256) && in_regs) {  // the selection gets a grid of its own
     launch_pdl(k_topk_tokens, dim3((B + TOPK_CTA_WARPS - 1) / TOPK_CTA_WARPS), dim3(TOPK_CTA_WARPS * 32), 0, s, L, B, ny,
                user_idx, user_w);
     topk_warps = 0;
