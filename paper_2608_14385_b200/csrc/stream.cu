@@ -473,9 +473,14 @@ static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stag
 // `s_excl` is shared-memory scratch for one int per unit (at most 2 m + 2 n + 2 of them).
 static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B, int* s_excl, bool early_done) {
   __shared__ int s_ubase[MAX_CAT + 1], s_segbase[MAX_CAT + 1], s_itembase[MAX_CAT + 1], s_wsum[32], s_carry;
-  CatInfo cats[MAX_CAT];
-  const int ncat = category_list(L, P, cats);
+  // the category list lives in shared memory: a per-thread array indexed with a run-time index would
+  // sit in local memory and give the kernel a stack frame
+  __shared__ CatInfo cats[MAX_CAT];
+  __shared__ int s_ncat;
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarp = nthr >> 5;
+  if (tid == 0) s_ncat = category_list(L, P, cats);
+  __syncthreads();
+  const int ncat = s_ncat;
   if (!early_done)  // else early_first_stage() has zeroed the counters, and the first stage may be running
 #pragma unroll 1
     for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
@@ -690,7 +695,7 @@ k_topk_tokens(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, fl
   else topk_one_token_regs<32>(L, t, B, kslices, lane, user_idx, user_w);
 }
 
-__global__ void __launch_bounds__(FINISH_THREADS)
+__global__ void __launch_bounds__(FINISH_THREADS, 1)
 k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   extern __shared__ uint32_t s_dyn[];
@@ -737,9 +742,9 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     unsigned char* base = reinterpret_cast<unsigned char*>(s_dyn) + (size_t)warp * per_warp;
 #pragma unroll 1
     for (int t = warp; t < B; t += topk_warps) {
+      // (wider routers that fit the register variants are ranked by k_topk_tokens: their 16 and 32
+      // logits per lane would set this kernel's register budget and give it a stack frame)
       if (regs_ok && L.n <= 256) topk_one_token_regs<8>(S, t, B, kslices, lane, user_idx, user_w);
-      else if (regs_ok && L.n <= 512) topk_one_token_regs<16>(S, t, B, kslices, lane, user_idx, user_w);
-      else if (regs_ok) topk_one_token_regs<32>(S, t, B, kslices, lane, user_idx, user_w);
       else topk_one_token(S, t, B, kslices, reinterpret_cast<float*>(base), base + (size_t)L.n * 4, lane, user_idx, user_w);
     }
   }
@@ -969,9 +974,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     // The shared expert (Eq. (1)) does not depend on the routing: in the fused schedule its items
     // are generated here, from the batch size alone, and stream while the routing kernel that
     // precedes this grid is still running.
+    int first_cta = 0;  // the CTA that takes the next dealt item
     if (P.sh_prefix && cat < 0) {
       Seg* stage_seg = reinterpret_cast<Seg*>(seg_stage);
-      int first_cta = 0;  // the CTA that takes the stage's first item
       for (int st = ST_SH1; ok && st <= PREFIX_LAST_STAGE; ++st) {
         const int ips = P.st[st].items_per_seg;
         const int n_items = groups_of(B, P.st[st].tg) * ips;
@@ -998,7 +1003,10 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     // longest, so the rest of the routing (expert lists, the other stages' records) hides behind
     // it.  Phase 2, after the routing kernel has completed: everything else.
     int ncat = 0, item_end = 0;
-    int cur_i = (int)blockIdx.x;  // item i of the launch's range goes to CTA i mod grid
+    // Item i of the launch's range goes to CTA (first_cta + i) mod grid: the dealing continues behind
+    // the CTAs that took the shared expert's prefix items (equal in size to the first stage's), so
+    // those do not start the routed stages one item behind the others.
+    int cur_i = ((int)blockIdx.x - first_cta + G) % G;
     auto seg_of = [&](int k, int item, int& it) -> const Seg* {
       const int ib = cat_tab[4 * k + 0], sb = cat_tab[4 * k + 1], ips = cat_tab[4 * k + 2];
       it = (item - ib) % ips;
