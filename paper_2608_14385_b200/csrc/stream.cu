@@ -630,6 +630,7 @@ static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, 
   }
   if (tid == 0) scr[A] = carry;
   __syncthreads();
+  TS_MIN(L, 18);
 #pragma unroll 1
   for (int a = tid; a < A; a += nthr) {
     const int id = unit_id(L, kind, a);
@@ -637,12 +638,16 @@ static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, 
 #pragma unroll 1
     for (int gi = 0; gi < gc; ++gi) write_seg(L, P, stage, id, gi, B, scr[a] + gi, (scr[a] + gi) * ips);
   }
+  TS_MIN(L, 19);
   __threadfence();  // every thread's records and zeroed counters, before the flag
   __syncthreads();
+  TS_MIN(L, 20);
   if (tid == 0) {
-    P.sync[SY_DEP + P.early_items] = (carry <= P.max_segs) ? carry * ips : 0;
-    __threadfence();
-    st_release(P.sync + SY_DEP + P.early_flag, 1);  // cleared again by the next step's router kernel
+    // the flag carries the item count (+ 1, so that it is never 0), which saves the streaming kernel
+    // a dependent load; it is cleared again by the next step's router kernel
+    const int items = (carry <= P.max_segs) ? carry * ips : 0;
+    P.sync[SY_DEP + P.early_items] = items;
+    st_release(P.sync + SY_DEP + P.early_flag, items + 1);
   }
 }
 
@@ -754,6 +759,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 12);
 #endif
   bucket_departments(S, B, s_dyn, FINISH_THREADS);
+  TS_MIN(L, 17);
   int* early_scr = reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B);  // after the masks and offsets
   if (P.early && P.early_stage == ST_S1) early_first_stage<ST_S1>(S, P, B, early_scr);
   bucket_experts(S, B, s_dyn, FINISH_THREADS);
@@ -1089,11 +1095,12 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         const int32_t* flag = P.sync + SY_DEP + P.early_flag;
         unsigned spins = 0;
         bool seen = true;
-        while (ld_acquire(flag) != 1) {
+        int fv;
+        while ((fv = ld_acquire(flag)) == 0) {
           __nanosleep(64);
           if (++spins > SPIN_LIMIT / 16 || *abort_flag) { seen = false; break; }
         }
-        n1 = seen ? __ldcg(P.sync + SY_DEP + P.early_items) : -1;
+        n1 = seen ? fv - 1 : -1;  // the flag is the first stage's item count + 1
       }
       n1 = __shfl_sync(0xffffffffu, n1, 0);
       if (n1 < 0) {
