@@ -564,19 +564,33 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
   }
   __syncthreads();
   TS_MIN(L, 14);
-  // pass 2: every unit's records
+  // pass 2: every unit's records.  A warp stays with one category (warp w takes category w mod the
+  // number of categories, and with the other warps of that category every unit of it): the record
+  // code differs by stage, and a warp whose lanes held units of different stages would run the
+  // stages' code one after the other, from a cold instruction cache.
+  const int first_c = (early_done && ncat > 1) ? 1 : 0;  // category 0 was written by early_first_stage()
+  const int nc = ncat - first_c;
 #pragma unroll 1
-  for (int flat = tid; flat < total; flat += nthr) {
-    const int c = category_of(flat);
-    if (early_done && c == 0) continue;  // written, with the same numbering, by early_first_stage()
-    const int stage = cats[c].stage;
-    const int id = unit_id(L, cats[c].unit_kind, flat - s_ubase[c]);
-    const int gc = groups_of(unit_tokens(L, stage, id, B), P.st[stage].tg);
-    const int ips = P.st[stage].items_per_seg;
+  for (int c0 = warp % (nc > 0 ? nc : 1); c0 < nc; c0 += nwarp) {  // (one pass unless there are fewer warps than categories)
+    const int c = first_c + c0;
+    const bool shared = nwarp >= nc;  // several warps share a category
+    const int rank = shared ? warp / nc : 0;
+    const int per_c = shared ? (nwarp - c0 + nc - 1) / nc : 1;  // this warp's place among the category's warps
+    if (!(early_done && c == 0)) {
+      const int stage = cats[c].stage;
+      const int nu = s_ubase[c + 1] - s_ubase[c];
+      const int ips = P.st[stage].items_per_seg;
 #pragma unroll 1
-    for (int gi = 0; gi < gc; ++gi) {
-      const int si = s_excl[flat] + gi;
-      write_seg(L, P, stage, id, gi, B, si, s_itembase[c] + (si - s_segbase[c]) * ips);
+      for (int u = rank * 32 + lane; u < nu; u += per_c * 32) {
+        const int flat = s_ubase[c] + u;
+        const int id = unit_id(L, cats[c].unit_kind, u);
+        const int gc = groups_of(unit_tokens(L, stage, id, B), P.st[stage].tg);
+#pragma unroll 1
+        for (int gi = 0; gi < gc; ++gi) {
+          const int si = s_excl[flat] + gi;
+          write_seg(L, P, stage, id, gi, B, si, s_itembase[c] + (si - s_segbase[c]) * ips);
+        }
+      }
     }
   }
 }
