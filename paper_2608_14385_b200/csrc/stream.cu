@@ -52,6 +52,7 @@ constexpr int MAX_CAT_INTS_PAD = 8;             // cat_tab: 4 ints for each of 8
 #define PREFIX_LAST_STAGE ST_SH1  // the shared expert's second stage waits for all of the first: it runs from the list
 #endif
 constexpr int CLAIM_MIN_PER_CTA = 16;            // lists with fewer items per CTA are dealt out, not claimed
+constexpr int PREFETCH_BYTES = 512 * 1024;       // per CTA: at most this much of its likely first routed item goes to L2 during the routing
 constexpr int CLAIM_AHEAD = 4;                   // unfinished items a CTA may hold while it claims from the last category
 constexpr int NRED = 2;                          // reduction buffers between consumers and epilogue warp
 constexpr int SLOT_BYTES = 32 * 1024;
@@ -1104,6 +1105,29 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     };
 
     if (P.early && cat < 0 && ok) {
+      // While the routing is still in progress HBM is nearly idle.  When almost every department
+      // will be active anyway (the host decides from the batch size), bring the weights of the
+      // item this CTA gets if the first departments are active into L2: whichever CTA ends up
+      // with an item of those departments then streams it from L2.  A wrong guess only costs
+      // reads nobody was waiting for.
+      if ((check_deps & 4) && lane == 0 && P.early_stage == ST_S1) {
+        const StageCfg& sc = P.st[ST_S1];
+        const int x = ((int)blockIdx.x - first_cta + G) % G;
+        const int dept = x / sc.items_per_seg, it = x - dept * sc.items_per_seg;
+        if (dept < L.m) {
+          const int tile0 = it * sc.q;
+          const int ntile = min(sc.q, sc.n_tiles - tile0);
+          const size_t tile_bytes = (size_t)(sc.C / 16) * 512;
+          const char* w = reinterpret_cast<const char*>(sc.w0 + (size_t)dept * sc.unit_elems) + (size_t)tile0 * tile_bytes;
+          size_t bytes = (size_t)ntile * tile_bytes;
+          if (bytes > (size_t)PREFETCH_BYTES) bytes = PREFETCH_BYTES;
+#pragma unroll 1
+          for (size_t o = 0; o < bytes; o += 32768) {
+            const unsigned chunk = (unsigned)((bytes - o < 32768) ? (bytes - o) : 32768);
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(w + o), "r"(chunk) : "memory");
+          }
+        }
+      }
       int n1 = 0;
       if (lane == 0) {
         const int32_t* flag = P.sync + SY_DEP + P.early_flag;
@@ -1861,7 +1885,15 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | dbgflag);
+    // expected share of active departments under uniform routing: prefetch when it is at least 0.9
+    int pf = 0;
+    if (!L.vanilla) {
+      const int c = (L.k_dept > 0 && L.k_dept < L.m) ? L.k_dept : (L.k < L.m ? L.k : L.m);
+      double miss = 1.0;
+      for (int t = 0; t < B; ++t) miss *= 1.0 - (double)c / L.m;
+      pf = (miss <= 0.1) ? 4 : 0;
+    }
+    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | pf | dbgflag);
     ++launches;
   } else {
     for (int c = 0; c < ncat; ++c) {
