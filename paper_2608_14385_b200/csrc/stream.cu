@@ -1885,13 +1885,14 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
 #ifdef DEAMOE_TRACE
     if (const char* ev = getenv("DEAMOE_DBG")) dbgflag = atoi(ev) << 8;
 #endif
-    // expected share of active departments under uniform routing: prefetch when it is at least 0.9
+    // expected share of active departments under uniform routing: prefetch when it is at least 0.65
+    // (measured on the DeepSeek-V3 shape: a gain from 4 tokens on, share 0.68; a loss at 2, share 0.44)
     int pf = 0;
     if (!L.vanilla) {
       const int c = (L.k_dept > 0 && L.k_dept < L.m) ? L.k_dept : (L.k < L.m ? L.k : L.m);
       double miss = 1.0;
       for (int t = 0; t < B; ++t) miss *= 1.0 - (double)c / L.m;
-      pf = (miss <= 0.1) ? 4 : 0;
+      pf = (miss <= 0.35) ? 4 : 0;
     }
     launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | pf | dbgflag);
     ++launches;
