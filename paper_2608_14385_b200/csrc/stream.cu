@@ -1110,21 +1110,25 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       // item this CTA gets if the first departments are active into L2: whichever CTA ends up
       // with an item of those departments then streams it from L2.  A wrong guess only costs
       // reads nobody was waiting for.
-      if ((check_deps & 4) && lane == 0 && P.early_stage == ST_S1) {
-        const StageCfg& sc = P.st[ST_S1];
+      // (The vanilla layer does the same with its experts when nearly all of them will be active.)
+      if ((check_deps & 4) && lane == 0) {
+        const StageCfg& sc = P.st[P.early_stage];
         const int x = ((int)blockIdx.x - first_cta + G) % G;
-        const int dept = x / sc.items_per_seg, it = x - dept * sc.items_per_seg;
-        if (dept < L.m) {
-          const int tile0 = it * sc.q;
-          const int ntile = min(sc.q, sc.n_tiles - tile0);
+        const int unit = x / sc.items_per_seg, it = x - unit * sc.items_per_seg;
+        if (unit < (L.vanilla ? L.n : L.m)) {
+          const int tile0 = sc.paired ? it : it * sc.q;
+          const int ntile = sc.paired ? 1 : min(sc.q, sc.n_tiles - tile0);
           const size_t tile_bytes = (size_t)(sc.C / 16) * 512;
-          const char* w = reinterpret_cast<const char*>(sc.w0 + (size_t)dept * sc.unit_elems) + (size_t)tile0 * tile_bytes;
+          const size_t off = (size_t)unit * sc.unit_elems * 2 + (size_t)tile0 * tile_bytes;
           size_t bytes = (size_t)ntile * tile_bytes;
-          if (bytes > (size_t)PREFETCH_BYTES) bytes = PREFETCH_BYTES;
+          const size_t cap = sc.paired ? PREFETCH_BYTES / 2 : PREFETCH_BYTES;  // a paired item has a tile of each matrix
+          if (bytes > cap) bytes = cap;
 #pragma unroll 1
           for (size_t o = 0; o < bytes; o += 32768) {
             const unsigned chunk = (unsigned)((bytes - o < 32768) ? (bytes - o) : 32768);
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(w + o), "r"(chunk) : "memory");
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(sc.w0) + off + o), "r"(chunk) : "memory");
+            if (sc.paired)
+              asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(sc.w1) + off + o), "r"(chunk) : "memory");
           }
         }
       }
@@ -1888,10 +1892,11 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
     // expected share of active departments under uniform routing: prefetch when it is at least 0.65
     // (measured on the DeepSeek-V3 shape: a gain from 4 tokens on, share 0.68; a loss at 2, share 0.44)
     int pf = 0;
-    if (!L.vanilla) {
-      const int c = (L.k_dept > 0 && L.k_dept < L.m) ? L.k_dept : (L.k < L.m ? L.k : L.m);
+    {
+      const int units = L.vanilla ? L.n : L.m;  // the first stage's units: experts (vanilla) or departments
+      const int c = L.vanilla ? L.k : ((L.k_dept > 0 && L.k_dept < L.m) ? L.k_dept : (L.k < L.m ? L.k : L.m));
       double miss = 1.0;
-      for (int t = 0; t < B; ++t) miss *= 1.0 - (double)c / L.m;
+      for (int t = 0; t < B; ++t) miss *= 1.0 - (double)c / units;
       pf = (miss <= 0.35) ? 4 : 0;
     }
     launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev, B, -1, 1 | pf | dbgflag);
