@@ -41,7 +41,8 @@ def test_dense_schedule_wide_layer(B):
     run_case(DENSE_WIDE, B, seed=12, schedule=binding.SCHED_DENSE, weights=_scaled(DENSE_WIDE, 12, scale=6.0))
 
 
-@pytest.mark.parametrize("variant", ["no_shared", "sigma_none", "gelu", "rmsnorm", "group_limited", "residual"])
+@pytest.mark.parametrize("variant", ["no_shared", "sigma_none", "gelu", "rmsnorm", "group_limited", "strict_rmsnorm",
+                                     "residual"])
 def test_dense_schedule_variants(variant):
     shape = {
         "no_shared": DENSE_SMALL.with_(n_shared=0, shared_ffn=0),
@@ -49,6 +50,7 @@ def test_dense_schedule_variants(variant):
         "gelu": DENSE_SMALL.with_(sigma=2),
         "rmsnorm": DENSE_SMALL.with_(sigma=3),
         "group_limited": DENSE_SMALL.with_(n_dept=4, top_k=4, k_dept=2),
+        "strict_rmsnorm": DENSE_SMALL.with_(n_dept=6, experts_per_dept=6, top_k=4, k_dept=4, strict_dept=1, sigma=3),
         "residual": DENSE_SMALL.with_(residual=1),
     }[variant]
     run_case(shape, 50, seed=13, schedule=binding.SCHED_DENSE, weights=_scaled(shape, 13))
@@ -65,7 +67,7 @@ def test_dense_schedule_is_refused_for_layers_it_cannot_run():
 
 
 def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
-    """One AUTO layer sized for 128 tokens: 16 tokens take the streaming schedule, 64 the dense one;
+    """One AUTO layer sized for 128 tokens: up to 47 tokens take the streaming schedule, 48 and more the dense one;
     each agrees with a layer fixed to that schedule bit for bit, and the two schedules agree within
     the tolerance (they round intermediates alike but sum in different orders)."""
     shape = DENSE_WIDE
@@ -74,7 +76,7 @@ def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
     fused = binding.Layer(shape, w, 128, binding.SCHED_FUSED)
     dense = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
     try:
-        for B in (16, 64, 128):
+        for B in (16, 47, 48, 64, 128):
             x = synth.make_tokens(shape, B, 14 + B, torch.device("cuda:0"))
             oa, of, od = auto.forward(x).float(), fused.forward(x).float(), dense.forward(x).float()
             torch.cuda.synchronize()
