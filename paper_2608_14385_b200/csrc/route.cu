@@ -42,7 +42,8 @@ k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float*
   // dependents, so a streaming kernel can never see the value of the step before.
   if (step_flag && blockIdx.x == 0 && blockIdx.y == 0) {
     if (threadIdx.x == 0) {
-      *step_flag = 0;
+      step_flag[0] = 0;
+      step_flag[2] = 0;  // two words further: the flag that the rest of the work list exists
       __threadfence();
     }
     __syncthreads();

@@ -127,7 +127,8 @@ struct StreamDev {
   int claim_items;              // fused schedule: the items of the list are claimed, not dealt
   int dense;                    // dense schedule: the list holds the private stages only (the rest runs on tcgen05 kernels)
   int early_stage;              // the stage handed over early (ST_S1 or ST_V1)
-  int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): step number, item count
+  int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): flag, item count;
+                                // early_flag + 2: flag that the rest of the work list exists
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
   // activations between stages, bf16 planes ([rows, width] each)
   __nv_bfloat16 *xh, *xl;      // tokens split (fp32 activations only; bf16 tokens are read in place)
@@ -745,6 +746,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 11);
 #endif
   for (int i = tid; i < CNT_COUNT; i += FINISH_THREADS) S.counts[i] = 0;
+  // The status word of the step starts at "ok" here; the streaming kernel may report into the
+  // global word while this kernel is still running, so the publication at the end only ever
+  // writes an error of this kernel's own into it.
+  if (tid == 0) L.counts[CNT_STATUS] = 0;
   if (L.sigma == DEAMOE_SIGMA_RMSNORM) {  // sums of squares of this step's G, U and Z vectors
     const int ngu = 2 * B * (L.k < L.m ? L.k : L.m), nz = B * L.k;
 #pragma unroll 1
@@ -785,12 +790,20 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 13);
 #endif
   worklist_block(S, P, B, reinterpret_cast<int*>(s_dyn), P.early != 0);
+  if (P.early) {
+    // the rest of the work list is complete: tell the streaming kernel now rather than through this
+    // kernel's completion, which comes only after the routing state has been published (on a small
+    // layer the streaming kernel has finished the first stage by then and would wait)
+    __threadfence();  // every thread's records, before the flag
+    __syncthreads();
+    if (tid == 0) st_release(P.sync + SY_DEP + P.early_flag + 2, 1);  // cleared again by the next step's router kernel
+  }
   __syncthreads();
   TS_MIN(L, 15);
   // publish the routing state: every array is a run of 32-bit words in the shared-memory copy.
   // One rolled loop over a small table, so that this once-per-step code stays short.
-  __shared__ uint32_t* s_dst[12];
-  __shared__ int s_src[12], s_cnt[12];
+  __shared__ uint32_t* s_dst[13];
+  __shared__ int s_src[13], s_cnt[13];
   if (tid == 0) {
     const int pk = B * L.k;
     int e = 0;
@@ -806,11 +819,13 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     add(L.active_dept, fl.active_dept, L.m);
     add(L.active_expert, fl.active_expert, L.n);
     add(L.dept_mask, fl.dept_mask, 2 * ((L.m + 63) / 64));
-    add(L.counts, fl.counts, CNT_COUNT);
+    add(L.counts, fl.counts, CNT_STATUS);                                              // counts below the status word
+    add(L.counts + CNT_STATUS + 1, fl.counts + CNT_STATUS + 1, CNT_COUNT - CNT_STATUS - 1);  // and above it
+    if (S.counts[CNT_STATUS] != 0) L.counts[CNT_STATUS] = S.counts[CNT_STATUS];
   }
   __syncthreads();
 #pragma unroll 1
-  for (int e = 0; e < 12; ++e) {
+  for (int e = 0; e < 13; ++e) {
     uint32_t* dst = s_dst[e];
     const uint32_t* src = state + s_src[e];
     const int cnt = s_cnt[e];
@@ -1157,13 +1172,29 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       }
     }
 
-    pdl_wait();  // the rest of the work list is complete when the routing kernel is
-    cat_tab[lane] = sy[SY_CAT + lane];  // 4 * MAX_CAT == 32 entries
+    // The rest of the work list is complete when the routing kernel says so (fused schedule of a
+    // layer with the early hand-over: a second flag) or when it has completed.
+    bool waited = false;  // for the routing kernel's completion
+    if (P.early && cat < 0) {
+      if (lane == 0) {
+        const int32_t* flag = P.sync + SY_DEP + P.early_flag + 2;
+        unsigned spins = 0;
+        while (ld_acquire(flag) == 0) {
+          __nanosleep(64);
+          if (++spins > SPIN_LIMIT / 16 || *abort_flag) { ok = false; break; }
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    } else {
+      pdl_wait();
+      waited = true;
+    }
+    cat_tab[lane] = __ldcg(sy + SY_CAT + lane);  // 4 * MAX_CAT == 32 entries
     __syncwarp();
     // item range of this launch: one category (staged) or everything (fused)
-    ncat = sy[SY_NCAT];
+    ncat = __ldcg(sy + SY_NCAT);
     if (cat >= 0) cur_i = cat_tab[4 * cat] + (int)blockIdx.x;
-    item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : sy[SY_NITEMS];
+    item_end = (cat >= 0) ? cat_tab[4 * (cat + 1)] : __ldcg(sy + SY_NITEMS);
     if (*abort_flag && lane == 0) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;  // set before the routing kernel reset it
     if (cat < 0 && P.claim_items && ncat >= 2 && item_end >= CLAIM_MIN_PER_CTA * G) claim_base = cat_tab[4];
     if (ok) walk();
@@ -1179,6 +1210,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       reinterpret_cast<int*>(descs + (size_t)e * DESC_BYTES + DESC_TAIL)[0] = 1;
       mbar_arrive(&dq_full[e]);
     }
+    // This grid must not complete before the routing kernel has: the combine kernel behind it
+    // reads the routing state that kernel publishes last.
+    if (!waited) pdl_wait();
     return;
   }
 
