@@ -935,16 +935,47 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     // memory latency of the bookkeeping is paid here, off the streaming path.  It is the only
     // warp that reads what the routing kernel wrote, so it alone waits for that kernel.
 #ifdef DEAMOE_TRACE
-    long long ptr_q = 0;
+    long long ptr_q = 0, ptr_dep = 0;
 #endif
     const int G = (int)gridDim.x;
     int e = 0;
     uint32_t eph = 0;
     bool ok = true;
     // Queue the item `it` of the segment record held as one int4 per lane (lane l < SEG_VEC holds
-    // bytes [16 l, 16 l + 16)).  The planner does not wait for the item's inputs: the issue warp
-    // starts the item's weights at once and holds back only its activation rows.
+    // bytes [16 l, 16 l + 16)).  The item is queued before its inputs exist: the issue warp
+    // starts the item's weights at once and holds back only its activation rows, until this warp
+    // has seen the item's dependency counter at its target and says so in the descriptor.  The
+    // poll is done here because an acquire load next to the SM's bulk copies takes microseconds
+    // to return, during which the issue warp would not refill the ring.  The next item is queued
+    // only after that: the ring holds less than one item's weights beyond the one that waits, and
+    // a CTA that claims its items should not hold more of them while it waits (queueing one item
+    // beyond the awaited one was measured 1-3 % slower at 16 and 32 tokens).
     int queued = 0;  // items this planner has queued
+    int dep_seen = -1;  // dependency counter last seen at its target
+    // wait for a queued item's inputs, then release its activation rows (`word` of its descriptor)
+    auto await_inputs = [&](volatile int* word, int dep_idx, int dep_target) -> bool {
+#ifdef DEAMOE_TRACE
+      const long long td0 = clock64();
+#endif
+      bool seen = true;
+      if (lane == 0) {
+        unsigned spins = 0;
+        while (ld_acquire(P.sync + SY_DEP + dep_idx) < dep_target) {
+          __nanosleep(32);
+          if (++spins > SPIN_LIMIT / 16 || *abort_flag) { seen = false; break; }
+        }
+        if (seen) {
+          __threadfence_block();  // what the acquire made visible, before the word the issue warp polls
+          *word = 1;
+        }
+      }
+      seen = __shfl_sync(0xffffffffu, (int)seen, 0) != 0;
+      dep_seen = dep_idx;
+#ifdef DEAMOE_TRACE
+      ptr_dep += clock64() - td0;
+#endif
+      return seen;
+    };
     auto emit = [&](const int4 v, const int it) -> bool {
 #ifdef DEAMOE_TRACE
       const long long tpq0 = clock64();
@@ -977,11 +1008,13 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       const int tile0 = paired ? it : it * sg->q;
       const int q_eff = paired ? 2 : min(sg->q, sg->n_tiles - tile0);
       const int nrows = sg->planes * nB * T;
+      const int dep_idx = sg->dep_idx, dep_target = sg->dep_target;
+      const bool inputs_exist = !(check_deps & 1) || dep_idx < 0 || dep_idx == dep_seen;
       if (lane == 31) {
         int* tail = reinterpret_cast<int*>(ent + DESC_TAIL);
         tail[0] = 0;      // kind: work
         tail[1] = tile0;
-        tail[2] = 0;
+        tail[2] = inputs_exist ? 1 : 0;  // set below otherwise
         tail[3] = q_eff;
         tail[4] = nrows;
       }
@@ -1002,9 +1035,10 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&dq_full[e]);
+      const bool seen = inputs_exist || await_inputs(reinterpret_cast<volatile int*>(ent + DESC_TAIL) + 2, dep_idx, dep_target);
       if (++e == DESC_DEPTH) { e = 0; eph ^= 1u; }
       ++queued;
-      return true;
+      return seen;
     };
 
     // The shared expert (Eq. (1)) does not depend on the routing: in the fused schedule its items
@@ -1201,6 +1235,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
 #ifdef DEAMOE_TRACE
     if (lane == 0 && P.trace) {
       P.trace[(size_t)blockIdx.x * TR_SLOTS + 15] = ptr_q;
+      P.trace[(size_t)blockIdx.x * TR_SLOTS + 7] = ptr_dep;
     }
 #endif
     if (!ok && lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
@@ -1235,10 +1270,11 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     bool w_loaded = false, end_seen = false;
     const __nv_bfloat16* wsrc_w = nullptr;
     // activation cursor
-    int e_a = 0, ca = 0, ch_a = 0, nch_a = 0, kc0_a = 0, C_a = 0, qeff_a = 0, nrows_a = 0, dep_idx_a = -1, dep_tgt_a = 0;
+    int e_a = 0, ca = 0, ch_a = 0, nch_a = 0, kc0_a = 0, C_a = 0, qeff_a = 0, nrows_a = 0, dep_idx_a = -1;
     bool a_loaded = false, a_ready = false;
+    const volatile int* ready_a = nullptr;
     const __nv_bfloat16* asrc_a[2] = {nullptr, nullptr};
-    int dep_ok = -1;  // dependency counter last seen at its target
+    int dep_ok = -1;  // dependency counter behind whose completion this warp has fenced
     unsigned idle = 0;
     bool ok = true;
 #ifdef DEAMOE_TRACE
@@ -1308,7 +1344,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
           const int* tail = reinterpret_cast<const int*>(ent + DESC_TAIL);
           qeff_a = tail[3]; nrows_a = tail[4];
           kc0_a = sg->kc; C_a = sg->C;
-          dep_idx_a = sg->dep_idx; dep_tgt_a = sg->dep_target;
+          dep_idx_a = sg->dep_idx;
 #pragma unroll
           for (int u = 0; u < 2; ++u)
             asrc_a[u] = (lane + 32 * u < nrows_a)
@@ -1317,6 +1353,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
           ch_a = 0;
           a_loaded = true;
           a_ready = !(check_deps & 1) || dep_idx_a < 0 || dep_idx_a == dep_ok;
+          ready_a = reinterpret_cast<const volatile int*>(tail + 2);
 #ifdef DEAMOE_TRACE
           if (lane == 0 && !routed_seen && sg->stage != ST_SH1 && sg->stage != ST_SH2 && L.ts) {
             routed_seen = true;
@@ -1329,8 +1366,10 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
 #ifdef DEAMOE_TRACE
           const long long td0 = clock64();
 #endif
-          const int seen = __shfl_sync(0xffffffffu, (lane == 0) ? ld_acquire(P.sync + SY_DEP + dep_idx_a) : 0, 0);
-          if (seen >= dep_tgt_a) {
+          // the planner warp polls the counter and sets this word of the descriptor
+          const int seen = __shfl_sync(0xffffffffu, (lane == 0) ? *ready_a : 0, 0);
+          if (seen) {
+            __threadfence_block();
             dep_ok = dep_idx_a;
             fence_proxy_async();  // the rows were written through the generic proxy; the copies read through the async proxy
             a_ready = true;
