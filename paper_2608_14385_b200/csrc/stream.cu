@@ -1256,9 +1256,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     // Two cursors walk the CTA's chunk stream.  The WEIGHT cursor runs ahead: weights depend on
     // nothing, so a chunk's header and weight tiles are issued as soon as a ring slot is free,
     // also while the item's inputs do not exist yet.  The ACTIVATION cursor follows: the (tiny)
-    // activation rows of a chunk are copied once the dependency counter of its item has reached
-    // its target (one acquire load per poll; then a proxy fence, because the rows were written
-    // with ordinary stores by other CTAs).  So at a stage boundary the HBM pipe keeps running and
+    // activation rows of a chunk are copied once the planner warp has seen the dependency counter
+    // of its item at its target and set the descriptor's word (then a proxy fence, because the
+    // rows were written with ordinary stores by other CTAs).  So at a stage boundary the HBM pipe keeps running and
     // a waiting item costs only the latency of its activation rows, not of its weights.
     // Issuing a chunk's copies keeps the warp busy for 600-1000 cycles (about 270 for a bulk-copy
     // instruction plus 55 for every further lane that takes part).
