@@ -24,7 +24,10 @@
  *   - ties in TopK go to the lowest expert index; the order of S(x) is
  *     (logit descending, index ascending);
  *   - p = route_scale * softmax over the selected logits (norm_topk = 1) or
- *     over all n logits without renormalisation (norm_topk = 0);
+ *     over all n logits without renormalisation (norm_topk = 0); norm_topk = 2
+ *     is a variant the paper does not have (Section 3.1 only says "softmax
+ *     normalization and scaling"): p_i = route_scale * s_i / sum of s over the
+ *     selection, s = 1 / (1 + exp(-logit)), the selection still by raw logit;
  *   - k_dept > 0 selects group-limited routing: department score = the largest
  *     logit in the department, the k_dept best departments (ties to the lowest
  *     department index) survive, TopK runs over their experts only;
@@ -309,6 +312,13 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
       }
     }
     for (int q = 0; q < k; ++q) topk_idx[(size_t)t * k + q] = key[q].i;
+    if (c->norm_topk == 2) { /* sigmoid scores, normalised over the selection */
+      double den = 0.0;
+      for (int q = 0; q < k; ++q) den += 1.0 / (1.0 + exp(-key[q].v));
+      for (int q = 0; q < k; ++q)
+        topk_w[(size_t)t * k + q] = c->route_scale * (1.0 / (1.0 + exp(-key[q].v))) / den;
+      continue;
+    }
     /* softmax (max-subtracted) over the selection, or over all n logits */
     double mx = key[0].v, den = 0.0;
     if (c->norm_topk) {

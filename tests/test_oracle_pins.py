@@ -85,6 +85,33 @@ def test_gate_weights_are_renormalised_full_softmax():
         np.testing.assert_allclose(got0["w"][t], full[t, got0["idx"][t]], rtol=1e-12)
 
 
+def test_sigmoid_gate_variant_against_the_library_routine_and_its_limits():
+    """norm_topk = 2 (a variant the paper does not have): the selection is unchanged, the weights
+    are the logistic function of the selected logits (scipy's routine) normalised over the
+    selection; they sum to route_scale, are ordered like the logits, and for very negative logits
+    (where the logistic function tends to exp) they tend to the softmax weights."""
+    from scipy.special import expit
+    shape = SMALL.with_(route_scale=2.5, norm_topk=2)
+    router = synth.normal((12, 48), 0.3, 1, "r").numpy()
+    tokens = synth.to_numpy(synth.make_tokens(shape, 5, 1))
+    got = ref.route(oracle_cfg(shape), router, tokens, want_logits=True)
+    soft = ref.route(oracle_cfg(shape.with_(norm_topk=1)), router, tokens)
+    assert (got["idx"] == soft["idx"]).all()
+    for t in range(5):
+        s = expit(got["logits"][t, got["idx"][t]])
+        np.testing.assert_allclose(got["w"][t], 2.5 * s / s.sum(), rtol=1e-12)
+        assert abs(got["w"][t].sum() - 2.5) < 1e-12
+        assert (np.diff(got["w"][t]) <= 0).all()  # selection order is logit descending
+        assert not np.allclose(got["w"][t], soft["w"][t], rtol=1e-3)
+    # shift every logit by -40 through one extra input column: logistic(l) -> exp(l) (1 - O(e^-40))
+    router2 = np.concatenate([router, np.full((12, 1), -40.0, np.float32)], axis=1)
+    tokens2 = np.concatenate([synth.normal((5, 48), 1.0, 2, "x").numpy(), np.ones((5, 1), np.float32)], axis=1)
+    shape2 = shape.with_(hidden=49, act_dtype=0)
+    far = ref.route(oracle_cfg(shape2), router2, tokens2)
+    far_soft = ref.route(oracle_cfg(shape2.with_(norm_topk=1)), router2, tokens2)
+    np.testing.assert_allclose(far["w"], far_soft["w"], rtol=1e-12)
+
+
 def test_group_limited_routing_bruteforce():
     """k_dept cap: the selection is the flat top-k restricted to the k_dept departments with the
     largest best logit, so it never spans more than k_dept departments; k_dept = m changes nothing."""
