@@ -89,7 +89,10 @@ typedef struct {
   int32_t n_shared;         /* 0 or 1 always-on shared SwiGLU expert (Eq. (1), weight 1) */
   int32_t shared_ffn;       /* its intermediate size */
   int32_t sigma;            /* deamoe_sigma_t */
-  int32_t norm_topk;        /* 1: p = softmax over the k selected logits; 0: softmax over all n */
+  int32_t norm_topk;        /* 1: p = softmax over the k selected logits; 0: softmax over all n, not
+                               renormalised; 2 (a variant the paper does not have): logistic
+                               function of the k selected logits divided by their sum.  The
+                               selection is by raw logit (Eq. (2)) in every case. */
   int32_t weight_dtype;     /* deamoe_dtype_t of department / private / shared matrices */
   int32_t act_dtype;        /* deamoe_dtype_t of tokens and out */
   int32_t residual;         /* 1: out = tokens + layer(tokens) */

@@ -64,6 +64,7 @@ deamoe_status_t check_config(const deamoe_config_t* c, const deamoe_weights_t* w
   if (c->weight_dtype != DEAMOE_F32 && c->weight_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
   if (c->act_dtype != DEAMOE_F32 && c->act_dtype != DEAMOE_BF16) return DEAMOE_ERR_INVALID_ARG;
   if (c->sigma < DEAMOE_SIGMA_NONE || c->sigma > DEAMOE_SIGMA_RMSNORM) return DEAMOE_ERR_INVALID_ARG;
+  if (c->norm_topk < 0 || c->norm_topk > 2) return DEAMOE_ERR_INVALID_ARG;
   if (!vanilla && c->sigma == DEAMOE_SIGMA_RMSNORM && c->priv <= 0) return DEAMOE_ERR_UNSUPPORTED;
   if (c->schedule < DEAMOE_SCHED_AUTO || c->schedule > DEAMOE_SCHED_DENSE) return DEAMOE_ERR_INVALID_ARG;
   if (!(c->route_scale == c->route_scale)) return DEAMOE_ERR_INVALID_ARG;

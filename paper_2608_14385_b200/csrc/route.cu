@@ -224,7 +224,7 @@ extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* r
   using namespace deamoe;
   if (n_dept <= 0 || experts_per_dept <= 0 || hidden <= 0 || top_k <= 0 || B < 0) return DEAMOE_ERR_INVALID_ARG;
   const long long n = (long long)n_dept * experts_per_dept;
-  if (top_k > n || !(route_scale == route_scale)) return DEAMOE_ERR_INVALID_ARG;
+  if (top_k > n || !(route_scale == route_scale) || norm_topk < 0 || norm_topk > 2) return DEAMOE_ERR_INVALID_ARG;
   if (n > DEAMOE_MAX_EXPERTS || top_k > DEAMOE_MAX_TOPK || (hidden & 3)) return DEAMOE_ERR_UNSUPPORTED;
   if (B == 0) return DEAMOE_OK;
   if (!router || !tokens || !topk_idx || !topk_w) return DEAMOE_ERR_INVALID_ARG;

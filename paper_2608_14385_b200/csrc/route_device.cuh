@@ -115,8 +115,8 @@ static __device__ void topk_one_token(const LayerDev& L, int t, int B, int kslic
   // gate weights
   const float top = __shfl_sync(0xffffffffu, my_v, 0);
   float e, den;
-  if (L.norm_topk) {
-    e = (lane < k) ? expf(my_v - top) : 0.f;
+  if (L.norm_topk) {  // 1: softmax over the selection; 2: logistic scores normalised over the selection
+    e = (lane < k) ? (L.norm_topk == 2 ? 1.f / (1.f + expf(-my_v)) : expf(my_v - top)) : 0.f;
     den = e;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
@@ -309,8 +309,8 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
     });
   const float top = __shfl_sync(0xffffffffu, my_v, 0);
   float e, den;
-  if (L.norm_topk) {
-    e = (lane < k) ? expf(my_v - top) : 0.f;
+  if (L.norm_topk) {  // 1: softmax over the selection; 2: logistic scores normalised over the selection
+    e = (lane < k) ? (L.norm_topk == 2 ? 1.f / (1.f + expf(-my_v)) : expf(my_v - top)) : 0.f;
     den = e;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);

@@ -43,3 +43,9 @@ def test_status_strings_and_host_side_argument_errors():
     cfg.max_batch = 4
     w.priv_gate = None
     assert L.deamoe_layer_create(ctypes.byref(cfg), ctypes.byref(w), None, ctypes.byref(out)) == binding.ERR_INVALID_ARG
+    w.priv_gate = 1
+    for field, bad in (("norm_topk", 3), ("norm_topk", -1), ("sigma", 4)):
+        good = getattr(cfg, field)
+        setattr(cfg, field, bad)
+        assert L.deamoe_layer_create(ctypes.byref(cfg), ctypes.byref(w), None, ctypes.byref(out)) == binding.ERR_INVALID_ARG
+        setattr(cfg, field, good)

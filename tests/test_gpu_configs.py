@@ -233,3 +233,32 @@ def test_routing_of_wide_and_group_limited_routers(m, g, k, k_dept, strict):
             tied.close()
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("m,g,k,norm", [(6, 16, 6, 2), (40, 40, 8, 2), (10, 32, 10, 0)])
+def test_gate_variants_on_every_topk_path(m, g, k, norm):
+    """The gate-weight variants (logistic scores normalised over the selection; full softmax without
+    renormalisation) through the register top-k (inside the routing tail and, for more tokens than it
+    has warps, in the grid of its own) and through the shared-memory top-k of very wide routers."""
+    shape = synth.LayerShape(f"gate{m}x{g}", hidden=256, n_dept=m, experts_per_dept=g, ffn=16, priv=16, top_k=k,
+                             norm_topk=norm, route_scale=1.5)
+    dev = torch.device("cuda:0")
+    w = synth.make_deamoe_weights(shape, 3, dev)
+    w["router"] = w["router"] * 8.0  # logits of order one, so the variants differ visibly
+    layer = binding.Layer(shape, w, 40)
+    try:
+        cfg = oracle_cfg(shape)
+        for B, seed in ((3, 8), (40, 9)):
+            tokens = synth.make_tokens(shape, B, seed, dev)
+            layer.route(tokens, want_outputs=False)
+            torch.cuda.synchronize()
+            want = ref.route(cfg, synth.to_numpy(w["router"]), synth.to_numpy(tokens), want_logits=True)
+            safe = want["gap"] > 1e-5 * np.abs(want["logits"]).max(axis=1)
+            got = layer.routing(B)
+            assert safe.mean() > 0.5
+            assert (got["idx"][safe] == want["idx"][safe]).all()
+            assert np.abs(got["w"][safe].astype(np.float64) - want["w"][safe]).max() <= 1e-5
+        assert layer.stats()["device_status"] == 0
+    finally:
+        layer.close()
+

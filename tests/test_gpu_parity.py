@@ -60,7 +60,7 @@ def test_vanilla_comparator(schedule):
 
 @pytest.mark.parametrize("schedule", ALL_SCHEDULES)
 @pytest.mark.parametrize("variant", ["no_private", "sigma_none", "gelu", "rmsnorm", "rmsnorm_shared_f32", "square_private", "g1", "k_eq_n",
-                                     "norm_all", "group_limited", "strict_coverage", "f32_tokens"])
+                                     "norm_all", "sigmoid_gates", "group_limited", "strict_coverage", "f32_tokens"])
 def test_variants(schedule, variant):
     shape = {
         "no_private": SMALL.with_(priv=0),
@@ -72,6 +72,7 @@ def test_variants(schedule, variant):
         "g1": SMALL.with_(n_dept=12, experts_per_dept=1),
         "k_eq_n": SMALL.with_(n_dept=2, experts_per_dept=2, top_k=4),
         "norm_all": SMALL.with_(norm_topk=0, route_scale=2.5),
+        "sigmoid_gates": SMALL.with_(norm_topk=2, route_scale=2.5),
         "group_limited": SMALL.with_(n_dept=4, experts_per_dept=4, top_k=4, k_dept=2),
         "strict_coverage": SMALL.with_(n_dept=6, experts_per_dept=6, top_k=4, k_dept=4, strict_dept=1),
         "f32_tokens": RAGGED.with_(act_dtype=0),
