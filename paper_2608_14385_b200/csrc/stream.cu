@@ -1435,7 +1435,10 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     while (true) {
       const int rb = n % NRED;
       const uint32_t par = (uint32_t)(n / NRED) & 1u;
-      bool have = mbar_try_wait(&red_full[rb], par);
+      // A test that never blocks: `mbarrier.try_wait` may suspend the thread for microseconds before it
+      // reports "not yet", and the completions of the items already finished would wait that long.
+      const bool have = __shfl_sync(0xffffffffu, (lane == 0) ? (int)mbar_test_wait(&red_full[rb], par) : 0, 0) != 0;
+      __syncwarp();  // orders the other lanes' reads after lane 0's acquire
       if (!have) {
         if (pend) {  // nothing ready: publish what is finished
           __syncwarp();
