@@ -86,15 +86,3 @@ def count_active(topk_idx, g):
         depts |= dt
         experts |= set(int(i) for i in row)
     return len(depts), len(experts), pairs
-
-
-def step_flops_deamoe(topk_idx, h, f, r, n, g, n_shared=0, shared_ffn=0):
-    """Algorithmic FLOPs of one step evaluated the two-stage way: department
-    gate/up once per (token, department), private transforms and the department
-    down projection once per (token, expert), router and shared expert per token."""
-    B = len(topk_idx)
-    _, _, token_depts = count_active(topk_idx, g)
-    pairs = sum(len(row) for row in topk_idx)
-    rr = r if r > 0 else 0
-    return 2 * (token_depts * 2 * h * f + pairs * 3 * rr * f + pairs * h * f
-                + B * n_shared * 3 * h * shared_ffn + B * n * h)

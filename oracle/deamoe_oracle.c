@@ -18,7 +18,7 @@
  * expert, with no bucketing; the SETS and LISTS of Section 3.2 are produced by a
  * separate plain routine.
  *
- * Readings where the paper is silent (each is listed in the design notes):
+ * Readings taken where the paper is silent:
  *   - private matrices are [priv, ffn]; the paper's own case is priv == ffn;
  *     priv == 0 means A_g = A_u = A_d = identity (nothing stored);
  *   - ties in TopK go to the lowest expert index; the order of S(x) is
@@ -236,12 +236,21 @@ static int cmp_desc_then_index(const void *a, const void *b) {
  *   topk_idx [B, k]   selected experts in (logit desc, index asc) order
  *   topk_w   [B, k]   gate weights p (fp64)
  *   logits   [B, n]   fp64 router logits
- *   gap      [B]      smallest difference between neighbours among the first
- *                     min(k+1, candidates) sorted logits: how far the selection
- *                     and its order are from a tie
+ *   gap      [B]      how far the token's selection and its order are from a tie: the
+ *                     smallest margin of any comparison that decided them, i.e. the
+ *                     minimum of the three entries of gap_parts
+ *   gap_parts [B, 3]  [0] smallest difference between neighbours among the first
+ *                         min(k+1, candidates) sorted candidate logits;
+ *                     [1] group limit: score of the k_dept-th best department minus the
+ *                         score of the first department left out (INFINITY without a cut);
+ *                     [2] strict coverage: over all replacements, the newcomer's logit minus
+ *                         the next-best logit among the experts of the departments not yet
+ *                         covered (INFINITY if nothing was replaced or nothing else competed)
+ * The gaps are diagnostics for the tests (an fp32 router may legitimately decide a
+ * comparison the other way when its margin is at rounding level); they change no result.
  */
 int oracle_route(const oracle_config_t *c, const float *router, const void *tokens, int B,
-                 int32_t *topk_idx, double *topk_w, double *logits, double *gap) {
+                 int32_t *topk_idx, double *topk_w, double *logits, double *gap, double *gap_parts) {
   const int h = c->hidden, g = c->experts_per_dept, m = c->n_dept, n = m * g, k = c->top_k;
   if (!router || !tokens || !topk_idx || !topk_w || k < 1 || k > n) return 1;
   double *x = (double *)malloc(sizeof(double) * ((size_t)h + n));
@@ -255,6 +264,7 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
     for (int q = 0; q < h; ++q) x[q] = ld(tokens, c->act_dtype, (size_t)t * h + q);
     matvec(router, ORACLE_F32, n, h, x, l);
     if (logits) memcpy(logits + (size_t)t * n, l, sizeof(double) * n);
+    double gap_sel = INFINITY, gap_dept = INFINITY, gap_strict = INFINITY;
     /* group limit: keep the k_dept departments with the largest best logit */
     memset(alive, 1, (size_t)m);
     if (c->k_dept > 0 && c->k_dept < m) {
@@ -266,20 +276,19 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
       qsort(dkey, (size_t)m, sizeof(keyed_t), cmp_desc_then_index);
       memset(alive, 0, (size_t)m);
       for (int q = 0; q < c->k_dept; ++q) alive[dkey[q].i] = 1;
+      gap_dept = dkey[c->k_dept - 1].v - dkey[c->k_dept].v;
     }
     int cand = 0;
     for (int i = 0; i < n; ++i)
       if (alive[i / g]) { key[cand].v = l[i]; key[cand].i = i; ++cand; }
     if (cand < k) { rc = 1; break; }
     qsort(key, (size_t)cand, sizeof(keyed_t), cmp_desc_then_index);
-    if (gap) { /* smallest difference between neighbours of the sorted order, up to the first expert left out */
+    { /* smallest difference between neighbours of the sorted order, up to the first expert left out */
       int upto = (k + 1 < cand) ? k + 1 : cand;
-      double gmin = INFINITY;
       for (int q = 1; q < upto; ++q) {
         double d = key[q - 1].v - key[q].v;
-        if (d < gmin) gmin = d;
+        if (d < gap_sel) gap_sel = d;
       }
-      gap[t] = gmin;
     }
     /* strict department coverage: swap duplicates out until min(k_dept, k) departments are covered */
     if (c->strict_dept && c->k_dept > 0) {
@@ -300,18 +309,36 @@ int oracle_route(const oracle_config_t *c, const float *router, const void *toke
         }
         if (victim < 0) break;
         int best = -1;
+        double runner_up = -INFINITY; /* diagnostic only: the largest logit the newcomer beat */
         for (int i = 0; i < n; ++i) {
           int used = 0;
           for (int q = 0; q < k; ++q) if (key[q].i / g == i / g) used = 1;
           if (used) continue;
-          if (best < 0 || l[i] > l[best]) best = i; /* ascending i: ties keep the lowest index */
+          if (best < 0 || l[i] > l[best]) { /* ascending i: ties keep the lowest index */
+            if (best >= 0 && l[best] > runner_up) runner_up = l[best];
+            best = i;
+          } else if (l[i] > runner_up) {
+            runner_up = l[i];
+          }
         }
         if (best < 0) break;
+        if (l[best] - runner_up < gap_strict) gap_strict = l[best] - runner_up;
         key[victim].i = best;
         key[victim].v = l[best];
       }
     }
     for (int q = 0; q < k; ++q) topk_idx[(size_t)t * k + q] = key[q].i;
+    if (gap_parts) {
+      gap_parts[(size_t)t * 3 + 0] = gap_sel;
+      gap_parts[(size_t)t * 3 + 1] = gap_dept;
+      gap_parts[(size_t)t * 3 + 2] = gap_strict;
+    }
+    if (gap) {
+      double gmin = gap_sel;
+      if (gap_dept < gmin) gmin = gap_dept;
+      if (gap_strict < gmin) gmin = gap_strict;
+      gap[t] = gmin;
+    }
     if (c->norm_topk == 2) { /* sigmoid scores, normalised over the selection */
       double den = 0.0;
       for (int q = 0; q < k; ++q) den += 1.0 / (1.0 + exp(-key[q].v));
@@ -402,7 +429,7 @@ int oracle_deamoe_forward(const oracle_config_t *c, const oracle_weights_t *w, c
   int32_t *idx = topk_idx ? topk_idx : (int32_t *)malloc(sizeof(int32_t) * (size_t)B * k);
   double *p = topk_w ? topk_w : (double *)malloc(sizeof(double) * (size_t)B * k);
   double *x = (double *)malloc(sizeof(double) * (size_t)h * 2);
-  int rc = (!idx || !p || !x) ? 3 : oracle_route(c, w->router, tokens, B, idx, p, NULL, NULL);
+  int rc = (!idx || !p || !x) ? 3 : oracle_route(c, w->router, tokens, B, idx, p, NULL, NULL, NULL);
   double *e = x ? x + h : NULL;
   const int count = rows ? n_rows : B;
   for (int s = 0; s < count && rc == 0; ++s) {
@@ -440,7 +467,7 @@ int oracle_vanilla_forward(const oracle_config_t *c, const oracle_weights_t *w, 
   int32_t *idx = topk_idx ? topk_idx : (int32_t *)malloc(sizeof(int32_t) * (size_t)B * k);
   double *p = topk_w ? topk_w : (double *)malloc(sizeof(double) * (size_t)B * k);
   double *x = (double *)malloc(sizeof(double) * (size_t)h * 2);
-  int rc = (!idx || !p || !x) ? 3 : oracle_route(c, w->router, tokens, B, idx, p, NULL, NULL);
+  int rc = (!idx || !p || !x) ? 3 : oracle_route(c, w->router, tokens, B, idx, p, NULL, NULL, NULL);
   double *e = x ? x + h : NULL;
   const int count = rows ? n_rows : B;
   for (int s = 0; s < count && rc == 0; ++s) {

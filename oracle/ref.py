@@ -127,19 +127,23 @@ def make_weights(cfg, w, per_expert_dept_tables=False):
 
 
 def route(cfg, router, tokens, want_logits=False):
-    """Eq. (2) + gate weights.  Returns dict(idx [B,k] i32, w [B,k] f64, gap [B] f64, logits?)."""
+    """Eq. (2) + gate weights.  Returns dict(idx [B,k] i32, w [B,k] f64, gap [B] f64, gap_parts [B,3]
+    f64, logits?).  gap is the smallest margin of any comparison that decided the token's selection
+    (gap_parts: among the sorted candidates / at the department cut / at a strict-coverage
+    replacement); a test that compares an fp32 router bit for bit requires it to be clear of zero."""
     tokens = _check(np.ascontiguousarray(tokens), cfg.act_dtype, "tokens")
     router = _check(np.ascontiguousarray(router), F32, "router")
     B, k, n = tokens.shape[0], cfg.top_k, cfg.n_dept * cfg.experts_per_dept
     idx = np.zeros((B, k), np.int32)
     p = np.zeros((B, k), np.float64)
     gap = np.zeros((B,), np.float64)
+    parts = np.zeros((B, 3), np.float64)
     logits = np.zeros((B, n), np.float64) if want_logits else None
     rc = lib().oracle_route(C.byref(cfg), _ptr(router), _ptr(tokens), C.c_int(B), _ptr(idx), _ptr(p),
-                            _ptr(logits) if want_logits else None, _ptr(gap))
+                            _ptr(logits) if want_logits else None, _ptr(gap), _ptr(parts))
     if rc:
         raise RuntimeError(f"oracle_route failed: {rc}")
-    out = {"idx": idx, "w": p, "gap": gap}
+    out = {"idx": idx, "w": p, "gap": gap, "gap_parts": parts}
     if want_logits:
         out["logits"] = logits
     return out

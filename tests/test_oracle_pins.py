@@ -460,3 +460,89 @@ def test_rmsnorm_sigma_against_the_library_routine_and_its_invariants():
     a = ref.deamoe_expert(s_cfg, Wg, Wu, Wd, Ag, Au, Ad, x)
     b = ref.deamoe_expert(s_cfg, synth.to_numpy(wt2["dept_gate"][j]), Wu, Wd, Ag, Au, Ad, x)
     assert np.abs(a - b).max() > 1e-3 * np.abs(a).max()
+
+
+# ---------------------------------------------------------------- sigma = GeLU (Section 3.4, Table 4)
+
+def test_gelu_sigma_against_the_library_routine_and_textbook_values():
+    """sigma = GeLU is the exact (erf) form x Phi(x).  Pinned by (1) the taps G, U, Z against
+    torch.nn.functional.gelu(approximate="none") and scipy's normal CDF applied to the
+    un-transformed vectors (sigma = none taps; Z re-built with dense numpy), (2) textbook values
+    of the standard normal CDF: GeLU(1) = Phi(1) = 0.8413447460685429, which the tanh
+    approximation (0.8411919906082768) misses in the fourth digit, so neither a switch to that
+    form nor a wrong 1/sqrt(2) passes."""
+    from scipy.special import ndtr
+    shape = SMALL.with_(sigma=ref.SIGMA_GELU)
+    cfg = oracle_cfg(shape)
+    wt = _layer(shape, 9, std=0.3)
+    x = widen(synth.make_tokens(shape, 1, 9))[0]
+    j, i = 2, 2 * shape.experts_per_dept + 1
+    Wg, Wu, Wd = (synth.to_numpy(wt[f"dept_{k}"][j]) for k in ("gate", "up", "down"))
+    Ag, Au, Ad = (synth.to_numpy(wt[f"priv_{k}"][i]) for k in ("gate", "up", "down"))
+    out, G, U, Y, Z = ref.deamoe_expert(cfg, Wg, Wu, Wd, Ag, Au, Ad, x, taps=True)
+    raw_cfg = oracle_cfg(shape.with_(sigma=ref.SIGMA_NONE))
+    _, G0, U0, _, _ = ref.deamoe_expert(raw_cfg, Wg, Wu, Wd, Ag, Au, Ad, x, taps=True)
+
+    def lib_gelu(v):
+        return torch.nn.functional.gelu(torch.from_numpy(v), approximate="none").numpy()
+
+    assert np.abs(G0).max() > 1.0 and np.abs(U0).max() > 1.0      # arguments where the forms differ
+    np.testing.assert_allclose(G, lib_gelu(G0), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(U, lib_gelu(U0), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(G, G0 * ndtr(G0), rtol=1e-12, atol=1e-15)
+    Z0 = widen(wt["priv_down"][i]).T @ Y          # (A_d)^T Y, before the last sigma
+    np.testing.assert_allclose(Z, lib_gelu(Z0), rtol=1e-10, atol=1e-14)
+    np.testing.assert_allclose(out, widen(wt["dept_down"][j]).T @ Z, rtol=1e-11, atol=1e-14)
+    tanh_form = 0.5 * G0 * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (G0 + 0.044715 * G0 ** 3)))
+    assert np.abs(G - tanh_form).max() > 1e-5      # the approximation is told apart
+    # textbook values through the oracle itself: identity department matrices (fp32, no private part),
+    # so the tap G is sigma applied to the token
+    eye = synth.LayerShape("eye", hidden=4, n_dept=1, experts_per_dept=1, ffn=4, priv=0, top_k=1,
+                           sigma=ref.SIGMA_GELU, weight_dtype=0, act_dtype=0)
+    I4 = np.eye(4, dtype=np.float32)
+    xs = np.array([1.0, -1.0, 0.5, 2.0])
+    _, Gt, Ut, _, _ = ref.deamoe_expert(oracle_cfg(eye), I4, I4, I4, None, None, None, xs, taps=True)
+    phi = np.array([0.8413447460685429, 0.15865525393145707, 0.6914624612740131, 0.9772498680518208])
+    np.testing.assert_allclose(Gt, xs * phi, rtol=1e-14)
+    np.testing.assert_allclose(Ut, xs * phi, rtol=1e-14)
+    assert abs(Gt[0] - 0.8411919906082768) > 1e-4   # not the tanh form
+
+
+# ---------------------------------------------------------------- the tie-guard diagnostics
+
+def test_routing_gaps_report_every_comparison_that_decides_a_selection():
+    """oracle.ref.route reports, per token, the smallest margin of any comparison its selection
+    rests on: neighbours among the sorted candidates, the department cut of the group limit
+    (Section 3.3) and the choice of a newcomer under strict coverage.  Hand-built logits (the router
+    is the identity, so the logits are the token) put a near-tie at each place in turn."""
+    g, m, k = 3, 4, 3
+    n = g * m
+    base = synth.LayerShape("gaps", hidden=n, n_dept=m, experts_per_dept=g, ffn=8, priv=0, top_k=k,
+                            weight_dtype=0, act_dtype=0)
+    router = np.eye(n, dtype=np.float32)
+    #          dept 0          dept 1          dept 2          dept 3
+    l = np.array([[9.0, 8.0, 1.0, 7.0, 0.5, 0.25, 6.5, 0.1, 0.2, 6.25, 0.3, 0.4]], np.float32)
+    flat = ref.route(oracle_cfg(base), router, l)
+    assert list(flat["idx"][0]) == [0, 1, 3]
+    np.testing.assert_allclose(flat["gap_parts"][0], [0.5, np.inf, np.inf])      # 7.0 against 6.5 left out
+    assert flat["gap"][0] == 0.5
+    cut = ref.route(oracle_cfg(base.with_(k_dept=2)), router, l)                 # departments 0, 1 stay (9, 7 | 6.5)
+    assert list(cut["idx"][0]) == [0, 1, 3]
+    np.testing.assert_allclose(cut["gap_parts"][0], [1.0, 0.5, np.inf])          # candidates 9 8 7 | 1; cut 7 - 6.5
+    assert cut["gap"][0] == 0.5
+    l2 = l.copy()
+    l2[0, 6] = np.float32(7.0) - np.float32(2.0 ** -20)                          # department 2 almost ties department 1
+    near = ref.route(oracle_cfg(base.with_(k_dept=2)), router, l2)
+    assert near["gap_parts"][0, 1] == pytest.approx(2.0 ** -20) and near["gap"][0] == near["gap_parts"][0, 1]
+    assert near["gap_parts"][0, 0] == 1.0                                        # the flat candidates are far apart
+    # strict coverage with k_dept = 3: selection 0, 1, 3 covers two departments; expert 1 (the lower
+    # duplicate of department 0) is replaced by the best expert of departments 2, 3: 6.5 against 6.25
+    strict = ref.route(oracle_cfg(base.with_(k_dept=3, strict_dept=1)), router, l)
+    assert list(strict["idx"][0]) == [0, 6, 3]
+    np.testing.assert_allclose(strict["gap_parts"][0], [0.5, 0.25, 0.25])        # 7 - 6.5; cut 6.5 - 6.25; newcomer 6.5 - 6.25
+    l3 = l.copy()
+    l3[0, 9] = 6.5                                                               # exact tie for the newcomer
+    tied = ref.route(oracle_cfg(base.with_(k_dept=4, strict_dept=1)), router, l3)
+    assert list(tied["idx"][0]) == [0, 6, 3]
+    assert tied["gap_parts"][0, 2] == 0.0 and tied["gap"][0] == 0.0
+    assert 9 not in tied["idx"][0]                                               # ties go to the lower index
