@@ -43,7 +43,7 @@ def measured_peaks():
     if os.path.exists(path):
         d = json.load(open(path))
         return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy read+write)"
-    return 6650.0, "fallback (earlier measurement on this pool)"
+    return 6650.0, "fallback (no MEASURED_PEAKS.json: an earlier copy measurement on a B200)"
 
 
 class ClockSampler:

@@ -14,7 +14,9 @@
  *  - Pointers marked DEVICE are CUDA device pointers of the current device; pointers
  *    marked HOST are ordinary host pointers.  `cuda_stream` is a cudaStream_t passed as
  *    void* (NULL = the legacy default stream).
- *  - All matrices are dense, row-major, 16-byte aligned.
+ *  - All matrices are dense, row-major, 16-byte aligned.  A device pointer to tokens, outputs or a
+ *    router matrix that is not 16-byte aligned is rejected with DEAMOE_ERR_INVALID_ARG (the kernels
+ *    use 16-byte accesses and bulk copies); topk_idx / topk_w need 4-byte alignment.
  *  - Every call returns a deamoe_status_t; nothing aborts, traps or throws.  Argument
  *    errors are detected on the host before anything is enqueued.
  *  - deamoe_route / deamoe_forward only ENQUEUE work on the given stream; they never
@@ -22,6 +24,15 @@
  *    Calls on one layer must be enqueued on one stream (or otherwise ordered): a layer has one
  *    workspace.  A step keeps no per-step state on the host, so it may be captured into a CUDA
  *    graph and replayed (Section 5 of the paper runs its steps that way).
+ *  - The weight-streaming and dense kernels are PERSISTENT grids sized to fill the device (every
+ *    SM, two thread blocks each) whose blocks wait for one another's results, so all blocks of a
+ *    launch must be resident at the same time.  Run one such step per device at a time: if another
+ *    kernel holds SMs while a step runs (a second layer driven from another stream, another process
+ *    under MPS, a long-running communication kernel), blocks that cannot become resident keep the
+ *    others waiting.  Nothing hangs or faults in that case -- every device-side wait is bounded --
+ *    but when a wait expires the step's output is invalid and deamoe_get_stats reports
+ *    DEAMOE_ERR_TIMEOUT in the device status word; the layer is usable again for the next call.
+ *    Layers enqueued one after another on ONE stream (a model's stack) are the intended use.
  *  - There is no CPU fallback and no other backend: without a CUDA device the create
  *    calls fail with DEAMOE_ERR_CUDA.
  */
@@ -233,23 +244,43 @@ deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t *layer, float *ms);
  *   tokens   DEVICE [B, hidden] fp32 (16-byte aligned)
  *   topk_idx DEVICE [B, top_k] out, topk_w DEVICE [B, top_k] out (fp32)
  *
- * Limits: slices * B * n * 4 bytes must fit the fixed array, where slices (1..16) is the number of
- * column slices the logits kernel uses for this n and hidden; a larger request returns
- * DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout, n = 256, hidden = 7168: 16 slices,
- * B up to 256; hidden <= 512: 1 slice.)  Other errors as for deamoe_route.
+ * Limits: slices * B * n * 4 bytes must fit the fixed array, where slices (1, 2, 4, 8 or 16) is the
+ * number of column slices the logits kernel uses for this n and hidden -- the same rule as a layer
+ * object's: doubled while a slice is wider than 512 columns and (n / 4) * slices < 1024.  A larger
+ * request returns DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout, n = 256, hidden =
+ * 7168: 16 slices, B up to 256; n = 2048, hidden = 7168: 2 slices, B up to 256; hidden <= 512: 1
+ * slice.)  Other errors as for deamoe_route.
  *
  * The first call on each device resolves the array's device address and sets one kernel
  * attribute (the device must be current); make that first call before any stream capture begins.
  * Later calls only enqueue two kernels on `cuda_stream`.  All calls share the one array and it
  * keeps the previous call's contents: nothing has to be cleared, because every entry a call reads
  * it has first written itself, but two calls that overlap on the GPU (different streams, or the
- * same array used from two threads) race on it -- serialise them.
+ * same array used from two threads) race on it -- serialise them.  The one-time set-up itself is
+ * safe to reach from several host threads at once.
  */
 #define DEAMOE_STATIC_ROUTE_SCRATCH_BYTES (4u << 20)
 deamoe_status_t deamoe_route_static(void *cuda_stream, const float *router, const float *tokens,
                                     int32_t n_dept, int32_t experts_per_dept, int32_t hidden, int32_t top_k,
                                     int32_t norm_topk, float route_scale, int32_t B, int32_t *topk_idx,
                                     float *topk_w);
+
+/*
+ * Failure-detection test aid.  (The paper has no counterpart.)  Every device-side wait of the
+ * library is bounded: after a number of polls it gives up, the kernel records DEAMOE_ERR_TIMEOUT
+ * in the device status word, waits (bounded) for its copies in flight, frees its tensor memory
+ * and returns.  This call lets a test see that path without faulting or hanging anything:
+ *   wait_limit  polls after which a wait gives up in later calls on this layer (0 = the default);
+ *   withhold    bit 0: the routing kernel does not raise the flags that hand the work list to the
+ *               fused streaming kernel, so that kernel's planners wait until the limit expires;
+ *               bit 1: the copy role of the dense (tcgen05) kernel issues no copies, so its MMA role
+ *               waits for the ring until the limit expires.  0 = normal operation.
+ * A step run with a withheld hand-over returns garbage in `out` and DEAMOE_ERR_TIMEOUT from
+ * deamoe_get_stats; after deamoe_failure_test(layer, 0, 0) the layer works normally again.
+ * Errors: INVALID_ARG; UNSUPPORTED if the layer's schedule has no such hand-over (plain / staged
+ * schedule for bit 0, no dense schedule for bit 1).
+ */
+deamoe_status_t deamoe_failure_test(deamoe_layer_t *layer, int32_t wait_limit, int32_t withhold);
 
 /* Number of kernels the last forward/route call of this layer launched (host-side count). */
 int32_t deamoe_last_launches(const deamoe_layer_t *layer);

@@ -13,7 +13,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdeamoe.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_BATCH, ERR_TIMEOUT = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_BATCH, ERR_TIMEOUT, ERR_INTERNAL = range(8)
 F32, BF16 = 0, 1
 SIGMA_NONE, SIGMA_SILU, SIGMA_GELU, SIGMA_RMSNORM = 0, 1, 2, 3
 SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4
@@ -21,7 +21,8 @@ SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4
 # every symbol include/deamoe.h declares
 SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",
            "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_get_routing",
-           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_route_static", "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
+           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_route_static", "deamoe_failure_test",
+           "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
 
 
 class Config(C.Structure):
@@ -73,6 +74,7 @@ def lib():
         L.deamoe_get_stats.argtypes = [C.c_void_p] * 7
         L.deamoe_route_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
+        L.deamoe_failure_test.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         L.deamoe_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.deamoe_profile_last_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
         _lib = L
@@ -222,6 +224,13 @@ class Layer:
             raise DeaMoEError(st, "deamoe_get_stats")
         return {"active_dept": nd.value, "active_expert": ne.value, "token_dept_pairs": ntd.value,
                 "unique_weight_bytes": ub.value, "device_status": st_.value}
+
+    def failure_test(self, wait_limit=0, withhold=0):
+        """Test aid (deamoe_failure_test): lower the poll limit of the bounded device-side waits
+        and / or withhold a hand-over so that a wait expires; (0, 0) restores normal operation."""
+        st = lib().deamoe_failure_test(self._h, int(wait_limit), int(withhold))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_failure_test")
 
     def profile(self, enable=True):
         """Record CUDA events around the weight-streaming launches of later forward calls."""

@@ -126,12 +126,7 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   const int MB = cfg->max_batch, k = d.k;
   const int tdmax = MB * (k < d.m ? k : d.m);  // (token, department) rows
   const int pmax = MB * k;                     // (token, expert) pairs
-  // router column slices: enough CTAs to cover the GPU a few times
-  L->kslices = 1;
-  // Column slices of the router product: at least 512 columns per thread block, and no more
-  // slices than it takes to fill the device with ~1024 blocks of four router rows (every slice
-  // is one more array of partial logits that the top-k has to read back).
-  while (L->kslices < 16 && d.h / L->kslices > 512 && (d.n / 4) * L->kslices < 1024) L->kslices *= 2;
+  L->kslices = router_kslices(d.n, d.h);
 
   bool ok = true;
   auto A = [&](deamoe_status_t r) { if (r != DEAMOE_OK && ok) { ok = false; st = r; } };
@@ -214,6 +209,10 @@ deamoe_status_t check_call(deamoe_layer_t* L, const void* tokens, int B) {
   return DEAMOE_OK;
 }
 
+// Device buffers are read and written with 16-byte accesses: a misaligned pointer is an argument
+// error reported here, before anything is enqueued, never a fault on the device.
+deamoe_status_t check_device_ptr(const void* p) { return aligned16(p) ? DEAMOE_OK : DEAMOE_ERR_INVALID_ARG; }
+
 LayerDev call_view(deamoe_layer_t* L, const void* tokens) {
   LayerDev d = L->dev;
   d.tokens_raw = tokens;
@@ -247,6 +246,9 @@ deamoe_status_t deamoe_route(deamoe_layer_t* L, void* cuda_stream, const void* t
                              float* topk_w) {
   deamoe_status_t st = check_call(L, tokens, B);
   if (st != DEAMOE_OK) return st;
+  if (B > 0 && check_device_ptr(tokens) != DEAMOE_OK) return DEAMOE_ERR_INVALID_ARG;
+  if (B > 0 && ((reinterpret_cast<uintptr_t>(topk_idx) | reinterpret_cast<uintptr_t>(topk_w)) & 3u))
+    return DEAMOE_ERR_INVALID_ARG;
   L->last_B = B;
   L->last_launches = 0;
   if (B == 0) return DEAMOE_OK;
@@ -263,6 +265,8 @@ deamoe_status_t deamoe_forward(deamoe_layer_t* L, void* cuda_stream, const void*
   deamoe_status_t st = check_call(L, tokens, B);
   if (st != DEAMOE_OK) return st;
   if (B > 0 && (!out || out == tokens)) return DEAMOE_ERR_INVALID_ARG;
+  if (B > 0 && (check_device_ptr(tokens) != DEAMOE_OK || check_device_ptr(out) != DEAMOE_OK))
+    return DEAMOE_ERR_INVALID_ARG;
   st = deamoe_route(L, cuda_stream, tokens, B, nullptr, nullptr);
   if (st != DEAMOE_OK || B == 0) return st;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -371,6 +375,12 @@ deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t* L, float* ms) {
   const cudaError_t e = stream_profile_last_ms(*L->plan, ms);
   if (e == cudaErrorInvalidValue) return DEAMOE_ERR_INVALID_ARG;
   return e == cudaSuccess ? DEAMOE_OK : DEAMOE_ERR_CUDA;
+}
+
+deamoe_status_t deamoe_failure_test(deamoe_layer_t* L, int32_t wait_limit, int32_t withhold) {
+  if (!L || wait_limit < 0 || withhold < 0 || withhold > 3) return DEAMOE_ERR_INVALID_ARG;
+  if (!L->plan) return withhold ? DEAMOE_ERR_UNSUPPORTED : DEAMOE_OK;  // the plain schedule has no device-side waits
+  return stream_set_failure_test(*L->plan, (unsigned)wait_limit, withhold) ? DEAMOE_OK : DEAMOE_ERR_UNSUPPORTED;
 }
 
 int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launches : 0; }

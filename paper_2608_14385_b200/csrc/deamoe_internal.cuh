@@ -90,13 +90,25 @@ struct LayerDev {
   float* Osh;          // [MB, h]
   int32_t* sh_done;    // counter the combine kernel resets at the end of a step, or null
   // sigma = RMSNorm: sums of squares of the un-normalised vectors, zeroed by the routing tail
-  float* ss_gu;        // [MB*min(k,m), 2]: G and U of every (token, department) row
-  float* ss_z;         // [MB*k]: Z of every pair
+  unsigned long long* ss_gu;  // [MB*min(k,m), 2]: G and U of every (token, department) row (fixed point, see ss_fixed)
+  unsigned long long* ss_z;   // [MB*k]: Z of every pair
 };
 
 constexpr float RMS_EPS = 1e-6f;
 // 1 / sqrt(mean(v^2) + eps) from a sum of squares over `width` elements
 static __device__ __forceinline__ float rms_scale(float ss, int width) { return rsqrtf(ss / (float)width + RMS_EPS); }
+// The streaming and dense kernels add the squares of a vector tile by tile, from many thread blocks
+// in no fixed order.  The partial sums are therefore accumulated as 64-bit fixed-point integers
+// (2^-30 resolution): integer addition is associative, so the total -- and with it the layer's
+// output -- does not depend on the order of arrival.  A vector of f values loses at most
+// f / 16 * 2^-31 of its sum of squares to the rounding of the partial sums, far below RMS_EPS * f.
+constexpr float SS_FIXED_ONE = 1073741824.f;  // 2^30
+static __device__ __forceinline__ unsigned long long ss_fixed(float sq) {
+  return __float2ull_rn(fminf(sq * SS_FIXED_ONE, 4.0e18f));
+}
+static __device__ __forceinline__ float rms_scale_fixed(unsigned long long ss, int width) {
+  return rms_scale(__ull2float_rn(ss) * (1.0f / SS_FIXED_ONE), width);
+}
 
 // Programmatic dependent launch: a kernel launched with launch_pdl() may start while its
 // predecessor in the stream is still running (after the predecessor called pdl_trigger()); it must
@@ -116,6 +128,20 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.attrs = attr; cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// Column slices of the router product (one grid row of k_router_logits per slice, one array of
+// partial logits each): at least 512 columns per thread block, and no more slices than it takes to
+// fill the device with ~1024 blocks of four router rows (every slice is one more array the top-k has
+// to read back).  The slices' partial sums are added in slice order, so every caller that wants the
+// same fp32 logits must use the same count: the layer object and deamoe_route_static both call this.
+static inline int router_kslices(int n, int h) {
+  int ks = 1;
+  while (ks < 16 && h / ks > 512 && (n / 4) * ks < 1024) ks *= 2;
+  return ks;
+}
+
+// The kernels read tokens and write outputs with 16-byte vector accesses and bulk copies.
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
 

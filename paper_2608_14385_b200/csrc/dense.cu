@@ -65,7 +65,7 @@ constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5;
 constexpr int DN_THREADS = (DN_WARP_MMA + 1) * 32;
 constexpr int DN_TMEM_COLS = 2 * DN_TILE;   // 2 accumulator buffers; the CTAs of an SM share its 512 columns
 constexpr size_t DN_SMEM = (size_t)DN_AST * DN_STAGE_BYTES + 512 /* barriers, control */;
-constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits; then an error status, never a hang
+constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits (default poll limit); then an error status, never a hang
 static_assert((DN_SMEM + 1024) * DN_CTAS_PER_SM <= 228 * 1024, "shared memory budget");
 // No more than DN_CTAS_PER_SM of these CTAs fit an SM's shared memory, and together they ask for no
 // more tensor memory than an SM has: the allocation below never waits for another CTA.
@@ -98,6 +98,8 @@ struct DensePhase {
 struct DenseArgs {
   DensePhase ph[2];
   int nph;
+  unsigned spin_limit;  // polls after which a bounded wait gives up
+  int withhold;         // failure tests: the copy role issues nothing
 };
 // tensor maps of the phases' input planes: [phase][box height 16 / 32 / 64 rows]
 struct DenseMaps {
@@ -126,8 +128,8 @@ __device__ __forceinline__ bool bar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  On expiry (or when another role has given up) the abort flag is raised and false
 // is returned; the caller leaves its loop and the CTA runs to its common end.
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (unsigned it = 0; it < DN_SPIN_LIMIT; ++it) {
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned limit) {
+  for (unsigned it = 0; it < limit; ++it) {
     if (bar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 63u && *abort_flag) return false;
   }
@@ -297,6 +299,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
       long long dn_acc[2] = {0, 0};
       const long long dn_start = clock64();
 #endif
+      if (A.withhold) ok = false;  // failure test: nothing is copied, the MMA role's wait for the ring expires
       for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
@@ -309,7 +312,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
           for (int c = 0; c < nch; ++c, ++g) {
             const int s = (int)(g % DN_AST);
             { DN_T0();
-            if (!bar_wait(&a_empty[s], ((g / DN_AST) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            if (!bar_wait(&a_empty[s], ((g / DN_AST) & 1u) ^ 1u, abort_flag, A.spin_limit)) { ok = false; break; }
             DN_ADD(0); }
             unsigned char* st = ring + (size_t)s * DN_STAGE_BYTES;
             bar_arrive_expect_tx(&a_full[s], bytes + box_bytes);
@@ -348,13 +351,13 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
           const uint64_t desc0_x = umma_smem_desc(smem_addr(ring + DN_A_BYTES), box_rows * 16, 128);
           const uint32_t xstep = (2 * box_rows * 16) >> 4;  // a k-step of 16 columns = two column blocks of the rows
           const uint32_t buf = a & 1u;
-          if (!bar_wait(&acc_empty[buf], ((a >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (!bar_wait(&acc_empty[buf], ((a >> 1) & 1u) ^ 1u, abort_flag, A.spin_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d0 = tmem_base + buf * (uint32_t)DN_TILE;
           for (int c = 0; c < nch; ++c, ++g) {
             const int sa_i = (int)(g % DN_AST);
             { DN_T0();
-            if (!bar_wait(&a_full[sa_i], (g / DN_AST) & 1u, abort_flag)) { ok = false; break; }
+            if (!bar_wait(&a_full[sa_i], (g / DN_AST) & 1u, abort_flag, A.spin_limit)) { ok = false; break; }
             DN_ADD(1); }
             // (no tcgen05 fence here: the barrier wait orders the copies' writes before the MMAs)
             DN_T0();
@@ -393,7 +396,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
       for (int gi = 0; ok && gi < groups; ++gi, ++a) {
         const int n0 = gi * DN_NMAX, Tg = min(DN_NMAX, j.T - n0);
         const uint32_t buf = a & 1u;
-        if (lane == 0 && !bar_wait(&acc_full[buf], (a >> 1) & 1u, abort_flag)) ok = false;
+        if (lane == 0 && !bar_wait(&acc_full[buf], (a >> 1) & 1u, abort_flag, A.spin_limit)) ok = false;
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         if (!ok) break;
         tc_fence_after();
@@ -404,7 +407,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
         const bool rms = L.sigma == DEAMOE_SIGMA_RMSNORM;
         const int grow = j.row0 + n0 + n;                 // row of this lane's token in the stage's planes
         float zscale = 1.f;
-        if (rms && mine && ph.stage == ST_S4) zscale = rms_scale(__ldcg(L.ss_z + grow), L.f);
+        if (rms && mine && ph.stage == ST_S4) zscale = rms_scale_fixed(__ldcg(L.ss_z + grow), L.f);
         if (16 * e < Tg) {                                // warp-uniform: some lane of the warp has a token
           const uint32_t t0 = tmem_base + ((uint32_t)(e * 32) << 16) + buf * (uint32_t)DN_TILE;
           const size_t o0 = (size_t)(j.row0 + n0 + n) * ph.out_stride + (size_t)j.col0;
@@ -425,7 +428,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
                 float sq = 0.f;
 #pragma unroll
                 for (int q = 0; q < 16; ++q) sq = fmaf(v[q], v[q], sq);
-                atomicAdd(L.ss_gu + (size_t)grow * 2 + ((j.col0 + c0) >= L.f ? 1 : 0), sq);
+                atomicAdd(L.ss_gu + (size_t)grow * 2 + ((j.col0 + c0) >= L.f ? 1 : 0), ss_fixed(sq));
               }
               if (ph.outf) {
                 float4* dst = reinterpret_cast<float4*>(ph.outf + o0 + c0);
@@ -455,6 +458,12 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   // common end: every role arrives here, also after an abort
   tc_fence_before();
   __syncthreads();
+  if (*abort_flag) {
+    // giving up: copies issued into the ring may still be in flight; stay (bounded: about 64 us)
+    // until they have landed before the CTA's shared memory is released
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
   if (tid == 0 && *abort_flag) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;
   if (warp == 0) {
     tc_fence_after();
@@ -513,6 +522,8 @@ struct DensePlan {
   size_t o_gu, o_d, o_sgu, o_sd;  // element offsets: stacked gate;up / down^T of the departments, shared expert
   size_t e_gu, e_d;        // elements per department
   int n_sm;
+  unsigned spin_limit;     // DN_SPIN_LIMIT unless a failure test lowered it
+  int withhold;
 };
 
 bool dense_supported(const LayerDev& L) {
@@ -533,6 +544,7 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->n_sm, cudaDevAttrMultiProcessorCount, dev);
   if (p->n_sm <= 0) p->n_sm = 148;
+  p->spin_limit = DN_SPIN_LIMIT;
   const size_t fh = (size_t)L.f * L.h;
   p->e_gu = 2 * fh; p->e_d = fh;
   size_t total = 0;
@@ -592,6 +604,11 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   return DEAMOE_OK;
 }
 
+void dense_set_failure_test(DensePlan& p, unsigned spin_limit, int withhold) {
+  p.spin_limit = spin_limit ? spin_limit : DN_SPIN_LIMIT;
+  p.withhold = withhold;
+}
+
 void dense_plan_destroy(DensePlan* p) {
   if (!p) return;
   if (p->tiles) cudaFree(p->tiles);
@@ -616,6 +633,7 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
   DenseArgs A;
   std::memset(&A, 0, sizeof(A));
   A.nph = n_stages;
+  A.spin_limit = p.spin_limit; A.withhold = p.withhold;
   DenseMaps maps;
   std::memset(&maps, 0, sizeof(maps));
   int launches = 0;

@@ -20,6 +20,10 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
                                   uint64_t* bytes);
 void dense_plan_destroy(DensePlan* p);
 
+// Failure-detection tests: poll limit of the kernel's bounded waits (0 = default); withhold = 1: the
+// copy role issues no copies, so the MMA role's wait for the ring must expire.
+void dense_set_failure_test(DensePlan& p, unsigned spin_limit, int withhold);
+
 // Enqueue one launch that runs the given stages (at most two, independent of each other) of one
 // step.  in / out planes are the bf16 activation planes of the streaming schedule.  Returns the
 // number of kernels launched or -1.

@@ -1,6 +1,8 @@
 // Router (Eq. (2)), gate weights (Eq. (3)) and the department / expert token lists of
 // Section 3.2, all on the device with no host round trip.
+#include <atomic>
 #include <cstring>
+#include <mutex>
 
 #include "deamoe_internal.cuh"
 #include "route_device.cuh"
@@ -195,12 +197,15 @@ static __device__ __align__(256) float g_route_scratch[STATIC_SCRATCH_FLOATS];
 
 constexpr int MAX_DEVICES = 64;
 float* g_route_scratch_ptr[MAX_DEVICES];  // device address of the array, per device, after set-up
-bool g_route_ready[MAX_DEVICES];
+std::atomic<bool> g_route_ready[MAX_DEVICES];
+std::mutex g_route_setup_mutex;           // first calls from several host threads set up one at a time
 
 // Once per device, with that device current: resolve the array's device address (in host code the
 // symbol is only a handle) and let the top-k kernel use its full dynamic shared memory.
 deamoe_status_t static_route_setup(int dev) {
-  if (g_route_ready[dev]) return DEAMOE_OK;
+  if (g_route_ready[dev].load(std::memory_order_acquire)) return DEAMOE_OK;
+  std::lock_guard<std::mutex> lock(g_route_setup_mutex);
+  if (g_route_ready[dev].load(std::memory_order_relaxed)) return DEAMOE_OK;
   float* p = nullptr;
   if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_route_scratch) != cudaSuccess || !p) {
     cudaGetLastError();
@@ -211,7 +216,7 @@ deamoe_status_t static_route_setup(int dev) {
     return DEAMOE_ERR_CUDA;
   }
   g_route_scratch_ptr[dev] = p;
-  g_route_ready[dev] = true;
+  g_route_ready[dev].store(true, std::memory_order_release);
   return DEAMOE_OK;
 }
 
@@ -228,9 +233,12 @@ extern "C" deamoe_status_t deamoe_route_static(void* cuda_stream, const float* r
   if (n > DEAMOE_MAX_EXPERTS || top_k > DEAMOE_MAX_TOPK || (hidden & 3)) return DEAMOE_ERR_UNSUPPORTED;
   if (B == 0) return DEAMOE_OK;
   if (!router || !tokens || !topk_idx || !topk_w) return DEAMOE_ERR_INVALID_ARG;
-  // column slices of the logits kernel, chosen as the layer object does
-  int kslices = 1;
-  while (kslices < 16 && hidden / kslices > 512) kslices *= 2;
+  // the logits kernel reads router rows and tokens as 16-byte vectors; the outputs are 4-byte words
+  if (!aligned16(router) || !aligned16(tokens)) return DEAMOE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(topk_idx) | reinterpret_cast<uintptr_t>(topk_w)) & 3u) return DEAMOE_ERR_INVALID_ARG;
+  // column slices of the logits kernel: the same rule as the layer object, so that the partial sums
+  // are added in the same grouping and the fp32 logits (hence near-ties and gate weights) are the same
+  const int kslices = router_kslices((int)n, hidden);
   const int kslice = (((hidden + kslices - 1) / kslices) + 3) & ~3;
   const int ny = (hidden + kslice - 1) / kslice;
   if ((size_t)ny * (size_t)B * (size_t)n > STATIC_SCRATCH_FLOATS) return DEAMOE_ERR_BATCH;  // beyond the fixed scratch

@@ -64,8 +64,8 @@ constexpr int RED_FLOATS = CONSUMER_WARPS * MAX_QP * 128;
 constexpr size_t STREAM_SMEM =
     (size_t)NSLOT * SLOT_BYTES + (size_t)NRED * RED_FLOATS * 4 + (size_t)DESC_DEPTH * DESC_BYTES + 1024;
 static_assert((STREAM_SMEM + 1024) * CTAS_PER_SM <= 228 * 1024, "shared memory budget");
-static_assert((2 * NSLOT + 2 * DESC_DEPTH + 2 * NRED) * 8 + 16 * MAX_CAT_INTS_PAD + 16 * NRED + 16 + 224 <= 1024, "control region");
-constexpr unsigned SPIN_LIMIT = 1u << 24;  // bounded waits; then an error status, never a hang
+static_assert((2 * NSLOT + 2 * DESC_DEPTH + 2 * NRED) * 8 + 16 * MAX_CAT_INTS_PAD + 16 * NRED + 32 + 224 <= 1024, "control region");
+constexpr unsigned SPIN_LIMIT = 1u << 24;  // bounded waits (default poll limit); then an error status, never a hang
 constexpr int MAX_CAT = 8;
 
 enum Epi : int { EPI_SIGMA = 0, EPI_SWIGLU = 1, EPI_NONE = 2 };
@@ -130,6 +130,8 @@ struct StreamDev {
   int early_flag, early_items;  // slots (relative to SY_DEP, outside the zeroed range): flag, item count;
                                 // early_flag + 2: flag that the rest of the work list exists
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
+  unsigned spin_limit;         // polls after which a bounded wait gives up (SPIN_LIMIT; lower only in failure tests)
+  int withhold;                // failure tests: bit 0 = the routing tail raises no hand-over flag
   // activations between stages, bf16 planes ([rows, width] each)
   __nv_bfloat16 *xh, *xl;      // tokens split (fp32 activations only; bf16 tokens are read in place)
   __nv_bfloat16 *GUh, *GUl, *Yh, *Yl, *Zh, *Zl, *Yshh, *Yshl;
@@ -202,9 +204,13 @@ static __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t par
 // Bounded wait.  Returns false if the limit expired or the CTA was told to stop.
 // `sleep_ns` > 0 backs off between polls: used by the roles whose wake-up latency is not critical,
 // so that their polling does not compete with the consumers for issue slots.
+// abort_flag points at the CTA's control words: [0] the abort flag, [CTL_LIMIT] the poll limit of
+// this launch (SPIN_LIMIT unless a test lowered it).
+constexpr int CTL_LIMIT = 4;
 static __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                                  unsigned sleep_ns = 0) {
-  for (unsigned it = 0; it < SPIN_LIMIT; ++it) {
+  const unsigned limit = (unsigned)abort_flag[CTL_LIMIT];
+  for (unsigned it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 1023u) == 1023u && *abort_flag) return false;
@@ -663,7 +669,8 @@ static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, 
     // a dependent load; it is cleared again by the next step's router kernel
     const int items = (carry <= P.max_segs) ? carry * ips : 0;
     P.sync[SY_DEP + P.early_items] = items;
-    st_release(P.sync + SY_DEP + P.early_flag, items + 1);
+    if (!(P.withhold & 1))  // (a failure test withholds the flag: the streaming kernel's bounded wait must expire)
+      st_release(P.sync + SY_DEP + P.early_flag, items + 1);
   }
 }
 
@@ -753,7 +760,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   if (L.sigma == DEAMOE_SIGMA_RMSNORM) {  // sums of squares of this step's G, U and Z vectors
     const int ngu = 2 * B * (L.k < L.m ? L.k : L.m), nz = B * L.k;
 #pragma unroll 1
-    for (int i = tid; i < ngu + nz; i += FINISH_THREADS) (i < ngu ? L.ss_gu[i] : L.ss_z[i - ngu]) = 0.f;
+    for (int i = tid; i < ngu + nz; i += FINISH_THREADS) (i < ngu ? L.ss_gu[i] : L.ss_z[i - ngu]) = 0ull;
   }
   const bool regs_ok = topk_in_registers(L);
   if (topk_warps == 0) {  // the selection was made by k_topk_tokens
@@ -796,7 +803,8 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     // layer the streaming kernel has finished the first stage by then and would wait)
     __threadfence();  // every thread's records, before the flag
     __syncthreads();
-    if (tid == 0) st_release(P.sync + SY_DEP + P.early_flag + 2, 1);  // cleared again by the next step's router kernel
+    if (tid == 0 && !(P.withhold & 1))
+      st_release(P.sync + SY_DEP + P.early_flag + 2, 1);  // cleared again by the next step's router kernel
   }
   __syncthreads();
   TS_MIN(L, 15);
@@ -910,9 +918,10 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
   uint64_t* red_empty = red_full + NRED;
   int* cat_tab = reinterpret_cast<int*>(red_empty + NRED);             // 4 * MAX_CAT ints
   int* red_info = cat_tab + 4 * MAX_CAT;                               // NRED x {e | tile0 << 8, q, T, 0}
-  volatile int* ctl = red_info + 4 * NRED;  // [0] abort, [1] closed, [2] items produced, [3] items completed
+  volatile int* ctl = red_info + 4 * NRED;  // [0] abort, [1] closed, [2] items produced, [3] items completed, [4] poll limit
   volatile int* abort_flag = ctl;
-  unsigned char* seg_stage = reinterpret_cast<unsigned char*>(red_info + 4 * NRED + 4);  // one Seg, planner only
+  unsigned char* seg_stage = reinterpret_cast<unsigned char*>(red_info + 4 * NRED + 8);  // one Seg, planner only
+  const unsigned spin_limit = P.spin_limit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int32_t* sy = P.sync;
@@ -920,7 +929,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     for (int s = 0; s < NSLOT; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], CONSUMER_WARPS); }
     for (int s = 0; s < DESC_DEPTH; ++s) { mbar_init(&dq_full[s], 1); mbar_init(&dq_empty[s], 1); }
     for (int s = 0; s < NRED; ++s) { mbar_init(&red_full[s], CONSUMER_WARPS); mbar_init(&red_empty[s], 1); }
-    ctl[0] = 0; ctl[1] = 0; ctl[2] = 0; ctl[3] = 0;
+    ctl[0] = 0; ctl[1] = 0; ctl[2] = 0; ctl[3] = 0; ctl[CTL_LIMIT] = (int)spin_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -962,7 +971,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         unsigned spins = 0;
         while (ld_acquire(P.sync + SY_DEP + dep_idx) < dep_target) {
           __nanosleep(32);
-          if (++spins > SPIN_LIMIT / 16 || *abort_flag) { seen = false; break; }
+          if (++spins > spin_limit / 16 || *abort_flag) { seen = false; break; }
         }
         if (seen) {
           __threadfence_block();  // what the acquire made visible, before the word the issue warp polls
@@ -1110,7 +1119,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
           unsigned spins = 0;
           while (queued - ctl[3] >= CLAIM_AHEAD) {  // throttle: stay close to what is actually finished
             __nanosleep(100);
-            if (++spins > SPIN_LIMIT / 16 || *abort_flag) break;
+            if (++spins > spin_limit / 16 || *abort_flag) break;
           }
           item = claim_base + atomicAdd(P.sync + SY_CLAIM, 1);
         }
@@ -1189,7 +1198,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         int fv;
         while ((fv = ld_acquire(flag)) == 0) {
           __nanosleep(64);
-          if (++spins > SPIN_LIMIT / 16 || *abort_flag) { seen = false; break; }
+          if (++spins > spin_limit / 16 || *abort_flag) { seen = false; break; }
         }
         n1 = seen ? fv - 1 : -1;  // the flag is the first stage's item count + 1
       }
@@ -1215,7 +1224,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         unsigned spins = 0;
         while (ld_acquire(flag) == 0) {
           __nanosleep(64);
-          if (++spins > SPIN_LIMIT / 16 || *abort_flag) { ok = false; break; }
+          if (++spins > spin_limit / 16 || *abort_flag) { ok = false; break; }
         }
       }
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -1402,11 +1411,18 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       if (progressed) {
         idle = 0;
       } else {
-        if (++idle > SPIN_LIMIT || *abort_flag) { ok = false; break; }
+        if (++idle > spin_limit || *abort_flag) { ok = false; break; }
         __nanosleep(20);
       }
     }
     if (!ok && lane == 0) { L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT; *abort_flag = 1; }
+    if (!ok) {
+      // giving up: the bulk copies this warp has issued may still be in flight towards the ring;
+      // stay (bounded: about 64 us, many times a copy's latency) until they have landed, so that
+      // the CTA's shared memory is not released under them
+#pragma unroll 1
+      for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
 #ifdef DEAMOE_TRACE
     tr[TR_PTOTAL] = clock64() - tp0;
     if (lane == 0 && P.trace)
@@ -1451,7 +1467,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
           pend = 0;
           continue;
         }
-        if ((ctl[1] && n >= ctl[2]) || *abort_flag || ++idle > SPIN_LIMIT) break;
+        if ((ctl[1] && n >= ctl[2]) || *abort_flag || ++idle > spin_limit) break;
         __nanosleep(32);
         continue;
       }
@@ -1504,8 +1520,8 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
 #pragma unroll
           for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
           if ((lane & 15) == 0 && x < count && s < T) {
-            if (stage == ST_S1) atomicAdd(L.ss_gu + (size_t)(out_row0 + s) * 2 + (row >= L.f ? 1 : 0), sq);
-            else atomicAdd(L.ss_z + (out_row0 + s), sq);
+            if (stage == ST_S1) atomicAdd(L.ss_gu + (size_t)(out_row0 + s) * 2 + (row >= L.f ? 1 : 0), ss_fixed(sq));
+            else atomicAdd(L.ss_z + (out_row0 + s), ss_fixed(sq));
           }
         }
         if (live) {
@@ -1513,14 +1529,14 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
           if (epi == EPI_SIGMA) r = sigma_f(L.sigma, v0);
           else if (epi == EPI_SWIGLU) {
             if (rms && stage == ST_S2) {  // inputs were the un-normalised G and U of this pair's row
-              const float* ss = L.ss_gu + (size_t)sg->rows16[s] * 2;
-              v0 *= rms_scale(__ldcg(ss), L.f);
-              v1 *= rms_scale(__ldcg(ss + 1), L.f);
+              const unsigned long long* ss = L.ss_gu + (size_t)sg->rows16[s] * 2;
+              v0 *= rms_scale_fixed(__ldcg(ss), L.f);
+              v1 *= rms_scale_fixed(__ldcg(ss + 1), L.f);
             }
             r = silu_f(v0) * v1;
           } else {
             r = v0;
-            if (rms && stage == ST_S4) r *= rms_scale(__ldcg(L.ss_z + sg->rows16[s]), L.f);
+            if (rms && stage == ST_S4) r *= rms_scale_fixed(__ldcg(L.ss_z + sg->rows16[s]), L.f);
           }
           const size_t o = (size_t)(out_row0 + s) * out_stride + row;
           if (outf) {
@@ -1791,6 +1807,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   d.claim_items = (schedule == DEAMOE_SCHED_FUSED && (L.vanilla || L.r > 0)) ? 1 : 0;
   d.early_flag = d.n_dep + 1; d.early_items = d.n_dep + 2;  // the allocation has 8 spare counters
   d.planes = (L.adt == DEAMOE_F32) ? 2 : 1;
+  d.spin_limit = SPIN_LIMIT; d.withhold = 0;
   {
     // activation planes between stages
     const size_t tdmax = (size_t)MB * (L.k < L.m ? L.k : L.m), pmax = (size_t)MB * L.k;
@@ -1989,6 +2006,18 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
   }
   if (p.ev1) { cudaEventRecord(p.ev1, s); p.ev_recorded = 1; }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+// Failure tests: lower the poll limit of every bounded wait and / or withhold a hand-over.
+// spin_limit 0 restores the default.  Returns false if the plan cannot honour `withhold`.
+bool stream_set_failure_test(StreamPlan& p, unsigned spin_limit, int withhold) {
+  if ((withhold & 1) && !p.dev.early) return false;   // only the fused schedule hands over through flags
+  if ((withhold & 2) && !p.dense) return false;
+  const unsigned lim = spin_limit ? spin_limit : SPIN_LIMIT;
+  p.dev.spin_limit = lim; p.dev.withhold = withhold & 1;
+  p.dev_dense.spin_limit = lim; p.dev_dense.withhold = 0;
+  if (p.dense) dense_set_failure_test(*p.dense, spin_limit, (withhold & 2) ? 1 : 0);
+  return true;
 }
 
 cudaError_t stream_profile_enable(StreamPlan& p, bool on) {

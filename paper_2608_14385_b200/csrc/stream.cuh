@@ -29,6 +29,11 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
 // Enqueue all stages of one step.  Returns the number of kernels launched or -1.
 int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
 
+// Failure-detection tests: poll limit of the bounded waits (0 = default) and withheld hand-overs
+// (bit 0: the routing tail raises no flag for the fused streaming kernel; bit 1: the dense kernel's
+// copy role issues nothing).  False if the plan has no such hand-over.
+bool stream_set_failure_test(StreamPlan& p, unsigned spin_limit, int withhold);
+
 // Event pair around the streaming launches of stream_forward (measurement aid).
 cudaError_t stream_profile_enable(StreamPlan& p, bool on);
 cudaError_t stream_profile_last_ms(StreamPlan& p, float* ms);

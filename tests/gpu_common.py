@@ -46,6 +46,23 @@ def check_routing(shape, layer, w, tokens, B, require_guard=True):
     return want, bk
 
 
+def deep_rows(count):
+    """Row chooser for run_case: the `count` tokens that sit deepest in a department's token list
+    X^j (position 8 and beyond is the second 8-token pass of the streaming kernel's tiles, position 16
+    and beyond a second token group), always with the first and the last token of the batch."""
+    def choose(want_r, bk):
+        B = want_r["idx"].shape[0]
+        depth = np.zeros(B, np.int64)
+        off = bk["dept_off"]
+        for j in range(len(off) - 1):
+            toks = bk["dept_tok"][off[j]:off[j + 1]]
+            depth[toks] = np.maximum(depth[toks], np.arange(len(toks)))
+        order = sorted(range(B), key=lambda t: (-depth[t], t))
+        rows = sorted(set(order[:max(0, count - 2)]) | {0, B - 1})
+        return rows, int(depth[rows].max())
+    return choose
+
+
 def run_case(shape, B, seed=0, schedule=binding.SCHED_AUTO, vanilla=False, rows=None, max_batch=None,
              weights=None, tokens=None, layer=None, require_guard=True):
     """Build (or reuse) a layer on cuda:0, run one forward, compare with the oracle.
@@ -70,6 +87,9 @@ def run_case(shape, B, seed=0, schedule=binding.SCHED_AUTO, vanilla=False, rows=
         experts = {int(i) for i in np.nonzero(np.diff(bk["expert_off"]))[0]}
         assert st["active_dept"] == len(depts) and st["active_expert"] == len(experts)
         assert st["token_dept_pairs"] == int(bk["dept_off"][-1])
+        deepest = None
+        if callable(rows):
+            rows, deepest = rows(want_r, bk)
         if rows is not None:
             sel = want_r["idx"][rows].reshape(-1)
             experts_needed = {int(i) for i in sel}
@@ -85,7 +105,8 @@ def run_case(shape, B, seed=0, schedule=binding.SCHED_AUTO, vanilla=False, rows=
         ok, err, bound = within_tolerance(got[r], want["out"][r])
         assert ok, f"max|diff| {err:.3e} > {bound:.3e}"
         assert np.abs(want["out"][r]).max() > 0
-        return {"out": out, "stats": st, "err": err, "bound": bound, "want": want, "layer": layer}
+        return {"out": out, "stats": st, "err": err, "bound": bound, "want": want, "layer": layer, "rows": r,
+                "deepest": deepest}
     finally:
         if own:
             layer.close()

@@ -49,3 +49,19 @@ def test_status_strings_and_host_side_argument_errors():
         setattr(cfg, field, bad)
         assert L.deamoe_layer_create(ctypes.byref(cfg), ctypes.byref(w), None, ctypes.byref(out)) == binding.ERR_INVALID_ARG
         setattr(cfg, field, good)
+
+
+def test_misaligned_device_pointers_are_argument_errors_without_a_gpu():
+    """deamoe_route_static checks its arguments before it touches CUDA: pointers that are not
+    aligned for the kernels' 16-byte accesses come back as INVALID_ARG and nothing is enqueued (the
+    same check in deamoe_route / deamoe_forward needs a layer object and runs in the GPU tests)."""
+    L = binding.lib()
+    p = ctypes.c_void_p
+
+    def call(router, tokens, idx, w):
+        return L.deamoe_route_static(None, p(router), p(tokens), 4, 4, 1024, 2, 1, 1.0, 4, p(idx), p(w))
+    assert call(4096 + 4, 8192, 12288, 16384) == binding.ERR_INVALID_ARG      # router
+    assert call(4096, 8192 + 8, 12288, 16384) == binding.ERR_INVALID_ARG      # tokens
+    assert call(4096, 8192, 12288 + 2, 16384) == binding.ERR_INVALID_ARG      # topk_idx
+    assert call(4096, 8192, 12288, 16384 + 1) == binding.ERR_INVALID_ARG      # topk_w
+    assert binding.ERR_INTERNAL == 7 and binding.status_string(binding.ERR_INTERNAL) not in ("", "ok", "unknown status")

@@ -150,14 +150,6 @@ def test_layers_of_both_schedules_enqueued_back_to_back():
             layer.close()
 
 
-@pytest.mark.parametrize("B,rows", [(64, [5, 63]), (128, [0, 77, 127])])
-def test_dense_schedule_deepseek_v3_full_size_sampled_rows(B, rows):
-    """The benchmark's layer at full size in the configuration `bench.py --mode large` times: created
-    with AUTO for 128 tokens, which takes the dense schedule at these batch sizes.  Routing and token
-    lists are compared for the whole batch, output values on sampled token rows."""
-    run_case(synth.DSV3, B, seed=0, rows=rows, max_batch=128)
-
-
 def test_7b_class_layer_dense_every_element():
     """7B-class layer (h 4096, f 1408: a stacked gate / up tile holds rows of both matrices), 64
     tokens, every output element against the oracle."""
