@@ -13,8 +13,10 @@ of its active departments and experts, far more than the L2 holds, and successiv
 different token batches (different routings).  A 256 MiB buffer is overwritten between steps to
 flush L2 (untimed).  Prints ONE JSON line.
 
-With N > 1 (torchrun) every rank runs an independent replica of the same layer on its own GPU --
-the path has no collective -- and the line reports the aggregate.
+With N > 1 every rank runs an independent replica of the same layer on its own GPU -- the path has
+no collective -- and the line reports the aggregate.  Under torchrun the ranks are already there
+(RANK / LOCAL_RANK / WORLD_SIZE in the environment); invoked plainly with --gpus N > 1 the script
+starts the N ranks itself (torchrun on 127.0.0.1) and passes its arguments through.
 """
 import argparse
 import json
@@ -94,6 +96,45 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def free_port():
+    import socket
+    sk = socket.socket()
+    sk.bind(("127.0.0.1", 0))
+    port = sk.getsockname()[1]
+    sk.close()
+    return port
+
+
+def spawn_ranks(n, argv):
+    """`python bench.py --gpus N` outside torchrun: start the N ranks (one per GPU) the way the driver
+    does, on 127.0.0.1, with this script's own arguments; NCCL's communicator log goes to stderr."""
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd, env=env)
+
+
+def selftest_cpu(args, rank, world):
+    """The multi-rank plumbing without a GPU: process group (gloo), barrier, max over ranks, aggregate."""
+    import torch
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        dist.barrier()
+    total_ms = max_over_ranks(10.0 * (rank + 1) * args.steps, dist, torch.device("cpu"))
+    us = us_per_layer_step(total_ms, args.steps, world)
+    if rank == 0:
+        print(json.dumps({"selftest": True, "metric": "us_per_step_deamoe_layer", "value": us, "unit": "us",
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3,
+                          "scaling": "weak", "slowest_rank_total_ms": total_ms}))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def max_over_ranks(value, dist=None, device=None):
     """The slowest rank's value (all ranks get it); identity without a process group."""
     if dist is None:
@@ -114,79 +155,106 @@ def pct(xs, q):
     return xs[min(len(xs) - 1, max(0, int(round(q * (len(xs) - 1)))))]
 
 
-def oracle_sample_seconds(shape, weights_fn, tokens, rows, vanilla=False, one_thread=None):
-    """Time the fp64 oracle (as it stands) on `rows` of this batch with all host cores."""
-    import numpy as np
+def workload_config(shape, B, schedule):
+    """The `config` object of the JSON line; both arms (the CUDA path and --impl reference) print the same."""
+    return {"workload": f"{shape.name}-shape DeaMoE layer, decode batch {B} (replica per GPU)",
+            "batch": B, "hidden": shape.hidden, "n_dept": shape.n_dept, "experts_per_dept": shape.experts_per_dept,
+            "ffn": shape.ffn, "priv": shape.priv, "top_k": shape.top_k, "n_shared": shape.n_shared,
+            "schedule": schedule, "l2": "256 MiB buffer overwritten between steps (untimed); "
+            "4 rotating token batches", "accumulate": "fp32"}
+
+
+class HostWeights:
+    """Host (numpy) copies of the synthetic layer's matrices for the oracle, generated unit by unit on
+    first use (any unit of the counter-based generator can be made alone) and kept."""
+
+    def __init__(self, shape, dev, router=None, shared=None):
+        import torch
+        from paper_2608_14385_b200 import synth
+        self.shape, self.dev, self.synth, self.torch = shape, dev, synth, torch
+        self.router = synth.to_numpy(router if router is not None else synth.make_router(shape, 0, dev))
+        self.shared = shared
+        self.cache = {}
+
+    def unit(self, name, u):
+        key = (name, u)
+        if key not in self.cache:
+            self.cache[key] = self.synth.to_numpy(self.synth.weight_slice(self.shape, name, u, 0, self.dev))
+        return self.cache[key]
+
+    def tables(self, depts, experts):
+        shape, synth, torch = self.shape, self.synth, self.torch
+        w = {"router": self.router}
+        for name in ("gate", "up", "down"):
+            tab = [None] * shape.n_dept
+            for j in depts:
+                tab[j] = self.unit(f"dept_{name}", j)
+            w[f"dept_{name}"] = tab
+            if shape.priv > 0:
+                tab = [None] * shape.n_expert
+                for i in experts:
+                    tab[i] = self.unit(f"priv_{name}", i)
+                w[f"priv_{name}"] = tab
+            if shape.n_shared:
+                key = f"shared_{name}"
+                if key not in self.cache:
+                    t = self.shared[key] if self.shared else synth.normal(
+                        (shape.shared_ffn, shape.hidden), synth.W_STD, 0, f"L0/{key}", self.dev,
+                        torch.bfloat16 if shape.weight_dtype else torch.float32)
+                    self.cache[key] = synth.to_numpy(t)
+                w[key] = self.cache[key]
+        return w
+
+
+def oracle_step_seconds(shape, host, tokens, threads, rows=None):
+    """Wall time of the fp64 oracle (as it stands) for ONE whole step on this batch: routing of all B
+    tokens once, then Eq. (4) / Eq. (3) for every token row (or only `rows`).  The weights it will touch
+    are fetched before the clock starts."""
     from oracle import ref
     from paper_2608_14385_b200 import synth
-    cores = ref.host_cores()
-    ref.set_threads(cores)
     cfg = ref.make_config(**shape.asdict())
-    router = synth.to_numpy(weights_fn("router", None))
     tok = synth.to_numpy(tokens)
-    r = ref.route(cfg, router, tok)
-    sel = r["idx"][rows].reshape(-1)
-    experts = sorted({int(i) for i in sel})
-    depts = sorted({int(i) // shape.experts_per_dept for i in sel})
-    m, n = shape.n_dept, shape.n_expert
-    w = {"router": router}
-    units = experts if vanilla else depts
-    for name in ("gate", "up", "down"):
-        tab = [None] * (n if vanilla else m)
-        for u in units:
-            tab[u] = synth.to_numpy(weights_fn(f"dept_{name}", u))
-        w[f"dept_{name}"] = tab
-        if not vanilla and shape.priv > 0:
-            tab = [None] * n
-            for i in experts:
-                tab[i] = synth.to_numpy(weights_fn(f"priv_{name}", i))
-            w[f"priv_{name}"] = tab
-        if shape.n_shared:
-            w[f"shared_{name}"] = synth.to_numpy(weights_fn(f"shared_{name}", None))
-    fwd = ref.vanilla_forward if vanilla else ref.deamoe_forward
+    ref.set_threads(ref.host_cores())
+    sel = ref.route(cfg, host.router, tok)["idx"]
+    if rows is not None:
+        sel = sel[rows]
+    experts = sorted({int(i) for i in sel.reshape(-1)})
+    depts = sorted({i // shape.experts_per_dept for i in experts})
+    w = host.tables(depts, experts)
+    ref.set_threads(threads)
     t0 = time.perf_counter()
-    fwd(cfg, w, tok, rows=rows)
-    t_all = time.perf_counter() - t0
-    if one_thread is not None:      # the same sample once more on a single core
-        ref.set_threads(1)
-        t0 = time.perf_counter()
-        fwd(cfg, w, tok, rows=rows)
-        one_thread.append(time.perf_counter() - t0)
-        ref.set_threads(cores)
-    return t_all, cores
+    ref.deamoe_forward(cfg, w, tok, rows=rows)
+    dt = time.perf_counter() - t0
+    ref.set_threads(ref.host_cores())
+    return dt
 
 
 def run_reference(args, shape, rank, world):
-    """--impl reference: the oracle on the host cores, rank 0 only."""
+    """--impl reference: the oracle on the host cores, rank 0 only.  Every step is one whole layer step
+    (all B token rows, routing once), so value x steps is the time the run really spent in the oracle."""
     if rank != 0:
         return
     import torch
+    from oracle import ref
     from paper_2608_14385_b200 import synth
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
     B = args.batch
-
-    def wfn(name, unit):
-        if name == "router":
-            return synth.make_router(shape, 0, dev)
-        if unit is None:
-            return synth.normal((shape.shared_ffn, shape.hidden), synth.W_STD, 0, f"L0/{name}", dev,
-                                torch.bfloat16 if shape.weight_dtype else torch.float32)
-        return synth.weight_slice(shape, name, unit, 0, dev)
-    rows = [0]
+    cores = ref.host_cores()
+    host = HostWeights(shape, dev)
     times = []
     for step in range(args.warmup + args.steps):
         tokens = synth.make_tokens(shape, B, 100 + step % 4, dev)
-        sec, cores = oracle_sample_seconds(shape, wfn, tokens, rows)
+        sec = oracle_step_seconds(shape, host, tokens, cores)
         if step >= args.warmup:
-            times.append(sec * B / len(rows))
+            times.append(sec)
     us = statistics.mean(times) * 1e6
     line = {
         "impl": "reference", "metric": "us_per_step_deamoe_layer", "value": us, "unit": "us", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{shape.name}-shape DeaMoE layer, decode batch {B}", "batch": B},
+        "config": workload_config(shape, B, args.schedule),
         "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
-                         "sample": f"{len(rows)} of {B} token rows per step, time scaled by {B}/{len(rows)}"},
+                         "sample": f"every step: all {B} token rows of one layer step (routing once), fp64"},
         "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -195,6 +263,26 @@ def run_reference(args, shape, rank, world):
 # dram__bytes_read.sum + dram__bytes_write.sum of k_stream divided by its algorithmic bytes, from
 # the committed ncu capture (profiles/k_stream_dsv3-mini_b4.md)
 DRAM_TRAFFIC_RATIO = 1.001
+
+
+def read_only_ceiling(binding, torch, dev, gib=4, reps=6):
+    """GB/s of a plain vectorised read of a `gib` GiB buffer (the library's deamoe_probe_read kernel),
+    best of `reps`, CUDA events: what a read-only HBM stream reaches on this GPU, measured in this run."""
+    buf = torch.empty(gib << 30, dtype=torch.uint8, device=dev)
+    buf.fill_(1)
+    sink = torch.zeros(binding.PROBE_BLOCKS, dtype=torch.int32, device=dev)
+    best = 0.0
+    for i in range(reps + 2):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        binding.probe_read(buf, sink)
+        b.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            best = max(best, buf.numel() / (a.elapsed_time(b) * 1e-3) / 1e9)
+    del buf
+    torch.cuda.empty_cache()
+    return best
 
 
 def stream_kernel_ms(layer, batches, steps, flush, torch):
@@ -248,7 +336,13 @@ def main():
                     help="layer: the contract line (default); locality: routing-locality sweep on the DeepSeek-V3 "
                          "shape; stack: 32 consecutive 7B-class layers with a residual add, DeaMoE vs vanilla; "
                          "large: 32-128 tokens on the DeepSeek-V3 shape, streaming vs dense (tcgen05) schedule")
+    ap.add_argument("--selftest-cpu", action="store_true",
+                    help="no GPU work: every rank reports a fixed made-up duration through the same rank start-up, "
+                         "barrier and max-over-ranks code (gloo); used by the CPU tests of the multi-rank path")
     args = ap.parse_args()
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
 
     from paper_2608_14385_b200 import synth
     shape = synth.SHAPES[args.shape]
@@ -257,6 +351,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, shape, rank, world)
+        return
+    if args.selftest_cpu:
+        selftest_cpu(args, rank, world)
         return
 
     import torch
@@ -300,6 +397,7 @@ def main():
         layer.forward(b)
         ubytes.append(layer.stats()["unique_weight_bytes"])
 
+    read_gbs = read_only_ceiling(binding, torch, dev)
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.5)      # nvidia-smi needs a moment before its first sample
@@ -328,14 +426,20 @@ def main():
         achieved = alg / (k_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": alg * DRAM_TRAFFIC_RATIO,
-                "traffic_note": "dram read+write bytes of k_stream from the ncu capture in profiles/ "
-                                "(smaller layer of the same matrices), scaled by algorithmic bytes",
+                "traffic_note": "ESTIMATE: dram read+write bytes of k_stream from the ncu capture in profiles/ "
+                                "(smaller layer of the same matrices), scaled by algorithmic bytes; L2 prefetches of "
+                                "departments that turn out inactive (at most 512 KB per thread block) not included",
                 "kernel": "k_stream (the weight-streaming launch(es) of one step)",
-                "kernel_ms": k_ms, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg}
+                "kernel_ms": k_ms, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg,
+                "read_only_ceiling_gbs": read_gbs,
+                "read_only_ceiling_note": "plain 16-byte-load read of 4 GiB by deamoe_probe_read, best of 6, this run; "
+                                          "`peak` is a read+write copy figure, which a read-only stream may exceed",
+                "frac_of_read_only_ceiling": achieved / read_gbs if read_gbs else None,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
         if args.schedule == "dense" or (args.schedule == "auto" and B >= 48):
             # dense schedule: the pair of events brackets k_dense, k_stream, k_dense (ordinary launches, back to back)
             roof["kernel"] = "k_dense + k_stream + k_dense (the three weight-streaming launches of a dense step)"
-            roof["traffic_note"] = ("dram read+write bytes from the ncu captures of k_stream (1.001 x algorithmic) and "
+            roof["traffic_note"] = ("ESTIMATE: dram read+write bytes from the ncu captures of k_stream (1.001 x algorithmic) and "
                                     "k_dense (1.02 x) in profiles/, scaled by algorithmic bytes")
             roof["traffic"] = alg * 1.01
     else:
@@ -364,11 +468,7 @@ def main():
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": us_per_step / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.weight_dtype else "f32",
         "data": "synthetic",
-        "config": {"workload": f"{shape.name}-shape DeaMoE layer, decode batch {B} (replica per GPU)",
-                   "batch": B, "hidden": shape.hidden, "n_dept": shape.n_dept, "experts_per_dept": shape.experts_per_dept,
-                   "ffn": shape.ffn, "priv": shape.priv, "top_k": shape.top_k, "n_shared": shape.n_shared,
-                   "schedule": args.schedule, "l2": "256 MiB buffer overwritten between steps (untimed); "
-                   "4 rotating token batches", "accumulate": "fp32"},
+        "config": workload_config(shape, B, args.schedule),
         "us_per_step_p10_p50_p90": [pct(times_ms, 0.1) * 1e3, pct(times_ms, 0.5) * 1e3, pct(times_ms, 0.9) * 1e3],
         "hbm_gbs_on_unique_bytes": {"mean": statistics.mean(gbs), "p50": pct(gbs, 0.5),
                                     "frac_of_measured_peak": statistics.mean(gbs) / peak,
@@ -387,18 +487,23 @@ def main():
         else:
             line["sweep"] = sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev)
     if rank == 0 and not args.no_cpu:
-        def wfn(name, unit):
-            if name == "router":
-                return router
-            if unit is None:
-                return shared[name]
-            return synth.weight_slice(shape, name, unit, 0, dev)
-        one = []
-        sec, cores = oracle_sample_seconds(shape, wfn, batches[0], [0], one_thread=one)
-        line["cpu_baseline"] = {"value": sec * B * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-                                "sample": f"1 of {B} token rows of one step, time scaled by {B}",
-                                "value_one_core": one[0] * B * 1e6}
-    layer.close()
+        from oracle import ref
+        host = HostWeights(shape, dev, router=router, shared=shared)
+        cores = ref.host_cores()
+        sec = oracle_step_seconds(shape, host, batches[0], cores)
+        few = list(range(min(B, 2)))
+        one = oracle_step_seconds(shape, host, batches[0], 1, rows=few)
+        line["cpu_baseline"] = {"value": sec * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+                                "sample": f"one whole layer step: all {B} token rows, routing once, fp64",
+                                "one_core_us_per_token_row": one * 1e6 / len(few),
+                                "one_core_sample": f"{len(few)} of {B} token rows on one core (not scaled)"}
+    if rank == 0 and not args.no_sweep and shape.name == "dsv3":
+        layer.close()
+        layer = None
+        torch.cuda.empty_cache()
+        line["other_workloads"] = other_workloads(args, sched, peak, torch, dev, flush)
+    if layer is not None:
+        layer.close()
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
@@ -406,15 +511,14 @@ def main():
         dist.destroy_process_group()
 
 
-def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev):
+def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev, batches_list=(4, 8, 16, 32, 64), steps=None):
     """The paper's own DeepSeek-V3-matched DeaMoE row (8 x 108 experts, square private matrices, top-10 in
     at most 5 departments) against the model it was matched to: a standard 256-expert top-8 MoE layer of
     the DeepSeek-V3 shape (no shared expert, as in the paper's Table 1 accounting), same token counts.
     Reports time, unique bytes, their ratio (the quantity of the paper's Fig. 2) and the speed-up."""
     import dataclasses
     from paper_2608_14385_b200 import binding, synth
-    batches_list = [4, 8, 16, 32, 64]
-    steps = max(10, args.steps // 2)
+    steps = steps or max(10, args.steps // 2)
     res = {}
     for B in batches_list:
         bs = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(4)]
@@ -503,17 +607,21 @@ def locality_sweep(args, sched, peak, torch, dev):
             "rows": rows}
 
 
-def stack_bench(args, sched, peak, torch, dev):
+def stack_bench(args, sched, peak, torch, dev, steps=None):
     """32 consecutive 7B-class layers, x <- x + Layer_l(x), every layer with its own seeded weights;
     MoE time per decode step of the DeaMoE stack and of the vanilla-MoE stack at B = 1 and 8.  The stacks
-    (6.6 GB and 17.7 GB) are far larger than L2, so no flush is needed between steps.  The 128
-    kernels of a step are enqueued back to back; a step is timed by one pair of events."""
+    (6.6 GB and 17.7 GB) are far larger than L2, so no flush is needed between steps.  A step (the
+    128 kernels of the 32 layers) is captured once in a CUDA graph and timed as ONE graph launch per
+    step, the way a serving runtime replays a decode step (Section 5 of the paper); the same step
+    enqueued kernel by kernel is reported beside it."""
     import dataclasses
     from paper_2608_14385_b200 import binding, synth
     shape = dataclasses.replace(synth.MOE7B, residual=1)
     n_layers = 32
+    steps = steps or max(10, args.steps // 2)
     out = {"metric": "us_per_decode_step_moe_stack", "unit": "us", "layers": n_layers, "shape": shape.name,
            "data": "synthetic", "config": {"workload": "stack of 32 7B-class layers with residual add",
+                                           "launch": "one CUDA-graph replay per step",
                                            "l2": "stack larger than L2, no flush"}, "rows": []}
     res = {}
     for vanilla in (False, True):
@@ -527,41 +635,88 @@ def stack_bench(args, sched, peak, torch, dev):
             # tokens scaled by 1/16: with N(0,1) tokens the vanilla stack (gain ~0.6 per layer, quadratic in |x|)
             # overflows bf16 within 32 layers without a normalisation; routing (an arg-max) is scale-invariant
             xs = [(synth.make_tokens(shape, B, 300 + i, dev).float() / 16).to(torch.bfloat16) for i in range(4)]
+            x_in = xs[0].clone()
             bufs = [torch.empty_like(xs[0]), torch.empty_like(xs[0])]
 
-            def step(x):
-                cur = x
+            def step():
+                cur = x_in
                 for l, layer in enumerate(layers):      # enqueued back to back, no host synchronisation
                     layer.forward(cur, bufs[l & 1])
                     cur = bufs[l & 1]
                 return cur
             for i in range(3):
-                step(xs[i % 4])
-            steps = max(10, args.steps // 2)
-            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+                x_in.copy_(xs[i % 4])
+                step()
             torch.cuda.synchronize()
-            for i in range(steps):
-                ev[i][0].record()
-                step(xs[i % 4])
-                ev[i][1].record()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
             torch.cuda.synchronize()
-            t = [a.elapsed_time(b) for a, b in ev]
+
+            def timed(run):
+                ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+                for i in range(2):
+                    x_in.copy_(xs[i % 4])
+                    run()
+                torch.cuda.synchronize()
+                for i in range(steps):
+                    x_in.copy_(xs[i % 4])
+                    ev[i][0].record()
+                    run()
+                    ev[i][1].record()
+                torch.cuda.synchronize()
+                return pct([a.elapsed_time(b) for a, b in ev], 0.5) * 1e3
+            t_graph = timed(graph.replay)
+            t_enq = timed(step)
             ub = 0
             for layer in layers:
                 ub += layer.stats()["unique_weight_bytes"]
+            ok = all(layer.stats()["device_status"] == 0 for layer in layers)
             finite = bool(torch.isfinite(bufs[(n_layers - 1) & 1].float()).all())
-            res[(vanilla, B)] = (pct(t, 0.5) * 1e3, ub / 1e6, finite)
+            res[(vanilla, B)] = (t_graph, ub / 1e6, finite and ok, t_enq)
+            del graph
         for layer in layers:
             layer.close()
         del layers
         torch.cuda.empty_cache()
     for B in (1, 8):
-        d_us, d_mb, d_fin = res[(False, B)]
-        v_us, v_mb, v_fin = res[(True, B)]
+        d_us, d_mb, d_fin, d_enq = res[(False, B)]
+        v_us, v_mb, v_fin, v_enq = res[(True, B)]
         out["rows"].append({"batch": B, "deamoe_us": d_us, "deamoe_mb_last_step": d_mb, "deamoe_gbs": d_mb / d_us * 1e3,
                             "vanilla_us": v_us, "vanilla_mb_last_step": v_mb, "vanilla_gbs": v_mb / v_us * 1e3,
                             "speedup_vs_vanilla": v_us / d_us, "byte_ratio_vanilla_over_deamoe": v_mb / d_mb,
-                            "deamoe_us_per_layer": d_us / n_layers, "outputs_finite": d_fin and v_fin})
+                            "deamoe_us_per_layer": d_us / n_layers, "outputs_finite_and_status_ok": d_fin and v_fin,
+                            "deamoe_us_enqueued_kernel_by_kernel": d_enq, "vanilla_us_enqueued_kernel_by_kernel": v_enq})
+    return out
+
+
+def other_workloads(args, sched, peak, torch, dev, flush):
+    """Compact rows for the other benchmark configurations, run after the headline so that one default
+    invocation measures them all: one 7B-class layer (configuration 2), the stack of 32 such layers
+    (configuration 5) and the paper's own DeepSeek-V3-matched row of Table 1 with group-limited routing."""
+    from paper_2608_14385_b200 import binding, synth
+    t0 = time.time()
+    out = {}
+    shape = synth.MOE7B
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    layer = binding.Layer(shape, w, 16, sched)
+    router = w["router"]
+    del w
+    rows = sweep(args, shape, layer, router, {}, flush, sched, peak, torch, dev, steps=12)
+    layer.close()
+    torch.cuda.empty_cache()
+    out["7b_layer"] = {"workload": "7b-shape DeaMoE layer vs vanilla MoE, L2 overwritten between steps", "rows": rows}
+    out["stack_32x7b"] = stack_bench(args, sched, peak, torch, dev, steps=10)
+    shape = synth.DSV3_PAPER
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    layer = binding.Layer(shape, w, 64, sched)
+    del w
+    torch.cuda.empty_cache()
+    out["dsv3_paper_row"] = paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev, batches_list=(4, 16, 64),
+                                            steps=10)
+    layer.close()
+    torch.cuda.empty_cache()
+    out["seconds"] = time.time() - t0
     return out
 
 
@@ -620,12 +775,12 @@ def large_batch_sweep(args, sched, peak, torch, dev):
             "l2": "256 MiB buffer overwritten between steps", "peak_gbs_measured": peak, "rows": rows}
 
 
-def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev):
+def sweep(args, shape, layer, router, shared, flush, sched, peak, torch, dev, steps=None):
     """DeaMoE layer and the in-library vanilla MoE at the same shape over the batch range."""
     from paper_2608_14385_b200 import binding, synth
     out = []
     batches_list = [1, 2, 4, 8, 16, 32, 64, 128] if shape.name == "dsv3" else [1, 4, 16]
-    steps = max(10, args.steps // 2)
+    steps = steps or max(10, args.steps // 2)
     res = {}
     for B in batches_list:
         bs = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(4)]

@@ -266,6 +266,17 @@ deamoe_status_t deamoe_route_static(void *cuda_stream, const float *router, cons
                                     float *topk_w);
 
 /*
+ * Measurement aid.  (The paper has no counterpart.)  Enqueues one kernel that reads `bytes` bytes
+ * of `buf` (DEVICE, 16-byte aligned; a trailing remainder of fewer than 16 bytes is ignored) exactly
+ * once with plain 16-byte loads and writes one word per thread block to sink (DEVICE,
+ * DEAMOE_PROBE_BLOCKS words, caller-owned).  Timed by the caller with events on a buffer much
+ * larger than the L2, it gives the read-only HBM bandwidth of this GPU: the ceiling a
+ * weight-streaming step is set against (the usual copy benchmark reads AND writes).  No layer needed.
+ */
+#define DEAMOE_PROBE_BLOCKS 2368
+deamoe_status_t deamoe_probe_read(void *cuda_stream, const void *buf, uint64_t bytes, uint32_t *sink);
+
+/*
  * Failure-detection test aid.  (The paper has no counterpart.)  Every device-side wait of the
  * library is bounded: after a number of polls it gives up, the kernel records DEAMOE_ERR_TIMEOUT
  * in the device status word, waits (bounded) for its copies in flight, frees its tensor memory

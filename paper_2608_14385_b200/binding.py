@@ -21,7 +21,7 @@ SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4
 # every symbol include/deamoe.h declares
 SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",
            "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_get_routing",
-           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_route_static", "deamoe_failure_test",
+           "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_route_static", "deamoe_failure_test", "deamoe_probe_read",
            "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
 
 
@@ -75,6 +75,7 @@ def lib():
         L.deamoe_route_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
         L.deamoe_failure_test.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.deamoe_probe_read.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         L.deamoe_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.deamoe_profile_last_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
         _lib = L
@@ -103,6 +104,17 @@ def make_config(shape, max_batch, schedule=SCHED_AUTO):
 
 
 STATIC_ROUTE_SCRATCH_BYTES = 4 << 20
+PROBE_BLOCKS = 2368
+
+
+def probe_read(buf, sink):
+    """Enqueue one plain read of the CUDA tensor `buf` (deamoe_probe_read); sink: int32 CUDA tensor of
+    at least PROBE_BLOCKS elements.  The caller times it with events."""
+    assert buf.is_cuda and buf.is_contiguous() and sink.is_cuda and sink.numel() >= PROBE_BLOCKS
+    st = lib().deamoe_probe_read(_stream(), _dptr(buf), buf.numel() * buf.element_size(), _dptr(sink))
+    if st != OK:
+        raise DeaMoEError(st, "deamoe_probe_read")
+
 
 
 def route_static(router, tokens, n_dept, experts_per_dept, top_k, norm_topk=1, route_scale=1.0, idx=None, w=None):

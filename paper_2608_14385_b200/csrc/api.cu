@@ -383,6 +383,12 @@ deamoe_status_t deamoe_failure_test(deamoe_layer_t* L, int32_t wait_limit, int32
   return stream_set_failure_test(*L->plan, (unsigned)wait_limit, withhold) ? DEAMOE_OK : DEAMOE_ERR_UNSUPPORTED;
 }
 
+deamoe_status_t deamoe_probe_read(void* cuda_stream, const void* buf, uint64_t bytes, uint32_t* sink) {
+  if (!buf || !sink || bytes < 16 || !aligned16(buf) || (reinterpret_cast<uintptr_t>(sink) & 3u)) return DEAMOE_ERR_INVALID_ARG;
+  return launch_probe_read(buf, (size_t)bytes, sink, DEAMOE_PROBE_BLOCKS, reinterpret_cast<cudaStream_t>(cuda_stream)) > 0
+             ? DEAMOE_OK : DEAMOE_ERR_CUDA;
+}
+
 int32_t deamoe_last_launches(const deamoe_layer_t* L) { return L ? L->last_launches : 0; }
 
 uint64_t deamoe_device_bytes(const deamoe_layer_t* L) { return L ? L->device_bytes : 0; }

@@ -160,5 +160,6 @@ int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStrea
 cudaError_t route_configure(const LayerDev& L);
 int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s);
 int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s);
+int launch_probe_read(const void* src, size_t bytes, uint32_t* sink, int blocks, cudaStream_t s);
 
 }  // namespace deamoe

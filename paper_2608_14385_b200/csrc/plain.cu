@@ -303,6 +303,47 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
   TS_MAX(L, 10);
 }
 
+// Measurement aid: read `n16` 16-byte words once, with plain vectorised loads that bypass L1, eight
+// independent loads in flight per thread; the xor of everything read goes to sink[block] so that the
+// loads cannot be dropped.  What a read-only stream of this GPU's HBM can reach without any of the
+// layer's machinery: the yardstick the weight-streaming kernel is set against.
+__global__ void __launch_bounds__(256) k_probe_read(const uint4* __restrict__ src, size_t n16, uint32_t* __restrict__ sink) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t acc = 0;
+  auto ld = [](const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+  };
+  for (; i + 7 * stride < n16; i += 8 * stride) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = ld(src + i + u * stride);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+  }
+  for (; i < n16; i += stride) {
+    const uint4 v = ld(src + i);
+    acc ^= v.x ^ v.y ^ v.z ^ v.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+  __shared__ uint32_t s_acc[8];
+  if ((threadIdx.x & 31) == 0) s_acc[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t a = 0;
+    for (int w = 0; w < 8; ++w) a ^= s_acc[w];
+    sink[blockIdx.x] = a;
+  }
+}
+
+int launch_probe_read(const void* src, size_t bytes, uint32_t* sink, int blocks, cudaStream_t s) {
+  k_probe_read<<<blocks, 256, 0, s>>>(reinterpret_cast<const uint4*>(src), bytes / 16, sink);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 template <typename WT>
 static int plain_forward_t(const LayerDev& L, int B, cudaStream_t s) {
   int launches = 0;

@@ -45,3 +45,22 @@ def test_single_process_is_identity():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.us_per_layer_step(2.0, 4, 1) == 500.0
+
+
+def test_bench_started_plainly_with_gpus_2_starts_two_ranks_itself():
+    """`python bench.py --gpus 2` outside torchrun (how the single-GPU arm is invoked) must not run one
+    replica and call it two: it starts the two ranks itself on 127.0.0.1.  Run here without a GPU through
+    the CPU self-test mode, which goes through the same start-up, process group (gloo), barrier, max
+    over ranks and aggregate; rank r pretends its timed region took 10 (r + 1) ms per step."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-cpu", "--steps", "5"],
+                       capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [ln for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                              # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["steps"] == 5
+    assert line["slowest_rank_total_ms"] == 100.0       # rank 1: 5 steps x 20 ms
+    assert abs(line["value"] - 100.0e3 / (5 * 2)) < 1e-9   # 2 replicas x 5 layer-steps in 100 ms
