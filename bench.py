@@ -336,6 +336,10 @@ def main():
                     help="layer: the contract line (default); locality: routing-locality sweep on the DeepSeek-V3 "
                          "shape; stack: 32 consecutive 7B-class layers with a residual add, DeaMoE vs vanilla; "
                          "large: 32-128 tokens on the DeepSeek-V3 shape, streaming vs dense (tcgen05) schedule")
+    ap.add_argument("--shard", default="replica", choices=["replica", "dept"],
+                    help="replica (default): every rank runs its own copy of the layer, no collective; dept: ONE layer "
+                         "spread over the ranks by department (each rank holds its departments' weights, computes "
+                         "their partial sum, one NCCL all-reduce of [B, h] fp32 completes Eq. (3)): strong scaling")
     ap.add_argument("--selftest-cpu", action="store_true",
                     help="no GPU work: every rank reports a fixed made-up duration through the same rank start-up, "
                          "barrier and max-over-ranks code (gloo); used by the CPU tests of the multi-rank path")
@@ -376,6 +380,14 @@ def main():
         if rank == 0:
             fn = {"locality": locality_sweep, "stack": stack_bench, "large": large_batch_sweep}[args.mode]
             print(json.dumps(fn(args, sched, peak, torch, dev)))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+    if args.shard == "dept":
+        line = sharded_bench(args, shape, sched, peak, peak_src, torch, dev, dist, rank, local, world)
+        if rank == 0:
+            print(json.dumps(line))
         if dist is not None:
             dist.barrier()
             dist.destroy_process_group()
@@ -509,6 +521,73 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def sharded_bench(args, shape, sched, peak, peak_src, torch, dev, dist, rank, local, world):
+    """--shard dept: one layer spread over the ranks by department (paper Section 3.1: a department and
+    its experts' private matrices are an independent unit).  A step = forward_partial on every rank, one
+    all-reduce (NCCL) of the [B, h] fp32 partial sums, finish_partial.  Total work is fixed as N grows."""
+    from paper_2608_14385_b200 import binding, shard, synth
+    B = args.batch
+    my_shape, (lo, hi) = shard.slice_shape(shape, rank, world)
+    w = synth.make_deamoe_weights(my_shape, 0, dev, dept_range=(lo, hi))
+    layer = binding.Layer(my_shape, w, max(B, 32), sched, dept_range=(lo, hi))
+    del w
+    torch.cuda.empty_cache()
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    NB = 4
+    batches = [synth.make_tokens(shape, B, 100 + i, dev) for i in range(NB)]
+    partial = torch.empty((B, shape.hidden), dtype=torch.float32, device=dev)
+    outs = [torch.empty_like(b) for b in batches]
+
+    def step(i):
+        layer.forward_partial(batches[i % NB], partial)
+        if dist is not None:
+            dist.all_reduce(partial)
+        layer.finish_partial(partial, batches[i % NB], outs[i % NB])
+
+    ubytes = []
+    for i in range(NB):
+        step(i)
+        t = torch.tensor([float(layer.stats()["unique_weight_bytes"])], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(t)
+        ubytes.append(float(t.item()))
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.5)
+    for i in range(args.warmup):
+        flush.add_(1)
+        step(i)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    for i in range(args.steps):
+        flush.add_(1)
+        ev[i][0].record()
+        step(i)
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    times_ms = [a.elapsed_time(b) for a, b in ev]
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(sum(times_ms), dist, dev)
+    us = total_ms * 1e3 / args.steps
+    mean_bytes = statistics.mean(ubytes[i % NB] for i in range(args.steps))
+    launches = args.steps * (layer.last_launches + 1)
+    layer.close()
+    cfg = workload_config(shape, B, args.schedule)
+    cfg["workload"] = f"{shape.name}-shape DeaMoE layer, decode batch {B}, ONE layer sharded by department over {world} GPU(s)"
+    cfg["parallelism"] = f"dept-shard x{world}: departments [{lo}, {hi}) on rank {rank}; all-reduce of [B, h] fp32"
+    return {"metric": "us_per_step_deamoe_layer", "value": us, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16" if shape.weight_dtype else "f32", "data": "synthetic", "config": cfg,
+            "unique_weight_mb_per_step_all_ranks": mean_bytes / 1e6,
+            "hbm_gbs_on_unique_bytes_all_ranks": mean_bytes / (us * 1e-6) / 1e9,
+            "frac_of_measured_peak_per_gpu": mean_bytes / (us * 1e-6) / 1e9 / (peak * world),
+            "clocks": clocks, "gpu_launches": launches, "peak_source": peak_src}
 
 
 def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev, batches_list=(4, 8, 16, 32, 64), steps=None):

@@ -116,6 +116,11 @@ typedef struct {
                                department holds another selected expert is replaced, in place, by
                                the expert with the largest logit (ties: lowest index) of the
                                departments not yet covered.  Needs n_dept <= 64.  0: the soft cap. */
+  int32_t dept_begin, dept_end; /* 0, 0: the whole layer.  Otherwise this object is the SLICE of the layer
+                               that holds departments [dept_begin, dept_end) and their experts -- a
+                               department with its experts' private matrices is an independent unit
+                               (Section 3.1 / 3.2), so a layer can be spread over several GPUs by
+                               department.  See deamoe_forward_partial. */
 } deamoe_config_t;
 
 #define DEAMOE_MAX_BATCH 128
@@ -134,6 +139,9 @@ typedef struct {
  *   priv_down                    [n, r, f]   A_d^i, applied transposed: (A_d^i)^T y
  *   shared_gate/up/down          [shared_ffn, h]
  * priv_* must be NULL iff priv == 0; shared_* must be NULL iff n_shared == 0.
+ * For a department slice (dept_begin, dept_end) the router is still the whole [n, h] matrix (every
+ * slice routes all tokens, identically), while dept_* hold only the slice's departments,
+ * [dept_end - dept_begin, f, h], and priv_* only their experts, [(dept_end - dept_begin) * g, r, f].
  * For deamoe_vanilla_create the dept_* pointers hold the n standard experts, [n, f, h].
  */
 typedef struct {
@@ -180,6 +188,32 @@ deamoe_status_t deamoe_route(deamoe_layer_t *layer, void *cuda_stream, const voi
  */
 deamoe_status_t deamoe_forward(deamoe_layer_t *layer, void *cuda_stream, const void *tokens, int32_t B,
                                void *out);
+
+/*
+ * Department-sharded execution (Section 3.1 / 3.2: the departments are independent units; Eq. (3) is a
+ * sum over the selected experts, so it splits over any partition of the departments).  Every GPU
+ * creates the slice of the layer that holds its departments (cfg.dept_begin / dept_end; exactly one
+ * slice is created with the shared expert, if there is one), gets the same tokens, and calls
+ *
+ *   deamoe_forward_partial: partial[B, h] (DEVICE, fp32, 16-byte aligned) =
+ *       sum over the token's selected experts THAT LIVE IN THIS SLICE of p_i Expert_i(x)
+ *       (+ the shared expert if this slice has it); no residual, no rounding to the activation dtype.
+ *       Routing is computed in full by every slice (same router, same tokens, same result); its
+ *       department sets, token lists and byte counters (deamoe_get_routing / deamoe_get_stats)
+ *       cover the slice's own departments only.
+ *
+ * The caller adds the partial sums of all slices element by element (one all-reduce of B * h
+ * floats; any order is correct up to fp32 rounding) and calls, on any slice object,
+ *
+ *   deamoe_finish_partial: out[B, h] (DEVICE, act_dtype) = sum (+ tokens if cfg.residual).
+ *
+ * Both only enqueue on the stream.  deamoe_forward_partial also works on a whole (unsliced) DeaMoE
+ * layer; deamoe_forward on a slice is INVALID_ARG (a slice alone does not compute the layer).
+ */
+deamoe_status_t deamoe_forward_partial(deamoe_layer_t *layer, void *cuda_stream, const void *tokens, int32_t B,
+                                       float *partial);
+deamoe_status_t deamoe_finish_partial(deamoe_layer_t *layer, void *cuda_stream, const float *sum,
+                                      const void *tokens, int32_t B, void *out);
 
 /* The same step for a layer made by deamoe_vanilla_create (INVALID_ARG for a DeaMoE layer). */
 deamoe_status_t deamoe_vanilla_forward(deamoe_layer_t *layer, void *cuda_stream, const void *tokens,

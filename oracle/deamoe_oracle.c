@@ -38,7 +38,9 @@
  *     whose department holds another selected expert is replaced, in place, by the expert with
  *     the largest logit (ties: lowest index) among the departments not yet covered;
  *   - sigma = RMSNorm (one of the operators of Section 3.4 / Table 4) acts on the whole
- *     length-f vector: v / sqrt(mean(v^2) + 1e-6), no learned gain.
+ *     length-f vector: v / sqrt(mean(v^2) + 1e-6), no learned gain;
+ *   - a department slice (dept_begin, dept_end) evaluates Eq. (3) over the selected experts of
+ *     those departments only; the slices of a partition add up to the layer.
  *
  * Only tests, the smoke check and the benchmark's cpu_baseline leg may call
  * this file.  It shares no code with the CUDA library.
@@ -76,6 +78,10 @@ typedef struct {
   int32_t residual;         /* 1: out = x + layer(x) */
   int32_t strict_dept;      /* 1: strict department coverage (Section 3.3, last paragraph) */
   double route_scale;
+  int32_t dept_begin, dept_end; /* 0, 0: the whole layer; else only the experts of departments
+                                   [dept_begin, dept_end) contribute to oracle_deamoe_forward: the
+                                   partial sum of one slice of a department-sharded layer (Eq. (3)
+                                   is a sum over experts, Section 3.1's departments are independent) */
 } oracle_config_t;
 
 /* Pointer tables: one pointer per department / per expert, so a caller may
@@ -439,6 +445,7 @@ int oracle_deamoe_forward(const oracle_config_t *c, const oracle_weights_t *w, c
     for (int q = 0; q < h; ++q) { x[q] = ld(tokens, c->act_dtype, (size_t)t * h + q); o[q] = 0.0; }
     for (int q = 0; q < k && rc == 0; ++q) {
       const int i = idx[(size_t)t * k + q], j = i / g;
+      if (c->dept_end > 0 && (j < c->dept_begin || j >= c->dept_end)) continue; /* another slice's expert */
       rc = oracle_deamoe_expert(c, w->dept_gate[j], w->dept_up[j], w->dept_down[j],
                                 c->priv > 0 ? w->priv_gate[i] : NULL,
                                 c->priv > 0 ? w->priv_up[i] : NULL,

@@ -24,7 +24,7 @@ class OracleConfig(C.Structure):
     _fields_ = [(k, C.c_int32) for k in (
         "hidden", "n_dept", "experts_per_dept", "ffn", "priv", "top_k", "k_dept", "n_shared",
         "shared_ffn", "sigma", "norm_topk", "weight_dtype", "act_dtype", "residual", "strict_dept")] + [
-        ("route_scale", C.c_double)]
+        ("route_scale", C.c_double), ("dept_begin", C.c_int32), ("dept_end", C.c_int32)]
 
 
 class OracleWeights(C.Structure):
@@ -64,10 +64,12 @@ def host_cores():
 
 def make_config(hidden, n_dept, experts_per_dept, ffn, priv, top_k, k_dept=0, n_shared=0,
                 shared_ffn=0, sigma=SIGMA_SILU, norm_topk=1, weight_dtype=BF16, act_dtype=BF16,
-                residual=0, route_scale=1.0, strict_dept=0, **_ignored):
+                residual=0, route_scale=1.0, strict_dept=0, dept_range=None, **_ignored):
+    """dept_range = (begin, end): the partial sum of that department slice (see deamoe_oracle.c)."""
+    lo, hi = dept_range if dept_range is not None else (0, 0)
     return OracleConfig(hidden, n_dept, experts_per_dept, ffn, priv, top_k, k_dept, n_shared,
                         shared_ffn, sigma, norm_topk, weight_dtype, act_dtype, residual, strict_dept,
-                        float(route_scale))
+                        float(route_scale), int(lo), int(hi))
 
 
 def _check(arr, dtype_code, what):

@@ -20,7 +20,8 @@ SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4
 
 # every symbol include/deamoe.h declares
 SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",
-           "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_get_routing",
+           "deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host", "deamoe_forward_partial",
+           "deamoe_finish_partial", "deamoe_get_routing",
            "deamoe_get_stats", "deamoe_profile_enable", "deamoe_profile_last_ms", "deamoe_route_static", "deamoe_failure_test", "deamoe_probe_read",
            "deamoe_last_launches", "deamoe_device_bytes", "deamoe_status_string")
 
@@ -29,7 +30,8 @@ class Config(C.Structure):
     _fields_ = [(k, C.c_int32) for k in (
         "hidden", "n_dept", "experts_per_dept", "ffn", "priv", "top_k", "k_dept", "n_shared",
         "shared_ffn", "sigma", "norm_topk", "weight_dtype", "act_dtype", "residual", "max_batch",
-        "schedule")] + [("route_scale", C.c_float), ("strict_dept", C.c_int32)]
+        "schedule")] + [("route_scale", C.c_float), ("strict_dept", C.c_int32), ("dept_begin", C.c_int32),
+                        ("dept_end", C.c_int32)]
 
 
 class Weights(C.Structure):
@@ -70,6 +72,8 @@ def lib():
         L.deamoe_route.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         for name in ("deamoe_forward", "deamoe_vanilla_forward", "deamoe_forward_host"):
             getattr(L, name).argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.deamoe_forward_partial.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.deamoe_finish_partial.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.deamoe_get_routing.argtypes = [C.c_void_p] * 9
         L.deamoe_get_stats.argtypes = [C.c_void_p] * 7
         L.deamoe_route_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
@@ -94,13 +98,14 @@ def _dptr(t):
     return C.c_void_p(t.data_ptr()) if t is not None else None
 
 
-def make_config(shape, max_batch, schedule=SCHED_AUTO):
+def make_config(shape, max_batch, schedule=SCHED_AUTO, dept_range=None):
     d = shape.asdict() if hasattr(shape, "asdict") else dict(shape)
+    lo, hi = dept_range if dept_range is not None else (0, 0)
     return Config(d["hidden"], d["n_dept"], d["experts_per_dept"], d["ffn"], d["priv"], d["top_k"],
                   d.get("k_dept", 0), d.get("n_shared", 0), d.get("shared_ffn", 0), d.get("sigma", 1),
                   d.get("norm_topk", 1), d.get("weight_dtype", 1), d.get("act_dtype", 1),
                   d.get("residual", 0), int(max_batch), int(schedule), float(d.get("route_scale", 1.0)),
-                  int(d.get("strict_dept", 0)))
+                  int(d.get("strict_dept", 0)), int(lo), int(hi))
 
 
 STATIC_ROUTE_SCRATCH_BYTES = 4 << 20
@@ -140,11 +145,13 @@ def route_static(router, tokens, n_dept, experts_per_dept, top_k, norm_topk=1, r
 class Layer:
     """One DeaMoE (or vanilla MoE) layer living on the current CUDA device."""
 
-    def __init__(self, shape, weights, max_batch, schedule=SCHED_AUTO, vanilla=False):
-        """weights: dict of CUDA tensors in the canonical layouts of include/deamoe.h."""
+    def __init__(self, shape, weights, max_batch, schedule=SCHED_AUTO, vanilla=False, dept_range=None):
+        """weights: dict of CUDA tensors in the canonical layouts of include/deamoe.h.
+        dept_range = (begin, end): this object is the slice of the layer holding those departments
+        (the dept_* / priv_* tensors then hold only them); use forward_partial / finish_partial."""
         self.shape = shape
         self.vanilla = vanilla
-        self.cfg = make_config(shape, max_batch, schedule)
+        self.cfg = make_config(shape, max_batch, schedule, dept_range)
         if vanilla:
             self.cfg.priv = 0
         w = Weights()
@@ -198,6 +205,28 @@ class Layer:
         st = fn(self._h, _stream(), _dptr(tokens), B, _dptr(out))
         if st != OK:
             raise DeaMoEError(st, "deamoe_forward")
+        return out
+
+    def forward_partial(self, tokens, partial=None):
+        """fp32 partial sum of this layer object (a department slice, or a whole layer): [B, h]."""
+        B = self._check_tokens(tokens)
+        if partial is None:
+            partial = torch.empty(tokens.shape, dtype=torch.float32, device=tokens.device)
+        assert partial.is_cuda and partial.is_contiguous() and partial.dtype == torch.float32
+        st = lib().deamoe_forward_partial(self._h, _stream(), _dptr(tokens), B, _dptr(partial))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_forward_partial")
+        return partial
+
+    def finish_partial(self, total, tokens, out=None):
+        """out = total (+ tokens if residual) in the activation dtype; total: the slices' partial sums added."""
+        B = self._check_tokens(tokens)
+        if out is None:
+            out = torch.empty_like(tokens)
+        assert total.is_cuda and total.is_contiguous() and total.dtype == torch.float32
+        st = lib().deamoe_finish_partial(self._h, _stream(), _dptr(total), _dptr(tokens), B, _dptr(out))
+        if st != OK:
+            raise DeaMoEError(st, "deamoe_finish_partial")
         return out
 
     def forward_host(self, tokens, out):

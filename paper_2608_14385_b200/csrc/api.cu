@@ -70,6 +70,10 @@ deamoe_status_t check_config(const deamoe_config_t* c, const deamoe_weights_t* w
   if (!(c->route_scale == c->route_scale)) return DEAMOE_ERR_INVALID_ARG;
   if (c->strict_dept != 0 && c->strict_dept != 1) return DEAMOE_ERR_INVALID_ARG;
   if (c->strict_dept && c->k_dept > 0 && c->n_dept > 64) return DEAMOE_ERR_UNSUPPORTED;
+  if (c->dept_begin != 0 || c->dept_end != 0) {  // a department slice of the layer (0, 0 = all of it)
+    if (vanilla) return DEAMOE_ERR_INVALID_ARG;
+    if (c->dept_begin < 0 || c->dept_end <= c->dept_begin || c->dept_end > c->n_dept) return DEAMOE_ERR_INVALID_ARG;
+  }
   if (c->max_batch < 1 || c->max_batch > DEAMOE_MAX_BATCH) return DEAMOE_ERR_BATCH;
   if (!w->router || !w->dept_gate || !w->dept_up || !w->dept_down) return DEAMOE_ERR_INVALID_ARG;
   if (vanilla && c->priv != 0) return DEAMOE_ERR_INVALID_ARG;
@@ -107,6 +111,8 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   d.residual = cfg->residual; d.vanilla = vanilla ? 1 : 0;
   d.wdt = cfg->weight_dtype; d.adt = cfg->act_dtype; d.max_batch = cfg->max_batch;
   d.strict_dept = cfg->strict_dept;
+  d.dept_lo = 0; d.dept_hi = d.m;
+  if (cfg->dept_end > 0) { d.dept_lo = cfg->dept_begin; d.dept_hi = cfg->dept_end; }
   d.rp = d.r > 0 ? d.r : d.f;
   d.route_scale = cfg->route_scale;
 
@@ -131,16 +137,17 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   bool ok = true;
   auto A = [&](deamoe_status_t r) { if (r != DEAMOE_OK && ok) { ok = false; st = r; } };
   const size_t ws = dtype_size(d.wdt);
-  const size_t units = vanilla ? (size_t)d.n : (size_t)d.m;
+  const size_t units = vanilla ? (size_t)d.n : (size_t)(d.dept_hi - d.dept_lo);
+  const size_t n_loc = (size_t)(d.dept_hi - d.dept_lo) * d.g;  // experts whose private matrices this object holds
   A(dev_copy(L, reinterpret_cast<const void**>(&d.router), w->router, (size_t)d.n * d.h * 4, s));
   if (ok && sched == DEAMOE_SCHED_PLAIN) {
     A(dev_copy(L, &d.dept_gate, w->dept_gate, units * d.f * d.h * ws, s));
     A(dev_copy(L, &d.dept_up, w->dept_up, units * d.f * d.h * ws, s));
     A(dev_copy(L, &d.dept_down, w->dept_down, units * d.f * d.h * ws, s));
     if (d.r > 0) {
-      A(dev_copy(L, &d.priv_gate, w->priv_gate, (size_t)d.n * d.r * d.f * ws, s));
-      A(dev_copy(L, &d.priv_up, w->priv_up, (size_t)d.n * d.r * d.f * ws, s));
-      A(dev_copy(L, &d.priv_down, w->priv_down, (size_t)d.n * d.r * d.f * ws, s));
+      A(dev_copy(L, &d.priv_gate, w->priv_gate, n_loc * d.r * d.f * ws, s));
+      A(dev_copy(L, &d.priv_up, w->priv_up, n_loc * d.r * d.f * ws, s));
+      A(dev_copy(L, &d.priv_down, w->priv_down, n_loc * d.r * d.f * ws, s));
     }
     if (d.n_shared) {
       A(dev_copy(L, &d.shared_gate, w->shared_gate, (size_t)d.fs * d.h * ws, s));
@@ -261,7 +268,37 @@ deamoe_status_t deamoe_route(deamoe_layer_t* L, void* cuda_stream, const void* t
   return DEAMOE_OK;
 }
 
+static deamoe_status_t forward_impl(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B, void* out,
+                                    int partial);
+
 deamoe_status_t deamoe_forward(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B, void* out) {
+  // a department slice alone does not compute the layer's output: its partial sum goes through
+  // deamoe_forward_partial, an all-reduce over the slices, and deamoe_finish_partial
+  if (L && (L->dev.dept_lo != 0 || L->dev.dept_hi != L->dev.m)) return DEAMOE_ERR_INVALID_ARG;
+  return forward_impl(L, cuda_stream, tokens, B, out, 0);
+}
+
+deamoe_status_t deamoe_forward_partial(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B,
+                                       float* partial) {
+  if (L && L->dev.vanilla) return DEAMOE_ERR_INVALID_ARG;
+  return forward_impl(L, cuda_stream, tokens, B, partial, 1);
+}
+
+deamoe_status_t deamoe_finish_partial(deamoe_layer_t* L, void* cuda_stream, const float* sum, const void* tokens,
+                                      int32_t B, void* out) {
+  deamoe_status_t st = check_call(L, tokens, B);
+  if (st != DEAMOE_OK) return st;
+  if (B == 0) return DEAMOE_OK;
+  if (!sum || !out || out == tokens || out == (const void*)sum) return DEAMOE_ERR_INVALID_ARG;
+  if (check_device_ptr(tokens) != DEAMOE_OK || check_device_ptr(out) != DEAMOE_OK || check_device_ptr(sum) != DEAMOE_OK)
+    return DEAMOE_ERR_INVALID_ARG;
+  LayerDev d = call_view(L, tokens);
+  return launch_finish_partial(d, sum, tokens, B, out, reinterpret_cast<cudaStream_t>(cuda_stream)) > 0 ? DEAMOE_OK
+                                                                                                         : DEAMOE_ERR_CUDA;
+}
+
+static deamoe_status_t forward_impl(deamoe_layer_t* L, void* cuda_stream, const void* tokens, int32_t B, void* out,
+                                    int partial) {
   deamoe_status_t st = check_call(L, tokens, B);
   if (st != DEAMOE_OK) return st;
   if (B > 0 && (!out || out == tokens)) return DEAMOE_ERR_INVALID_ARG;
@@ -278,7 +315,7 @@ deamoe_status_t deamoe_forward(deamoe_layer_t* L, void* cuda_stream, const void*
     nl = stream_forward(*L->plan, d, B, s);
   }
   if (nl < 0) return DEAMOE_ERR_CUDA;
-  const int nc = launch_combine(d, tokens, B, out, s);
+  const int nc = launch_combine(d, tokens, B, out, s, partial);
   if (nc < 0) return DEAMOE_ERR_CUDA;
   L->last_launches += nl + nc;
   return DEAMOE_OK;

@@ -59,6 +59,8 @@ struct LayerDev {
   int h, m, g, n, f, r, k, k_dept, n_shared, fs, sigma, norm_topk, residual, vanilla;
   int wdt, adt, max_batch;
   int strict_dept;  // 1: strict department coverage routing (with k_dept > 0)
+  int dept_lo, dept_hi;  // departments [dept_lo, dept_hi) live in this layer object (all of them: 0, m); the
+                         // weight arrays hold only those, the routing state lists only their tokens
   int rp;  // rows of Y per pair: r, or f when there are no private parameters
   float route_scale;
   // canonical weights (PLAIN schedule and fp32); element type per wdt
@@ -159,7 +161,9 @@ int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStrea
                          int32_t* step_flag = nullptr);
 cudaError_t route_configure(const LayerDev& L);
 int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s);
-int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s);
+// partial != 0: fp32 output without the residual (the partial sum of a department-sharded layer)
+int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s, int partial = 0);
+int launch_finish_partial(const LayerDev& L, const float* sum, const void* tokens, int B, void* out, cudaStream_t s);
 int launch_probe_read(const void* src, size_t bytes, uint32_t* sink, int blocks, cudaStream_t s);
 
 }  // namespace deamoe

@@ -231,12 +231,12 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
     const int id = L.active_dept[u];
     j.row0 = L.dept_off[id];
     j.T = L.dept_off[id + 1] - j.row0;
-    woff = (size_t)id * ph.unit_elems;
+    woff = (size_t)(id - L.dept_lo) * ph.unit_elems;  // the tile arrays start at this object's first department
   } else if (ph.stage == ST_S4) {
     const int id = L.active_dept[u];
     j.row0 = L.expert_off[id * L.g];
     j.T = L.expert_off[(id + 1) * L.g] - j.row0;
-    woff = (size_t)id * ph.unit_elems;
+    woff = (size_t)(id - L.dept_lo) * ph.unit_elems;
   } else {
     j.row0 = u * DN_NMAX;  // shared expert: unit u = token group u
     j.T = min(DN_NMAX, B - j.row0);
@@ -548,8 +548,9 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   const size_t fh = (size_t)L.f * L.h;
   p->e_gu = 2 * fh; p->e_d = fh;
   size_t total = 0;
-  p->o_gu = total; total += (size_t)L.m * p->e_gu;
-  p->o_d = total; total += (size_t)L.m * p->e_d;
+  const int m_loc = L.dept_hi - L.dept_lo;  // departments this layer object holds
+  p->o_gu = total; total += (size_t)m_loc * p->e_gu;
+  p->o_d = total; total += (size_t)m_loc * p->e_d;
   if (L.n_shared) {
     const size_t sh = (size_t)L.fs * L.h;
     p->o_sgu = total; total += 2 * sh;
@@ -583,9 +584,9 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
                                                  cs, su, du, dst_row0, spt, tstride);
   };
   // departments: gate rows [0, f) and up rows [f, 2f) of one stacked matrix; down applied as W_d^T
-  pack(w.dept_gate, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, 0, NOSPLIT, 0);
-  pack(w.dept_up, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, L.m, L.f, NOSPLIT, 0);
-  pack(w.dept_down, p->o_d, L.h, L.f, 1, L.h, (long long)fh, (long long)p->e_d, L.m, 0, NOSPLIT, 0);
+  pack(w.dept_gate, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, m_loc, 0, NOSPLIT, 0);
+  pack(w.dept_up, p->o_gu, L.f, L.h, L.h, 1, (long long)fh, (long long)p->e_gu, m_loc, L.f, NOSPLIT, 0);
+  pack(w.dept_down, p->o_d, L.h, L.f, 1, L.h, (long long)fh, (long long)p->e_d, m_loc, 0, NOSPLIT, 0);
   if (L.n_shared) {
     // shared expert: tile t = half a tile of gate rows followed by the same rows of up
     pack(w.shared_gate, p->o_sgu, L.fs, L.h, L.h, 1, 0, 0, 1, 0, DN_TILE / 2, DN_TILE);

@@ -30,12 +30,13 @@ static __device__ __forceinline__ const void* woff(const void* base, int wdt, si
 // Resolve unit `u` (an index into the active list of the stage) of `stage`.
 static __device__ bool resolve(const LayerDev& L, int stage, int u, int B, UnitView& v) {
   const size_t fh = (size_t)L.f * L.h, rf = (size_t)L.r * L.f;
+  const int e_lo = L.dept_lo * L.g;  // the weight arrays start at department dept_lo / expert e_lo
   v.Wb = nullptr; v.in_b = nullptr; v.in_rows = nullptr; v.in_row0 = 0; v.out_row0 = 0;
   switch (stage) {
     case ST_S1: {  // rows [0,f): W_g^j, rows [f,2f): W_u^j  (handled as two matrices of f rows)
       if (u >= L.counts[CNT_ACTIVE_DEPT]) return false;
       const int j = L.active_dept[u];
-      v.Wa = woff(L.dept_gate, L.wdt, j * fh); v.Wb = woff(L.dept_up, L.wdt, j * fh);
+      v.Wa = woff(L.dept_gate, L.wdt, (j - L.dept_lo) * fh); v.Wb = woff(L.dept_up, L.wdt, (j - L.dept_lo) * fh);
       v.rows = L.f; v.cols = L.h;
       v.T = L.dept_off[j + 1] - L.dept_off[j];
       v.in_a = L.x32; v.in_b = L.x32; v.in_stride = L.h; v.in_rows = L.dept_tok + L.dept_off[j];
@@ -46,7 +47,7 @@ static __device__ bool resolve(const LayerDev& L, int stage, int u, int B, UnitV
     case ST_S2: {
       if (u >= L.counts[CNT_ACTIVE_EXPERT]) return false;
       const int i = L.active_expert[u];
-      v.Wa = woff(L.priv_gate, L.wdt, i * rf); v.Wb = woff(L.priv_up, L.wdt, i * rf);
+      v.Wa = woff(L.priv_gate, L.wdt, (i - e_lo) * rf); v.Wb = woff(L.priv_up, L.wdt, (i - e_lo) * rf);
       v.rows = L.r; v.cols = L.f;
       v.T = L.expert_off[i + 1] - L.expert_off[i];
       v.in_a = L.GU; v.in_b = L.GU + L.f; v.in_stride = 2 * L.f; v.in_rows = L.pair_gurow + L.expert_off[i];
@@ -57,7 +58,7 @@ static __device__ bool resolve(const LayerDev& L, int stage, int u, int B, UnitV
     case ST_S3: {  // Z = sigma(A_d^T Y): A_d stored [r, f]
       if (u >= L.counts[CNT_ACTIVE_EXPERT]) return false;
       const int i = L.active_expert[u];
-      v.Wa = woff(L.priv_down, L.wdt, i * rf);
+      v.Wa = woff(L.priv_down, L.wdt, (i - e_lo) * rf);
       v.rows = L.r; v.cols = L.f;
       v.T = L.expert_off[i + 1] - L.expert_off[i];
       v.in_a = L.Y; v.in_stride = L.rp; v.in_row0 = L.expert_off[i];
@@ -68,7 +69,7 @@ static __device__ bool resolve(const LayerDev& L, int stage, int u, int B, UnitV
     case ST_S4: {  // O = W_d^T Z over the pairs of the department (contiguous in pair order)
       if (u >= L.counts[CNT_ACTIVE_DEPT]) return false;
       const int j = L.active_dept[u];
-      v.Wa = woff(L.dept_down, L.wdt, j * fh);
+      v.Wa = woff(L.dept_down, L.wdt, (j - L.dept_lo) * fh);
       v.rows = L.f; v.cols = L.h;
       const int p0 = L.expert_off[j * L.g], p1 = L.expert_off[(j + 1) * L.g];
       v.T = p1 - p0;
@@ -253,7 +254,10 @@ __global__ void k_plain_rmsnorm(LayerDev L, float* __restrict__ buf, int count_i
 }
 
 // Eq. (3): out[t] = sum_q p[t,q] * O[slot(t,q)] (+ shared expert) (+ x[t]), written in act dtype.
-__global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void* __restrict__ out) {
+// partial != 0 (department-sharded layer): the sum over this layer object's pairs only (+ its shared
+// expert if it has one), written as fp32 without the residual; the partial sums of all shards are
+// added by the caller (an all-reduce) and finished by k_finish_partial.
+__global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void* __restrict__ out, int partial) {
   TS_MIN(L, 8);
   pdl_wait();  // stage outputs of the preceding kernel
   TS_MIN(L, 9);
@@ -266,6 +270,7 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int q = 0; q < L.k; ++q) {
       const int slot = L.pair_slot[t * L.k + q];
+      if (slot == -1) continue;  // the pair's department lives in another layer object (sharded layer)
       if ((unsigned)slot >= (unsigned)(L.max_batch * L.k)) {  // consistency check: skip the access, report
         L.counts[CNT_STATUS] = DEAMOE_ERR_INTERNAL;
         continue;
@@ -277,6 +282,10 @@ __global__ void k_combine(LayerDev L, int B, const float* __restrict__ x32, void
     if (L.n_shared) {
       const float4 o = __ldcg(reinterpret_cast<const float4*>(L.Osh) + i);
       acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+    }
+    if (partial) {
+      reinterpret_cast<float4*>(out)[i] = acc;
+      continue;
     }
     if (L.residual) {
       if (L.adt == DEAMOE_F32) {
@@ -391,13 +400,52 @@ int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s) {
   return L.wdt == DEAMOE_F32 ? plain_forward_t<float>(L, B, s) : plain_forward_t<__nv_bfloat16>(L, B, s);
 }
 
-int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s) {
+int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s, int partial) {
   (void)tokens;
   const size_t total = (size_t)B * (L.h / 4);  // four columns per thread
   int blocks = (int)((total + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  const cudaError_t e = launch_pdl(k_combine, dim3(blocks), dim3(256), 0, s, L, B, (const float*)L.x32, out);
+  const cudaError_t e = launch_pdl(k_combine, dim3(blocks), dim3(256), 0, s, L, B, (const float*)L.x32, out, partial);
   return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? 1 : -1;
+}
+
+// out[t] = sum[t] (+ x[t] if residual), written in the activation dtype: the last step of Eq. (3) for a
+// department-sharded layer, after the shards' partial sums have been added.
+__global__ void k_finish_partial(LayerDev L, int B, const float* __restrict__ sum, void* __restrict__ out) {
+  const size_t total = (size_t)B * (L.h >> 2);
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    float4 acc = reinterpret_cast<const float4*>(sum)[i];
+    if (L.residual) {
+      if (L.adt == DEAMOE_F32) {
+        const float4 x = reinterpret_cast<const float4*>(L.tokens_raw)[i];
+        acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+      } else {
+        const uint2 raw = reinterpret_cast<const uint2*>(L.tokens_raw)[i];
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+        acc.x += __bfloat162float(a.x); acc.y += __bfloat162float(a.y);
+        acc.z += __bfloat162float(b.x); acc.w += __bfloat162float(b.y);
+      }
+    }
+    if (L.adt == DEAMOE_F32) {
+      reinterpret_cast<float4*>(out)[i] = acc;
+    } else {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(out)[i] = pk;
+    }
+  }
+}
+
+int launch_finish_partial(const LayerDev& L, const float* sum, const void* tokens, int B, void* out, cudaStream_t s) {
+  (void)tokens;
+  const size_t total = (size_t)B * (L.h / 4);
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  k_finish_partial<<<blocks, 256, 0, s>>>(L, B, sum, out);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace deamoe

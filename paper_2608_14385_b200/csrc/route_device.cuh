@@ -400,8 +400,10 @@ static __device__ void bucket_departments(const LayerDev& L, int B, uint32_t* s_
   for (int p = tid; p < B * k; p += nthr) {
     const int t = p / k;
     const int i = L.topk_idx[p];
+    const int j = i / g;
+    if (j < L.dept_lo || j >= L.dept_hi) continue;  // a department another layer object (another GPU) holds
     atomicOr(&b.emask[(size_t)i * W + (t >> 5)], 1u << (t & 31));
-    atomicOr(&b.dmask[(size_t)(i / g) * W + (t >> 5)], 1u << (t & 31));
+    atomicOr(&b.dmask[(size_t)j * W + (t >> 5)], 1u << (t & 31));
   }
   __syncthreads();
   // department counts; the active-department bitmask falls out of a warp ballot (32 departments
@@ -483,6 +485,10 @@ static __device__ void bucket_experts(const LayerDev& L, int B, uint32_t* s_u32,
     const int t = p / k;
     const int i = L.topk_idx[p];
     const int j = i / g;
+    if (j < L.dept_lo || j >= L.dept_hi) {  // not this layer object's pair: the combine skips it
+      L.pair_slot[p] = -1;
+      continue;
+    }
     int re = 0, rd = 0;
 #pragma unroll 1
     for (int w = 0; w < (t >> 5); ++w) {

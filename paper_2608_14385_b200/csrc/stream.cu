@@ -345,6 +345,9 @@ static __device__ __forceinline__ int unit_tokens(const LayerDev& L, int stage, 
   }
 }
 static __device__ __forceinline__ int groups_of(int T, int tg) { return (T + tg - 1) / tg; }
+static __device__ __forceinline__ int stage_kind(int stage) {  // 0 single unit, 1 departments, 2 experts
+  return (stage == ST_SH1 || stage == ST_SH2) ? 0 : ((stage == ST_S1 || stage == ST_S4) ? 1 : 2);
+}
 
 static __device__ __forceinline__ int chunk_k(int C, int q, int act_rows) {
   const int avail = SLOT_BYTES - SLOT_HDR - act_rows * ACT_PAD * 2;
@@ -458,7 +461,10 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
   o[2] = make_int4(kc, sc.C, sc.rows, sc.n_tiles);
   o[3] = make_int4(in_stride, out_stride, out_row0, dep_idx);
   o[4] = make_int4(dep_target, done_idx, planes, 0);
-  o[5] = ptr2(sc.w0 + (size_t)id * sc.unit_elems, sc.w1 ? sc.w1 + (size_t)id * sc.unit_elems : nullptr);
+  // the packed arrays hold only this layer object's departments [dept_lo, dept_hi) and their experts
+  const int sk = stage_kind(stage);
+  const size_t wu = (size_t)(id - (sk == 1 ? L.dept_lo : (sk == 2 ? L.dept_lo * L.g : 0)));
+  o[5] = ptr2(sc.w0 + wu * sc.unit_elems, sc.w1 ? sc.w1 + wu * sc.unit_elems : nullptr);
   o[6] = ptr2(in0h, in0l);
   o[7] = ptr2(in1h, in1l);
   o[8] = ptr2(outh, outl);
@@ -603,9 +609,6 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
   }
 }
 
-static __device__ __forceinline__ int stage_kind(int stage) {  // 0 single unit, 1 departments, 2 experts
-  return (stage == ST_SH1 || stage == ST_SH2) ? 0 : ((stage == ST_S1 || stage == ST_S4) ? 1 : 2);
-}
 
 // Hand the first stage (department gate / up; for the vanilla layer the experts' gate / up) to the
 // streaming kernel as soon as its token lists exist: zero the dependency counters, write the stage's segment records (the same
@@ -1173,7 +1176,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         const StageCfg& sc = P.st[P.early_stage];
         const int x = ((int)blockIdx.x - first_cta + G) % G;
         const int unit = x / sc.items_per_seg, it = x - unit * sc.items_per_seg;
-        if (unit < (L.vanilla ? L.n : L.m)) {
+        if (unit < (L.vanilla ? L.n : L.dept_hi - L.dept_lo)) {  // (offsets below are relative to this object's first unit)
           const int tile0 = sc.paired ? it : it * sc.q;
           const int ntile = sc.paired ? 1 : min(sc.q, sc.n_tiles - tile0);
           const size_t tile_bytes = (size_t)(sc.C / 16) * 512;
@@ -1724,7 +1727,8 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&p->n_sm, cudaDevAttrMultiProcessorCount, dev);
   if (p->n_sm <= 0) p->n_sm = 148;
-  const size_t units = L.vanilla ? (size_t)L.n : (size_t)L.m;
+  const int m_loc = L.dept_hi - L.dept_lo, n_loc = m_loc * L.g;  // departments / experts this object holds
+  const size_t units = L.vanilla ? (size_t)L.n : (size_t)m_loc;
   const size_t e_gu = packed_elems(2 * L.f, L.h);  // stacked gate;up (DeaMoE stage 1)
   const size_t e_fh = packed_elems(L.f, L.h), e_hf = packed_elems(L.h, L.f);
   const size_t e_rf = packed_elems(L.r, L.f), e_fr = packed_elems(L.f, L.r);
@@ -1739,9 +1743,9 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
     o_a = total; total += units * e_gu;
     o_c = total; total += units * e_hf;
     if (L.r > 0) {
-      o_pg = total; total += (size_t)L.n * e_rf;
-      o_pu = total; total += (size_t)L.n * e_rf;
-      o_pd = total; total += (size_t)L.n * e_fr;
+      o_pg = total; total += (size_t)n_loc * e_rf;
+      o_pu = total; total += (size_t)n_loc * e_rf;
+      o_pd = total; total += (size_t)n_loc * e_fr;
     }
   }
   if (L.n_shared) {
@@ -1779,9 +1783,9 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
     fill_stage(d.st[ST_S1], base + o_a, nullptr, e_gu, L.h, 2 * L.f, 0, EPI_SIGMA);
     fill_stage(d.st[ST_S4], base + o_c, nullptr, e_hf, L.f, L.h, 0, EPI_NONE);
     if (L.r > 0) {
-      P(w.priv_gate, o_pg, L.r, L.f, L.f, 1, rf, (long long)e_rf, L.n);
-      P(w.priv_up, o_pu, L.r, L.f, L.f, 1, rf, (long long)e_rf, L.n);
-      P(w.priv_down, o_pd, L.f, L.r, 1, L.f, rf, (long long)e_fr, L.n);
+      P(w.priv_gate, o_pg, L.r, L.f, L.f, 1, rf, (long long)e_rf, n_loc);
+      P(w.priv_up, o_pu, L.r, L.f, L.f, 1, rf, (long long)e_rf, n_loc);
+      P(w.priv_down, o_pd, L.f, L.r, 1, L.f, rf, (long long)e_fr, n_loc);
       fill_stage(d.st[ST_S2], base + o_pg, base + o_pu, e_rf, L.f, L.r, 1, EPI_SWIGLU);
       fill_stage(d.st[ST_S3], base + o_pd, nullptr, e_fr, L.r, L.f, 0, EPI_SIGMA);
     }

@@ -546,3 +546,43 @@ def test_routing_gaps_report_every_comparison_that_decides_a_selection():
     assert list(tied["idx"][0]) == [0, 6, 3]
     assert tied["gap_parts"][0, 2] == 0.0 and tied["gap"][0] == 0.0
     assert 9 not in tied["idx"][0]                                               # ties go to the lower index
+
+
+# ---------------------------------------------------------------- department slices (sharded layer)
+
+def test_department_slices_add_up_to_the_layer():
+    """Eq. (3) is a sum over the selected experts and the departments are independent units
+    (Section 3.1), so for ANY partition of the departments the slices' partial sums (the shared expert
+    on exactly one of them, the residual on none) add up to the layer's output.  Also: a slice that
+    holds no selected expert of a token contributes exactly zero for it, and the slice generator gives
+    the same numbers as indexing the full tensors."""
+    shape = synth.LayerShape("sl", hidden=48, n_dept=5, experts_per_dept=3, ffn=40, priv=24, top_k=4,
+                             n_shared=1, shared_ffn=32, residual=1)
+    wt = _layer(shape, 11, std=0.3)
+    w = oracle_weights(wt)
+    tokens = synth.to_numpy(synth.make_tokens(shape, 6, 11))
+    full = ref.deamoe_forward(oracle_cfg(shape), w, tokens)
+    x = widen(synth.make_tokens(shape, 6, 11))
+    for cuts in ([0, 2, 5], [0, 1, 2, 5], [0, 5], [0, 4, 5]):
+        total = np.zeros_like(full["out"])
+        for r, (lo, hi) in enumerate(zip(cuts[:-1], cuts[1:])):
+            own_shared = r == len(cuts) - 2
+            sl = shape.with_(n_shared=1 if own_shared else 0, residual=0)
+            cfg = ref.make_config(**sl.asdict(), dept_range=(lo, hi))
+            wr = dict(w)
+            for name in ("dept_gate", "dept_up", "dept_down"):        # a slice only has its own departments
+                wr[name] = [w[name][j] if lo <= j < hi else None for j in range(shape.n_dept)]
+            for name in ("priv_gate", "priv_up", "priv_down"):
+                wr[name] = [w[name][i] if lo <= i // 3 < hi else None for i in range(shape.n_expert)]
+            part = ref.deamoe_forward(cfg, wr, tokens)
+            assert (part["idx"] == full["idx"]).all()                 # every slice routes all tokens alike
+            for t in range(6):
+                if not any(lo <= i // 3 < hi for i in full["idx"][t]) and not own_shared:
+                    assert (part["out"][t] == 0).all()
+            total += part["out"]
+        np.testing.assert_allclose(total + x, full["out"], rtol=1e-12, atol=1e-13)
+    sliced = synth.make_deamoe_weights(shape, 11, dept_range=(1, 4))
+    whole = synth.make_deamoe_weights(shape, 11)
+    assert torch.equal(sliced["dept_down"], whole["dept_down"][1:4])
+    assert torch.equal(sliced["priv_gate"], whole["priv_gate"][3:12])
+    assert torch.equal(sliced["router"], whole["router"])
