@@ -319,7 +319,11 @@ deamoe_status_t deamoe_probe_read(void *cuda_stream, const void *buf, uint64_t b
  *   withhold    bit 0: the routing kernel does not raise the flags that hand the work list to the
  *               fused streaming kernel, so that kernel's planners wait until the limit expires;
  *               bit 1: the copy role of the dense (tcgen05) kernel issues no copies, so its MMA role
- *               waits for the ring until the limit expires.  0 = normal operation.
+ *               waits for the ring until the limit expires;
+ *               bit 2: the routing kernel publishes an out-of-range slot for the first (token,
+ *               expert) pair, which the combine kernel's consistency check must skip and report
+ *               as DEAMOE_ERR_INTERNAL (that pair's term is then missing from the output).
+ *               0 = normal operation.
  * A step run with a withheld hand-over returns garbage in `out` and DEAMOE_ERR_TIMEOUT from
  * deamoe_get_stats; after deamoe_failure_test(layer, 0, 0) the layer works normally again.
  * Errors: INVALID_ARG; UNSUPPORTED if the layer's schedule has no such hand-over (plain / staged

@@ -415,7 +415,7 @@ deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t* L, float* ms) {
 }
 
 deamoe_status_t deamoe_failure_test(deamoe_layer_t* L, int32_t wait_limit, int32_t withhold) {
-  if (!L || wait_limit < 0 || withhold < 0 || withhold > 3) return DEAMOE_ERR_INVALID_ARG;
+  if (!L || wait_limit < 0 || withhold < 0 || withhold > 7) return DEAMOE_ERR_INVALID_ARG;
   if (!L->plan) return withhold ? DEAMOE_ERR_UNSUPPORTED : DEAMOE_OK;  // the plain schedule has no device-side waits
   return stream_set_failure_test(*L->plan, (unsigned)wait_limit, withhold) ? DEAMOE_OK : DEAMOE_ERR_UNSUPPORTED;
 }

@@ -131,7 +131,8 @@ struct StreamDev {
                                 // early_flag + 2: flag that the rest of the work list exists
   int planes;                  // 1: activations carried as bf16; 2: as bf16 hi + lo (fp32 activations)
   unsigned spin_limit;         // polls after which a bounded wait gives up (SPIN_LIMIT; lower only in failure tests)
-  int withhold;                // failure tests: bit 0 = the routing tail raises no hand-over flag
+  int withhold;                // failure tests: bit 0 = the routing tail raises no hand-over flag; bit 2 = it
+                               // publishes an out-of-range slot for the first (token, expert) pair
   // activations between stages, bf16 planes ([rows, width] each)
   __nv_bfloat16 *xh, *xl;      // tokens split (fp32 activations only; bf16 tokens are read in place)
   __nv_bfloat16 *GUh, *GUl, *Yh, *Yl, *Zh, *Zl, *Yshh, *Yshl;
@@ -842,6 +843,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     const int cnt = s_cnt[e];
 #pragma unroll 1
     for (int i = tid; i < cnt; i += FINISH_THREADS) dst[i] = src[i];
+  }
+  if (P.withhold & 4) {  // failure test: an out-of-range pair slot, which the combine must skip and report
+    __syncthreads();
+    if (tid == 0) L.pair_slot[0] = 0x7fff0000;
   }
 #ifdef DEAMOE_TRACE
   __syncthreads();
@@ -2018,8 +2023,8 @@ bool stream_set_failure_test(StreamPlan& p, unsigned spin_limit, int withhold) {
   if ((withhold & 1) && !p.dev.early) return false;   // only the fused schedule hands over through flags
   if ((withhold & 2) && !p.dense) return false;
   const unsigned lim = spin_limit ? spin_limit : SPIN_LIMIT;
-  p.dev.spin_limit = lim; p.dev.withhold = withhold & 1;
-  p.dev_dense.spin_limit = lim; p.dev_dense.withhold = 0;
+  p.dev.spin_limit = lim; p.dev.withhold = withhold & 5;
+  p.dev_dense.spin_limit = lim; p.dev_dense.withhold = withhold & 4;
   if (p.dense) dense_set_failure_test(*p.dense, spin_limit, (withhold & 2) ? 1 : 0);
   return true;
 }

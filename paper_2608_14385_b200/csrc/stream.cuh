@@ -31,7 +31,8 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s);
 
 // Failure-detection tests: poll limit of the bounded waits (0 = default) and withheld hand-overs
 // (bit 0: the routing tail raises no flag for the fused streaming kernel; bit 1: the dense kernel's
-// copy role issues nothing).  False if the plan has no such hand-over.
+// copy role issues nothing; bit 2: the routing tail publishes an out-of-range pair slot for the
+// combine's consistency check).  False if the plan has no such hand-over.
 bool stream_set_failure_test(StreamPlan& p, unsigned spin_limit, int withhold);
 
 // Event pair around the streaming launches of stream_forward (measurement aid).

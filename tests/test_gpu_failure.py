@@ -82,6 +82,32 @@ def test_dense_kernel_wait_expires_when_its_copies_are_withheld():
         layer.close()
 
 
+@pytest.mark.parametrize("schedule", [binding.SCHED_STAGED, binding.SCHED_FUSED])
+def test_out_of_range_pair_slot_is_skipped_and_reported(schedule):
+    """The combine kernel checks every pair slot before it uses it as a row index.  With a planted
+    out-of-range slot for pair (token 0, first expert) it must skip that row (no access), report
+    DEAMOE_ERR_INTERNAL, and leave every other token's output exactly as in a normal step."""
+    w = _weights(SHAPE, 36)
+    layer = binding.Layer(SHAPE, w, 8, schedule)
+    try:
+        tokens = synth.make_tokens(SHAPE, 6, 36, "cuda:0")
+        good = layer.forward(tokens).clone()
+        torch.cuda.synchronize()
+        layer.failure_test(0, 4)
+        bad = layer.forward(tokens).clone()
+        torch.cuda.synchronize()
+        assert layer.stats()["device_status"] == binding.ERR_INTERNAL
+        assert torch.equal(bad[1:], good[1:])             # the other tokens are untouched
+        assert not torch.equal(bad[0], good[0])           # token 0 lost one expert's term
+        assert torch.isfinite(bad.float()).all()
+        layer.failure_test(0, 0)
+        assert torch.equal(layer.forward(tokens), good)
+        torch.cuda.synchronize()
+        assert layer.stats()["device_status"] == binding.OK
+    finally:
+        layer.close()
+
+
 def test_failure_test_is_refused_where_there_is_no_such_hand_over():
     w = _weights(SHAPE, 34)
     for sched, withhold in ((binding.SCHED_PLAIN, 1), (binding.SCHED_STAGED, 1), (binding.SCHED_FUSED, 2)):
