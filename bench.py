@@ -510,10 +510,14 @@ def main():
                                 "one_core_us_per_token_row": one * 1e6 / len(few),
                                 "one_core_sample": f"{len(few)} of {B} token rows on one core (not scaled)"}
     if rank == 0 and not args.no_sweep and shape.name == "dsv3":
+        locality = locality_rows(shape, layer, router, flush, peak, torch, dev, cs=(1, 2, 4, 8), batches_list=(1, 16), steps=10)
         layer.close()
         layer = None
         torch.cuda.empty_cache()
         line["other_workloads"] = other_workloads(args, sched, peak, torch, dev, flush)
+        line["other_workloads"]["locality_dsv3"] = {
+            "workload": "dsv3-shape DeaMoE layer, every token's top-8 planted in exactly c departments (configuration 4)",
+            "rows": locality}
     if layer is not None:
         layer.close()
     if rank == 0:
@@ -637,25 +641,18 @@ def paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev, batches_
             "paper_context": ctx}
 
 
-def locality_sweep(args, sched, peak, torch, dev):
-    """Routing-locality sweep on the DeepSeek-V3 shape: every token's top-8 is planted (through the real
-    router) in exactly c departments; c = 8 with random tokens is the uniform case.  Unique bytes are set
-    against the closed form |D| ~ m (1 - (1 - c/m)^B) with 8 B distinct experts at most."""
-    from paper_2608_14385_b200 import binding, synth
-    shape = synth.DSV3
-    w = synth.make_deamoe_weights(shape, 0, dev)
-    layer = binding.Layer(shape, w, 32, sched)
-    router = w["router"]
-    del w
-    torch.cuda.empty_cache()
-    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-    m, g, k = shape.n_dept, shape.experts_per_dept, shape.top_k
+def locality_rows(shape, layer, router, flush, peak, torch, dev, cs, batches_list, steps):
+    """Rows of the routing-locality sweep on an existing layer: every token's top-k is planted (through the
+    real router) in exactly c departments (c = 0: no planting, uniform routing).  Unique bytes are set against
+    the closed form |D| ~ m (1 - (1 - c/m)^B) with k B distinct experts at most."""
+    from paper_2608_14385_b200 import synth
+    m, k = shape.n_dept, shape.top_k
     dept_b = 3 * shape.hidden * shape.ffn * 2
     exp_b = 3 * shape.priv * shape.ffn * 2
     fixed_b = shape.n_shared * 3 * shape.hidden * shape.shared_ffn * 2 + shape.n_expert * shape.hidden * 4
     rows = []
-    for c in (1, 2, 4, 8, 0):                      # 0 = uniform (no planting)
-        for B in (1, 4, 16, 32):
+    for c in cs:
+        for B in batches_list:
             bs = []
             for i in range(4):
                 t = synth.make_tokens(shape, B, 200 + i, dev)
@@ -667,7 +664,7 @@ def locality_sweep(args, sched, peak, torch, dev):
                 layer.forward(b)
                 st = layer.stats()
                 ub.append(st["unique_weight_bytes"]); nd.append(st["active_dept"]); ne.append(st["active_expert"])
-            t_ms, _ = time_layer(layer, bs, max(10, args.steps // 2), 3, flush, torch, lambda: None)
+            t_ms, _ = time_layer(layer, bs, steps, 3, flush, torch, lambda: None)
             us = pct(t_ms, 0.5) * 1e3
             mb = statistics.mean(ub) / 1e6
             row = {"c": c if c else "uniform", "batch": B, "us": us, "unique_mb": mb, "gbs": mb / us * 1e3,
@@ -679,6 +676,22 @@ def locality_sweep(args, sched, peak, torch, dev):
                 row["closed_form_mb"] = (e_d * dept_b + e_e * exp_b + fixed_b) / 1e6
                 row["closed_form_active_dept"] = e_d
             rows.append(row)
+    return rows
+
+
+def locality_sweep(args, sched, peak, torch, dev):
+    """Routing-locality sweep on the DeepSeek-V3 shape (BASELINE configuration 4): c = 1, 2, 4, 8 and uniform
+    routing at B = 1, 4, 16, 32."""
+    from paper_2608_14385_b200 import binding, synth
+    shape = synth.DSV3
+    w = synth.make_deamoe_weights(shape, 0, dev)
+    layer = binding.Layer(shape, w, 32, sched)
+    router = w["router"]
+    del w
+    torch.cuda.empty_cache()
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    rows = locality_rows(shape, layer, router, flush, peak, torch, dev, cs=(1, 2, 4, 8, 0), batches_list=(1, 4, 16, 32),
+                         steps=max(10, args.steps // 2))
     layer.close()
     return {"metric": "routing_locality_sweep", "unit": "us", "shape": shape.name, "data": "synthetic",
             "config": {"workload": "dsv3-shape DeaMoE layer, top-8 planted in c departments per token",
