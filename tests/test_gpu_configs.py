@@ -34,6 +34,43 @@ def test_locality_sweep_planted_routing(c):
 
 
 @pytest.mark.parametrize("B", [1, 8])
+def test_stack_of_32_layers_teacher_forced(B):
+    """Benchmark configuration 5 at its full depth: 32 consecutive 7B-class layers with a residual add,
+    every layer with its own seeded weights, tokens scaled as `bench.py` scales them (1/16, so that the
+    un-normalised stack stays finite).  Teacher forced: GPU layer l gets the oracle's x_l rounded to
+    bf16; routing bit-exact (on tokens clear of a tie) and every output element in tolerance, layer by
+    layer."""
+    n_layers = 32
+    shape = synth.MOE7B.with_(residual=1)
+    dev = torch.device("cuda:0")
+    cfg = oracle_cfg(shape)
+    x = (synth.make_tokens(shape, B, 300, dev).float() / 16).to(torch.bfloat16)
+    worst = 0.0
+    for l in range(n_layers):
+        w = synth.make_deamoe_weights(shape, 0, dev, layer=l)
+        layer = binding.Layer(shape, w, 8)
+        try:
+            hostw = {k: synth.to_numpy(v) for k, v in w.items()}
+            want = ref.deamoe_forward(cfg, hostw, synth.to_numpy(x))
+            r = ref.route(cfg, hostw["router"], synth.to_numpy(x), want_logits=True)
+            safe = r["gap"] > 1e-5 * np.abs(r["logits"]).max(axis=1)
+            got = layer.forward(x)
+            torch.cuda.synchronize()
+            assert layer.stats()["device_status"] == 0
+            assert (layer.routing(B)["idx"][safe] == want["idx"][safe]).all(), f"layer {l}"
+            ok, err, bound = within_tolerance(got.float().cpu().numpy()[safe], want["out"][safe])
+            assert ok, (l, err, bound)
+            worst = max(worst, err / bound)
+            assert safe.mean() >= 0.75
+            x = torch.from_numpy(want["out"]).to(torch.bfloat16).to(dev)
+            assert torch.isfinite(x.float()).all()
+        finally:
+            layer.close()
+        del w
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("B", [1, 8])
 def test_stack_of_layers_teacher_forced_and_free_running(B):
     """x_{l+1} = x_l + Layer_l(x_l), every layer with its own seeded weights.  Teacher forced: GPU layer l
     is fed the oracle's x_l (rounded to the activation dtype) and must match routing bit-exactly and

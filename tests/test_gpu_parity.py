@@ -204,8 +204,10 @@ def test_7b_class_layer(B):
     run_case(synth.MOE7B, B, seed=0)
 
 
-def test_7b_class_vanilla():
-    run_case(synth.MOE7B, 4, seed=0, vanilla=True)
+@pytest.mark.parametrize("B", [1, 4, 16])
+def test_7b_class_vanilla(B):
+    """The comparator of benchmark configuration 2 at the batch sizes `bench.py` times, every element."""
+    run_case(synth.MOE7B, B, seed=0, vanilla=True, max_batch=16)
 
 
 def test_dsv3_shape_vanilla_sampled_row():
