@@ -221,8 +221,10 @@ deamoe_status_t deamoe_vanilla_forward(deamoe_layer_t *layer, void *cuda_stream,
 
 /*
  * End-to-end step on HOST buffers: copies tokens (HOST [B, h], act_dtype, ideally pinned) to a
- * device staging buffer owned by the layer, runs deamoe_forward, copies the result to `out`
- * (HOST [B, h]) and synchronises the stream before returning.
+ * device staging buffer owned by the layer, runs deamoe_forward, brings the result to `out`
+ * (HOST [B, h]) and synchronises the stream before returning.  When `out` is pinned memory the
+ * device can address, the last kernel of the step writes into it directly; otherwise the result is
+ * copied from a staging buffer.
  */
 deamoe_status_t deamoe_forward_host(deamoe_layer_t *layer, void *cuda_stream, const void *tokens,
                                     int32_t B, void *out);

@@ -336,9 +336,22 @@ deamoe_status_t deamoe_forward_host(deamoe_layer_t* L, void* cuda_stream, const 
   const size_t bytes = (size_t)B * L->dev.h * dtype_size(L->dev.adt);
   if (cudaMemcpyAsync(L->stage_tokens, tokens, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
     return DEAMOE_ERR_CUDA;
-  st = deamoe_forward(L, cuda_stream, L->stage_tokens, B, L->stage_out);
+  // If `out` is pinned host memory that the device can address (cudaHostAlloc / cudaHostRegister under
+  // unified addressing), the combine kernel writes the result straight into it: one pass of B * h
+  // values over the bus, and no separate copy behind the step.  Pageable memory takes the copy.
+  void* direct = nullptr;
+  {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, out) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer &&
+        aligned16(at.devicePointer))
+      direct = at.devicePointer;
+    else
+      cudaGetLastError();
+  }
+  st = deamoe_forward(L, cuda_stream, L->stage_tokens, B, direct ? direct : L->stage_out);
   if (st != DEAMOE_OK) return st;
-  if (cudaMemcpyAsync(out, L->stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return DEAMOE_ERR_CUDA;
+  if (!direct && cudaMemcpyAsync(out, L->stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return DEAMOE_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return DEAMOE_ERR_CUDA;
   return DEAMOE_OK;
 }
