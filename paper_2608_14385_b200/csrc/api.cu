@@ -157,7 +157,18 @@ deamoe_status_t create_impl(const deamoe_config_t* cfg, const deamoe_weights_t* 
   }
   if (ok) {
     if (d.adt == DEAMOE_BF16) A(dev_alloc(L, &d.x32, (size_t)MB * d.h));
-    A(dev_alloc(L, &d.logit_part, (size_t)L->kslices * MB * d.n));
+    // bf16 tokens on a streaming schedule: the router product runs on the tensor cores, on a three-piece
+    // bf16 copy of the router (route.cu); its partial-logit arrays may be more than the scalar kernel's
+    int part_slices = L->kslices;
+    if (sched != DEAMOE_SCHED_PLAIN && d.adt == DEAMOE_BF16 && (d.h & 15) == 0) {
+      __nv_bfloat16* r3 = nullptr;
+      A(dev_alloc(L, &r3, router3_elems(d.n, d.h)));
+      if (ok && pack_router3(d.router, r3, d.n, d.h, s) != cudaSuccess) A(DEAMOE_ERR_CUDA);
+      d.router3 = r3;
+      d.router3_slices = router3_kslices(d.n, d.h);
+      if (d.router3_slices > part_slices) part_slices = d.router3_slices;
+    }
+    A(dev_alloc(L, &d.logit_part, (size_t)part_slices * MB * d.n));
     A(dev_alloc(L, &d.topk_idx, (size_t)pmax));
     A(dev_alloc(L, &d.topk_w, (size_t)pmax));
     A(dev_alloc(L, &d.dept_mask, (size_t)(d.m + 63) / 64));

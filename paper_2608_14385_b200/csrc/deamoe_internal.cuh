@@ -65,6 +65,10 @@ struct LayerDev {
   float route_scale;
   // canonical weights (PLAIN schedule and fp32); element type per wdt
   const float* router;
+  // the router matrix once more, for the tensor-core logits kernel of bf16-token layers: every fp32 value as
+  // the exact sum of three bf16 pieces, in mma fragment order (k_pack_router3 in route.cu); or null
+  const __nv_bfloat16* router3;
+  int router3_slices;   // column slices that kernel uses (its partial-logit arrays)
   const void *dept_gate, *dept_up, *dept_down;
   const void *priv_gate, *priv_up, *priv_down;
   const void *shared_gate, *shared_up, *shared_down;
@@ -160,6 +164,11 @@ size_t bucket_smem_bytes(const LayerDev& L, int B);
 int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices,
                          int32_t* step_flag = nullptr);
 cudaError_t route_configure(const LayerDev& L);
+// Tensor-core router product (bf16 tokens): elements of the packed three-piece router, the column slices it is run
+// with, and the packing itself (enqueued on s).
+size_t router3_elems(int n, int h);
+int router3_kslices(int n, int h);
+cudaError_t pack_router3(const float* router, __nv_bfloat16* out, int n, int h, cudaStream_t s);
 int launch_plain_forward(const LayerDev& L, int B, cudaStream_t s);
 // partial != 0: fp32 output without the residual (the partial sum of a department-sharded layer)
 int launch_combine(const LayerDev& L, const void* tokens, int B, void* out, cudaStream_t s, int partial = 0);

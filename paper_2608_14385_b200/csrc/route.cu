@@ -121,6 +121,160 @@ k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float*
 #endif
 }
 
+// ---------------------------------------------------------------- logits = W_r x on the tensor cores
+// For bf16 tokens the fp32 product of Eq. (2) can run on mma.sync without losing a bit of the router: at
+// create every fp32 router value w is split into three bf16 pieces, w = hi + mid + lo exactly (8 + 8 + 8
+// mantissa bits), stored in the per-lane order of the m16n8k16 A fragment.  A bf16 token times a bf16 piece
+// is exact in fp32, so the only rounding is the fp32 accumulation, as in the scalar kernel above (in a
+// different, equally fixed order).  One CTA takes 16 router rows x all tokens x one column slice; its four
+// warps split the slice's 16-column steps, each accumulating 16 x B partial logits in registers (B / 8
+// accumulator tiles), which are then added across the warps through shared memory in a fixed order.
+// The scalar kernel needs ~1.5 us of dependent latency per group of 8 tokens (44 us at 128 tokens, 13 at
+// 32); this one issues three 16-byte loads and 2 x B / 8 4-byte loads per step and has no per-token-group
+// barrier.  It is used for calls of more than 16 tokens.
+constexpr int R3_ROWS = 16, R3_WARPS = 4;
+
+size_t router3_elems(int n, int h) { return (size_t)((n + R3_ROWS - 1) / R3_ROWS) * (h / 16) * 3 * 32 * 8; }
+
+int router3_kslices(int n, int h) {
+  const int tiles = (n + R3_ROWS - 1) / R3_ROWS, ksteps = h / 16;
+  int ks = 1;
+  // more slices while every warp keeps at least two 16-column steps and the grid stays within ~256 CTAs; at
+  // most 16, because every slice is one more array of partial logits for the top-k to add up
+  while (ks < 16 && ksteps / (2 * ks) >= 2 * R3_WARPS && tiles * (2 * ks) <= 256) ks *= 2;
+  return ks;
+}
+
+// out[((tile * (h / 16) + kt) * 3 + piece) * 32 + lane][8]: the A fragment (rows tile * 16 .., columns kt * 16 ..)
+// of piece `piece` of the router; rows beyond n are zero.
+__global__ void k_pack_router3(const float* __restrict__ Wr, __nv_bfloat16* __restrict__ out, int n, int h) {
+  const int nk = h / 16;
+  const long long total = (long long)((n + R3_ROWS - 1) / R3_ROWS) * nk * 32;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
+    const int lane = (int)(idx & 31);
+    const long long tk = idx >> 5;
+    const int kt = (int)(tk % nk), tile = (int)(tk / nk);
+    const int g = lane >> 2, tig = lane & 3;
+    const int rr[4] = {tile * 16 + g, tile * 16 + g + 8, tile * 16 + g, tile * 16 + g + 8};
+    const int kk[4] = {kt * 16 + tig * 2, kt * 16 + tig * 2, kt * 16 + tig * 2 + 8, kt * 16 + tig * 2 + 8};
+    __align__(16) __nv_bfloat16 v[3][8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+      for (int d = 0; d < 2; ++d) {
+        const float w = rr[e] < n ? Wr[(size_t)rr[e] * h + kk[e] + d] : 0.f;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+        const float r1 = w - __bfloat162float(hi);          // exact: at most 16 significant bits are left
+        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+        const float r2 = r1 - __bfloat162float(mid);        // exact: at most 8 are left, so lo is exact too
+        v[0][e * 2 + d] = hi; v[1][e * 2 + d] = mid; v[2][e * 2 + d] = __float2bfloat16_rn(r2);
+      }
+    const size_t base = (((size_t)tile * nk + kt) * 3) * 32 + lane;
+#pragma unroll
+    for (int pc = 0; pc < 3; ++pc)
+      *reinterpret_cast<uint4*>(out + (base + (size_t)pc * 32) * 8) = *reinterpret_cast<const uint4*>(v[pc]);
+  }
+}
+
+cudaError_t pack_router3(const float* router, __nv_bfloat16* out, int n, int h, cudaStream_t s) {
+  const long long total = (long long)((n + R3_ROWS - 1) / R3_ROWS) * (h / 16) * 32;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 2048) blocks = 2048;
+  k_pack_router3<<<blocks, 256, 0, s>>>(router, out, n, h);
+  return cudaGetLastError();
+}
+
+static __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint4& a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
+}
+
+// NT = accumulator tiles of 8 tokens (a power of two, ceil(B / 8) rounded up).
+template <int NT>
+__global__ void __launch_bounds__(R3_WARPS * 32)
+k_router_logits_mma(const __nv_bfloat16* __restrict__ W3, const __nv_bfloat16* __restrict__ X, float* __restrict__ part,
+                    int n, int h, int B, int ksteps_per_slice, int32_t* __restrict__ step_flag TS_PARAM) {
+#ifdef DEAMOE_TRACE
+  if (threadIdx.x == 0 && ts) atomicMin(ts + 0, gtime());
+#endif
+  if (step_flag && blockIdx.x == 0 && blockIdx.y == 0) {  // see k_router_logits
+    if (threadIdx.x == 0) {
+      step_flag[0] = 0;
+      step_flag[2] = 0;
+      __threadfence();
+    }
+    __syncthreads();
+  }
+  pdl_trigger();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, tig = lane & 3;
+  const int nk = h / 16;
+  const int k_begin = blockIdx.y * ksteps_per_slice, k_end = min(nk, k_begin + ksteps_per_slice);
+  float acc[NT][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) acc[t][x] = 0.f;
+  const uint4* wp = reinterpret_cast<const uint4*>(W3) + ((size_t)blockIdx.x * nk * 3) * 32 + lane;
+  // token row of this lane in accumulator tile t: 8 t + g (clamped; rows past B are never stored)
+  const __nv_bfloat16* xrow[NT];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) xrow[t] = X + (size_t)min(8 * t + g, B - 1) * h + 2 * tig;
+  // G steps at a time: every load of the group is issued before its first MMA (the router comes from HBM,
+  // the tokens from the L2; with few tokens a warp's steps would otherwise be a chain of memory latencies)
+  constexpr int G = NT <= 2 ? 4 : (NT <= 4 ? 2 : 1);
+  for (int kt0 = k_begin + warp; kt0 < k_end; kt0 += R3_WARPS * G) {
+    uint4 a[G][3];
+    uint32_t b0[G][NT], b1[G][NT];
+#pragma unroll
+    for (int u = 0; u < G; ++u) {
+      const int kt = min(kt0 + u * R3_WARPS, k_end - 1);  // clamped: a step past the end is loaded but not used
+#pragma unroll
+      for (int pc = 0; pc < 3; ++pc) a[u][pc] = __ldg(wp + (size_t)kt * 96 + pc * 32);
+#pragma unroll
+      for (int t = 0; t < NT; ++t) {
+        b0[u][t] = *reinterpret_cast<const uint32_t*>(xrow[t] + kt * 16);
+        b1[u][t] = *reinterpret_cast<const uint32_t*>(xrow[t] + kt * 16 + 8);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < G; ++u) {
+      if (kt0 + u * R3_WARPS < k_end) {
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          mma_bf16_16816(acc[t], a[u][0], b0[u][t], b1[u][t]);
+          mma_bf16_16816(acc[t], a[u][1], b0[u][t], b1[u][t]);
+          mma_bf16_16816(acc[t], a[u][2], b0[u][t], b1[u][t]);
+        }
+      }
+    }
+  }
+  // add the four warps' partial sums in warp order and store part[slice][token][row]
+  __shared__ float red[R3_WARPS][R3_ROWS][NT * 8 + 1];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) {
+    red[warp][g][t * 8 + 2 * tig] = acc[t][0];
+    red[warp][g][t * 8 + 2 * tig + 1] = acc[t][1];
+    red[warp][g + 8][t * 8 + 2 * tig] = acc[t][2];
+    red[warp][g + 8][t * 8 + 2 * tig + 1] = acc[t][3];
+  }
+  __syncthreads();
+  const int row0 = blockIdx.x * R3_ROWS;
+  for (int i = threadIdx.x; i < R3_ROWS * B; i += R3_WARPS * 32) {
+    const int row = i % R3_ROWS, t = i / R3_ROWS;
+    if (row0 + row < n) {
+      float v = red[0][row][t];
+#pragma unroll
+      for (int w = 1; w < R3_WARPS; ++w) v += red[w][row][t];
+      part[((size_t)blockIdx.y * B + t) * n + row0 + row] = v;
+    }
+  }
+#ifdef DEAMOE_TRACE
+  if (threadIdx.x == 0 && ts) atomicMax(ts + 1, gtime());
+#endif
+}
+
 // ---------------------------------------------------------------- top-k, gate weights, bucketing
 __global__ void __launch_bounds__(TOPK_WARPS * 32)
 k_topk(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
@@ -152,6 +306,25 @@ cudaError_t route_configure(const LayerDev& L) {
 // Router logits straight from the caller's tokens (no fp32 copy): used by the streaming schedules.
 // Returns the number of column slices written (the second grid dimension), or -1.
 int launch_router_logits(const LayerDev& L, const void* tokens, int B, cudaStream_t s, int kslices, int32_t* step_flag) {
+  // More than 16 tokens (three and more groups of eight for the scalar kernel, whose time grows by ~1.5 us per
+  // group: 13 us at 32 tokens, 44 at 128): the tensor-core product on the three-piece router, 7.5 us at 32
+  // tokens.  Up to 16 tokens the scalar kernel's 1024 small CTAs bring the router in faster (4.9 against 6.3 us
+  // for one token on the DeepSeek-V3 shape).
+  if (L.adt == DEAMOE_BF16 && L.router3 && B > 16) {
+    const int nk = L.h / 16, ks = L.router3_slices;
+    const int per = (nk + ks - 1) / ks;
+    dim3 grid((L.n + R3_ROWS - 1) / R3_ROWS, (nk + per - 1) / per);
+    const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(tokens);
+    const int nt = (B + 7) / 8;
+#define DEAMOE_R3(NT) k_router_logits_mma<NT><<<grid, R3_WARPS * 32, 0, s>>>(L.router3, X, L.logit_part, L.n, L.h, B, per, step_flag TS_ARG(L))
+    if (nt <= 1) DEAMOE_R3(1);
+    else if (nt <= 2) DEAMOE_R3(2);
+    else if (nt <= 4) DEAMOE_R3(4);
+    else if (nt <= 8) DEAMOE_R3(8);
+    else DEAMOE_R3(16);
+#undef DEAMOE_R3
+    return cudaGetLastError() == cudaSuccess ? (int)grid.y : -1;
+  }
   const int kslice = (((L.h + kslices - 1) / kslices) + 3) & ~3;
   dim3 grid((L.n + RG - 1) / RG, (L.h + kslice - 1) / kslice);
   if (L.adt == DEAMOE_BF16)
