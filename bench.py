@@ -260,9 +260,11 @@ def run_reference(args, shape, rank, world):
     print(json.dumps(line))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of k_stream divided by its algorithmic bytes, from
-# the committed ncu capture (profiles/k_stream_dsv3-mini_b4.md)
-DRAM_TRAFFIC_RATIO = 1.001
+# dram__bytes_read.sum + dram__bytes_write.sum of the weight-streaming launches divided by their algorithmic
+# bytes, from the committed one-pass ncu captures of the benchmark's own full-size launches
+# (profiles/dram_traffic_full_size_dsv3_b16_b128.md): k_stream at B = 16, and k_dense + k_stream + k_dense at B = 128
+DRAM_TRAFFIC_RATIO = 1.0013
+DRAM_TRAFFIC_RATIO_DENSE = 1.0127
 
 
 def read_only_ceiling(binding, torch, dev, gib=4, reps=6):
@@ -438,9 +440,9 @@ def main():
         achieved = alg / (k_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": alg * DRAM_TRAFFIC_RATIO,
-                "traffic_note": "ESTIMATE: dram read+write bytes of k_stream from the ncu capture in profiles/ "
-                                "(smaller layer of the same matrices), scaled by algorithmic bytes; L2 prefetches of "
-                                "departments that turn out inactive (at most 512 KB per thread block) not included",
+                "traffic_note": "ESTIMATE for this run: its algorithmic bytes x 1.0013, the (dram read + write) / algorithmic "
+                                "ratio that ncu measured on this workload's own k_stream launches (one-pass capture of four "
+                                "full-size launches at B = 16, profiles/dram_traffic_full_size_dsv3_b16_b128.md)",
                 "kernel": "k_stream (the weight-streaming launch(es) of one step)",
                 "kernel_ms": k_ms, "peak_source": peak_src, "algorithmic_bytes_per_launch": alg,
                 "read_only_ceiling_gbs": read_gbs,
@@ -451,9 +453,10 @@ def main():
         if args.schedule == "dense" or (args.schedule == "auto" and B >= 48):
             # dense schedule: the pair of events brackets k_dense, k_stream, k_dense (ordinary launches, back to back)
             roof["kernel"] = "k_dense + k_stream + k_dense (the three weight-streaming launches of a dense step)"
-            roof["traffic_note"] = ("ESTIMATE: dram read+write bytes from the ncu captures of k_stream (1.001 x algorithmic) and "
-                                    "k_dense (1.02 x) in profiles/, scaled by algorithmic bytes")
-            roof["traffic"] = alg * 1.01
+            roof["traffic_note"] = ("ESTIMATE for this run: its algorithmic bytes x 1.0127, the ratio ncu measured on the three "
+                                    "full-size launches of a dense step at B = 128 "
+                                    "(profiles/dram_traffic_full_size_dsv3_b16_b128.md)")
+            roof["traffic"] = alg * DRAM_TRAFFIC_RATIO_DENSE
     else:
         achieved = mean_bytes / (statistics.mean(times_ms) * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -403,7 +403,9 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
       outh = P.Zh; outl = P.Zl; out_stride = L.f; out_row0 = in_row0;
       dep_idx = P.dep_s2 + id;
       dep_target = groups_of(Tall, P.st[ST_S2].tg) * P.st[ST_S2].n_tiles;
-      done_idx = P.dep_s3 + j;
+      // (dense schedule: the last stage runs in a later kernel, nobody polls this counter, and an item
+      // without one spares the epilogue warp its fence and atomic)
+      done_idx = P.dense ? -1 : P.dep_s3 + j;
       break;
     case ST_S4: {
       const int p0 = L.expert_off[id * L.g];
