@@ -40,8 +40,11 @@
 // so a chunk is one contiguous bulk copy.  Layout of an operand chunk (R rows x 64 columns, bf16,
 // "K-major, no swizzle"): 8 x 8 core matrices of 128 contiguous bytes; byte offset of element
 // (r, k) = (r / 8) * 1024 + (k / 8) * 128 + (r % 8) * 16 + (k % 8) * 2.
-// The jobs are dealt round-robin.  Whole tiles fill as many complete rounds as there are; the
-// tiles left over are split into two 64-row halves each, so that the last round is half as long.
+// A job is one tile of one unit.  The CTAs claim the jobs from a counter, one at a time and shortly
+// before their current job's last chunks are issued: CTAs are not served by the memory system at
+// one rate (dealt round-robin, the first CTA was done 95 us before the last of a 320 us launch), and
+// a claimed list ends when the work ends.  The copy role claims and posts each job to the other
+// roles through a small queue in shared memory; the last CTA to finish clears the counter.
 #include "dense.cuh"
 
 #include <cuda.h>  // CUtensorMap and the encode function's signature; the entry point is looked up at run time
@@ -63,6 +66,8 @@ constexpr int DN_B_BYTES = DN_NMAX * DN_BK * 2;   // 8 KB
 constexpr int DN_STAGE_BYTES = DN_A_BYTES + DN_B_BYTES;
 constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5;
 constexpr int DN_THREADS = (DN_WARP_MMA + 1) * 32;
+constexpr int DN_JQ = 4;                    // slots of the CTA's queue of claimed jobs
+constexpr int DN_CLAIM_AHEAD = 6;           // chunks left to issue of a job when the copy role claims the next one
 constexpr int DN_TMEM_COLS = 2 * DN_TILE;   // 2 accumulator buffers; the CTAs of an SM share its 512 columns
 constexpr size_t DN_SMEM = (size_t)DN_AST * DN_STAGE_BYTES + 512 /* barriers, control */;
 constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits (default poll limit); then an error status, never a hang
@@ -100,6 +105,7 @@ struct DenseArgs {
   int nph;
   unsigned spin_limit;  // polls after which a bounded wait gives up
   int withhold;         // failure tests: the copy role issues nothing
+  int32_t* claim;       // [0]: next job of this launch; [1]: CTAs that have finished (the last one clears both)
 };
 // tensor maps of the phases' input planes: [phase][box height 16 / 32 / 64 rows]
 struct DenseMaps {
@@ -187,16 +193,14 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // ---------------------------------------------------------------- job decoding (all roles alike)
 struct Sched {
-  int jobs0;   // whole-tile jobs of phase 0
-  int jobs;    // whole-tile jobs of both phases
-  int full;    // of which this many, a multiple of the grid, are done as whole tiles
-  int n_idx;   // job indices: full + 2 * (jobs - full)
+  int jobs0;   // tile jobs of phase 0
+  int jobs;    // tile jobs of both phases, claimed in this order
 };
 struct Job {
   int phase;
   int T;          // token rows of the unit (0: nothing to do)
   int row0;       // first row of the unit's bucket, in its input plane and in its output
-  int ncols;      // weight rows of the job = accumulator columns: DN_TILE, or half of it for half a tile
+  int ncols;      // weight rows of the job = accumulator columns (DN_TILE)
   int col0;       // output column of accumulator column 0
   const __nv_bfloat16* w;    // the job's part of the tile's first chunk; the next chunk is DN_TILE * DN_BK further
 };
@@ -209,19 +213,15 @@ __device__ __forceinline__ int phase_units(const LayerDev& L, const DensePhase& 
   return (ph.stage == ST_S1 || ph.stage == ST_S4) ? L.counts[CNT_ACTIVE_DEPT] : (B + DN_NMAX - 1) / DN_NMAX;
 }
 
-__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int G, int B) {
+__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int B) {
   Sched s;
   s.jobs0 = phase_units(L, A.ph[0], B) * A.ph[0].tiles;
   s.jobs = s.jobs0 + (A.nph > 1 ? phase_units(L, A.ph[1], B) * A.ph[1].tiles : 0);
-  s.full = (s.jobs / G) * G;
-  s.n_idx = s.full + 2 * (s.jobs - s.full);
   return s;
 }
 
-__device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A, const Sched& sc, int idx, int B) {
+__device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A, const Sched& sc, int tjob, int B) {
   Job j;
-  int tjob = idx, half = -1;
-  if (idx >= sc.full) { tjob = sc.full + ((idx - sc.full) >> 1); half = (idx - sc.full) & 1; }
   j.phase = (tjob >= sc.jobs0) ? 1 : 0;
   const DensePhase& ph = A.ph[j.phase];
   const int local = tjob - (j.phase ? sc.jobs0 : 0);
@@ -244,15 +244,6 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
   j.w = ph.w + woff + (size_t)tile * DN_TILE * ph.K;
   j.ncols = DN_TILE;
   j.col0 = ph.dual ? tile * (DN_TILE / 2) : tile * DN_TILE;
-  if (half >= 0) {
-    if (ph.dual) {
-      if (half == 1) j.T = 0;  // a gate / up tile is not split: its first half-job does all of it
-    } else {
-      j.ncols = DN_TILE / 2;
-      j.col0 += half * (DN_TILE / 2);
-      j.w += (size_t)half * (DN_TILE / 2) * DN_BK;  // the second half of the row groups of every chunk
-    }
-  }
   return j;
 }
 
@@ -264,14 +255,18 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   uint64_t* a_empty = a_full + DN_AST;
   uint64_t* acc_full = a_empty + DN_AST;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* jq_full = acc_empty + 2;     // queue of claimed jobs: the copy role posts, the five other warps read
+  uint64_t* jq_empty = jq_full + DN_JQ;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(jq_empty + DN_JQ);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  static_assert((2 * DN_AST + 4) * 8 + 8 <= 512, "control region");
+  volatile int* jq = abort_flag + 1;     // [DN_JQ] job index, -1: no more jobs
+  static_assert((2 * DN_AST + 4 + 2 * DN_JQ) * 8 + 8 + 4 * DN_JQ <= 512, "control region");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < DN_AST; ++s) { bar_init(&a_full[s], 1); bar_init(&a_empty[s], 1); }
     for (int b = 0; b < 2; ++b) { bar_init(&acc_full[b], 1); bar_init(&acc_empty[b], 4); }
+    for (int q = 0; q < DN_JQ; ++q) { bar_init(&jq_full[q], 1); bar_init(&jq_empty[q], 5); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -287,7 +282,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   const uint32_t tmem_base = *tmem_slot;
 
   const int G = (int)gridDim.x;
-  const Sched sc = make_sched(L, A, G, B);
+  const Sched sc = make_sched(L, A, B);
 
   if (warp == DN_WARP_TMA) {
     // ============================================================ weight chunks -> weight ring
@@ -299,17 +294,30 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
       long long dn_acc[2] = {0, 0};
       const long long dn_start = clock64();
 #endif
-      if (A.withhold) ok = false;  // failure test: nothing is copied, the MMA role's wait for the ring expires
-      for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
+      // failure test: nothing is claimed, posted or copied, and the other roles' wait for a job expires
+      if (A.withhold) ok = false;
+      int idx = ok ? atomicAdd(A.claim, 1) : 0;
+      for (uint32_t jn = 0; ok; ++jn) {
+        // post the claimed job (or the end of the list) to the other roles
+        const int q = (int)(jn % DN_JQ);
+        if (!bar_wait(&jq_empty[q], ((jn / DN_JQ) & 1u) ^ 1u, abort_flag, A.spin_limit)) { ok = false; break; }
+        jq[q] = idx < sc.jobs ? idx : -1;
+        bar_arrive(&jq_full[q]);
+        if (idx >= sc.jobs) break;
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t bytes = (uint32_t)j.ncols * DN_BK * 2;
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
+        int left = groups * nch;   // chunks of this job still to issue
+        int next = -1;
         for (int gi = 0; ok && gi < groups; ++gi) {
           const int bi = box_index(min(DN_NMAX, j.T - gi * DN_NMAX));
           const CUtensorMap* tm = &maps.tm[j.phase][bi];
           const uint32_t box_bytes = (16u << bi) * DN_BK * 2;
-          for (int c = 0; c < nch; ++c, ++g) {
+          for (int c = 0; c < nch; ++c, ++g, --left) {
+            // the next job is claimed shortly before this one's last chunks are issued: late enough that the
+            // CTAs share the end of the list by their speed, early enough that the answer is there in time
+            if (left == DN_CLAIM_AHEAD) next = atomicAdd(A.claim, 1);
             const int s = (int)(g % DN_AST);
             { DN_T0();
             if (!bar_wait(&a_empty[s], ((g / DN_AST) & 1u) ^ 1u, abort_flag, A.spin_limit)) { ok = false; break; }
@@ -320,6 +328,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
             tensor_load_3d(st + DN_A_BYTES, tm, 0, j.row0 + gi * DN_NMAX, c * (DN_BK / 8), &a_full[s]);
           }
         }
+        idx = next >= 0 ? next : atomicAdd(A.claim, 1);  // (a job of fewer chunks than the claim runs ahead)
       }
 #ifdef DEAMOE_TRACE
       dn_trace[blockIdx.x * 16 + 0] = dn_acc[0];
@@ -341,7 +350,12 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
       const uint64_t desc0_w = umma_smem_desc(smem_addr(ring), 128, DN_BK * 16);
       // activation rows as the TMA box leaves them: (box rows x 16) bytes between neighbours along K,
       // 128 between 8-row groups; built per token group below
-      for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
+      for (uint32_t jn = 0; ok; ++jn) {
+        const int q = (int)(jn % DN_JQ);
+        if (!bar_wait(&jq_full[q], (jn / DN_JQ) & 1u, abort_flag, A.spin_limit)) { ok = false; break; }
+        const int idx = jq[q];
+        bar_arrive(&jq_empty[q]);
+        if (idx < 0) break;
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t idesc = umma_instr_desc(DN_NMAX, j.ncols);  // tokens: M operand; weight rows: N operand
@@ -388,7 +402,20 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
     const int e = warp;
     uint32_t a = 0;
     bool ok = true;
-    for (int idx = (int)blockIdx.x; ok && idx < sc.n_idx; idx += G) {
+    for (uint32_t jn = 0; ok; ++jn) {
+      const int q = (int)(jn % DN_JQ);
+      int idx = -1;
+      if (lane == 0) {
+        if (bar_wait(&jq_full[q], (jn / DN_JQ) & 1u, abort_flag, A.spin_limit)) {
+          idx = jq[q];
+          bar_arrive(&jq_empty[q]);
+        } else {
+          ok = false;
+        }
+      }
+      idx = __shfl_sync(0xffffffffu, idx, 0);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (!ok || idx < 0) break;
       const Job j = decode_job(L, A, sc, idx, B);
       const DensePhase& ph = A.ph[j.phase];
       const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
@@ -465,6 +492,10 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
   }
   if (tid == 0 && *abort_flag) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;
+  if (tid == 0 && atomicAdd(A.claim + 1, 1) == G - 1) {  // the last CTA to finish: nobody claims any more
+    A.claim[0] = 0;
+    A.claim[1] = 0;
+  }
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(DN_TMEM_COLS) : "memory");
@@ -524,6 +555,7 @@ struct DensePlan {
   int n_sm;
   unsigned spin_limit;     // DN_SPIN_LIMIT unless a failure test lowered it
   int withhold;
+  int32_t* claim;          // the launches' job counter and count of finished CTAs (zero between launches)
 };
 
 bool dense_supported(const LayerDev& L) {
@@ -558,7 +590,9 @@ deamoe_status_t dense_plan_create(const LayerDev& L, const deamoe_weights_t& w, 
   }
   p->xg_rows = L.max_batch * (L.k < L.m ? L.k : L.m);
   if (cudaMalloc(&p->tiles, total * 2) != cudaSuccess ||
-      cudaMalloc(&p->Xg, (size_t)p->xg_rows * L.h * 2) != cudaSuccess) {
+      cudaMalloc(&p->Xg, (size_t)p->xg_rows * L.h * 2) != cudaSuccess ||
+      cudaMalloc(&p->claim, 2 * sizeof(int32_t)) != cudaSuccess ||
+      cudaMemset(p->claim, 0, 2 * sizeof(int32_t)) != cudaSuccess) {
     cudaGetLastError();
     dense_plan_destroy(p);
     return DEAMOE_ERR_ALLOC;
@@ -614,6 +648,7 @@ void dense_plan_destroy(DensePlan* p) {
   if (!p) return;
   if (p->tiles) cudaFree(p->tiles);
   if (p->Xg) cudaFree(p->Xg);
+  if (p->claim) cudaFree(p->claim);
   delete p;
 }
 
@@ -635,6 +670,7 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
   std::memset(&A, 0, sizeof(A));
   A.nph = n_stages;
   A.spin_limit = p.spin_limit; A.withhold = p.withhold;
+  A.claim = p.claim;
   DenseMaps maps;
   std::memset(&maps, 0, sizeof(maps));
   int launches = 0;
