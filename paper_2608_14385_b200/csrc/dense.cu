@@ -69,6 +69,7 @@ constexpr int DN_THREADS = (DN_WARP_MMA + 1) * 32;
 constexpr int DN_JQ = 4;                    // slots of the CTA's queue of claimed jobs
 constexpr int DN_CLAIM_AHEAD = 6;           // chunks left to issue of a job when the copy role claims the next one
 constexpr int DN_TMEM_COLS = 2 * DN_TILE;   // 2 accumulator buffers; the CTAs of an SM share its 512 columns
+static_assert(DN_TILE == DENSE_TILE_ROWS, "tile height");
 constexpr size_t DN_SMEM = (size_t)DN_AST * DN_STAGE_BYTES + 512 /* barriers, control */;
 constexpr unsigned DN_SPIN_LIMIT = 1u << 22;  // bounded waits (default poll limit); then an error status, never a hang
 static_assert((DN_SMEM + 1024) * DN_CTAS_PER_SM <= 228 * 1024, "shared memory budget");
@@ -106,6 +107,7 @@ struct DenseArgs {
   unsigned spin_limit;  // polls after which a bounded wait gives up
   int withhold;         // failure tests: the copy role issues nothing
   int32_t* claim;       // [0]: next job of this launch; [1]: CTAs that have finished (the last one clears both)
+  int32_t* s1_done;     // first stage: per department, every epilogue warp adds one per finished tile (null: nobody listens)
 };
 // tensor maps of the phases' input planes: [phase][box height 16 / 32 / 64 rows]
 struct DenseMaps {
@@ -198,6 +200,7 @@ struct Sched {
 };
 struct Job {
   int phase;
+  int unit;       // department of the job (first and last stage)
   int T;          // token rows of the unit (0: nothing to do)
   int row0;       // first row of the unit's bucket, in its input plane and in its output
   int ncols;      // weight rows of the job = accumulator columns (DN_TILE)
@@ -227,13 +230,16 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
   const int local = tjob - (j.phase ? sc.jobs0 : 0);
   const int u = local / ph.tiles, tile = local - u * ph.tiles;
   size_t woff = 0;
+  j.unit = 0;
   if (ph.stage == ST_S1) {
     const int id = L.active_dept[u];
+    j.unit = id;
     j.row0 = L.dept_off[id];
     j.T = L.dept_off[id + 1] - j.row0;
     woff = (size_t)(id - L.dept_lo) * ph.unit_elems;  // the tile arrays start at this object's first department
   } else if (ph.stage == ST_S4) {
     const int id = L.active_dept[u];
+    j.unit = id;
     j.row0 = L.expert_off[id * L.g];
     j.T = L.expert_off[(id + 1) * L.g] - j.row0;
     woff = (size_t)(id - L.dept_lo) * ph.unit_elems;
@@ -263,6 +269,9 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   static_assert((2 * DN_AST + 4 + 2 * DN_JQ) * 8 + 8 + 4 * DN_JQ <= 512, "control region");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // The kernel behind this one in the stream may become resident as this grid's CTAs leave (it waits for
+  // what it needs of this grid's results through counters, or for the whole grid).
+  pdl_trigger();
   if (tid == 0) {
     for (int s = 0; s < DN_AST; ++s) { bar_init(&a_full[s], 1); bar_init(&a_empty[s], 1); }
     for (int b = 0; b < 2; ++b) { bar_init(&acc_full[b], 1); bar_init(&acc_empty[b], 4); }
@@ -479,6 +488,13 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
         __syncwarp();
         if (lane == 0) bar_arrive(&acc_empty[buf]);
       }
+      // a finished tile of the first stage counts towards its department: the streaming kernel that runs the
+      // private stages may already be resident and starts an expert when its department's rows are complete
+      if (ok && A.s1_done && ph.stage == ST_S1) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(A.s1_done + j.unit, 1);
+      }
     }
   }
 
@@ -671,6 +687,7 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
   A.nph = n_stages;
   A.spin_limit = p.spin_limit; A.withhold = p.withhold;
   A.claim = p.claim;
+  A.s1_done = io.s1_done;
   DenseMaps maps;
   std::memset(&maps, 0, sizeof(maps));
   int launches = 0;

@@ -32,7 +32,12 @@ struct DenseIO {
   __nv_bfloat16* GU;            // [token-departments, 2f]
   const __nv_bfloat16* Z;       // [pairs, f]
   __nv_bfloat16* Ysh;           // [B, fs]
+  int32_t* s1_done;             // per department: counts DENSE_S1_ARRIVALS per finished tile of its first stage
 };
+// Tile height of the dense kernels and what one finished first-stage tile adds to its department's counter: a
+// department's first stage is complete at DENSE_S1_ARRIVALS * (2 f / DENSE_TILE_ROWS).
+constexpr int DENSE_TILE_ROWS = 128;
+constexpr int DENSE_S1_ARRIVALS = 4;
 int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* stages, int n_stages, int B,
                  cudaStream_t s);
 

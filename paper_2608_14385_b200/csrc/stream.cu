@@ -392,10 +392,11 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
       in_stride = 2 * L.f;
       in_list = L.pair_gurow + L.expert_off[id] + t0;
       outh = P.Yh; outl = P.Yl; out_stride = L.rp; out_row0 = L.expert_off[id] + t0;
-      if (!P.dense) {  // (dense schedule: the first stage ran in an earlier kernel)
-        dep_idx = P.dep_s1 + j;
+      dep_idx = P.dep_s1 + j;
+      if (P.dense)  // the first stage runs in the tensor-core kernel, which may still be running: its count per department
+        dep_target = DENSE_S1_ARRIVALS * (2 * L.f / DENSE_TILE_ROWS);
+      else
         dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
-      }
       done_idx = P.dep_s2 + id;
       break;
     case ST_S3:
@@ -1238,6 +1239,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         }
       }
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    } else if (check_deps & 16) {
+      // dense schedule: the preceding kernel is the first tensor-core launch, which started after the routing
+      // had completed; the list is there, and what the items need of that launch they await item by item
     } else {
       pdl_wait();
       waited = true;
@@ -1981,13 +1985,15 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
     DenseIO io;
     io.tokens = reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw);
     io.GU = p.dev.GUh; io.Z = p.dev.Zh; io.Ysh = p.dev.Yshh;
+    io.s1_done = p.dev.sync + SY_DEP + p.dev.dep_s1;
     // (the shared expert's tiles first: every token passes through them, which makes them the longest jobs, and
     // jobs claimed from a counter finish closest together when the longest are claimed first)
     const int first[2] = {ST_SH1, ST_S1}, last[2] = {ST_SH2, ST_S4};
     const int o = L.n_shared ? 0 : 1;
     const int n1 = dense_launch(*p.dense, L, io, first + o, 2 - o, B, s);
     if (n1 < 0) return -1;
-    k_stream<<<p.grid, STREAM_THREADS, STREAM_SMEM, s>>>(L, p.dev_dense, B, -1, 1);
+    // resident as soon as the tensor-core kernel's CTAs leave room; an expert's items wait for its department's rows
+    launch_pdl(k_stream, dim3(p.grid), dim3(STREAM_THREADS), STREAM_SMEM, s, L, p.dev_dense, B, -1, 1 | 16);
     const int n2 = dense_launch(*p.dense, L, io, last + o, 2 - o, B, s);
     if (n2 < 0) return -1;
     launches += n1 + 1 + n2;
