@@ -108,6 +108,8 @@ struct DenseArgs {
   int withhold;         // failure tests: the copy role issues nothing
   int32_t* claim;       // [0]: next job of this launch; [1]: CTAs that have finished (the last one clears both)
   int32_t* s1_done;     // first stage: per department, every epilogue warp adds one per finished tile (null: nobody listens)
+  const int32_t* gathered;  // launched beside the routing: CTAs of the gather kernel that are done (null: an ordinary launch)
+  int gather_ctas;
 };
 // tensor maps of the phases' input planes: [phase][box height 16 / 32 / 64 rows]
 struct DenseMaps {
@@ -191,12 +193,18 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
 }
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---------------------------------------------------------------- job decoding (all roles alike)
 struct Sched {
-  int jobs0;   // tile jobs of phase 0
-  int jobs;    // tile jobs of both phases, claimed in this order
+  int free_jobs;  // jobs at the head of the list that need nothing of the routing (the shared expert's, as phase 0)
+  int jobs0;      // tile jobs of phase 0
+  int jobs;       // tile jobs of both phases, claimed in this order
 };
 struct Job {
   int phase;
@@ -212,12 +220,22 @@ struct Job {
 // of the batch.  (A department's bucket of more than DN_NMAX rows is rare and stays one job that
 // passes over its tile once per group; the shared expert sees every token, so from 65 tokens on
 // each of its groups is a job of its own: jobs of one length deal out evenly.)
+__device__ __forceinline__ bool phase_routed(const DensePhase& ph) { return ph.stage == ST_S1 || ph.stage == ST_S4; }
 __device__ __forceinline__ int phase_units(const LayerDev& L, const DensePhase& ph, int B) {
-  return (ph.stage == ST_S1 || ph.stage == ST_S4) ? L.counts[CNT_ACTIVE_DEPT] : (B + DN_NMAX - 1) / DN_NMAX;
+  return phase_routed(ph) ? __ldcg(L.counts + CNT_ACTIVE_DEPT) : (B + DN_NMAX - 1) / DN_NMAX;
 }
 
-__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int B) {
+// The list as far as it is known before the routing: the shared expert's jobs, if they come first.
+__device__ __forceinline__ Sched head_sched(const LayerDev& L, const DenseArgs& A, int B) {
   Sched s;
+  s.free_jobs = phase_routed(A.ph[0]) ? 0 : phase_units(L, A.ph[0], B) * A.ph[0].tiles;
+  s.jobs0 = s.free_jobs;
+  s.jobs = s.free_jobs;
+  return s;
+}
+// The whole list (reads the routing state).
+__device__ __forceinline__ Sched make_sched(const LayerDev& L, const DenseArgs& A, int B) {
+  Sched s = head_sched(L, A, B);
   s.jobs0 = phase_units(L, A.ph[0], B) * A.ph[0].tiles;
   s.jobs = s.jobs0 + (A.nph > 1 ? phase_units(L, A.ph[1], B) * A.ph[1].tiles : 0);
   return s;
@@ -232,16 +250,16 @@ __device__ __forceinline__ Job decode_job(const LayerDev& L, const DenseArgs& A,
   size_t woff = 0;
   j.unit = 0;
   if (ph.stage == ST_S1) {
-    const int id = L.active_dept[u];
+    const int id = __ldcg(L.active_dept + u);
     j.unit = id;
-    j.row0 = L.dept_off[id];
-    j.T = L.dept_off[id + 1] - j.row0;
+    j.row0 = __ldcg(L.dept_off + id);
+    j.T = __ldcg(L.dept_off + id + 1) - j.row0;
     woff = (size_t)(id - L.dept_lo) * ph.unit_elems;  // the tile arrays start at this object's first department
   } else if (ph.stage == ST_S4) {
-    const int id = L.active_dept[u];
+    const int id = __ldcg(L.active_dept + u);
     j.unit = id;
-    j.row0 = L.expert_off[id * L.g];
-    j.T = L.expert_off[(id + 1) * L.g] - j.row0;
+    j.row0 = __ldcg(L.expert_off + id * L.g);
+    j.T = __ldcg(L.expert_off + (id + 1) * L.g) - j.row0;
     woff = (size_t)(id - L.dept_lo) * ph.unit_elems;
   } else {
     j.row0 = u * DN_NMAX;  // shared expert: unit u = token group u
@@ -291,7 +309,14 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   const uint32_t tmem_base = *tmem_slot;
 
   const int G = (int)gridDim.x;
-  const Sched sc = make_sched(L, A, B);
+  // Launched programmatically behind the kernel that gathers the first stage's token rows, this grid may be
+  // running before the routing is done.  It starts with the jobs that need nothing of the routing; before the
+  // first job that does, the copy role waits (bounded) until every CTA of the gather kernel has counted itself
+  // done, which also says that the departments' token lists are published.  (Not griddepcontrol.wait: that
+  // waits for the routing kernel's end as well, and the first stage needs only what that kernel publishes early.)
+  // The other roles learn of a job from the copy role, so what it has seen they may read.
+  Sched sc = head_sched(L, A, B);
+  bool routed = false;
 
   if (warp == DN_WARP_TMA) {
     // ============================================================ weight chunks -> weight ring
@@ -310,6 +335,19 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
         // post the claimed job (or the end of the list) to the other roles
         const int q = (int)(jn % DN_JQ);
         if (!bar_wait(&jq_empty[q], ((jn / DN_JQ) & 1u) ^ 1u, abort_flag, A.spin_limit)) { ok = false; break; }
+        if (idx >= sc.free_jobs && !routed) {
+          if (A.gathered) {
+            unsigned spins = 0;
+            while (ld_acquire_gpu(A.gathered) < A.gather_ctas) {
+              __nanosleep(64);
+              if (++spins > A.spin_limit / 16 || *abort_flag) { *abort_flag = 1; ok = false; break; }
+            }
+            if (!ok) break;
+            asm volatile("fence.proxy.async;" ::: "memory");  // the gathered rows were stored, the boxes are read by TMA
+          }
+          routed = true;
+          sc = make_sched(L, A, B);
+        }
         jq[q] = idx < sc.jobs ? idx : -1;
         bar_arrive(&jq_full[q]);
         if (idx >= sc.jobs) break;
@@ -365,6 +403,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
         const int idx = jq[q];
         bar_arrive(&jq_empty[q]);
         if (idx < 0) break;
+        if (idx >= sc.free_jobs && !routed) { routed = true; sc = make_sched(L, A, B); }
         const Job j = decode_job(L, A, sc, idx, B);
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t idesc = umma_instr_desc(DN_NMAX, j.ncols);  // tokens: M operand; weight rows: N operand
@@ -425,6 +464,7 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
       idx = __shfl_sync(0xffffffffu, idx, 0);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       if (!ok || idx < 0) break;
+      if (idx >= sc.free_jobs && !routed) { routed = true; sc = make_sched(L, A, B); }
       const Job j = decode_job(L, A, sc, idx, B);
       const DensePhase& ph = A.ph[j.phase];
       const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
@@ -545,13 +585,36 @@ __global__ void k_pack_tiles(const __nv_bfloat16* __restrict__ src, __nv_bfloat1
 
 // First stage's input: the tokens of every department's bucket X^j (Section 3.2), in bucket order.
 // Row r of Xg = token dept_tok[r]; one block per row, 16 bytes per thread and step.
-__global__ void k_gather_buckets(LayerDev L, const __nv_bfloat16* __restrict__ tokens, __nv_bfloat16* __restrict__ Xg) {
-  const int rows = L.counts[CNT_TOKEN_DEPT];
+// Launched programmatically behind the routing kernel: waits (bounded) for that kernel's word that the
+// departments' token lists are published, which is well before its end.
+__global__ void k_gather_buckets(LayerDev L, const __nv_bfloat16* __restrict__ tokens, __nv_bfloat16* __restrict__ Xg,
+                                 const int32_t* __restrict__ routed_flag, int32_t* __restrict__ gathered,
+                                 unsigned spin_limit) {
+  pdl_trigger();
+  __shared__ int s_ok;
+  if (threadIdx.x == 0) {
+    int ok = 1;
+    unsigned spins = 0;
+    while (routed_flag && ld_acquire_gpu(routed_flag) == 0) {
+      __nanosleep(64);
+      if (++spins > spin_limit / 16) { ok = 0; break; }
+    }
+    if (!ok) L.counts[CNT_STATUS] = DEAMOE_ERR_TIMEOUT;
+    s_ok = ok;
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  const int rows = __ldcg(L.counts + CNT_TOKEN_DEPT);
   const int v = L.h / 8;
   for (int r = (int)blockIdx.x; r < rows; r += (int)gridDim.x) {
-    const int4* src = reinterpret_cast<const int4*>(tokens + (size_t)L.dept_tok[r] * L.h);
+    const int4* src = reinterpret_cast<const int4*>(tokens + (size_t)__ldcg(L.dept_tok + r) * L.h);
     int4* dst = reinterpret_cast<int4*>(Xg + (size_t)r * L.h);
     for (int i = (int)threadIdx.x; i < v; i += (int)blockDim.x) dst[i] = src[i];
+  }
+  if (gathered) {  // this CTA's rows are stored: count it in for the tensor-core kernel that may already be waiting
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) atomicAdd(gathered, 1);
   }
 }
 
@@ -691,6 +754,7 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
   DenseMaps maps;
   std::memset(&maps, 0, sizeof(maps));
   int launches = 0;
+  bool chained = false;
   for (int i = 0; i < n_stages; ++i) {
     DensePhase& ph = A.ph[i];
     ph.stage = stages[i];
@@ -701,7 +765,11 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
         ph.K = L.h; ph.tiles = 2 * L.f / DN_TILE; ph.dual = 0; ph.epi = DE_SIGMA;
         ph.w = p.tiles + p.o_gu; ph.unit_elems = p.e_gu;
         in = p.Xg; in_rows = p.xg_rows; ph.outh = io.GU; ph.out_stride = 2 * L.f;
-        k_gather_buckets<<<2 * p.n_sm, 256, 0, s>>>(L, io.tokens, p.Xg);
+        if (launch_pdl(k_gather_buckets, dim3(2 * p.n_sm), dim3(256), 0, s, L, io.tokens, p.Xg, io.routed_flag,
+                       io.gathered, io.spin_limit ? io.spin_limit : DN_SPIN_LIMIT) != cudaSuccess)
+          return -1;
+        chained = io.routed_flag != nullptr && io.gathered != nullptr;
+        if (chained) { A.gathered = io.gathered; A.gather_ctas = 2 * p.n_sm; }
         ++launches;
         break;
       case ST_S4:
@@ -726,7 +794,11 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
       if (!encode_rows_map(p, &maps.tm[i][b], in, in_rows, ph.K, 16 << b)) return -1;
   }
   if (n_stages == 1) std::memcpy(maps.tm[1], maps.tm[0], sizeof(maps.tm[0]));
-  k_dense<<<p.n_sm * DN_CTAS_PER_SM, DN_THREADS, DN_SMEM, s>>>(L, A, B, maps);
+  if (chained) {  // behind the gather kernel, possibly beside the end of the routing
+    if (launch_pdl(k_dense, dim3(p.n_sm * DN_CTAS_PER_SM), dim3(DN_THREADS), DN_SMEM, s, L, A, B, maps) != cudaSuccess) return -1;
+  } else {
+    k_dense<<<p.n_sm * DN_CTAS_PER_SM, DN_THREADS, DN_SMEM, s>>>(L, A, B, maps);
+  }
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }

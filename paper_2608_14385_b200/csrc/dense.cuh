@@ -33,6 +33,9 @@ struct DenseIO {
   const __nv_bfloat16* Z;       // [pairs, f]
   __nv_bfloat16* Ysh;           // [B, fs]
   int32_t* s1_done;             // per department: counts DENSE_S1_ARRIVALS per finished tile of its first stage
+  const int32_t* routed_flag;   // set by the routing kernel once the departments' token lists are published
+  int32_t* gathered;            // cleared by the step's router kernel: CTAs of the gather kernel that are done
+  unsigned spin_limit;          // polls after which the wait for that flag gives up
 };
 // Tile height of the dense kernels and what one finished first-stage tile adds to its department's counter: a
 // department's first stage is complete at DENSE_S1_ARRIVALS * (2 f / DENSE_TILE_ROWS).

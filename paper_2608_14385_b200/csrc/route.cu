@@ -46,6 +46,7 @@ k_router_logits(const float* __restrict__ Wr, const XT* __restrict__ x32, float*
     if (threadIdx.x == 0) {
       step_flag[0] = 0;
       step_flag[2] = 0;  // two words further: the flag that the rest of the work list exists
+      step_flag[3] = 0;  // and the dense schedule's count of finished CTAs of its gather kernel
       __threadfence();
     }
     __syncthreads();
@@ -203,6 +204,7 @@ k_router_logits_mma(const __nv_bfloat16* __restrict__ W3, const __nv_bfloat16* _
     if (threadIdx.x == 0) {
       step_flag[0] = 0;
       step_flag[2] = 0;
+      step_flag[3] = 0;
       __threadfence();
     }
     __syncthreads();

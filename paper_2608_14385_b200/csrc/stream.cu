@@ -489,7 +489,8 @@ static __device__ void write_seg(const LayerDev& L, const StreamDev& P, int stag
 // category after category, a block-wide exclusive scan of their token-group counts gives each
 // unit the index of its first segment record, and the thread writes the unit's records.
 // `s_excl` is shared-memory scratch for one int per unit (at most 2 m + 2 n + 2 of them).
-static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B, int* s_excl, bool early_done) {
+static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int B, int* s_excl, bool counters_zeroed,
+                                      bool early_done) {
   __shared__ int s_ubase[MAX_CAT + 1], s_segbase[MAX_CAT + 1], s_itembase[MAX_CAT + 1], s_wsum[32], s_carry;
   // the category list lives in shared memory: a per-thread array indexed with a run-time index would
   // sit in local memory and give the kernel a stack frame
@@ -499,7 +500,7 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
   if (tid == 0) s_ncat = category_list(L, P, cats);
   __syncthreads();
   const int ncat = s_ncat;
-  if (!early_done)  // else early_first_stage() has zeroed the counters, and the first stage may be running
+  if (!counters_zeroed)  // else an early hand-over has zeroed the counters, and the first stage may be running
 #pragma unroll 1
     for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
   if (tid == 0) {
@@ -711,6 +712,27 @@ static __host__ __device__ FinishSmem finish_layout(int n, int m, int k, int B) 
   return f;
 }
 
+// Dense schedule: the tensor-core kernel of the first stage needs the departments' token lists and nothing
+// else of the routing.  Publish those as soon as they exist (the rest of the routing state follows at this
+// kernel's end, as always), zero the step's counters, which that kernel counts into, and raise the flag that
+// the kernels queued behind this one wait for.  S: the routing arrays in shared memory; L: in global memory.
+static __device__ void dense_hand_over(const LayerDev& S, const LayerDev& L, const StreamDev& P) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+#pragma unroll 1
+  for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
+  const int td = S.counts[CNT_TOKEN_DEPT], na = S.counts[CNT_ACTIVE_DEPT];
+#pragma unroll 1
+  for (int j = tid; j <= L.m; j += nthr) L.dept_off[j] = S.dept_off[j];
+#pragma unroll 1
+  for (int j = tid; j < td; j += nthr) L.dept_tok[j] = S.dept_tok[j];
+#pragma unroll 1
+  for (int j = tid; j < na; j += nthr) L.active_dept[j] = S.active_dept[j];
+  if (tid == 0) { L.counts[CNT_ACTIVE_DEPT] = na; L.counts[CNT_TOKEN_DEPT] = td; }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) st_release(P.sync + SY_DEP + P.early_flag, 1);  // cleared again by the next step's router kernel
+}
+
 // Top-k + gate weights in a grid of their own: one warp per token over as many CTAs as it takes,
 // instead of the routing tail's one CTA ranking its tokens sixteen at a time.  Used when a call has
 // more tokens than the tail has warps, in the dense schedule, and for routers of more than 256
@@ -795,6 +817,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   bucket_departments(S, B, s_dyn, FINISH_THREADS);
   TS_MIN(L, 17);
   int* early_scr = reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B);  // after the masks and offsets
+  if (P.dense) dense_hand_over(S, L, P);
   if (P.early && P.early_stage == ST_S1) early_first_stage<ST_S1>(S, P, B, early_scr);
   bucket_experts(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
@@ -803,8 +826,8 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   long long tt2 = clock64();
   TS_MIN(L, 13);
 #endif
-  worklist_block(S, P, B, reinterpret_cast<int*>(s_dyn), P.early != 0);
-  if (P.early) {
+  worklist_block(S, P, B, reinterpret_cast<int*>(s_dyn), P.early != 0 || P.dense != 0, P.early != 0);
+  if (P.early || P.dense) {
     // the rest of the work list is complete: tell the streaming kernel now rather than through this
     // kernel's completion, which comes only after the routing state has been published (on a small
     // layer the streaming kernel has finished the first stage by then and would wait)
@@ -1229,7 +1252,9 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
     // The rest of the work list is complete when the routing kernel says so (fused schedule of a
     // layer with the early hand-over: a second flag) or when it has completed.
     bool waited = false;  // for the routing kernel's completion
-    if (P.early && cat < 0) {
+    if ((P.early && cat < 0) || (check_deps & 16)) {
+      // (dense schedule, check_deps & 16: the kernel in front of this one is the first tensor-core launch, which
+      // runs beside the end of the routing; what the items need of that launch they await item by item)
       if (lane == 0) {
         const int32_t* flag = P.sync + SY_DEP + P.early_flag + 2;
         unsigned spins = 0;
@@ -1239,9 +1264,6 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
         }
       }
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-    } else if (check_deps & 16) {
-      // dense schedule: the preceding kernel is the first tensor-core launch, which started after the routing
-      // had completed; the list is there, and what the items need of that launch they await item by item
     } else {
       pdl_wait();
       waited = true;
@@ -1919,7 +1941,7 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
                  int32_t* user_idx, float* user_w) {
   const StreamDev& dv = takes_dense(p, B) ? p.dev_dense : p.dev;
   const int ny = launch_router_logits(L, tokens, B, s, kslices,
-                                      dv.early ? dv.sync + SY_DEP + dv.early_flag : nullptr);
+                                      (dv.early || dv.dense) ? dv.sync + SY_DEP + dv.early_flag : nullptr);
   if (ny < 0) return -1;
   const int per_warp = (L.n * 5 + 15) & ~15;
   const bool in_regs = topk_in_registers(L);
@@ -1986,6 +2008,9 @@ int stream_forward(StreamPlan& p, const LayerDev& L, int B, cudaStream_t s) {
     io.tokens = reinterpret_cast<const __nv_bfloat16*>(L.tokens_raw);
     io.GU = p.dev.GUh; io.Z = p.dev.Zh; io.Ysh = p.dev.Yshh;
     io.s1_done = p.dev.sync + SY_DEP + p.dev.dep_s1;
+    io.routed_flag = p.dev.sync + SY_DEP + p.dev.early_flag;
+    io.gathered = p.dev.sync + SY_DEP + p.dev.early_flag + 3;  // cleared by the step's router kernel, like the flags
+    io.spin_limit = p.dev_dense.spin_limit;
     // (the shared expert's tiles first: every token passes through them, which makes them the longest jobs, and
     // jobs claimed from a counter finish closest together when the longest are claimed first)
     const int first[2] = {ST_SH1, ST_S1}, last[2] = {ST_SH2, ST_S4};
