@@ -395,7 +395,7 @@ def main():
             dist.destroy_process_group()
         return
     B = args.batch
-    # (sized for the largest batch of the sweep; from 48 tokens on AUTO takes the dense schedule)
+    # (sized for the largest batch of the sweep; from 32 tokens on AUTO takes the dense schedule)
     max_batch = max(64 if shape.name in synth.PAPER_BASELINES else (128 if shape.name == "dsv3" and not args.no_sweep else 32), B)
     w = synth.make_deamoe_weights(shape, 0, dev)
     layer = binding.Layer(shape, w, max_batch, sched)
@@ -450,7 +450,7 @@ def main():
                                           "`peak` is a read+write copy figure, which a read-only stream may exceed",
                 "frac_of_read_only_ceiling": achieved / read_gbs if read_gbs else None,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
-        if args.schedule == "dense" or (args.schedule == "auto" and B >= 48):
+        if args.schedule == "dense" or (args.schedule == "auto" and B >= binding.DENSE_MIN_BATCH):
             # dense schedule: the pair of events brackets k_dense, k_stream, k_dense (ordinary launches, back to back)
             roof["kernel"] = "k_dense + k_stream + k_dense (the three weight-streaming launches of a dense step)"
             roof["traffic_note"] = ("ESTIMATE for this run: its algorithmic bytes x 1.0127, the ratio ncu measured on the three "

@@ -79,7 +79,7 @@ typedef enum {
                               cores, private matrices in the streaming kernel.  bf16 weights and
                               tokens, a DeaMoE layer with private matrices, h a multiple of 256,
                               f and shared_ffn of 128; else UNSUPPORTED.  AUTO takes this schedule by
-                              itself for calls of 48 tokens and more on layers that support it. */
+                              itself for calls of 32 tokens and more on layers that support it. */
 } deamoe_schedule_t;
 
 /*

@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdeamoe.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_BATCH, ERR_TIMEOUT, ERR_INTERNAL = range(8)
+DENSE_MIN_BATCH = 32   # calls of this many tokens and more take the dense schedule under SCHED_AUTO (DENSE_MIN_BATCH in csrc/dense.cuh)
 F32, BF16 = 0, 1
 SIGMA_NONE, SIGMA_SILU, SIGMA_GELU, SIGMA_RMSNORM = 0, 1, 2, 3
 SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4

@@ -216,6 +216,15 @@ struct Job {
   const __nv_bfloat16* w;    // the job's part of the tile's first chunk; the next chunk is DN_TILE * DN_BK further
 };
 
+__device__ __forceinline__ void put_job(volatile Job* q, const Job& j) {
+  q->phase = j.phase; q->unit = j.unit; q->T = j.T; q->row0 = j.row0; q->ncols = j.ncols; q->col0 = j.col0; q->w = j.w;
+}
+__device__ __forceinline__ Job get_job(const volatile Job* q) {
+  Job j;
+  j.phase = q->phase; j.unit = q->unit; j.T = q->T; j.row0 = q->row0; j.ncols = q->ncols; j.col0 = q->col0; j.w = q->w;
+  return j;
+}
+
 // Units of a phase: the active departments, or, for the shared expert, the groups of DN_NMAX tokens
 // of the batch.  (A department's bucket of more than DN_NMAX rows is rare and stays one job that
 // passes over its tile once per group; the shared expert sees every token, so from 65 tokens on
@@ -283,8 +292,10 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
   uint64_t* jq_empty = jq_full + DN_JQ;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(jq_empty + DN_JQ);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* jq = abort_flag + 1;     // [DN_JQ] job index, -1: no more jobs
-  static_assert((2 * DN_AST + 4 + 2 * DN_JQ) * 8 + 8 + 4 * DN_JQ <= 512, "control region");
+  // [DN_JQ] decoded jobs (phase -1: no more jobs): the copy role reads the routing state, the other roles
+  // have no global-memory latency at a job's start
+  volatile Job* jq = reinterpret_cast<volatile Job*>(abort_flag + 1);
+  static_assert(sizeof(Job) == 32 && (2 * DN_AST + 4 + 2 * DN_JQ) * 8 + 8 + sizeof(Job) * DN_JQ <= 512, "control region");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // The kernel behind this one in the stream may become resident as this grid's CTAs leave (it waits for
@@ -348,10 +359,12 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
           routed = true;
           sc = make_sched(L, A, B);
         }
-        jq[q] = idx < sc.jobs ? idx : -1;
+        Job j;
+        j.phase = -1;
+        if (idx < sc.jobs) j = decode_job(L, A, sc, idx, B);
+        put_job(&jq[q], j);
         bar_arrive(&jq_full[q]);
-        if (idx >= sc.jobs) break;
-        const Job j = decode_job(L, A, sc, idx, B);
+        if (j.phase < 0) break;
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t bytes = (uint32_t)j.ncols * DN_BK * 2;
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
@@ -400,11 +413,9 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
       for (uint32_t jn = 0; ok; ++jn) {
         const int q = (int)(jn % DN_JQ);
         if (!bar_wait(&jq_full[q], (jn / DN_JQ) & 1u, abort_flag, A.spin_limit)) { ok = false; break; }
-        const int idx = jq[q];
+        const Job j = get_job(&jq[q]);
         bar_arrive(&jq_empty[q]);
-        if (idx < 0) break;
-        if (idx >= sc.free_jobs && !routed) { routed = true; sc = make_sched(L, A, B); }
-        const Job j = decode_job(L, A, sc, idx, B);
+        if (j.phase < 0) break;
         const int nch = A.ph[j.phase].K / DN_BK;
         const uint32_t idesc = umma_instr_desc(DN_NMAX, j.ncols);  // tokens: M operand; weight rows: N operand
         const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
@@ -452,20 +463,13 @@ __global__ void __launch_bounds__(DN_THREADS, DN_CTAS_PER_SM) k_dense(LayerDev L
     bool ok = true;
     for (uint32_t jn = 0; ok; ++jn) {
       const int q = (int)(jn % DN_JQ);
-      int idx = -1;
-      if (lane == 0) {
-        if (bar_wait(&jq_full[q], (jn / DN_JQ) & 1u, abort_flag, A.spin_limit)) {
-          idx = jq[q];
-          bar_arrive(&jq_empty[q]);
-        } else {
-          ok = false;
-        }
-      }
-      idx = __shfl_sync(0xffffffffu, idx, 0);
-      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-      if (!ok || idx < 0) break;
-      if (idx >= sc.free_jobs && !routed) { routed = true; sc = make_sched(L, A, B); }
-      const Job j = decode_job(L, A, sc, idx, B);
+      if (lane == 0 && !bar_wait(&jq_full[q], (jn / DN_JQ) & 1u, abort_flag, A.spin_limit)) ok = false;
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;   // (also orders lane 0's wait before every lane's read)
+      if (!ok) break;
+      const Job j = get_job(&jq[q]);
+      __syncwarp();
+      if (lane == 0) bar_arrive(&jq_empty[q]);
+      if (j.phase < 0) break;
       const DensePhase& ph = A.ph[j.phase];
       const int groups = (j.T + DN_NMAX - 1) / DN_NMAX;
       const int nout = ph.dual ? DN_TILE / 2 : j.ncols;  // outputs per token
@@ -604,12 +608,28 @@ __global__ void k_gather_buckets(LayerDev L, const __nv_bfloat16* __restrict__ t
   }
   __syncthreads();
   if (!s_ok) return;
+  // 16-byte words of all rows dealt over all threads, four loads in flight per thread (this copy sits between
+  // the routing and the first stage, with nothing to overlap it but the shared expert's tiles)
   const int rows = __ldcg(L.counts + CNT_TOKEN_DEPT);
   const int v = L.h / 8;
-  for (int r = (int)blockIdx.x; r < rows; r += (int)gridDim.x) {
-    const int4* src = reinterpret_cast<const int4*>(tokens + (size_t)__ldcg(L.dept_tok + r) * L.h);
-    int4* dst = reinterpret_cast<int4*>(Xg + (size_t)r * L.h);
-    for (int i = (int)threadIdx.x; i < v; i += (int)blockDim.x) dst[i] = src[i];
+  const int total = rows * v, nthr = (int)(gridDim.x * blockDim.x);
+  const int4* src = reinterpret_cast<const int4*>(tokens);
+  int4* dst = reinterpret_cast<int4*>(Xg);
+  for (int i0 = (int)(blockIdx.x * blockDim.x + threadIdx.x); i0 < total; i0 += 4 * nthr) {
+    int4 val[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * nthr;
+      if (i < total) {
+        const int r = i / v, c = i - r * v;
+        val[u] = __ldg(src + (size_t)__ldcg(L.dept_tok + r) * v + c);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * nthr;
+      if (i < total) dst[i] = val[u];
+    }
   }
   if (gathered) {  // this CTA's rows are stored: count it in for the tensor-core kernel that may already be waiting
     __threadfence();

@@ -8,7 +8,7 @@ namespace deamoe {
 struct DensePlan;
 
 // Batches from this size on take the dense schedule when the layer has one (DEAMOE_SCHED_AUTO).
-constexpr int DENSE_MIN_BATCH = 48;  // measured crossover on the DeepSeek-V3 shape: about 46 tokens
+constexpr int DENSE_MIN_BATCH = 32;  // measured crossover on the DeepSeek-V3 shape: about 28 tokens
 
 // True if the layer's shapes and dtypes fit the dense kernels (bf16 weights and activations, a
 // DeaMoE layer with private matrices, h a multiple of 256, f and shared_ffn of 128).

@@ -67,7 +67,7 @@ def test_dense_schedule_is_refused_for_layers_it_cannot_run():
 
 
 def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
-    """One AUTO layer sized for 128 tokens: up to 47 tokens take the streaming schedule, 48 and more the dense one;
+    """One AUTO layer sized for 128 tokens: up to 31 tokens take the streaming schedule, 32 and more the dense one;
     each agrees with a layer fixed to that schedule bit for bit, and the two schedules agree within
     the tolerance (they round intermediates alike but sum in different orders)."""
     shape = DENSE_WIDE
@@ -76,13 +76,13 @@ def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
     fused = binding.Layer(shape, w, 128, binding.SCHED_FUSED)
     dense = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
     try:
-        for B in (16, 47, 48, 64, 128):
+        for B in (16, 31, 32, 64, 128):
             x = synth.make_tokens(shape, B, 14 + B, torch.device("cuda:0"))
             oa, of, od = auto.forward(x).float(), fused.forward(x).float(), dense.forward(x).float()
             torch.cuda.synchronize()
             for layer in (auto, fused, dense):
                 assert layer.stats()["device_status"] == 0
-            same = of if B < 48 else od
+            same = of if B < binding.DENSE_MIN_BATCH else od
             assert torch.equal(oa, same)
             ok, err, bound = within_tolerance(od.cpu().numpy().astype(np.float64), of.cpu().numpy().astype(np.float64))
             assert ok, f"{err:.3e} > {bound:.3e}"
