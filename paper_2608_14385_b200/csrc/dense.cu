@@ -608,27 +608,20 @@ __global__ void k_gather_buckets(LayerDev L, const __nv_bfloat16* __restrict__ t
   }
   __syncthreads();
   if (!s_ok) return;
-  // 16-byte words of all rows dealt over all threads, four loads in flight per thread (this copy sits between
-  // the routing and the first stage, with nothing to overlap it but the shared expert's tiles)
   const int rows = __ldcg(L.counts + CNT_TOKEN_DEPT);
   const int v = L.h / 8;
-  const int total = rows * v, nthr = (int)(gridDim.x * blockDim.x);
-  const int4* src = reinterpret_cast<const int4*>(tokens);
-  int4* dst = reinterpret_cast<int4*>(Xg);
-  for (int i0 = (int)(blockIdx.x * blockDim.x + threadIdx.x); i0 < total; i0 += 4 * nthr) {
-    int4 val[4];
+  for (int r = (int)blockIdx.x; r < rows; r += (int)gridDim.x) {
+    const int4* src = reinterpret_cast<const int4*>(tokens + (size_t)__ldcg(L.dept_tok + r) * L.h);
+    int4* dst = reinterpret_cast<int4*>(Xg + (size_t)r * L.h);
+    // four loads in flight per thread (this copy sits between the routing and the first stage)
+    for (int i0 = (int)threadIdx.x; i0 < v; i0 += 4 * (int)blockDim.x) {
+      int4 val[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = i0 + u * nthr;
-      if (i < total) {
-        const int r = i / v, c = i - r * v;
-        val[u] = __ldg(src + (size_t)__ldcg(L.dept_tok + r) * v + c);
-      }
-    }
+      for (int u = 0; u < 4; ++u)
+        if (i0 + u * (int)blockDim.x < v) val[u] = __ldg(src + i0 + u * (int)blockDim.x);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = i0 + u * nthr;
-      if (i < total) dst[i] = val[u];
+      for (int u = 0; u < 4; ++u)
+        if (i0 + u * (int)blockDim.x < v) dst[i0 + u * (int)blockDim.x] = val[u];
     }
   }
   if (gathered) {  // this CTA's rows are stored: count it in for the tensor-core kernel that may already be waiting

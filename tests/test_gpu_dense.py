@@ -127,6 +127,34 @@ def test_dense_step_can_be_captured_in_a_cuda_graph_and_replayed():
         layer.close()
 
 
+def test_dense_steps_of_changing_batch_on_one_layer_leave_no_state_behind():
+    """Steps of very different token counts queued on one dense layer without a synchronisation in between:
+    the hand-over words of a step (the routing kernel's flags, the count of finished gather CTAs, the job
+    counter of the tensor-core launches, the departments' completion counters) are all reused by the next,
+    which may start while the previous step's last kernels drain.  Every output must equal, bit for bit, the
+    one a fresh layer gives for that batch alone."""
+    shape = DENSE_WIDE
+    w = _scaled(shape, 16, scale=6.0)
+    layer = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
+    try:
+        seq = [(100, 61), (5, 62), (64, 63), (33, 64), (128, 65), (1, 66), (128, 67), (17, 68)]
+        xs = [synth.make_tokens(shape, B, seed, "cuda:0") for B, seed in seq]
+        outs = [layer.forward(x).clone() for x in xs]     # (clone is enqueued on the same stream)
+        torch.cuda.synchronize()
+        assert layer.stats()["device_status"] == 0
+        for (B, seed), x, got in zip(seq, xs, outs):
+            fresh = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
+            try:
+                want = fresh.forward(x).clone()
+                torch.cuda.synchronize()
+            finally:
+                fresh.close()
+            assert torch.equal(got, want), (B, seed)
+        run_case(shape, 128, weights=w, tokens=xs[4], layer=layer)   # and the layer still agrees with the oracle
+    finally:
+        layer.close()
+
+
 def test_layers_of_both_schedules_enqueued_back_to_back():
     """Dense and streaming steps of different layers queued on one stream without a synchronisation
     in between (a decoder stack): every output equals the one the layer gives when run alone."""
