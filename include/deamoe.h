@@ -26,7 +26,9 @@
  *    graph and replayed (Section 5 of the paper runs its steps that way).
  *  - The weight-streaming and dense kernels are PERSISTENT grids sized to fill the device (every
  *    SM, two thread blocks each) whose blocks wait for one another's results, so all blocks of a
- *    launch must be resident at the same time.  Run one such step per device at a time: if another
+ *    launch must be resident at the same time; consecutive kernels of one step are launched
+ *    programmatically and run beside one another, handing over through counters in device memory
+ *    rather than at kernel boundaries.  Run one such step per device at a time: if another
  *    kernel holds SMs while a step runs (a second layer driven from another stream, another process
  *    under MPS, a long-running communication kernel), blocks that cannot become resident keep the
  *    others waiting.  Nothing hangs or faults in that case -- every device-side wait is bounded --
