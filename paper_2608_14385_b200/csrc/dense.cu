@@ -66,6 +66,7 @@ constexpr int DN_B_BYTES = DN_NMAX * DN_BK * 2;   // 8 KB
 constexpr int DN_STAGE_BYTES = DN_A_BYTES + DN_B_BYTES;
 constexpr int DN_WARP_TMA = 4, DN_WARP_MMA = 5;
 constexpr int DN_THREADS = (DN_WARP_MMA + 1) * 32;
+constexpr int DN_GATHER_CTAS_PER_SM = 2;     // CTAs (of 256 threads) of the kernel that gathers the token rows: all resident at once
 constexpr int DN_JQ = 4;                    // slots of the CTA's queue of claimed jobs
 constexpr int DN_CLAIM_AHEAD = 6;           // chunks left to issue of a job when the copy role claims the next one
 constexpr int DN_TMEM_COLS = 2 * DN_TILE;   // 2 accumulator buffers; the CTAs of an SM share its 512 columns
@@ -613,16 +614,7 @@ __global__ void k_gather_buckets(LayerDev L, const __nv_bfloat16* __restrict__ t
   for (int r = (int)blockIdx.x; r < rows; r += (int)gridDim.x) {
     const int4* src = reinterpret_cast<const int4*>(tokens + (size_t)__ldcg(L.dept_tok + r) * L.h);
     int4* dst = reinterpret_cast<int4*>(Xg + (size_t)r * L.h);
-    // four loads in flight per thread (this copy sits between the routing and the first stage)
-    for (int i0 = (int)threadIdx.x; i0 < v; i0 += 4 * (int)blockDim.x) {
-      int4 val[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (i0 + u * (int)blockDim.x < v) val[u] = __ldg(src + i0 + u * (int)blockDim.x);
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (i0 + u * (int)blockDim.x < v) dst[i0 + u * (int)blockDim.x] = val[u];
-    }
+    for (int i = (int)threadIdx.x; i < v; i += (int)blockDim.x) dst[i] = src[i];
   }
   if (gathered) {  // this CTA's rows are stored: count it in for the tensor-core kernel that may already be waiting
     __threadfence();
@@ -778,11 +770,11 @@ int dense_launch(DensePlan& p, const LayerDev& L, const DenseIO& io, const int* 
         ph.K = L.h; ph.tiles = 2 * L.f / DN_TILE; ph.dual = 0; ph.epi = DE_SIGMA;
         ph.w = p.tiles + p.o_gu; ph.unit_elems = p.e_gu;
         in = p.Xg; in_rows = p.xg_rows; ph.outh = io.GU; ph.out_stride = 2 * L.f;
-        if (launch_pdl(k_gather_buckets, dim3(2 * p.n_sm), dim3(256), 0, s, L, io.tokens, p.Xg, io.routed_flag,
+        if (launch_pdl(k_gather_buckets, dim3(DN_GATHER_CTAS_PER_SM * p.n_sm), dim3(256), 0, s, L, io.tokens, p.Xg, io.routed_flag,
                        io.gathered, io.spin_limit ? io.spin_limit : DN_SPIN_LIMIT) != cudaSuccess)
           return -1;
         chained = io.routed_flag != nullptr && io.gathered != nullptr;
-        if (chained) { A.gathered = io.gathered; A.gather_ctas = 2 * p.n_sm; }
+        if (chained) { A.gathered = io.gathered; A.gather_ctas = DN_GATHER_CTAS_PER_SM * p.n_sm; }
         ++launches;
         break;
       case ST_S4:
