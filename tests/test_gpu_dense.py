@@ -135,24 +135,27 @@ def test_dense_steps_of_changing_batch_on_one_layer_leave_no_state_behind():
     one a fresh layer gives for that batch alone."""
     shape = DENSE_WIDE
     w = _scaled(shape, 16, scale=6.0)
-    layer = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
-    try:
-        seq = [(100, 61), (5, 62), (64, 63), (33, 64), (128, 65), (1, 66), (128, 67), (17, 68)]
-        xs = [synth.make_tokens(shape, B, seed, "cuda:0") for B, seed in seq]
-        outs = [layer.forward(x).clone() for x in xs]     # (clone is enqueued on the same stream)
-        torch.cuda.synchronize()
-        assert layer.stats()["device_status"] == 0
-        for (B, seed), x, got in zip(seq, xs, outs):
-            fresh = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
-            try:
-                want = fresh.forward(x).clone()
-                torch.cuda.synchronize()
-            finally:
-                fresh.close()
-            assert torch.equal(got, want), (B, seed)
-        run_case(shape, 128, weights=w, tokens=xs[4], layer=layer)   # and the layer still agrees with the oracle
-    finally:
-        layer.close()
+    seq = [(100, 61), (5, 62), (64, 63), (33, 64), (128, 65), (1, 66), (128, 67), (17, 68)]
+    xs = [synth.make_tokens(shape, B, seed, "cuda:0") for B, seed in seq]
+    # DENSE: every step takes the dense schedule; AUTO: the steps of fewer than 32 tokens take the fused one, whose
+    # hand-over flags are the same words with another meaning
+    for sched in (binding.SCHED_DENSE, binding.SCHED_AUTO):
+        layer = binding.Layer(shape, w, 128, sched)
+        try:
+            outs = [layer.forward(x).clone() for x in xs]     # (clone is enqueued on the same stream)
+            torch.cuda.synchronize()
+            assert layer.stats()["device_status"] == 0
+            for (B, seed), x, got in zip(seq, xs, outs):
+                fresh = binding.Layer(shape, w, 128, sched)
+                try:
+                    want = fresh.forward(x).clone()
+                    torch.cuda.synchronize()
+                finally:
+                    fresh.close()
+                assert torch.equal(got, want), (sched, B, seed)
+            run_case(shape, 128, weights=w, tokens=xs[4], layer=layer)   # and the layer still agrees with the oracle
+        finally:
+            layer.close()
 
 
 def test_layers_of_both_schedules_enqueued_back_to_back():
