@@ -81,7 +81,8 @@ typedef enum {
                               cores, private matrices in the streaming kernel.  bf16 weights and
                               tokens, a DeaMoE layer with private matrices, h a multiple of 256,
                               f and shared_ffn of 128; else UNSUPPORTED.  AUTO takes this schedule by
-                              itself for calls of 32 tokens and more on layers that support it. */
+                              itself for calls of 32 tokens and more (64 and more on layers of fewer than 64 experts) on
+                              layers that support it. */
 } deamoe_schedule_t;
 
 /*

@@ -14,10 +14,19 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdeamoe.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_BATCH, ERR_TIMEOUT, ERR_INTERNAL = range(8)
-DENSE_MIN_BATCH = 32   # calls of this many tokens and more take the dense schedule under SCHED_AUTO (DENSE_MIN_BATCH in csrc/dense.cuh)
+DENSE_MIN_BATCH = 32   # calls of this many tokens and more take the dense schedule under SCHED_AUTO (csrc/dense.cuh) ...
+DENSE_SMALL_ROUTER = 64  # ... twice as many on layers of fewer experts than this
+
 F32, BF16 = 0, 1
 SIGMA_NONE, SIGMA_SILU, SIGMA_GELU, SIGMA_RMSNORM = 0, 1, 2, 3
 SCHED_AUTO, SCHED_PLAIN, SCHED_STAGED, SCHED_FUSED, SCHED_DENSE = 0, 1, 2, 3, 4
+
+
+def dense_min_batch(shape):
+    """Smallest call that SCHED_AUTO runs in the dense schedule on a layer of this shape (if it supports it)."""
+    n = shape.n_dept * shape.experts_per_dept
+    return DENSE_MIN_BATCH if n >= DENSE_SMALL_ROUTER else 2 * DENSE_MIN_BATCH
+
 
 # every symbol include/deamoe.h declares
 SYMBOLS = ("deamoe_layer_create", "deamoe_vanilla_create", "deamoe_layer_destroy", "deamoe_route",

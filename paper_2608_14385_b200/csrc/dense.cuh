@@ -8,7 +8,11 @@ namespace deamoe {
 struct DensePlan;
 
 // Batches from this size on take the dense schedule when the layer has one (DEAMOE_SCHED_AUTO).
-constexpr int DENSE_MIN_BATCH = 32;  // measured crossover on the DeepSeek-V3 shape: about 28 tokens
+// Measured crossover: about 28 tokens on the DeepSeek-V3 shape, 16 - 32 on the layers of the paper's Table 1
+// (256 - 1280 experts); a 7B-class layer of 4 x 4 experts crosses over near 64 (its first stage has fewer tile
+// jobs than the device has CTAs), so layers of fewer than DENSE_SMALL_ROUTER experts switch at twice the size.
+constexpr int DENSE_MIN_BATCH = 32;
+constexpr int DENSE_SMALL_ROUTER = 64;
 
 // True if the layer's shapes and dtypes fit the dense kernels (bf16 weights and activations, a
 // DeaMoE layer with private matrices, h a multiple of 256, f and shared_ffn of 128).

@@ -67,7 +67,7 @@ def test_dense_schedule_is_refused_for_layers_it_cannot_run():
 
 
 def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
-    """One AUTO layer sized for 128 tokens: up to 31 tokens take the streaming schedule, 32 and more the dense one;
+    """One AUTO layer sized for 128 tokens: below `binding.dense_min_batch(shape)` tokens (64 for this 16-expert layer) calls take the streaming schedule, from there on the dense one;
     each agrees with a layer fixed to that schedule bit for bit, and the two schedules agree within
     the tolerance (they round intermediates alike but sum in different orders)."""
     shape = DENSE_WIDE
@@ -76,13 +76,13 @@ def test_auto_switches_to_the_dense_schedule_by_batch_and_both_agree():
     fused = binding.Layer(shape, w, 128, binding.SCHED_FUSED)
     dense = binding.Layer(shape, w, 128, binding.SCHED_DENSE)
     try:
-        for B in (16, 31, 32, 64, 128):
+        for B in (16, 32, 63, 64, 128):
             x = synth.make_tokens(shape, B, 14 + B, torch.device("cuda:0"))
             oa, of, od = auto.forward(x).float(), fused.forward(x).float(), dense.forward(x).float()
             torch.cuda.synchronize()
             for layer in (auto, fused, dense):
                 assert layer.stats()["device_status"] == 0
-            same = of if B < binding.DENSE_MIN_BATCH else od
+            same = of if B < binding.dense_min_batch(shape) else od
             assert torch.equal(oa, same)
             ok, err, bound = within_tolerance(od.cpu().numpy().astype(np.float64), of.cpu().numpy().astype(np.float64))
             assert ok, f"{err:.3e} > {bound:.3e}"
@@ -137,7 +137,7 @@ def test_dense_steps_of_changing_batch_on_one_layer_leave_no_state_behind():
     w = _scaled(shape, 16, scale=6.0)
     seq = [(100, 61), (5, 62), (64, 63), (33, 64), (128, 65), (1, 66), (128, 67), (17, 68)]
     xs = [synth.make_tokens(shape, B, seed, "cuda:0") for B, seed in seq]
-    # DENSE: every step takes the dense schedule; AUTO: the steps of fewer than 32 tokens take the fused one, whose
+    # DENSE: every step takes the dense schedule; AUTO: the steps of fewer than 64 tokens (a 16-expert layer) take the fused one, whose
     # hand-over flags are the same words with another meaning
     for sched in (binding.SCHED_DENSE, binding.SCHED_AUTO):
         layer = binding.Layer(shape, w, 128, sched)
