@@ -327,6 +327,197 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
   }
 }
 
+// Wide routers (more than 256 experts): a token's top-k by ONE CTA of ceil(n / 256) warps.  Warp w holds experts
+// 256 w ... 256 w + 255, eight per lane, and picks its own k best; warp 0 then picks the k best of the warps'
+// candidates.  Same selection as topk_one_token_regs (largest logit first, ties to the lower expert index, the same
+// fixed-order sums of the partial logits), but every loop over more than eight values is rolled: the 16- and
+// 32-logits-per-lane variants of the one-warp routine are 30 - 60 KB of straight-line code, and a step starts with
+// cold instruction caches (they took 13 - 25 us, of which the warps stood waiting for instructions five cycles in
+// six).  Not for strict department coverage, whose repair step scans all logits.
+constexpr int WIDE_MAX_WARPS = 8;
+static __host__ __device__ inline bool topk_wide_fits(const LayerDev& L) {
+  const bool grouped = L.k_dept > 0 && L.k_dept < L.m;
+  return L.n > 256 && L.n <= 256 * WIDE_MAX_WARPS && L.k <= 32 && (!grouped || L.m <= 32) &&
+         !(L.strict_dept && L.k_dept > 0);
+}
+static __device__ void topk_one_token_wide(const LayerDev& L, int t, int B, int kslices, int32_t* __restrict__ user_idx,
+                                           float* __restrict__ user_w) {
+  __shared__ float s_dmax[WIDE_MAX_WARPS][32];
+  __shared__ float s_mx[WIDE_MAX_WARPS], s_den[WIDE_MAX_WARPS];
+  __shared__ unsigned s_ckey[WIDE_MAX_WARPS][32];
+  __shared__ int s_cidx[WIDE_MAX_WARPS][32];
+  const int n = L.n, k = L.k;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int base = 256 * warp;
+  float v[8];
+  unsigned taken = 0;
+  {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = 0.f;
+    const float* __restrict__ src = L.logit_part + (size_t)t * n;
+    const size_t slice = (size_t)B * n;
+    // (eight slices' loads in flight at a time: a round of loads costs 1.5 us here, right behind the kernel that
+    // wrote the partial logits, whatever its width)
+#pragma unroll 8
+    for (int sl = 0; sl < kslices; ++sl, src += slice) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] += __ldg(src + min(base + lane + 32 * j, n - 1));
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (!(v[j] == v[j])) v[j] = -INFINITY;  // a NaN logit (non-finite input) must still yield valid indices
+      if (base + lane + 32 * j >= n) { v[j] = -INFINITY; taken |= 1u << j; }
+    }
+  }
+  float mx_all = -INFINITY, den_all = 0.f;
+  if (!L.norm_topk) {  // gate weights by softmax over ALL experts: maximum and denominator across the warps
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mx = fmaxf(mx, v[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) s_mx[warp] = mx;
+    __syncthreads();
+#pragma unroll 1
+    for (int w = 0; w < nw; ++w) mx_all = fmaxf(mx_all, s_mx[w]);
+    float den = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (!((taken >> j) & 1u)) den += expf(v[j] - mx_all);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    if (lane == 0) s_den[warp] = den;
+    __syncthreads();
+#pragma unroll 1
+    for (int w = 0; w < nw; ++w) den_all += s_den[w];  // warp order: the same sum on every run
+  }
+  if (L.k_dept > 0 && L.k_dept < L.m) {
+    // Group limit (Section 3.3; m <= 32): the score of a department is its largest logit; a department is dropped
+    // when at least k_dept departments rank ahead of it (score descending, index ascending).
+    const int g = L.g, m = L.m;
+    float dloc = -INFINITY;  // lane d: largest logit of department d among this warp's experts
+#pragma unroll 1
+    for (int d = 0; d < m; ++d) {
+      const int lo = d * g, hi = lo + g;
+      if (hi <= base || lo >= base + 256) continue;  // (warp-uniform) none of this warp's experts
+      float loc = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int idx = base + lane + 32 * j;
+        if (idx >= lo && idx < hi && idx < n) loc = fmaxf(loc, v[j]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) loc = fmaxf(loc, __shfl_xor_sync(0xffffffffu, loc, o));
+      if (lane == d) dloc = loc;
+    }
+    s_dmax[warp][lane] = dloc;
+    __syncthreads();
+    float dscore = -INFINITY;
+#pragma unroll 1
+    for (int w = 0; w < nw; ++w) dscore = fmaxf(dscore, s_dmax[w][lane]);
+    int ahead = 0;
+#pragma unroll 1
+    for (int d2 = 0; d2 < m; ++d2) {
+      const float s2 = __shfl_sync(0xffffffffu, dscore, d2);
+      ahead += better(s2, d2, dscore, lane) ? 1 : 0;
+    }
+    const unsigned alive = __ballot_sync(0xffffffffu, lane < m && ahead < L.k_dept);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int idx = base + lane + 32 * j;
+      if (idx < n && !((alive >> (idx / g)) & 1u)) taken |= 1u << j;
+    }
+  }
+  // this warp's k best (order-preserving integer keys, 0 = not a candidate)
+  unsigned key[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const unsigned bits = __float_as_uint(v[j] + 0.f);  // + 0.f: -0 and +0 are one value, so they get one key
+    key[j] = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+  }
+  {
+    unsigned gmax;
+    int gj;
+    rescan_group<0, 8>(key, taken, gmax, gj);
+    unsigned ck = 0u;
+    int ci = 0x7fffffff;
+#pragma unroll 1
+    for (int q = 0; q < k; ++q) {
+      const unsigned wmax = __reduce_max_sync(0xffffffffu, gmax);
+      if (wmax == 0u) break;  // (warp-uniform) this warp has no candidate left
+      const unsigned cand = (gmax == wmax) ? (unsigned)(base + lane + 32 * gj) : 0x7fffffffu;
+      const unsigned widx = __reduce_min_sync(0xffffffffu, cand);
+      if (lane == q) { ck = wmax; ci = (int)widx; }
+      if (lane == (int)((widx - (unsigned)base) & 31u)) {  // the owner masks the element and rescans
+        taken |= 1u << ((widx - (unsigned)base) >> 5);
+        rescan_group<0, 8>(key, taken, gmax, gj);
+      }
+    }
+    s_ckey[warp][lane] = ck;
+    s_cidx[warp][lane] = ci;
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  // warp 0: the k best of the warps' candidates.  Lane l holds every warp's l-th candidate; the warps' expert
+  // ranges ascend, so among equal keys the first one in a lane's scan is the lower expert index.
+  unsigned ckey[WIDE_MAX_WARPS];
+  int cidx[WIDE_MAX_WARPS];
+#pragma unroll
+  for (int w = 0; w < WIDE_MAX_WARPS; ++w) {
+    ckey[w] = (w < nw) ? s_ckey[w][lane] : 0u;
+    cidx[w] = (w < nw) ? s_cidx[w][lane] : 0x7fffffff;
+  }
+  unsigned used = 0;
+  auto scan = [&](unsigned& bk, int& bi) {
+    bk = 0u; bi = 0x7fffffff;
+#pragma unroll
+    for (int w = 0; w < WIDE_MAX_WARPS; ++w) {
+      const unsigned kq = ((used >> w) & 1u) ? 0u : ckey[w];
+      if (kq > bk) { bk = kq; bi = cidx[w]; }
+    }
+  };
+  unsigned bk;
+  int bi;
+  scan(bk, bi);
+  float my_v = 0.f;  // lane q keeps the q-th selected logit (k <= 32)
+  int my_i = 0;
+#pragma unroll 1
+  for (int q = 0; q < k; ++q) {
+    const unsigned wmax = __reduce_max_sync(0xffffffffu, bk);
+    const unsigned cand = (bk == wmax && wmax != 0u) ? (unsigned)bi : 0x7fffffffu;
+    const unsigned widx = __reduce_min_sync(0xffffffffu, cand);
+    if (lane == q) {
+      my_i = (int)widx;
+      my_v = __uint_as_float((wmax & 0x80000000u) ? (wmax ^ 0x80000000u) : ~wmax);
+    }
+    if (widx != 0x7fffffffu && bk == wmax && (unsigned)bi == widx) {  // the owner drops the candidate and rescans
+#pragma unroll
+      for (int w = 0; w < WIDE_MAX_WARPS; ++w)
+        if (cidx[w] == (int)widx) used |= 1u << w;
+      scan(bk, bi);
+    }
+  }
+  // gate weights
+  const float top = __shfl_sync(0xffffffffu, my_v, 0);
+  float e, den;
+  if (L.norm_topk) {  // 1: softmax over the selection; 2: logistic scores normalised over the selection
+    e = (lane < k) ? (L.norm_topk == 2 ? 1.f / (1.f + expf(-my_v)) : expf(my_v - top)) : 0.f;
+    den = e;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+  } else {
+    e = (lane < k) ? expf(my_v - mx_all) : 0.f;
+    den = den_all;
+  }
+  if (lane < k) {
+    const float p = L.route_scale * e / den;
+    L.topk_idx[(size_t)t * k + lane] = my_i;
+    L.topk_w[(size_t)t * k + lane] = p;
+    if (user_idx) user_idx[(size_t)t * k + lane] = my_i;
+    if (user_w) user_w[(size_t)t * k + lane] = p;
+  }
+}
+
 // ---------------------------------------------------------------- department bucketing
 // One CTA.  Token-membership bitmasks per department and per expert are built with shared
 // atomics, then counts, offsets (warp ballot/popc scans), ascending token lists, the pair

@@ -752,6 +752,14 @@ k_topk_tokens(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, fl
   else topk_one_token_regs<32>(L, t, B, kslices, lane, user_idx, user_w);
 }
 
+// The same for routers of more than 256 experts: one CTA per token (see topk_one_token_wide).
+__global__ void __launch_bounds__(WIDE_MAX_WARPS * 32)
+k_topk_wide(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
+  pdl_trigger();
+  pdl_wait();  // the router logits of the preceding kernel
+  topk_one_token_wide(L, (int)blockIdx.x, B, kslices, user_idx, user_w);
+}
+
 __global__ void __launch_bounds__(FINISH_THREADS, 1)
 k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
@@ -1950,13 +1958,17 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   if (topk_warps > B) topk_warps = B;
   if (topk_warps < 1) topk_warps = 1;
   int extra = 0;
-  if ((takes_dense(p, B) || B > FINISH_THREADS / 32 || L.n > 256) && in_regs) {  // the selection gets a grid of its own
+  if (topk_wide_fits(L)) {  // wide router: the selection by one CTA per token, in a grid of its own
+    launch_pdl(k_topk_wide, dim3(B), dim3(((L.n + 255) / 256) * 32), 0, s, L, B, ny, user_idx, user_w);
+    topk_warps = 0;
+    extra = 1;
+  } else if ((takes_dense(p, B) || B > FINISH_THREADS / 32 || L.n > 256) && in_regs) {  // the selection gets a grid of its own
     launch_pdl(k_topk_tokens, dim3((B + TOPK_CTA_WARPS - 1) / TOPK_CTA_WARPS), dim3(TOPK_CTA_WARPS * 32), 0, s, L, B, ny,
                user_idx, user_w);
     topk_warps = 0;
     extra = 1;
   }
-  size_t scratch = in_regs ? 0 : (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
+  size_t scratch = (in_regs || topk_warps == 0) ? 0 : (size_t)topk_warps * per_warp;   // top-k scratch, reused by the bucketing masks
   const size_t bs = bucket_smem_bytes(L, B) + (size_t)((L.vanilla ? L.n : L.m) + 2) * sizeof(int);  // + early_first_stage()'s scan
   if (bs > scratch) scratch = bs;
   scratch = (scratch + 15) & ~(size_t)15;
