@@ -285,10 +285,10 @@ deamoe_status_t deamoe_profile_last_ms(deamoe_layer_t *layer, float *ms);
  *
  * Limits: slices * B * n * 4 bytes must fit the fixed array, where slices (1, 2, 4, 8 or 16) is the
  * number of column slices the logits kernel uses for this n and hidden -- the same rule as a layer
- * object's: doubled while a slice is wider than 512 columns and (n / 4) * slices < 1024.  A larger
- * request returns DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout, n = 256, hidden =
- * 7168: 16 slices, B up to 256; n = 2048, hidden = 7168: 2 slices, B up to 256; hidden <= 512: 1
- * slice.)  Other errors as for deamoe_route.
+ * object's: doubled while a slice is wider than 512 columns and (n / 4) * slices, doubled, stays at or
+ * below 740.  A larger request returns DEAMOE_ERR_BATCH and enqueues nothing.  (DeepSeek-V3 layout,
+ * n = 256, hidden = 7168: 8 slices, B up to 512; n = 2048, hidden = 7168: 1 slice, B up to 512;
+ * hidden <= 512: 1 slice.)  Other errors as for deamoe_route.
  *
  * The first call on each device resolves the array's device address and sets one kernel
  * attribute (the device must be current); make that first call before any stream capture begins.

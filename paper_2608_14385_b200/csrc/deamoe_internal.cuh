@@ -135,14 +135,16 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// Column slices of the router product (one grid row of k_router_logits per slice, one array of
-// partial logits each): at least 512 columns per thread block, and no more slices than it takes to
-// fill the device with ~1024 blocks of four router rows (every slice is one more array the top-k has
-// to read back).  The slices' partial sums are added in slice order, so every caller that wants the
+// Column slices of the router product (one grid row of k_router_logits per slice, one array of partial logits
+// each): doubled while a slice is wider than 512 columns and the grid, blocks of four router rows times the slices,
+// still fits the device in ONE wave (the 128-thread blocks are resident five to an SM, by their registers: 740 on a
+// B200).  Measured on routers of 256 / 864 / 1280 experts and 7168 columns: 8 / 2 / 2 slices bring the logits in
+// 3.9 / 8.9 / 10.9 us, the 16 / 8 / 4 of a second wave in 4.9 / 10.1 / 12.2 (and every slice is one more array
+// the top-k has to read back).  The slices' partial sums are added in slice order, so every caller that wants the
 // same fp32 logits must use the same count: the layer object and deamoe_route_static both call this.
 static inline int router_kslices(int n, int h) {
   int ks = 1;
-  while (ks < 16 && h / ks > 512 && (n / 4) * ks < 1024) ks *= 2;
+  while (ks < 16 && h / ks > 512 && (n / 4) * (2 * ks) <= 740) ks *= 2;
   return ks;
 }
 

@@ -61,17 +61,17 @@ def test_static_routing_matches_layer_routing_on_two_consecutive_calls():
 
 
 def test_static_routing_on_the_multi_slice_layout_against_the_oracle():
-    """The documented large use: the DeepSeek-V3 router (256 experts, hidden 7168, top-8) takes 16
+    """The documented large use: the DeepSeek-V3 router (256 experts, hidden 7168, top-8) takes 8
     column slices, so the fixed array holds part[slice][B][n] with a stride that depends on the call's
-    B.  256 tokens fill the 4 MiB exactly; a call with 3 tokens right behind it (no synchronisation)
+    B.  512 tokens fill the 4 MiB exactly; a call with 3 tokens right behind it (no synchronisation)
     reads slices that lie between leftovers of the first.  Both are compared bit for bit with the
-    oracle and with a layer object's routing (same slice rule, so the same fp32 sums); 257 tokens do
+    oracle and with a layer object's routing (same slice rule, so the same fp32 sums); 513 tokens do
     not fit and are refused."""
     shape = synth.LayerShape("noalloc-dsv3", hidden=7168, n_dept=32, experts_per_dept=8, ffn=16, priv=16, top_k=8,
                              act_dtype=0)
     dev = torch.device("cuda:0")
     weights = synth.make_deamoe_weights(shape, 24, dev)
-    big, small = synth.make_tokens(shape, 256, 25, dev), synth.make_tokens(shape, 3, 26, dev)
+    big, small = synth.make_tokens(shape, 512, 25, dev), synth.make_tokens(shape, 3, 26, dev)
     outs = [(torch.full((b.shape[0], shape.top_k), -1, dtype=torch.int32, device=dev),
              torch.full((b.shape[0], shape.top_k), -1.0, dtype=torch.float32, device=dev)) for b in (big, small)]
     for b, (idx, w) in zip((big, small), outs):
@@ -83,7 +83,7 @@ def test_static_routing_on_the_multi_slice_layout_against_the_oracle():
         for b, (idx, w) in zip((big, small), outs):
             o = ref.route(cfg, synth.to_numpy(weights["router"]), synth.to_numpy(b), want_logits=True)
             safe = o["gap"] > 1e-5 * np.abs(o["logits"]).max(axis=1)
-            assert safe.mean() > 0.97                  # 256 tokens: a few may sit within rounding of a tie
+            assert safe.mean() > 0.97                  # 512 tokens: a few may sit within rounding of a tie
             assert (idx.cpu().numpy()[safe] == o["idx"][safe]).all()
             assert np.abs(w.cpu().numpy().astype(np.float64) - o["w"])[safe].max() <= 1e-5
             for s0 in range(0, b.shape[0], 128):       # the layer object takes at most 128 tokens per call
@@ -94,7 +94,7 @@ def test_static_routing_on_the_multi_slice_layout_against_the_oracle():
                 assert (lw - w[s0:s0 + 128]).abs().max().item() <= 1e-6
     finally:
         layer.close()
-    too_many = torch.zeros((257, shape.hidden), dtype=torch.float32, device=dev)
+    too_many = torch.zeros((513, shape.hidden), dtype=torch.float32, device=dev)
     with pytest.raises(binding.DeaMoEError) as e:
         binding.route_static(weights["router"], too_many, shape.n_dept, shape.experts_per_dept, shape.top_k)
     assert e.value.status == binding.ERR_BATCH
