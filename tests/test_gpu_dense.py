@@ -158,6 +158,41 @@ def test_dense_steps_of_changing_batch_on_one_layer_leave_no_state_behind():
             layer.close()
 
 
+def test_many_steps_of_random_batch_sizes_repeat_bit_for_bit():
+    """400 steps of random token counts (1 - 128) on one AUTO layer, queued without a synchronisation, a second
+    layer's steps in between: every (batch, tokens) pair must give the same bits each time it comes up, and the
+    device status must stay 0.  (The chained kernels of a step overlap differently from step to step; nothing
+    they hand over may depend on that.)"""
+    import random
+    shape = DENSE_WIDE
+    a = binding.Layer(shape, _scaled(shape, 17, scale=6.0), 128, binding.SCHED_AUTO)
+    b = binding.Layer(DENSE_SMALL, _scaled(DENSE_SMALL, 18), 128, binding.SCHED_DENSE)
+    try:
+        rng = random.Random(5)
+        sizes = [1, 2, 7, 16, 31, 32, 33, 63, 64, 65, 100, 128]
+        pool = {(B, i): synth.make_tokens(shape, B, 300 + 10 * B + i, "cuda:0") for B in sizes for i in range(2)}
+        pool_b = {B: synth.make_tokens(DENSE_SMALL, B, 500 + B, "cuda:0") for B in sizes}
+        first, first_b = {}, {}
+        for _ in range(400):
+            key = (rng.choice(sizes), rng.randrange(2))
+            out = a.forward(pool[key])
+            if key not in first:
+                first[key] = out.clone()
+            else:
+                assert torch.equal(out, first[key]), key
+            if rng.random() < 0.3:
+                B = rng.choice(sizes)
+                out = b.forward(pool_b[B])
+                if B not in first_b:
+                    first_b[B] = out.clone()
+                else:
+                    assert torch.equal(out, first_b[B]), B
+        torch.cuda.synchronize()
+        assert a.stats()["device_status"] == 0 and b.stats()["device_status"] == 0
+    finally:
+        a.close(); b.close()
+
+
 def test_layers_of_both_schedules_enqueued_back_to_back():
     """Dense and streaming steps of different layers queued on one stream without a synchronisation
     in between (a decoder stack): every output equals the one the layer gives when run alone."""
