@@ -45,6 +45,13 @@
 // one rate (dealt round-robin, the first CTA was done 95 us before the last of a 320 us launch), and
 // a claimed list ends when the work ends.  The copy role claims and posts each job to the other
 // roles through a small queue in shared memory; the last CTA to finish clears the counter.
+//
+// The first launch of a step (shared expert's and departments' gate / up) is launched programmatically behind the
+// kernel that gathers the token rows, which itself sits behind the routing kernel: its CTAs are resident while the
+// routing runs, do the shared expert's jobs (they need nothing of the routing) and start the departments' jobs when
+// every CTA of the gather kernel has counted itself done.  Every finished department tile is counted into that
+// department's completion counter, which the streaming kernel of the private stages, resident as this grid's CTAs
+// leave, tests expert by expert.  The second launch (down projections) is an ordinary launch.
 #include "dense.cuh"
 
 #include <cuda.h>  // CUtensorMap and the encode function's signature; the entry point is looked up at run time
