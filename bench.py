@@ -799,7 +799,8 @@ def stack_bench(args, sched, peak, torch, dev, steps=None):
 def other_workloads(args, sched, peak, torch, dev, flush):
     """Compact rows for the other benchmark configurations, run after the headline so that one default
     invocation measures them all: one 7B-class layer (configuration 2), the stack of 32 such layers
-    (configuration 5) and the paper's own DeepSeek-V3-matched row of Table 1 with group-limited routing."""
+    (configuration 5), the paper's own DeepSeek-V3-matched row of Table 1 with group-limited routing, and the
+    table's other four rows."""
     from paper_2608_14385_b200 import binding, synth
     t0 = time.time()
     out = {}
@@ -822,6 +823,18 @@ def other_workloads(args, sched, peak, torch, dev, flush):
                                             steps=10)
     layer.close()
     torch.cuda.empty_cache()
+    # the other rows of the paper's Table 1, each against the standard MoE layer it was matched to
+    out["table1_rows"] = {}
+    for name in ("dsv2-paper", "qwen3-paper", "kimi-k2-paper", "b7-paper"):
+        shape = synth.SHAPES[name]
+        w = synth.make_deamoe_weights(shape, 0, dev)
+        layer = binding.Layer(shape, w, 64, sched)
+        del w
+        torch.cuda.empty_cache()
+        out["table1_rows"][name] = paper_row_sweep(args, shape, layer, flush, sched, peak, torch, dev,
+                                                   batches_list=(4, 16, 64), steps=8)
+        layer.close()
+        torch.cuda.empty_cache()
     out["seconds"] = time.time() - t0
     return out
 
