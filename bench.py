@@ -461,7 +461,7 @@ def main():
                 "frac_of_read_only_ceiling": achieved / read_gbs if read_gbs else None,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
         if args.schedule == "dense" or (args.schedule == "auto" and B >= binding.dense_min_batch(shape)):
-            # dense schedule: the pair of events brackets k_dense, k_stream, k_dense (ordinary launches, back to back)
+            # dense schedule: the pair of events brackets the gather kernel and k_dense, k_stream, k_dense (a chain that hands over through counters)
             roof["kernel"] = "k_dense + k_stream + k_dense (the three weight-streaming launches of a dense step)"
             roof["traffic_note"] = ("ESTIMATE for this run: its algorithmic bytes x 1.0127, the ratio ncu measured on the three "
                                     "full-size launches of a dense step at B = 128 "
