@@ -206,17 +206,17 @@ def test_layers_enqueued_back_to_back_match_layers_run_one_by_one(vanilla):
 WIDE_ROUTERS = [
     # n_dept, experts_per_dept, top_k, k_dept, strict department coverage
     (6, 16, 6, 0, 0),       # 96 experts: 8 logits per lane
-    (10, 32, 10, 0, 0),     # 320 experts: 16 logits per lane
+    (10, 32, 10, 0, 0),     # 320 experts: the wide top-k (one CTA of two warps per token)
     (10, 32, 10, 4, 0),     # group limited
     (8, 108, 10, 5, 0),     # the paper's DeepSeek-V3 router (Table 1)
     (8, 64, 10, 5, 0),      # ... DeepSeek-V2 router
     (8, 40, 8, 5, 0),       # ... Qwen3-235B router
-    (16, 80, 10, 5, 0),     # ... Kimi-K2 router: 1280 experts, the shared-memory top-k with a group limit
+    (16, 80, 10, 5, 0),     # ... Kimi-K2 router: 1280 experts, five warps per token, with a group limit
     (8, 84, 10, 4, 0),      # ... Baseline-7B router
-    (32, 32, 32, 0, 0),     # 1024 experts, top-32: the widest the register top-k takes
+    (32, 32, 32, 0, 0),     # 1024 experts, top-32: every lane of the merging warp holds a selection
     (32, 32, 8, 3, 0),
-    (40, 40, 8, 6, 0),      # 1600 experts, 40 departments: the shared-memory top-k
-    (32, 64, 8, 0, 0),      # 2048 experts: the most a layer may have
+    (40, 40, 8, 6, 0),      # 1600 experts, a group limit over 40 departments (more than a warp has lanes): the shared-memory top-k
+    (32, 64, 8, 0, 0),      # 2048 experts: the most a layer may have (eight warps per token)
     (6, 16, 6, 4, 1),       # strict department coverage (Section 3.3, last paragraph)
     (8, 108, 10, 5, 1),     # ... on the paper's DeepSeek-V3 router
     (40, 40, 8, 6, 1),      # ... in the shared-memory top-k
@@ -226,8 +226,10 @@ WIDE_ROUTERS = [
 @pytest.mark.parametrize("m,g,k,k_dept,strict", WIDE_ROUTERS)
 def test_routing_of_wide_and_group_limited_routers(m, g, k, k_dept, strict):
     """Routing only (indices, gate weights, department and expert lists) on layers with tiny experts but
-    wide routers, so that every top-k variant (8 / 16 / 32 logits per lane, group limit in registers,
-    shared-memory fallback) is compared with the oracle, with random logits and with exact ties."""
+    wide routers, so that every top-k variant (one warp with 8 logits per lane; the wide kernel of 2 - 8 warps per
+    token, with and without a group limit; the one-warp variants with 16 / 32 logits per lane, which strict
+    coverage still takes; the shared-memory fallback) is compared with the oracle, with random logits and with
+    exact ties."""
     shape = synth.LayerShape(f"wide{m}x{g}", hidden=256, n_dept=m, experts_per_dept=g, ffn=16, priv=16, top_k=k,
                              k_dept=k_dept, strict_dept=strict)
     dev = torch.device("cuda:0")
@@ -272,13 +274,15 @@ def test_routing_of_wide_and_group_limited_routers(m, g, k, k_dept, strict):
         layer.close()
 
 
-@pytest.mark.parametrize("m,g,k,norm", [(6, 16, 6, 2), (40, 40, 8, 2), (10, 32, 10, 0)])
-def test_gate_variants_on_every_topk_path(m, g, k, norm):
+@pytest.mark.parametrize("m,g,k,norm,k_dept", [(6, 16, 6, 2, 0), (40, 40, 8, 2, 0), (10, 32, 10, 0, 0),
+                                                (16, 80, 10, 0, 5), (40, 40, 8, 2, 6), (40, 40, 8, 0, 6)])
+def test_gate_variants_on_every_topk_path(m, g, k, norm, k_dept):
     """The gate-weight variants (logistic scores normalised over the selection; full softmax without
-    renormalisation) through the register top-k (inside the routing tail and, for more tokens than it
-    has warps, in the grid of its own) and through the shared-memory top-k of very wide routers."""
+    renormalisation) through the one-warp register top-k (inside the routing tail and, for more tokens than it
+    has warps, in the grid of its own), through the wide kernel of several warps per token (whose softmax over all
+    experts sums across warps; with and without a group limit) and through the shared-memory top-k."""
     shape = synth.LayerShape(f"gate{m}x{g}", hidden=256, n_dept=m, experts_per_dept=g, ffn=16, priv=16, top_k=k,
-                             norm_topk=norm, route_scale=1.5)
+                             norm_topk=norm, route_scale=1.5, k_dept=k_dept)
     dev = torch.device("cuda:0")
     w = synth.make_deamoe_weights(shape, 3, dev)
     w["router"] = w["router"] * 8.0  # logits of order one, so the variants differ visibly
