@@ -760,6 +760,11 @@ k_topk_wide(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, floa
   topk_one_token_wide(L, (int)blockIdx.x, B, kslices, user_idx, user_w);
 }
 
+// TOPK: who selects (0: a kernel in front of this one; 1: this kernel's warps with the logits in registers; 2: with
+// the logits in shared memory); VAN: a vanilla layer.  Compile-time, so that an instantiation holds only the code its
+// steps run: the kernel waits for its instructions most of the time (a step runs it once, from cold caches), and
+// code that is never executed but sits between code that is costs fetches.
+template <int TOPK, bool VAN>
 __global__ void __launch_bounds__(FINISH_THREADS, 1)
 k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int scratch_words,
                int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
@@ -799,8 +804,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
 #pragma unroll 1
     for (int i = tid; i < ngu + nz; i += FINISH_THREADS) (i < ngu ? L.ss_gu[i] : L.ss_z[i - ngu]) = 0ull;
   }
-  const bool regs_ok = topk_in_registers(L);
-  if (topk_warps == 0) {  // the selection was made by k_topk_tokens
+  if (TOPK == 0) {  // the selection was made by a kernel of its own
 #pragma unroll 1
     for (int i = tid; i < B * L.k; i += FINISH_THREADS) {
       S.topk_idx[i] = __ldcg(L.topk_idx + i);
@@ -813,7 +817,7 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     for (int t = warp; t < B; t += topk_warps) {
       // (wider routers that fit the register variants are ranked by k_topk_tokens: their 16 and 32
       // logits per lane would set this kernel's register budget and give it a stack frame)
-      if (regs_ok && L.n <= 256) topk_one_token_regs<8>(S, t, B, kslices, lane, user_idx, user_w);
+      if (TOPK == 1) topk_one_token_regs<8>(S, t, B, kslices, lane, user_idx, user_w);
       else topk_one_token(S, t, B, kslices, reinterpret_cast<float*>(base), base + (size_t)L.n * 4, lane, user_idx, user_w);
     }
   }
@@ -826,10 +830,10 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
   TS_MIN(L, 17);
   int* early_scr = reinterpret_cast<int*>(s_dyn) + bucket_smem_words(L.n, L.m, B);  // after the masks and offsets
   if (P.dense) dense_hand_over(S, L, P);
-  if (P.early && P.early_stage == ST_S1) early_first_stage<ST_S1>(S, P, B, early_scr);
+  if (!VAN && P.early) early_first_stage<ST_S1>(S, P, B, early_scr);
   bucket_experts(S, B, s_dyn, FINISH_THREADS);
   __syncthreads();
-  if (P.early && P.early_stage != ST_S1) early_first_stage<ST_V1>(S, P, B, early_scr);
+  if (VAN && P.early) early_first_stage<ST_V1>(S, P, B, early_scr);
 #ifdef DEAMOE_TRACE
   long long tt2 = clock64();
   TS_MIN(L, 13);
@@ -1758,6 +1762,15 @@ static cudaError_t pack(const void* src, __nv_bfloat16* dst, int rows, int C, lo
   return cudaGetLastError();
 }
 
+static cudaError_t finish_smem_attribute() {  // every instantiation may need more than the default 48 KB
+  cudaError_t e = cudaSuccess;
+#define DEAMOE_ATTR(T, V) if (e == cudaSuccess) e = cudaFuncSetAttribute(k_route_finish<T, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+  DEAMOE_ATTR(0, false); DEAMOE_ATTR(1, false); DEAMOE_ATTR(2, false);
+  DEAMOE_ATTR(0, true); DEAMOE_ATTR(1, true); DEAMOE_ATTR(2, true);
+#undef DEAMOE_ATTR
+  return e;
+}
+
 deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w, int schedule, int dense_mode,
                                    cudaStream_t s, StreamPlan** out, uint64_t* bytes) {
   StreamPlan* p = new (std::nothrow) StreamPlan();
@@ -1896,7 +1909,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
     if (schedule == DEAMOE_SCHED_FUSED && p->n_sm > 1) p->grid -= per_sm;
   }
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_route_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    e = finish_smem_attribute();
   p->bytes += seg_bytes + sync_bytes;
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -1975,8 +1988,12 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   const size_t smem = scratch + (size_t)fl.total * 4;
   if (smem > 200 * 1024) return -1;
-  launch_pdl(k_route_finish, dim3(1), dim3(FINISH_THREADS), smem, s, L, dv, B, ny, topk_warps, (int)(scratch / 4),
-             user_idx, user_w);
+  const int mode = topk_warps == 0 ? 0 : ((in_regs && L.n <= 256) ? 1 : 2);
+#define DEAMOE_FINISH(T, V) launch_pdl(k_route_finish<T, V>, dim3(1), dim3(FINISH_THREADS), smem, s, L, dv, B, ny, topk_warps, \
+                                       (int)(scratch / 4), user_idx, user_w)
+  if (L.vanilla) { if (mode == 0) DEAMOE_FINISH(0, true); else if (mode == 1) DEAMOE_FINISH(1, true); else DEAMOE_FINISH(2, true); }
+  else { if (mode == 0) DEAMOE_FINISH(0, false); else if (mode == 1) DEAMOE_FINISH(1, false); else DEAMOE_FINISH(2, false); }
+#undef DEAMOE_FINISH
   return cudaGetLastError() == cudaSuccess ? 2 + extra : -1;
 }
 
