@@ -153,7 +153,9 @@ static __device__ __forceinline__ void rescan_group(const unsigned (&key)[VPL], 
   mj_out = mj;
 }
 
-template <int VPL>
+// FEAT: 0 = neither a group limit nor strict coverage nor the softmax over all experts can occur (their code is
+// left out of the instantiation); 1 = whatever the layer's configuration says.
+template <int VPL, int FEAT = 1>
 static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int kslices, int lane,
                                            int32_t* __restrict__ user_idx, float* __restrict__ user_w) {
   const int n = L.n, k = L.k;
@@ -194,7 +196,7 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
   if (chk == 12345.678f) L.counts[15] = 1;
 #endif
   float mx_all = -INFINITY, den_all = 0.f;
-  if (!L.norm_topk) {
+  if (FEAT && !L.norm_topk) {
 #pragma unroll
     for (int j = 0; j < VPL; ++j) mx_all = fmaxf(mx_all, v[j]);
 #pragma unroll
@@ -205,7 +207,7 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) den_all += __shfl_xor_sync(0xffffffffu, den_all, o);
   }
-  if (L.k_dept > 0 && L.k_dept < L.m) {
+  if (FEAT && L.k_dept > 0 && L.k_dept < L.m) {
     // Group limit (Section 3.3; needs m <= 32): the score of a department is its largest logit;
     // a department is dropped when at least k_dept departments rank ahead of it (score
     // descending, index ascending).  Lane d ends up holding the score of department d.
@@ -290,7 +292,7 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
 #ifdef DEAMOE_TRACE
   if (lane == 0 && t == 0) { L.counts[11] = (int)(clock64() - ta); L.counts[12] = (int)(ta & 0x7fffffff); }
 #endif
-  if (L.strict_dept && L.k_dept > 0)
+  if (FEAT && L.strict_dept && L.k_dept > 0)
     strict_coverage(L, lane, my_v, my_i, [&](unsigned long long covered, float& cv, int& ci) {
       float bv = -INFINITY;
       int bi = 0x7fffffff;
@@ -309,7 +311,7 @@ static __device__ void topk_one_token_regs(const LayerDev& L, int t, int B, int 
     });
   const float top = __shfl_sync(0xffffffffu, my_v, 0);
   float e, den;
-  if (L.norm_topk) {  // 1: softmax over the selection; 2: logistic scores normalised over the selection
+  if (!FEAT || L.norm_topk) {  // 1: softmax over the selection; 2: logistic scores normalised over the selection
     e = (lane < k) ? (L.norm_topk == 2 ? 1.f / (1.f + expf(-my_v)) : expf(my_v - top)) : 0.f;
     den = e;
 #pragma unroll
@@ -529,6 +531,7 @@ static __device__ __forceinline__ int warp_exclusive_offsets(const int* cnt, int
   // exclusive prefix sum of cnt[0..count) into off[0..count], compaction of the non-empty
   // indices into active[]; executed by one warp.
   int run = 0, nact = 0;
+#pragma unroll 1
   for (int base = 0; base < count; base += 32) {
     const int i = base + lane;
     const int c = (i < count) ? cnt[i] : 0;

@@ -761,7 +761,8 @@ k_topk_wide(LayerDev L, int B, int kslices, int32_t* __restrict__ user_idx, floa
 }
 
 // TOPK: who selects (0: a kernel in front of this one; 1: this kernel's warps with the logits in registers; 2: with
-// the logits in shared memory); VAN: a vanilla layer.  Compile-time, so that an instantiation holds only the code its
+// the logits in shared memory; 3: as 1 on a layer without group limit, strict coverage or softmax over all experts,
+// whose code is then left out); VAN: a vanilla layer.  Compile-time, so that an instantiation holds only the code its
 // steps run: the kernel waits for its instructions most of the time (a step runs it once, from cold caches), and
 // code that is never executed but sits between code that is costs fetches.
 template <int TOPK, bool VAN>
@@ -817,7 +818,8 @@ k_route_finish(LayerDev L, StreamDev P, int B, int kslices, int topk_warps, int 
     for (int t = warp; t < B; t += topk_warps) {
       // (wider routers that fit the register variants are ranked by k_topk_tokens: their 16 and 32
       // logits per lane would set this kernel's register budget and give it a stack frame)
-      if (TOPK == 1) topk_one_token_regs<8>(S, t, B, kslices, lane, user_idx, user_w);
+      if (TOPK == 3) topk_one_token_regs<8, 0>(S, t, B, kslices, lane, user_idx, user_w);
+      else if (TOPK == 1) topk_one_token_regs<8, 1>(S, t, B, kslices, lane, user_idx, user_w);
       else topk_one_token(S, t, B, kslices, reinterpret_cast<float*>(base), base + (size_t)L.n * 4, lane, user_idx, user_w);
     }
   }
@@ -1765,8 +1767,8 @@ static cudaError_t pack(const void* src, __nv_bfloat16* dst, int rows, int C, lo
 static cudaError_t finish_smem_attribute() {  // every instantiation may need more than the default 48 KB
   cudaError_t e = cudaSuccess;
 #define DEAMOE_ATTR(T, V) if (e == cudaSuccess) e = cudaFuncSetAttribute(k_route_finish<T, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
-  DEAMOE_ATTR(0, false); DEAMOE_ATTR(1, false); DEAMOE_ATTR(2, false);
-  DEAMOE_ATTR(0, true); DEAMOE_ATTR(1, true); DEAMOE_ATTR(2, true);
+  DEAMOE_ATTR(0, false); DEAMOE_ATTR(1, false); DEAMOE_ATTR(2, false); DEAMOE_ATTR(3, false);
+  DEAMOE_ATTR(0, true); DEAMOE_ATTR(1, true); DEAMOE_ATTR(2, true); DEAMOE_ATTR(3, true);
 #undef DEAMOE_ATTR
   return e;
 }
@@ -1988,11 +1990,17 @@ int stream_route(StreamPlan& p, const LayerDev& L, const void* tokens, int B, cu
   const FinishSmem fl = finish_layout(L.n, L.m, L.k, B);
   const size_t smem = scratch + (size_t)fl.total * 4;
   if (smem > 200 * 1024) return -1;
-  const int mode = topk_warps == 0 ? 0 : ((in_regs && L.n <= 256) ? 1 : 2);
+  const bool plain_router = !(L.k_dept > 0 && L.k_dept < L.m) && !(L.strict_dept && L.k_dept > 0) && L.norm_topk != 0;
+  const int mode = topk_warps == 0 ? 0 : ((in_regs && L.n <= 256) ? (plain_router ? 3 : 1) : 2);
 #define DEAMOE_FINISH(T, V) launch_pdl(k_route_finish<T, V>, dim3(1), dim3(FINISH_THREADS), smem, s, L, dv, B, ny, topk_warps, \
                                        (int)(scratch / 4), user_idx, user_w)
-  if (L.vanilla) { if (mode == 0) DEAMOE_FINISH(0, true); else if (mode == 1) DEAMOE_FINISH(1, true); else DEAMOE_FINISH(2, true); }
-  else { if (mode == 0) DEAMOE_FINISH(0, false); else if (mode == 1) DEAMOE_FINISH(1, false); else DEAMOE_FINISH(2, false); }
+  if (L.vanilla) {
+    if (mode == 0) DEAMOE_FINISH(0, true); else if (mode == 1) DEAMOE_FINISH(1, true); else if (mode == 2) DEAMOE_FINISH(2, true);
+    else DEAMOE_FINISH(3, true);
+  } else {
+    if (mode == 0) DEAMOE_FINISH(0, false); else if (mode == 1) DEAMOE_FINISH(1, false); else if (mode == 2) DEAMOE_FINISH(2, false);
+    else DEAMOE_FINISH(3, false);
+  }
 #undef DEAMOE_FINISH
   return cudaGetLastError() == cudaSuccess ? 2 + extra : -1;
 }
