@@ -60,6 +60,7 @@ constexpr int SLOT_HDR = 128;
 constexpr int NSLOT = 3;
 constexpr int ACT_PAD = 8;   // floats of padding per activation row in shared memory
 constexpr int MAX_QP = 2;    // 8-token passes a consumer warp accumulates for its tile (16 tokens per segment)
+constexpr int SEG_TOKENS = 8 * MAX_QP;   // token rows of a segment: a warp accumulates up to MAX_QP passes of 8 tokens for its tile
 constexpr int RED_FLOATS = CONSUMER_WARPS * MAX_QP * 128;
 constexpr size_t STREAM_SMEM =
     (size_t)NSLOT * SLOT_BYTES + (size_t)NRED * RED_FLOATS * 4 + (size_t)DESC_DEPTH * DESC_BYTES + 1024;
@@ -369,8 +370,8 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
                                  Seg& dst) {
   const StageCfg& sc = P.st[stage];
   const int Tall = unit_tokens(L, stage, id, B);
-  const int t0 = gi * sc.tg;
-  const int T = min(sc.tg, Tall - t0);
+  const int t0 = gi * SEG_TOKENS;
+  const int T = min(SEG_TOKENS, Tall - t0);
   int nB = 1, in_stride = 0, out_stride = 0, out_row0 = 0, dep_idx = -1, dep_target = 0, done_idx = -1, in_row0 = 0;
   const __nv_bfloat16* in0h = nullptr; const __nv_bfloat16* in0l = nullptr;
   const __nv_bfloat16* in1h = nullptr; const __nv_bfloat16* in1l = nullptr;
@@ -396,14 +397,14 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
       if (P.dense)  // the first stage runs in the tensor-core kernel, which may still be running: its count per department
         dep_target = DENSE_S1_ARRIVALS * (2 * L.f / DENSE_TILE_ROWS);
       else
-        dep_target = groups_of(unit_tokens(L, ST_S1, j, B), P.st[ST_S1].tg) * P.st[ST_S1].n_tiles;
+        dep_target = groups_of(unit_tokens(L, ST_S1, j, B), SEG_TOKENS) * P.st[ST_S1].n_tiles;
       done_idx = P.dep_s2 + id;
       break;
     case ST_S3:
       in0h = P.Yh; in0l = P.Yl; in_stride = L.rp; in_row0 = L.expert_off[id] + t0;
       outh = P.Zh; outl = P.Zl; out_stride = L.f; out_row0 = in_row0;
       dep_idx = P.dep_s2 + id;
-      dep_target = groups_of(Tall, P.st[ST_S2].tg) * P.st[ST_S2].n_tiles;
+      dep_target = groups_of(Tall, SEG_TOKENS) * P.st[ST_S2].n_tiles;
       // (dense schedule: the last stage runs in a later kernel, nobody polls this counter, and an item
       // without one spares the epilogue warp its fence and atomic)
       done_idx = P.dense ? -1 : P.dep_s3 + j;
@@ -416,7 +417,7 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
 #pragma unroll 1
         for (int e = 0; e < L.g; ++e) {
           const int Te = L.expert_off[id * L.g + e + 1] - L.expert_off[id * L.g + e];
-          dep_target += groups_of(Te, P.st[ST_S3].tg) * P.st[ST_S3].n_tiles;
+          dep_target += groups_of(Te, SEG_TOKENS) * P.st[ST_S3].n_tiles;
         }
         dep_idx = P.dep_s3 + id;
       }
@@ -431,7 +432,7 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
       in0h = P.Yshh; in0l = P.Yshl; in_stride = L.fs; in_row0 = t0;
       outf = L.Osh; out_stride = L.h; out_row0 = t0;
       dep_idx = P.dep_sh1;
-      dep_target = groups_of(B, P.st[ST_SH1].tg) * P.st[ST_SH1].n_tiles;
+      dep_target = groups_of(B, SEG_TOKENS) * P.st[ST_SH1].n_tiles;
       break;
     case ST_V1:
       in0h = tokh; in0l = tokl; in_stride = L.h; in_list = L.expert_tok + L.expert_off[id] + t0;
@@ -442,7 +443,7 @@ static __device__ void build_seg(const LayerDev& L, const StreamDev& P, int stag
       in0h = P.Yh; in0l = P.Yl; in_stride = L.f; in_row0 = L.expert_off[id] + t0;
       outf = L.O; out_stride = L.h; out_row0 = in_row0;
       dep_idx = P.dep_s2 + id;
-      dep_target = groups_of(Tall, P.st[ST_V1].tg) * P.st[ST_V1].n_tiles;
+      dep_target = groups_of(Tall, SEG_TOKENS) * P.st[ST_V1].n_tiles;
       break;
   }
   const int planes = in0l ? P.planes : 1;
@@ -527,7 +528,7 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
     if (flat < total) {
       const int c = category_of(flat);
       const int stage = cats[c].stage;
-      gc = groups_of(unit_tokens(L, stage, unit_id(L, cats[c].unit_kind, flat - s_ubase[c]), B), P.st[stage].tg);
+      gc = groups_of(unit_tokens(L, stage, unit_id(L, cats[c].unit_kind, flat - s_ubase[c]), B), SEG_TOKENS);
     }
     int incl = gc;
 #pragma unroll
@@ -603,7 +604,7 @@ static __device__ void worklist_block(const LayerDev& L, const StreamDev& P, int
       for (int u = rank * 32 + lane; u < nu; u += per_c * 32) {
         const int flat = s_ubase[c] + u;
         const int id = unit_id(L, cats[c].unit_kind, u);
-        const int gc = groups_of(unit_tokens(L, stage, id, B), P.st[stage].tg);
+        const int gc = groups_of(unit_tokens(L, stage, id, B), SEG_TOKENS);
 #pragma unroll 1
         for (int gi = 0; gi < gc; ++gi) {
           const int si = s_excl[flat] + gi;
@@ -628,7 +629,7 @@ static __device__ void early_first_stage(const LayerDev& L, const StreamDev& P, 
 #pragma unroll 1
   for (int i = tid; i < P.n_dep + MAX_CAT + 8; i += nthr) P.sync[SY_CLAIM + i] = 0;
   const int A = unit_count(L, kind);
-  const int tg = P.st[stage].tg, ips = P.st[stage].items_per_seg;
+  const int tg = SEG_TOKENS, ips = P.st[stage].items_per_seg;
   int carry = 0;  // exclusive scan of the departments' group counts, 'nthr' departments at a time
 #pragma unroll 1
   for (int base = 0; base < A; base += nthr) {
@@ -1106,7 +1107,7 @@ k_stream(LayerDev L, StreamDev P, int B, int cat, int check_deps) {
       Seg* stage_seg = reinterpret_cast<Seg*>(seg_stage);
       for (int st = ST_SH1; ok && st <= PREFIX_LAST_STAGE; ++st) {
         const int ips = P.st[st].items_per_seg;
-        const int n_items = groups_of(B, P.st[st].tg) * ips;
+        const int n_items = groups_of(B, SEG_TOKENS) * ips;
         int have_seg = -1;
         int4 v = make_int4(0, 0, 0, 0);
         for (int x = ((int)blockIdx.x - first_cta + G) % G; ok && x < n_items; x += G) {
@@ -1747,7 +1748,7 @@ static void fill_stage(StageCfg& s, const __nv_bfloat16* w0, const __nv_bfloat16
   s.paired = paired;
   s.q = 2;                      // two 16-row tiles per item: (gate, up) of paired stages, else rows r, r+16
   s.epi = epi;
-  s.tg = 8 * MAX_QP;            // a warp accumulates up to MAX_QP passes of 8 tokens for its tile
+  s.tg = SEG_TOKENS;            // (the kernels use the constant: a run-time divisor costs a division per use)
   s.items_per_seg = paired ? s.n_tiles : (s.n_tiles + s.q - 1) / s.q;
   s.enabled = 1; s.pad = 0;
 }
