@@ -424,10 +424,12 @@ static __device__ void topk_one_token_wide(const LayerDev& L, int t, int B, int 
       ahead += better(s2, d2, dscore, lane) ? 1 : 0;
     }
     const unsigned alive = __ballot_sync(0xffffffffu, lane < m && ahead < L.k_dept);
+    const unsigned inv = (g > 1) ? (unsigned)((0x100000000ull + (unsigned)g - 1u) / (unsigned)g) : 0u;  // ceil(2^32 / g)
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int idx = base + lane + 32 * j;
-      if (idx < n && !((alive >> (idx / g)) & 1u)) taken |= 1u << j;
+      const unsigned idx = (unsigned)(base + lane + 32 * j);
+      const unsigned d = (g > 1) ? __umulhi(idx, inv) : idx;  // idx / g, exact for idx * g < 2^32
+      if (idx < (unsigned)n && !((alive >> d) & 1u)) taken |= 1u << j;
     }
   }
   // this warp's k best (order-preserving integer keys, 0 = not a candidate)
