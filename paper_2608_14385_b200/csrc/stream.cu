@@ -1923,7 +1923,7 @@ deamoe_status_t stream_plan_create(const LayerDev& L, const deamoe_weights_t& w,
   // that can be called with that many).  Its routing and its streaming launch see the plan with
   // the fused schedule's hand-overs switched off and the private stages as the whole list.
   p->dense_min = dense_mode == 2 ? 1 : (L.n >= DENSE_SMALL_ROUTER ? DENSE_MIN_BATCH : 2 * DENSE_MIN_BATCH);
-  if (dense_mode == 2 || (dense_mode == 1 && dense_supported(L) && L.max_batch >= DENSE_MIN_BATCH)) {
+  if (dense_mode == 2 || (dense_mode == 1 && dense_supported(L) && L.max_batch >= p->dense_min)) {
     uint64_t db = 0;
     const deamoe_status_t ds = dense_plan_create(L, w, s, &p->dense, &db);
     if (ds != DEAMOE_OK) {
